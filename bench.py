@@ -1,0 +1,372 @@
+#!/usr/bin/env python
+"""Benchmark of the rollout denoising step (attention -> LM head/confidence -> unmask selection).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+A "step" is one pass of the whole hot path over one batch: dare_denoise_block on the LLaDA-8B-shaped
+workload (batch 16 rollouts, prompt 512 + generation 256 in blocks of 32, top-k = 2 per step, so 16 steps
+per block and 128 steps per generation; after 128 steps the token state is re-masked and the prefix length
+returns to the prompt).  The metric is denoised (committed) tokens per second.
+
+N > 1 (torchrun): every rank runs the same workload on its own rollouts (batch rows are independent, no
+data-path collective); value = tokens of all ranks / max-over-ranks time ("weak" scaling).
+
+`--impl reference` times the CPU oracle (oracle/dare_oracle.py) as it stands on a bounded sample of the same
+workload, on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2604_04215_b200 import inputs as I  # noqa: E402
+
+METRIC = "denoised_tokens_per_sec"
+UNIT = "tokens/s"
+NPOOL = 4   # distinct activation sets cycled through the steps
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unsampled"]}
+        time.sleep(0.15)
+        self.proc.terminate()       # the exact child started above
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, mx, reasons = [], [], set()
+        for ts, line in self.lines:
+            if ts < t0 or ts > t1 + 0.1:
+                continue
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unsampled"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def lm_rows_masked(wl, s_in_block):
+    """Masked rows entering step s of a block under top-k: every rollout still has L - k*s masks."""
+    return wl.batch * max(0, wl.block_len - wl.k * s_in_block)
+
+
+def run_ours(args):
+    from paper_2604_04215_b200 import binding as dare
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback for the product path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    wl = I.scaled(I.WORKLOADS[args.workload], seed=rank)
+    ctx = dare.Context(local)
+    B, L = wl.batch, wl.block_len
+    steps_per_block = -(-L // wl.k) if wl.mode == I.SELECT_TOPK else L
+    steps_per_gen = steps_per_block * wl.n_blocks
+
+    # ---- resident state: weights, in-place KV cache (filled over its whole capacity), pristine tokens
+    w_h = I.normal_bf16(0, I.TID_W, (wl.vocab, wl.hidden), 0.02)           # same weights on every rank
+    k_pre_h, v_pre_h, k_suf_h, v_suf_h = I.make_caches(wl)
+    tok0_h = I.fresh_tokens(wl)
+    w = w_h.cuda(); k_pre = k_pre_h.cuda(); v_pre = v_pre_h.cuda()
+    k_suf = k_suf_h.cuda() if k_suf_h is not None else None
+    v_suf = v_suf_h.cuda() if v_suf_h is not None else None
+    suffix_len = torch.full((B,), wl.suffix_cap, dtype=torch.int32, device="cuda") if wl.suffix_cap else None
+    tok0 = tok0_h.cuda()
+    tokens = tok0.clone()
+    plen_blocks = [torch.full((B,), wl.prompt_len + b * L, dtype=torch.int32, device="cuda") for b in range(wl.n_blocks)]
+    # ---- per-step activations: a small pool, pinned on the host for the end-to-end leg
+    pool_h = []
+    for i in range(NPOOL):
+        q, _, _, x = I.make_step_activations(wl, i, inplace_block=True)
+        pool_h.append((q.pin_memory(), x.pin_memory()))
+    pool = [(q.cuda(), x.cuda()) for q, x in pool_h]
+    attn_out = torch.empty(B, L, wl.n_q_heads, wl.head_dim, dtype=torch.bfloat16, device="cuda")
+    pred = torch.empty(B * L, dtype=torch.int32, device="cuda")
+    conf = torch.empty(B * L, dtype=torch.float32, device="cuda")
+    n_total = args.steps + args.warmup
+    nc_all = torch.zeros(max(n_total, 1), B, dtype=torch.int32, device="cuda")
+    nr = torch.zeros(B, dtype=torch.int32, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def step(t, q, x, nc):
+        g = t % steps_per_gen
+        b = g // steps_per_block
+        if g == 0:
+            tokens.copy_(tok0)                                  # new generation: re-mask (one small copy)
+        dare.dare_denoise_block(ctx, q, k_pre, v_pre, plen_blocks[b], None, None, k_suf, v_suf, suffix_len,
+                                attn_out, None, x, w, wl.mask_id, True, tokens, wl.prompt_len + b * L,
+                                wl.mode, wl.threshold, wl.k, pred, conf, nc, nr, stream=stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    # ---- device-resident timed region
+    for t in range(args.warmup):
+        q, x = pool[t % NPOOL]
+        step(t, q, x, nc_all[t])
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    w0 = time.time()
+    e0.record(stream)
+    for t in range(args.warmup, n_total):
+        q, x = pool[t % NPOOL]
+        step(t, q, x, nc_all[t])
+    e1.record(stream)
+    barrier()
+    w1 = time.time()
+    clocks = sampler.stop(w0, w1) if rank == 0 else None
+    ms = e0.elapsed_time(e1)
+    committed = int(nc_all[args.warmup:n_total].sum().item())
+    if ctx.device_status() != 0:
+        raise RuntimeError("device status word is non-zero after the timed region")
+    t_ms = torch.tensor([ms], dtype=torch.float64, device="cuda")
+    tot = torch.tensor([committed], dtype=torch.float64, device="cuda")
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t_ms, op=dist.ReduceOp.MAX)
+        dist.all_reduce(tot, op=dist.ReduceOp.SUM)
+    ms_max, committed_all = float(t_ms.item()), float(tot.item())
+    value = committed_all / (ms_max * 1e-3)
+
+    # ---- instrumented pass: the same steps issued as the three entry points with events between them, to
+    #      attribute time to the dominant kernel (LM head) for the roofline
+    n_inst = min(args.steps, 2 * steps_per_gen)
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(n_inst)]
+    tokens.copy_(tok0)
+    torch.cuda.synchronize()
+    for t in range(n_inst):
+        g = t % steps_per_gen
+        b = g // steps_per_block
+        if g == 0:
+            tokens.copy_(tok0)
+        q, x = pool[t % NPOOL]
+        bs = wl.prompt_len + b * L
+        ev[t][0].record(stream)
+        dare.dare_attn_block(ctx, q, k_pre, v_pre, plen_blocks[b], None, None, k_suf, v_suf, suffix_len, attn_out,
+                             None, stream=stream)
+        ev[t][1].record(stream)
+        rt = tokens[:, bs:bs + L].contiguous().view(-1)
+        ev[t][1].record(stream)
+        dare.dare_lmhead_confidence(ctx, x, w, rt, wl.mask_id, True, pred, conf, stream=stream)
+        ev[t][2].record(stream)
+        dare.dare_unmask_select(ctx, tokens, bs, L, pred, conf, wl.mask_id, wl.mode, wl.threshold, wl.k, nr, nr,
+                                stream=stream)
+        ev[t][3].record(stream)
+    torch.cuda.synchronize()
+    lm_ms = float(np.mean([ev[t][1].elapsed_time(ev[t][2]) for t in range(n_inst)]))
+    attn_ms = float(np.mean([ev[t][0].elapsed_time(ev[t][1]) for t in range(n_inst)]))
+    sel_ms = float(np.mean([ev[t][2].elapsed_time(ev[t][3]) for t in range(n_inst)]))
+    if wl.mode == I.SELECT_TOPK:
+        masked_avg = float(np.mean([lm_rows_masked(wl, (t % steps_per_gen) % steps_per_block) for t in range(n_inst)]))
+    else:
+        masked_avg = float(B * L)
+    peaks = _peaks()
+    lm_flops = 2.0 * masked_avg * wl.hidden * wl.vocab          # algorithmic: masked rows only
+    achieved = lm_flops / (lm_ms * 1e-3) / 1e12
+    peak = peaks["bf16_tflops_sustained"]
+    roofline = {"bound": "tensor", "kernel": "lmhead_partial_kernel(+merge)", "achieved": achieved, "peak": peak,
+                "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None, "peak_source": peaks["source"] + " sustained",
+                "executed_tflops": 2.0 * B * L * wl.hidden * wl.vocab / (lm_ms * 1e-3) / 1e12,
+                "ms_per_launch": lm_ms, "masked_rows_avg": masked_avg,
+                "frac_of_nominal_2250": achieved / 2250.0}
+    kv_bytes = 2.0 * 2 * B * wl.n_kv_heads * wl.head_dim * (
+        float(np.mean([wl.prompt_len + ((t % steps_per_gen) // steps_per_block) * L + L for t in range(n_inst)])) + wl.suffix_cap)
+    qo_bytes = 2.0 * 2 * B * L * wl.n_q_heads * wl.head_dim
+    attn_gbs = (kv_bytes + qo_bytes) / (attn_ms * 1e-3) / 1e9
+    breakdown = {"attn_ms": attn_ms, "lmhead_ms": lm_ms, "select_ms": sel_ms, "attn_GBps": attn_gbs,
+                 "attn_frac_hbm": attn_gbs / peaks["hbm_gbs"]}
+
+    # ---- end to end: the step's activations come from pinned host memory, results go back to the host
+    n_e2e = min(args.steps, 4 * steps_per_gen)
+    q_d, x_d = torch.empty_like(pool[0][0]), torch.empty_like(pool[0][1])
+    nc_h = torch.zeros(B, dtype=torch.int32).pin_memory()
+    nr_h = torch.zeros(B, dtype=torch.int32).pin_memory()
+    tok_blk_h = torch.zeros(B, L, dtype=torch.int32).pin_memory()
+    nc_d = torch.zeros(B, dtype=torch.int32, device="cuda")
+    barrier()
+    e2e_tokens = 0
+    ta = time.perf_counter()
+    for t in range(n_e2e):
+        qh, xh = pool_h[t % NPOOL]
+        q_d.copy_(qh, non_blocking=True)
+        x_d.copy_(xh, non_blocking=True)
+        step(t, q_d, x_d, nc_d)
+        g = t % steps_per_gen
+        bs = wl.prompt_len + (g // steps_per_block) * L
+        nc_h.copy_(nc_d, non_blocking=True)
+        nr_h.copy_(nr, non_blocking=True)
+        tok_blk_h.copy_(tokens[:, bs:bs + L], non_blocking=True)
+        torch.cuda.synchronize()
+        e2e_tokens += int(nc_h.sum())
+    tb = time.perf_counter()
+    e2e_t = torch.tensor([tb - ta], dtype=torch.float64, device="cuda")
+    e2e_n = torch.tensor([e2e_tokens], dtype=torch.float64, device="cuda")
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(e2e_t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(e2e_n, op=dist.ReduceOp.SUM)
+    h2d = pool_h[0][0].numel() * 2 + pool_h[0][1].numel() * 2
+    d2h = 4 * (B + B + B * L)
+    e2e = {"value": float(e2e_n.item()) / float(e2e_t.item()), "unit": UNIT, "h2d_bytes_per_step": h2d,
+           "d2h_bytes_per_step": d2h, "steps": n_e2e}
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu_baseline = time_oracle(wl, w_h, (k_pre_h, v_pre_h, k_suf_h, v_suf_h), budget_s=20.0)
+
+    if rank == 0:
+        attn_launches = 1   # + 1 combine launch when the attention plan splits KV (not in this workload)
+        out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+               "warmup": args.warmup, "ms_per_step": ms_max / args.steps, "higher_is_better": True,
+               "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+               "config": {"workload": f"{wl.name}: B{B} L{L} Hq{wl.n_q_heads}/Hkv{wl.n_kv_heads} d{wl.head_dim} "
+                                      f"D{wl.hidden} V{wl.vocab} prompt{wl.prompt_len}+gen{wl.gen_len} "
+                                      f"{'top-k ' + str(wl.k) if wl.mode == I.SELECT_TOPK else 'tau ' + str(wl.threshold)}",
+                          "l2": "inputs larger than L2 (W 1.04 GB and KV cache 0.2 GB are re-read every step)",
+                          "parallelism": f"dp{world} (independent rollouts per GPU, no collective)"},
+               "clocks": clocks, "e2e": e2e, "gpu_launches": (attn_launches + 3) * args.steps,
+               "roofline": roofline, "breakdown": breakdown, "cpu_baseline": cpu_baseline}
+        print(json.dumps(out))
+    ctx.close()
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def time_oracle(wl, w_h, caches_h, budget_s=20.0, max_steps=64):
+    """Times the oracle, as it stands, on a bounded sample: ONE rollout (of the batch) per step."""
+    from oracle import dare_oracle as O
+    sub = I.scaled(wl, batch=1)
+    k_pre, v_pre, k_suf, v_suf = [None if c is None else c[:1].to(torch.float64).numpy() for c in caches_h]
+    w64 = w_h.to(torch.float64).numpy()
+    tokens = I.fresh_tokens(sub).numpy()
+    L = wl.block_len
+    plen = np.array([wl.prompt_len])
+    slen = np.array([wl.suffix_cap]) if wl.suffix_cap else None
+    committed, steps = 0, 0
+    t0 = time.perf_counter()
+    while steps < max_steps and (time.perf_counter() - t0 < budget_s or steps == 0):
+        q, _, _, x = I.make_step_activations(sub, steps % NPOOL, inplace_block=True)
+        res = O.denoise_step(q.to(torch.float64).numpy(), k_pre, v_pre, plen, None, None, k_suf, v_suf, slen,
+                             x.to(torch.float64).numpy(), w64, tokens, wl.prompt_len, L, wl.mask_id, wl.mode,
+                             wl.threshold, wl.k)
+        committed += int(res["n_committed"].sum())
+        tokens = res["tokens"]
+        if (tokens[:, wl.prompt_len:wl.prompt_len + L] != wl.mask_id).all():
+            tokens = I.fresh_tokens(sub).numpy()
+        steps += 1
+    dt = time.perf_counter() - t0
+    return {"value": committed / dt, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
+            "sample": f"{steps} steps of 1 rollout out of {wl.batch} (all heads, full vocabulary), {dt:.1f} s; "
+                      f"tokens/s of that single rollout, not scaled",
+            "seconds_per_step_one_rollout": dt / steps}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl = I.WORKLOADS[args.workload]
+    w_h = I.normal_bf16(0, I.TID_W, (wl.vocab, wl.hidden), 0.02)
+    caches = I.make_caches(I.scaled(wl, batch=1))
+    n = max(1, min(args.steps, 16))
+    nw = max(0, min(args.warmup, 2))
+    if nw:
+        time_oracle(wl, w_h, caches, budget_s=0.0, max_steps=nw)
+    res = time_oracle(wl, w_h, caches, budget_s=1e9, max_steps=n)
+    out = {"impl": "reference", "metric": METRIC, "value": res["value"], "unit": UNIT, "n_gpus": args.gpus,
+           "steps": n, "warmup": nw, "ms_per_step": res["seconds_per_step_one_rollout"] * 1e3,
+           "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+           "config": {"workload": f"{wl.name} (bounded sample: one rollout of the batch per step)"},
+           "cpu_baseline": {"value": res["value"], "unit": UNIT, "cores": res["cores"], "kind": "oracle",
+                            "sample": res["sample"]},
+           "e2e": {"value": res["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(out))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1536)
+    ap.add_argument("--warmup", type=int, default=32)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llada8b", choices=sorted(I.WORKLOADS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,158 @@
+/*
+ * dare.h -- C ABI of the B200 (sm_100a) rollout denoising step for diffusion LLMs.
+ *
+ * One denoising step of the cached rollout the paper describes in Section 3.4
+ * ("Rollout-side optimization for MDLMs": KV-cache reuse and repeated denoising on
+ * partially fixed states) and Section 2.1 (block diffusion: bidirectional inside a
+ * block, earlier blocks fixed):
+ *
+ *     dare_attn_block         block queries x (prefix cache + block + optional suffix cache), GQA
+ *     dare_lmhead_confidence  LM head + vocabulary softmax -> (argmax token, max probability) per row,
+ *                             logits never written to memory
+ *     dare_unmask_select      confidence-threshold / per-block top-k commit on the int32 token state
+ *     dare_denoise_block      the three above, enqueued back to back
+ *
+ * Conventions
+ *   - Every data pointer is a DEVICE pointer unless the comment says "host".  The caller owns every
+ *     buffer; the library neither frees nor keeps them after the call's stream work has run.
+ *   - All entry points enqueue work on `stream` (a cudaStream_t passed as void*, NULL = default
+ *     stream) and return without synchronising.  They allocate nothing; the only allocation is the
+ *     workspace made once by dare_create.
+ *   - bf16 tensors are dense, row-major, 16-byte aligned.
+ *   - Return value: DARE_OK (0) or a negative dare_status.  On any error nothing has been launched.
+ *   - Data-dependent anomalies (a per-row length beyond its capacity, a wait inside a kernel that
+ *     ran out of its bounded time) never trap: they set bits in a device status word that
+ *     dare_device_status reads.
+ *   - One ctx serves one stream at a time (the workspace is shared by consecutive calls).
+ */
+#ifndef DARE_H_
+#define DARE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dare_ctx dare_ctx;
+
+typedef enum {
+    DARE_OK = 0,
+    DARE_ERR_NULL = -1,        /* a required pointer is NULL                                   */
+    DARE_ERR_SHAPE = -2,       /* unsupported or inconsistent dimensions                       */
+    DARE_ERR_ALIGN = -3,       /* pointer not 16-byte aligned / row size not a 16-byte multiple */
+    DARE_ERR_RANGE = -4,       /* scalar out of range (k < 1, NaN threshold, mask id, window)   */
+    DARE_ERR_WORKSPACE = -5,   /* ctx workspace too small for this call                         */
+    DARE_ERR_CUDA = -6,        /* a CUDA runtime/driver call failed                             */
+    DARE_ERR_UNSUPPORTED = -7  /* device is not sm_100                                          */
+} dare_status;
+
+/* bits of the device status word */
+#define DARE_DEV_LEN_CLAMPED 1u   /* a prefix/suffix length exceeded its capacity and was clamped */
+#define DARE_DEV_WAIT_EXPIRED 2u  /* a bounded wait inside a kernel gave up; outputs are invalid  */
+
+enum { DARE_SELECT_THRESHOLD = 0, DARE_SELECT_TOPK = 1 };
+
+/* Create a context on `device` with a workspace of `workspace_bytes` (0 = library default, 256 MiB).
+ * *out (host) receives the handle.  Allocates device memory; call outside any stream capture. */
+int dare_create(dare_ctx** out, int device, size_t workspace_bytes);
+int dare_destroy(dare_ctx* ctx);
+
+/* Static string for a status code (host pointer, never NULL). */
+const char* dare_status_string(int status);
+
+/* Synchronises `stream`, copies the device status word to *host_out (host) and clears it. */
+int dare_device_status(dare_ctx* ctx, void* stream, uint32_t* host_out);
+
+/* Number of SMs the ctx's device reports (launch shapes are sized from it). */
+int dare_sm_count(const dare_ctx* ctx);
+
+/*
+ * Block-bidirectional attention against the caches (Section 2.1; Section 3.4).
+ * For every row r, query head h (KV head h / (Hq/Hkv)) and block position i:
+ *     o = softmax_j(scale * <q, k_j>) . v_j   over all visible keys j:
+ *         prefix [0, prefix_len[r])  U  the block's own L keys  U  suffix [0, suffix_len[r]).
+ * No mask inside the visible set (bidirectional).  bf16 in, fp32 accumulate, bf16 out.
+ *
+ *   q            bf16 [B, L, Hq, d]
+ *   k_pre,v_pre  bf16 [B, Hkv, prefix_cap, d]
+ *   prefix_len   int32 [B] or NULL (= prefix_cap, or prefix_cap - L when the block is in place)
+ *   k_blk,v_blk  bf16 [B, Hkv, L, d]; both NULL => the block's K/V live in k_pre/v_pre at
+ *                [prefix_len, prefix_len + L)
+ *   k_suf,v_suf  bf16 [B, Hkv, suffix_cap, d] or both NULL (no dual cache)
+ *   suffix_len   int32 [B] or NULL (= suffix_cap)
+ *   out          bf16 [B, L, Hq, d]
+ *   lse          fp32 [B, Hq, L] or NULL: natural-log sum of exp(scale * score)
+ *   scale        softmax scale; 0 => 1/sqrt(d)
+ * Supported: d in {64, 128}; Hq % Hkv == 0; L >= 1; L * (Hq/Hkv) <= 1024.
+ * Lengths beyond capacity are clamped and flagged in the device status word.
+ */
+int dare_attn_block(dare_ctx* ctx,
+                    int B, int L, int Hq, int Hkv, int d, int prefix_cap, int suffix_cap, float scale,
+                    const void* q,
+                    const void* k_pre, const void* v_pre, const int32_t* prefix_len,
+                    const void* k_blk, const void* v_blk,
+                    const void* k_suf, const void* v_suf, const int32_t* suffix_len,
+                    void* out, float* lse, void* stream);
+
+/*
+ * Fused LM head + vocabulary softmax (Section 3.4, the logits-free idea the paper cites for its fused
+ * loss kernels, applied to decoding): for each row m,
+ *     z = hidden[m] . w^T  (V logits, kept on chip);  z[mask_id] = -inf if exclude_mask_column;
+ *     pred[m] = lowest index attaining max z;  conf[m] = exp(max z - logsumexp z).
+ *
+ *   hidden       bf16 [M, D]        w  bf16 [V, D]  (one row per vocabulary entry)
+ *   row_tokens   int32 [M] or NULL: rows whose token != mask_id are already committed and get
+ *                pred = that token, conf = -inf
+ *   pred         int32 [M] out      conf  fp32 [M] out
+ * Supported: D % 8 == 0, D >= 8; V >= 2; M >= 1.  Needs ctx workspace of 12 * ceil(V/256) *
+ * roundup(M,128) bytes.
+ */
+int dare_lmhead_confidence(dare_ctx* ctx,
+                           const void* hidden, int M, int D, const void* w, int V,
+                           const int32_t* row_tokens, int32_t mask_id, int exclude_mask_column,
+                           int32_t* pred, float* conf, void* stream);
+
+/*
+ * Parallel unmask selection, in place on the token state (Section 3.4, "partially fixed states";
+ * Section 4.2: block length 32, two tokens per step).  Per row, U = block positions whose token is
+ * mask_id.  THRESHOLD: commit every i in U with conf > threshold, or the single most confident one
+ * (lowest i on ties) if none passes.  TOPK: commit the min(k, #U) most confident (lower i first on
+ * ties).  Committed: tokens[r, block_start + i] = pred[r, i].  Everything else is left as it is.
+ * Comparisons are in fp32; NaN counts as -inf.
+ *
+ *   tokens       int32 [B, row_stride] in/out     pred int32 [B, L]     conf fp32 [B, L]
+ *   n_committed, n_remaining   int32 [B] out, each may be NULL
+ * Supported: 1 <= L <= 4096; 0 <= block_start, block_start + L <= row_stride.
+ */
+int dare_unmask_select(dare_ctx* ctx,
+                       int32_t* tokens, int B, int64_t row_stride, int block_start, int L,
+                       const int32_t* pred, const float* conf,
+                       int32_t mask_id, int mode, float threshold, int k,
+                       int32_t* n_committed, int32_t* n_remaining, void* stream);
+
+/*
+ * One whole denoising step: dare_attn_block, then dare_lmhead_confidence on the block's rows
+ * (row_tokens taken from tokens[:, block_start : block_start + L], M = B * L), then
+ * dare_unmask_select.  `hidden` is the LM-head input for the B*L block positions.  pred/conf are
+ * caller-provided [B*L] buffers that also serve as the step's intermediate results.
+ */
+int dare_denoise_block(dare_ctx* ctx,
+                       int B, int L, int Hq, int Hkv, int d, int prefix_cap, int suffix_cap, float scale,
+                       const void* q,
+                       const void* k_pre, const void* v_pre, const int32_t* prefix_len,
+                       const void* k_blk, const void* v_blk,
+                       const void* k_suf, const void* v_suf, const int32_t* suffix_len,
+                       void* attn_out, float* lse,
+                       const void* hidden, int D, const void* w, int V,
+                       int32_t mask_id, int exclude_mask_column,
+                       int32_t* tokens, int64_t row_stride, int block_start,
+                       int mode, float threshold, int k,
+                       int32_t* pred, float* conf,
+                       int32_t* n_committed, int32_t* n_remaining, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DARE_H_ */

@@ -1,0 +1,190 @@
+"""ctypes binding of libdare.so: argument marshalling only.
+
+The functions carry the names of the C entry points (include/dare.h).  Tensors are torch CUDA tensors
+used purely as device memory; every step runs inside the library's kernels.  There is no fallback: if
+the shared library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdare.so")
+
+SELECT_THRESHOLD = 0
+SELECT_TOPK = 1
+DEV_LEN_CLAMPED = 1
+DEV_WAIT_EXPIRED = 2
+
+EXPORTS = ["dare_create", "dare_destroy", "dare_status_string", "dare_device_status", "dare_sm_count",
+           "dare_attn_block", "dare_lmhead_confidence", "dare_unmask_select", "dare_denoise_block"]
+
+_lib = None
+
+
+class DareError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = load().dare_status_string(code).decode()
+        super().__init__(f"{where}: {msg} ({code})")
+
+
+def load():
+    """Load the shared library (built in-tree by paper_2604_04215_b200.build); raises if it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2604_04215_b200.build` "
+                           "(there is no fallback path)")
+    lib = C.CDLL(LIB_PATH)
+    vp, i32, i64, f32 = C.c_void_p, C.c_int, C.c_int64, C.c_float
+    lib.dare_create.argtypes = [C.POINTER(vp), i32, C.c_size_t]
+    lib.dare_create.restype = i32
+    lib.dare_destroy.argtypes = [vp]
+    lib.dare_destroy.restype = i32
+    lib.dare_status_string.argtypes = [i32]
+    lib.dare_status_string.restype = C.c_char_p
+    lib.dare_device_status.argtypes = [vp, vp, C.POINTER(C.c_uint32)]
+    lib.dare_device_status.restype = i32
+    lib.dare_sm_count.argtypes = [vp]
+    lib.dare_sm_count.restype = i32
+    attn_args = [i32] * 7 + [f32] + [vp] * 12
+    lib.dare_attn_block.argtypes = [vp] + attn_args
+    lib.dare_attn_block.restype = i32
+    lib.dare_lmhead_confidence.argtypes = [vp, vp, i32, i32, vp, i32, vp, i32, i32, vp, vp, vp]
+    lib.dare_lmhead_confidence.restype = i32
+    lib.dare_unmask_select.argtypes = [vp, vp, i32, i64, i32, i32, vp, vp, i32, i32, f32, i32, vp, vp, vp]
+    lib.dare_unmask_select.restype = i32
+    lib.dare_denoise_block.argtypes = ([vp] + [i32] * 7 + [f32] + [vp] * 11 +   # attention operands .. lse
+                                       [vp, i32, vp, i32, i32, i32,              # hidden, D, w, V, mask, excl
+                                        vp, i64, i32, i32, f32, i32,             # tokens, stride, start, mode, thr, k
+                                        vp, vp, vp, vp, vp])                     # pred, conf, n_comm, n_rem, stream
+    lib.dare_denoise_block.restype = i32
+    _lib = lib
+    return lib
+
+
+def _ptr(t: Optional[torch.Tensor], dtype=None):
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("expected a contiguous CUDA tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError(f"expected dtype {dtype}, got {t.dtype}")
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> C.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+class Context:
+    """Owns a dare_ctx (workspace + device status word) on one device."""
+
+    def __init__(self, device: int = 0, workspace_bytes: int = 0):
+        lib = load()
+        h = C.c_void_p()
+        rc = lib.dare_create(C.byref(h), int(device), int(workspace_bytes))
+        if rc != 0:
+            raise DareError(rc, "dare_create")
+        self.handle = h
+        self.device = device
+
+    def close(self):
+        if getattr(self, "handle", None):
+            load().dare_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @property
+    def sm_count(self) -> int:
+        return load().dare_sm_count(self.handle)
+
+    def device_status(self, stream=None) -> int:
+        out = C.c_uint32(0)
+        rc = load().dare_device_status(self.handle, _stream(stream), C.byref(out))
+        if rc != 0:
+            raise DareError(rc, "dare_device_status")
+        return int(out.value)
+
+
+def dare_attn_block(ctx: Context, q, k_pre, v_pre, prefix_len=None, k_blk=None, v_blk=None, k_suf=None, v_suf=None,
+                    suffix_len=None, out=None, lse=None, scale: float = 0.0, stream=None, check: bool = True):
+    B, L, Hq, d = q.shape
+    Hkv, prefix_cap = k_pre.shape[1], k_pre.shape[2]
+    suffix_cap = k_suf.shape[2] if k_suf is not None else 0
+    if out is None:
+        out = torch.empty_like(q)
+    bf = torch.bfloat16
+    rc = load().dare_attn_block(ctx.handle, B, L, Hq, Hkv, d, prefix_cap, suffix_cap, float(scale),
+                                _ptr(q, bf), _ptr(k_pre, bf), _ptr(v_pre, bf), _ptr(prefix_len, torch.int32),
+                                _ptr(k_blk, bf), _ptr(v_blk, bf), _ptr(k_suf, bf), _ptr(v_suf, bf),
+                                _ptr(suffix_len, torch.int32), _ptr(out, bf), _ptr(lse, torch.float32),
+                                _stream(stream))
+    if rc != 0 and check:
+        raise DareError(rc, "dare_attn_block")
+    return out if check else rc
+
+
+def dare_lmhead_confidence(ctx: Context, hidden, w, row_tokens=None, mask_id: int = -1,
+                           exclude_mask_column: bool = True, pred=None, conf=None, stream=None, check: bool = True):
+    M, D = hidden.shape
+    V = w.shape[0]
+    if pred is None:
+        pred = torch.empty(M, dtype=torch.int32, device=hidden.device)
+    if conf is None:
+        conf = torch.empty(M, dtype=torch.float32, device=hidden.device)
+    rc = load().dare_lmhead_confidence(ctx.handle, _ptr(hidden, torch.bfloat16), M, D, _ptr(w, torch.bfloat16), V,
+                                       _ptr(row_tokens, torch.int32), int(mask_id), int(bool(exclude_mask_column)),
+                                       _ptr(pred, torch.int32), _ptr(conf, torch.float32), _stream(stream))
+    if rc != 0 and check:
+        raise DareError(rc, "dare_lmhead_confidence")
+    return (pred, conf) if check else rc
+
+
+def dare_unmask_select(ctx: Context, tokens, block_start: int, L: int, pred, conf, mask_id: int, mode: int,
+                       threshold: float = 0.0, k: int = 1, n_committed=None, n_remaining=None, stream=None,
+                       check: bool = True):
+    B, row_stride = tokens.shape
+    rc = load().dare_unmask_select(ctx.handle, _ptr(tokens, torch.int32), B, row_stride, int(block_start), int(L),
+                                   _ptr(pred, torch.int32), _ptr(conf, torch.float32), int(mask_id), int(mode),
+                                   float(threshold), int(k), _ptr(n_committed, torch.int32),
+                                   _ptr(n_remaining, torch.int32), _stream(stream))
+    if rc != 0 and check:
+        raise DareError(rc, "dare_unmask_select")
+    return rc
+
+
+def dare_denoise_block(ctx: Context, q, k_pre, v_pre, prefix_len, k_blk, v_blk, k_suf, v_suf, suffix_len,
+                       attn_out, lse, hidden, w, mask_id: int, exclude_mask_column: bool, tokens, block_start: int,
+                       mode: int, threshold: float, k: int, pred, conf, n_committed=None, n_remaining=None,
+                       scale: float = 0.0, stream=None, check: bool = True):
+    B, L, Hq, d = q.shape
+    Hkv, prefix_cap = k_pre.shape[1], k_pre.shape[2]
+    suffix_cap = k_suf.shape[2] if k_suf is not None else 0
+    D = hidden.shape[1]
+    V = w.shape[0]
+    bf = torch.bfloat16
+    rc = load().dare_denoise_block(
+        ctx.handle, B, L, Hq, Hkv, d, prefix_cap, suffix_cap, float(scale),
+        _ptr(q, bf), _ptr(k_pre, bf), _ptr(v_pre, bf), _ptr(prefix_len, torch.int32), _ptr(k_blk, bf), _ptr(v_blk, bf),
+        _ptr(k_suf, bf), _ptr(v_suf, bf), _ptr(suffix_len, torch.int32), _ptr(attn_out, bf), _ptr(lse, torch.float32),
+        _ptr(hidden, bf), D, _ptr(w, bf), V, int(mask_id), int(bool(exclude_mask_column)),
+        _ptr(tokens, torch.int32), tokens.shape[1], int(block_start), int(mode), float(threshold), int(k),
+        _ptr(pred, torch.int32), _ptr(conf, torch.float32), _ptr(n_committed, torch.int32),
+        _ptr(n_remaining, torch.int32), _stream(stream))
+    if rc != 0 and check:
+        raise DareError(rc, "dare_denoise_block")
+    return rc

@@ -1,0 +1,211 @@
+// C-ABI entry points: argument validation, context/workspace, tensor-map encoding, launches.
+// Nothing here computes; every step of the path runs in the kernels of lmhead.cu, attn.cu and select.cu.
+#include <math.h>
+#include <new>
+#include <stdlib.h>
+
+#include "internal.h"
+
+namespace dare {
+
+int make_tmap_bf16_2d(const dare_ctx* ctx, CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols,
+                      uint32_t box_rows, uint32_t box_cols) {
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * 2};   // bytes, dimension 1
+    cuuint32_t box[2] = {box_cols, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = ctx->encode_tiled(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides,
+                                   box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? DARE_OK : DARE_ERR_CUDA;
+}
+
+}  // namespace dare
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_attn(const dare_ctx* ctx, int B, int L, int Hq, int Hkv, int d, int prefix_cap, int suffix_cap, float scale,
+               const void* q, const void* k_pre, const void* v_pre, const void* k_blk, const void* v_blk,
+               const void* k_suf, const void* v_suf, const void* out, dare::AttnArgs* a) {
+    if (!ctx || !q || !k_pre || !v_pre || !out) return DARE_ERR_NULL;
+    if ((k_blk == nullptr) != (v_blk == nullptr)) return DARE_ERR_NULL;
+    if ((k_suf == nullptr) != (v_suf == nullptr)) return DARE_ERR_NULL;
+    if (B < 1 || L < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv != 0) return DARE_ERR_SHAPE;
+    if (d != 64 && d != 128) return DARE_ERR_SHAPE;
+    if (static_cast<long long>(L) * (Hq / Hkv) > 1024) return DARE_ERR_SHAPE;
+    if (prefix_cap < (k_blk ? 1 : L) || suffix_cap < 0) return DARE_ERR_SHAPE;
+    if (k_suf && suffix_cap < 1) return DARE_ERR_SHAPE;
+    if (static_cast<long long>(B) * Hkv * prefix_cap > 0x7fffffffLL) return DARE_ERR_SHAPE;
+    if (!(scale >= 0.f) || isinf(scale)) return DARE_ERR_RANGE;
+    if (!aligned16(q) || !aligned16(k_pre) || !aligned16(v_pre) || !aligned16(out) || !aligned16(k_blk) ||
+        !aligned16(v_blk) || !aligned16(k_suf) || !aligned16(v_suf))
+        return DARE_ERR_ALIGN;
+    a->B = B; a->L = L; a->Hq = Hq; a->Hkv = Hkv; a->d = d; a->prefix_cap = prefix_cap; a->suffix_cap = suffix_cap;
+    a->scale = scale; a->q = q; a->k_pre = k_pre; a->v_pre = v_pre; a->k_blk = k_blk; a->v_blk = v_blk;
+    a->k_suf = k_suf; a->v_suf = v_suf; a->out = const_cast<void*>(out);
+    const int splits = dare::attn_plan_splits(ctx, *a);
+    if (dare::attn_workspace_bytes(*a, splits) > ctx->workspace_bytes) return DARE_ERR_WORKSPACE;
+    return DARE_OK;
+}
+
+int check_lmhead(const dare_ctx* ctx, const void* hidden, int M, int D, const void* w, int V, int32_t mask_id,
+                 const void* pred, const void* conf) {
+    if (!ctx || !hidden || !w || !pred || !conf) return DARE_ERR_NULL;
+    if (M < 1 || D < 8 || D % 8 != 0 || V < 2) return DARE_ERR_SHAPE;
+    if (!aligned16(hidden) || !aligned16(w)) return DARE_ERR_ALIGN;
+    (void)mask_id;
+    if (dare::lmhead_workspace_bytes(M, V) > ctx->workspace_bytes) return DARE_ERR_WORKSPACE;
+    return DARE_OK;
+}
+
+int check_select(const void* tokens, int B, int64_t row_stride, int block_start, int L, const void* pred,
+                 const void* conf, int mode, float threshold, int k) {
+    if (!tokens || !pred || !conf) return DARE_ERR_NULL;
+    if (B < 1 || L < 1 || L > 4096) return DARE_ERR_SHAPE;
+    if (block_start < 0 || row_stride < 1 || static_cast<int64_t>(block_start) + L > row_stride) return DARE_ERR_RANGE;
+    if (mode != DARE_SELECT_THRESHOLD && mode != DARE_SELECT_TOPK) return DARE_ERR_RANGE;
+    if (mode == DARE_SELECT_THRESHOLD && threshold != threshold) return DARE_ERR_RANGE;
+    if (mode == DARE_SELECT_TOPK && k < 1) return DARE_ERR_RANGE;
+    return DARE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int dare_create(dare_ctx** out, int device, size_t workspace_bytes) {
+    if (!out) return DARE_ERR_NULL;
+    *out = nullptr;
+    int n_dev = 0;
+    if (cudaGetDeviceCount(&n_dev) != cudaSuccess || device < 0 || device >= n_dev) return DARE_ERR_CUDA;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return DARE_ERR_CUDA;
+    if (prop.major != 10) return DARE_ERR_UNSUPPORTED;
+    if (cudaSetDevice(device) != cudaSuccess) return DARE_ERR_CUDA;
+    dare_ctx* ctx = new (std::nothrow) dare_ctx();
+    if (!ctx) return DARE_ERR_CUDA;
+    ctx->device = device;
+    ctx->sm_count = prop.multiProcessorCount;
+    ctx->workspace_bytes = workspace_bytes ? workspace_bytes : (size_t(256) << 20);
+    ctx->workspace = nullptr;
+    ctx->dev_status = nullptr;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess || fn == nullptr) {
+        delete ctx;
+        return DARE_ERR_CUDA;
+    }
+    ctx->encode_tiled = reinterpret_cast<dare_encode_tiled_fn>(fn);
+    if (cudaMalloc(&ctx->workspace, ctx->workspace_bytes) != cudaSuccess ||
+        cudaMalloc(reinterpret_cast<void**>(&ctx->dev_status), sizeof(uint32_t)) != cudaSuccess ||
+        cudaMemset(ctx->dev_status, 0, sizeof(uint32_t)) != cudaSuccess) {
+        if (ctx->workspace) cudaFree(ctx->workspace);
+        if (ctx->dev_status) cudaFree(ctx->dev_status);
+        delete ctx;
+        return DARE_ERR_CUDA;
+    }
+    *out = ctx;
+    return DARE_OK;
+}
+
+int dare_destroy(dare_ctx* ctx) {
+    if (!ctx) return DARE_ERR_NULL;
+    cudaSetDevice(ctx->device);
+    cudaFree(ctx->workspace);
+    cudaFree(ctx->dev_status);
+    delete ctx;
+    return DARE_OK;
+}
+
+const char* dare_status_string(int status) {
+    switch (status) {
+        case DARE_OK: return "ok";
+        case DARE_ERR_NULL: return "a required pointer is NULL";
+        case DARE_ERR_SHAPE: return "unsupported or inconsistent dimensions";
+        case DARE_ERR_ALIGN: return "pointer or row size not 16-byte aligned";
+        case DARE_ERR_RANGE: return "scalar argument out of range";
+        case DARE_ERR_WORKSPACE: return "context workspace too small";
+        case DARE_ERR_CUDA: return "CUDA call failed";
+        case DARE_ERR_UNSUPPORTED: return "device is not sm_100";
+        default: return "unknown status";
+    }
+}
+
+int dare_device_status(dare_ctx* ctx, void* stream, uint32_t* host_out) {
+    if (!ctx || !host_out) return DARE_ERR_NULL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(host_out, ctx->dev_status, sizeof(uint32_t), cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return DARE_ERR_CUDA;
+    if (cudaMemsetAsync(ctx->dev_status, 0, sizeof(uint32_t), s) != cudaSuccess) return DARE_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return DARE_ERR_CUDA;
+    return DARE_OK;
+}
+
+int dare_sm_count(const dare_ctx* ctx) { return ctx ? ctx->sm_count : DARE_ERR_NULL; }
+
+int dare_attn_block(dare_ctx* ctx, int B, int L, int Hq, int Hkv, int d, int prefix_cap, int suffix_cap, float scale,
+                    const void* q, const void* k_pre, const void* v_pre, const int32_t* prefix_len, const void* k_blk,
+                    const void* v_blk, const void* k_suf, const void* v_suf, const int32_t* suffix_len, void* out,
+                    float* lse, void* stream) {
+    dare::AttnArgs a;
+    int rc = check_attn(ctx, B, L, Hq, Hkv, d, prefix_cap, suffix_cap, scale, q, k_pre, v_pre, k_blk, v_blk, k_suf,
+                        v_suf, out, &a);
+    if (rc != DARE_OK) return rc;
+    a.prefix_len = prefix_len; a.suffix_len = suffix_len; a.lse = lse;
+    return dare::launch_attn(ctx, a, static_cast<cudaStream_t>(stream));
+}
+
+int dare_lmhead_confidence(dare_ctx* ctx, const void* hidden, int M, int D, const void* w, int V,
+                           const int32_t* row_tokens, int32_t mask_id, int exclude_mask_column, int32_t* pred,
+                           float* conf, void* stream) {
+    int rc = check_lmhead(ctx, hidden, M, D, w, V, mask_id, pred, conf);
+    if (rc != DARE_OK) return rc;
+    return dare::launch_lmhead(ctx, ctx->workspace, hidden, M, D, w, V, row_tokens, M, 0, mask_id, exclude_mask_column,
+                               pred, conf, static_cast<cudaStream_t>(stream));
+}
+
+int dare_unmask_select(dare_ctx* ctx, int32_t* tokens, int B, int64_t row_stride, int block_start, int L,
+                       const int32_t* pred, const float* conf, int32_t mask_id, int mode, float threshold, int k,
+                       int32_t* n_committed, int32_t* n_remaining, void* stream) {
+    if (!ctx) return DARE_ERR_NULL;
+    int rc = check_select(tokens, B, row_stride, block_start, L, pred, conf, mode, threshold, k);
+    if (rc != DARE_OK) return rc;
+    return dare::launch_unmask_select(tokens, B, row_stride, block_start, L, pred, conf, mask_id, mode, threshold, k,
+                                      n_committed, n_remaining, static_cast<cudaStream_t>(stream));
+}
+
+int dare_denoise_block(dare_ctx* ctx, int B, int L, int Hq, int Hkv, int d, int prefix_cap, int suffix_cap,
+                       float scale, const void* q, const void* k_pre, const void* v_pre, const int32_t* prefix_len,
+                       const void* k_blk, const void* v_blk, const void* k_suf, const void* v_suf,
+                       const int32_t* suffix_len, void* attn_out, float* lse, const void* hidden, int D, const void* w,
+                       int V, int32_t mask_id, int exclude_mask_column, int32_t* tokens, int64_t row_stride,
+                       int block_start, int mode, float threshold, int k, int32_t* pred, float* conf,
+                       int32_t* n_committed, int32_t* n_remaining, void* stream) {
+    // validate everything first: on any error nothing is launched
+    dare::AttnArgs a;
+    int rc = check_attn(ctx, B, L, Hq, Hkv, d, prefix_cap, suffix_cap, scale, q, k_pre, v_pre, k_blk, v_blk, k_suf,
+                        v_suf, attn_out, &a);
+    if (rc != DARE_OK) return rc;
+    a.prefix_len = prefix_len; a.suffix_len = suffix_len; a.lse = lse;
+    if (static_cast<long long>(B) * L > 0x7fffffffLL) return DARE_ERR_SHAPE;
+    const int M = B * L;
+    rc = check_lmhead(ctx, hidden, M, D, w, V, mask_id, pred, conf);
+    if (rc != DARE_OK) return rc;
+    rc = check_select(tokens, B, row_stride, block_start, L, pred, conf, mode, threshold, k);
+    if (rc != DARE_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    rc = dare::launch_attn(ctx, a, s);
+    if (rc != DARE_OK) return rc;
+    // The LM head reads each row's current token straight from the token state: row m = (r, i) lives at
+    // tokens[r * row_stride + block_start + i].
+    rc = dare::launch_lmhead(ctx, ctx->workspace, hidden, M, D, w, V, tokens + block_start, L, row_stride, mask_id,
+                             exclude_mask_column, pred, conf, s);
+    if (rc != DARE_OK) return rc;
+    return dare::launch_unmask_select(tokens, B, row_stride, block_start, L, pred, conf, mask_id, mode, threshold, k,
+                                      n_committed, n_remaining, s);
+}
+
+}  // extern "C"

@@ -1,0 +1,57 @@
+// Internal declarations shared by the translation units of libdare (not part of the ABI).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/dare.h"
+
+typedef CUresult (*dare_encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                         const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                         CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                         CUtensorMapFloatOOBfill);
+
+struct dare_ctx {
+    int device;
+    int sm_count;
+    void* workspace;
+    size_t workspace_bytes;
+    uint32_t* dev_status;   // device word, bits DARE_DEV_*
+    dare_encode_tiled_fn encode_tiled;
+};
+
+namespace dare {
+
+// bf16 2-D row-major tensor [rows, cols] -> tensor map with a [box_rows, 64] box and 128-byte swizzle.
+int make_tmap_bf16_2d(const dare_ctx* ctx, CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols,
+                      uint32_t box_rows, uint32_t box_cols);
+
+int launch_unmask_select(int32_t* tokens, int B, int64_t row_stride, int block_start, int L, const int32_t* pred,
+                         const float* conf, int32_t mask_id, int mode, float threshold, int k, int32_t* n_committed,
+                         int32_t* n_remaining, cudaStream_t stream);
+
+size_t lmhead_workspace_bytes(int M, int V);
+// Token of LM-head row m (to skip committed rows) = row_tokens[(m / tok_L) * tok_row_stride + m % tok_L].
+int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M, int D, const void* w, int V,
+                  const int32_t* row_tokens, int tok_L, int64_t tok_row_stride, int32_t mask_id, int exclude_mask_column, int32_t* pred, float* conf,
+                  cudaStream_t stream);
+
+struct AttnArgs {
+    int B, L, Hq, Hkv, d, prefix_cap, suffix_cap;
+    float scale;
+    const void* q;
+    const void *k_pre, *v_pre;
+    const int32_t* prefix_len;
+    const void *k_blk, *v_blk;
+    const void *k_suf, *v_suf;
+    const int32_t* suffix_len;
+    void* out;
+    float* lse;
+};
+int attn_plan_splits(const dare_ctx* ctx, const AttnArgs& a);
+size_t attn_workspace_bytes(const AttnArgs& a, int splits);
+int launch_attn(const dare_ctx* ctx, const AttnArgs& a, cudaStream_t stream);
+
+}  // namespace dare

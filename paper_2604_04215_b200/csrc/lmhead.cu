@@ -1,0 +1,295 @@
+// Fused LM head + vocabulary softmax: per row the argmax token and its probability, logits kept on chip.
+//
+// z = X W^T is a dense bf16 contraction (M x V x D), so it runs on the tcgen05 tensor cores:
+//   warp 0      TMA producer: X tile [128 x 64] and W tile [256 x 64] per pipeline stage (128-byte swizzle)
+//   warp 1      UMMA issuer: 128 x 256 x 16 MMAs into one of two 128 x 256 fp32 accumulators in TMEM
+//   warps 2..5  epilogue: each thread owns one row (one TMEM lane), streams the 256 logits of the tile
+//               through registers and keeps (running max, sum of exp, argmax); no cross-thread traffic
+// The two accumulators let the epilogue of tile i overlap the MMAs of tile i+1.  Each tile writes one
+// (max, sumexp, argmax) triple per row; a small second kernel merges the triples of a row across the
+// vocabulary tiles into (token, confidence).  Consecutive tile ids share a W tile (row-tile index runs
+// fastest), so the CTAs that need the same W tile run at the same time and W leaves HBM once.
+#include <math.h>
+
+#include "internal.h"
+#include "ptx.cuh"
+
+namespace dare {
+namespace {
+
+constexpr int BM = 128;
+constexpr int BN = 256;
+constexpr int BK = 64;
+constexpr int STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2;
+constexpr int B_BYTES = BN * BK * 2;
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int LM_THREADS = 192;
+constexpr uint32_t TMEM_COLS = 512;
+constexpr float LOG2E = 1.4426950408889634f;
+
+struct LmBarriers {
+    uint64_t full[STAGES];
+    uint64_t empty[STAGES];
+    uint64_t tmem_full[2];
+    uint64_t tmem_empty[2];
+    uint32_t tmem_base;
+    uint32_t abort_flag;
+};
+constexpr int LM_SMEM_BYTES = STAGES * STAGE_BYTES + static_cast<int>(sizeof(LmBarriers)) + 1024;
+
+__global__ void __launch_bounds__(LM_THREADS, 1)
+lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
+                      int M, int D, int V, int mask_col, int m_tiles, int n_tiles,
+                      float* __restrict__ part_max, float* __restrict__ part_sum, int32_t* __restrict__ part_arg,
+                      uint32_t* __restrict__ dev_status) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    LmBarriers* bars = reinterpret_cast<LmBarriers*>(tiles + STAGES * STAGE_BYTES);
+    volatile uint32_t* abort_flag = &bars->abort_flag;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(&bars->full[s], 1);
+            mbar_init(&bars->empty[s], 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(&bars->tmem_full[a], 1);
+            mbar_init(&bars->tmem_empty[a], 128);
+        }
+        bars->abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(&bars->tmem_base, TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = bars->tmem_base;
+
+    const int total_tiles = m_tiles * n_tiles;
+    const int num_k = (D + BK - 1) / BK;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            prefetch_tensormap(&tmap_x);
+            prefetch_tensormap(&tmap_w);
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                const int m_tile = tile % m_tiles;
+                const int n_tile = tile / m_tiles;
+                for (int kb = 0; kb < num_k; ++kb) {
+                    if (!mbar_wait(&bars->empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
+                    uint8_t* a_dst = tiles + stage * STAGE_BYTES;
+                    uint8_t* b_dst = a_dst + A_BYTES;
+                    mbar_arrive_expect_tx(&bars->full[stage], STAGE_BYTES);
+                    tma_load_2d(a_dst, &tmap_x, &bars->full[stage], kb * BK, m_tile * BM);
+                    tma_load_2d(b_dst, &tmap_w, &bars->full[stage], kb * BK, n_tile * BN);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(BM, BN);
+            int stage = 0;
+            uint32_t phase = 0;
+            int it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+                const int acc = it & 1;
+                const uint32_t acc_phase = (it >> 1) & 1;
+                if (!mbar_wait(&bars->tmem_empty[acc], acc_phase ^ 1, abort_flag)) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + acc * BN;
+                for (int kb = 0; kb < num_k; ++kb) {
+                    if (!mbar_wait(&bars->full[stage], phase, abort_flag)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    const uint32_t a_addr = smem_u32(tiles + stage * STAGE_BYTES);
+                    const uint64_t a_desc = umma_desc_sw128_kmajor(a_addr);
+                    const uint64_t b_desc = umma_desc_sw128_kmajor(a_addr + A_BYTES);
+#pragma unroll
+                    for (int kk = 0; kk < BK / 16; ++kk) {
+                        // 16 bf16 = 32 bytes further along K inside the 128-byte swizzled row: +2 in the
+                        // descriptor's 16-byte address units
+                        umma_bf16(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0);
+                    }
+                    umma_commit(&bars->empty[stage]);   // frees the stage when these MMAs have read it
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+                if (ok) umma_commit(&bars->tmem_full[acc]);
+            }
+        }
+    } else {
+        // epilogue: warp w may touch TMEM lanes [32 * (w % 4), +32)
+        const int lq = warp & 3;
+        const int row_in_tile = lq * 32 + lane;
+        int it = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+            const int m_tile = tile % m_tiles;
+            const int n_tile = tile / m_tiles;
+            const int acc = it & 1;
+            const uint32_t acc_phase = (it >> 1) & 1;
+            if (!mbar_wait(&bars->tmem_full[acc], acc_phase, abort_flag)) { ok = false; break; }
+            tc_fence_after_sync();
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(lq * 32) << 16) + acc * BN;
+            const int col0 = n_tile * BN;
+            float run_max = -INFINITY;
+            float run_sum = 0.f;
+            int run_arg = 0x7fffffff;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t v[32];
+                tmem_ld_32cols(taddr + c * 32, v);
+                tmem_ld_wait();
+                const int cbase = col0 + c * 32;
+                float cmax = -INFINITY;
+                int carg = 0x7fffffff;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    float z = __uint_as_float(v[j]);
+                    const int col = cbase + j;
+                    if (col >= V || col == mask_col) z = -INFINITY;
+                    v[j] = __float_as_uint(z);
+                    if (z > cmax) { cmax = z; carg = col; }   // strict '>' keeps the lowest index
+                }
+                if (cmax > -INFINITY) {
+                    if (cmax > run_max) {
+                        run_sum *= fast_exp2((run_max - cmax) * LOG2E);   // exp2(-inf) = 0 on the first chunk
+                        run_max = cmax;
+                        run_arg = carg;
+                    }
+                    const float mb = run_max * LOG2E;
+                    float s = 0.f;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) s += fast_exp2(fmaf(__uint_as_float(v[j]), LOG2E, -mb));
+                    run_sum += s;
+                }
+            }
+            tc_fence_before_sync();
+            mbar_arrive(&bars->tmem_empty[acc]);
+            const int row = m_tile * BM + row_in_tile;
+            if (row < M) {
+                const size_t o = static_cast<size_t>(row) * n_tiles + n_tile;
+                part_max[o] = run_max;
+                part_sum[o] = run_sum;
+                part_arg[o] = run_arg;
+            }
+        }
+    }
+
+    // teardown
+    tc_fence_before_sync();
+    __syncthreads();
+    if (*abort_flag) {
+        // give copies still in flight time to land before the shared memory is released
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) {}
+        if (threadIdx.x == 0) atomicOr(dev_status, DEV_WAIT_EXPIRED);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+// One warp per row: fold the per-tile triples into (token, confidence).
+__global__ void lmhead_merge_kernel(const float* __restrict__ part_max, const float* __restrict__ part_sum,
+                                    const int32_t* __restrict__ part_arg, int n_tiles, int M,
+                                    const int32_t* __restrict__ row_tokens, int tok_L, int64_t tok_row_stride,
+                                    int32_t mask_id, int32_t* __restrict__ pred, float* __restrict__ conf) {
+    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= M) return;
+    if (row_tokens != nullptr) {
+        const int32_t t = row_tokens[static_cast<int64_t>(row / tok_L) * tok_row_stride + row % tok_L];
+        if (t != mask_id) {
+            if (lane == 0) { pred[row] = t; conf[row] = -INFINITY; }
+            return;
+        }
+    }
+    float m = -INFINITY, s = 0.f;
+    int a = 0x7fffffff;
+    const size_t base = static_cast<size_t>(row) * n_tiles;
+    for (int t = lane; t < n_tiles; t += 32) {
+        const float m2 = part_max[base + t];
+        const float s2 = part_sum[base + t];
+        const int a2 = part_arg[base + t];
+        if (m2 > -INFINITY) {
+            if (m2 > m) { s = s * exp2f((m - m2) * LOG2E) + s2; m = m2; a = a2; }
+            else { s += s2 * exp2f((m2 - m) * LOG2E); if (m2 == m && a2 < a) a = a2; }
+        }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const float m2 = __shfl_xor_sync(0xffffffffu, m, off);
+        const float s2 = __shfl_xor_sync(0xffffffffu, s, off);
+        const int a2 = __shfl_xor_sync(0xffffffffu, a, off);
+        if (m2 > -INFINITY) {
+            if (m2 > m) { s = s * exp2f((m - m2) * LOG2E) + s2; m = m2; a = a2; }
+            else { s += s2 * exp2f((m2 - m) * LOG2E); if (m2 == m && a2 < a) a = a2; }
+        }
+    }
+    if (lane == 0) {
+        pred[row] = a;
+        conf[row] = 1.0f / s;   // exp(max - logsumexp) with the sum taken relative to the max
+    }
+}
+
+}  // namespace
+
+size_t lmhead_workspace_bytes(int M, int V) {
+    const size_t n_tiles = (static_cast<size_t>(V) + BN - 1) / BN;
+    return 3 * sizeof(float) * n_tiles * static_cast<size_t>(M);
+}
+
+int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M, int D, const void* w, int V,
+                  const int32_t* row_tokens, int tok_L, int64_t tok_row_stride, int32_t mask_id,
+                  int exclude_mask_column, int32_t* pred, float* conf, cudaStream_t stream) {
+    CUtensorMap tmap_x, tmap_w;
+    int rc = make_tmap_bf16_2d(ctx, &tmap_x, hidden, static_cast<uint64_t>(M), static_cast<uint64_t>(D), BM, BK);
+    if (rc != DARE_OK) return rc;
+    rc = make_tmap_bf16_2d(ctx, &tmap_w, w, static_cast<uint64_t>(V), static_cast<uint64_t>(D), BN, BK);
+    if (rc != DARE_OK) return rc;
+
+    const int m_tiles = (M + BM - 1) / BM;
+    const int n_tiles = (V + BN - 1) / BN;
+    const size_t n_part = static_cast<size_t>(M) * n_tiles;
+    float* part_max = static_cast<float*>(scratch);
+    float* part_sum = part_max + n_part;
+    int32_t* part_arg = reinterpret_cast<int32_t*>(part_sum + n_part);
+
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(lmhead_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, LM_SMEM_BYTES) !=
+            cudaSuccess)
+            return DARE_ERR_CUDA;
+        attr_set = true;
+    }
+    const int total = m_tiles * n_tiles;
+    // a multiple of m_tiles so that the CTAs sharing a W tile always run in the same wave
+    int grid = ctx->sm_count;
+    if (grid > total) grid = total;
+    if (grid >= m_tiles) grid -= grid % m_tiles;
+    const int mask_col = (exclude_mask_column && mask_id >= 0 && mask_id < V) ? mask_id : -1;
+    lmhead_partial_kernel<<<grid, LM_THREADS, LM_SMEM_BYTES, stream>>>(tmap_x, tmap_w, M, D, V, mask_col, m_tiles,
+                                                                       n_tiles, part_max, part_sum, part_arg,
+                                                                       ctx->dev_status);
+    if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
+    const int rows_per_block = 8;
+    lmhead_merge_kernel<<<(M + rows_per_block - 1) / rows_per_block, rows_per_block * 32, 0, stream>>>(
+        part_max, part_sum, part_arg, n_tiles, M, row_tokens, tok_L, tok_row_stride, mask_id, pred, conf);
+    if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
+    return DARE_OK;
+}
+
+}  // namespace dare

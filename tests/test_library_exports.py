@@ -1,0 +1,46 @@
+"""CPU-only: the C-ABI library builds, loads and exports every symbol the public header declares."""
+import ctypes
+import os
+import re
+
+from paper_2604_04215_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared():
+    names = set()
+    for fn in os.listdir(os.path.join(ROOT, "include")):
+        if fn.endswith(".h"):
+            text = open(os.path.join(ROOT, "include", fn)).read()
+            text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+            names |= set(re.findall(r"\b(dare_[a-z_0-9]+)\s*\(", text))
+    return names
+
+
+def test_library_exports_every_declared_symbol():
+    build.build()
+    lib = ctypes.CDLL(binding.LIB_PATH)
+    declared = _declared()
+    assert {"dare_attn_block", "dare_lmhead_confidence", "dare_unmask_select", "dare_denoise_block"} <= declared
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert set(binding.EXPORTS) <= declared
+
+
+def test_status_strings_need_no_gpu():
+    lib = binding.load()
+    assert lib.dare_status_string(0) == b"ok"
+    for code in range(-7, 0):
+        assert lib.dare_status_string(code) not in (b"ok", b"unknown status")
+    assert lib.dare_status_string(-99) == b"unknown status"
+
+
+def test_product_path_never_touches_the_oracle():
+    """The package may not import or read anything under oracle/ (the oracle is test infrastructure)."""
+    pkg = os.path.join(ROOT, "paper_2604_04215_b200")
+    for base, _, files in os.walk(pkg):
+        for fn in files:
+            if fn.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(base, fn)).read()
+                assert not re.search(r"(from|import)\s+oracle|oracle[/.]\w|dare_oracle", text), fn
