@@ -152,6 +152,33 @@ int dare_denoise_block(dare_ctx* ctx,
                        int32_t* pred, float* conf,
                        int32_t* n_committed, int32_t* n_remaining, void* stream);
 
+/*
+ * Allocation-free variant of dare_lmhead_confidence.  (The paper has no counterpart for this entry
+ * point; it exists for callers of this library that are not allowed to allocate device memory.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside another framework's allocator
+ * or memory-budget hooks, in a plug-in that does not own the process's memory pool, or at a point of a
+ * program where allocation would synchronise or fail.  Such callers cannot hold a dare_ctx, because
+ * dare_create allocates the workspace.  Here the per-tile scratch of the LM head lives in a fixed array
+ * of DARE_LMHEAD_STATIC_SCRATCH_BYTES inside the library's device image, which every GPU that loads the
+ * library keeps resident until the process exits.  The call allocates nothing and frees nothing.
+ *
+ * Same arguments, results and arithmetic as dare_lmhead_confidence, without the ctx; it runs on the
+ * CURRENT device.  Limits and rules:
+ *   - 12 * M * ceil(V/256) must not exceed DARE_LMHEAD_STATIC_SCRATCH_BYTES, else DARE_ERR_WORKSPACE is
+ *     returned and nothing is launched (use the ctx variant for larger problems).
+ *   - The first call on each device looks up the device address of the scratch array and a driver entry
+ *     point; make that first call before starting any stream capture.
+ *   - All calls on a device share the one scratch array.  Nothing in it needs to start at zero (every
+ *     entry that is read has been written by the same call), but two calls whose GPU work overlaps
+ *     (different streams, or several host threads) race on it: serialise them on one stream.
+ *   - Data-dependent status bits of this variant go to an internal word that is not exposed.
+ */
+#define DARE_LMHEAD_STATIC_SCRATCH_BYTES (8u << 20)
+int dare_lmhead_confidence_static(const void* hidden, int M, int D, const void* w, int V,
+                                  const int32_t* row_tokens, int32_t mask_id, int exclude_mask_column,
+                                  int32_t* pred, float* conf, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

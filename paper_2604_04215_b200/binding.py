@@ -21,7 +21,8 @@ DEV_LEN_CLAMPED = 1
 DEV_WAIT_EXPIRED = 2
 
 EXPORTS = ["dare_create", "dare_destroy", "dare_status_string", "dare_device_status", "dare_sm_count",
-           "dare_attn_block", "dare_lmhead_confidence", "dare_unmask_select", "dare_denoise_block"]
+           "dare_attn_block", "dare_lmhead_confidence", "dare_unmask_select", "dare_denoise_block",
+           "dare_lmhead_confidence_static"]
 
 _lib = None
 
@@ -58,6 +59,8 @@ def load():
     lib.dare_attn_block.restype = i32
     lib.dare_lmhead_confidence.argtypes = [vp, vp, i32, i32, vp, i32, vp, i32, i32, vp, vp, vp]
     lib.dare_lmhead_confidence.restype = i32
+    lib.dare_lmhead_confidence_static.argtypes = [vp, i32, i32, vp, i32, vp, i32, i32, vp, vp, vp]
+    lib.dare_lmhead_confidence_static.restype = i32
     lib.dare_unmask_select.argtypes = [vp, vp, i32, i64, i32, i32, vp, vp, i32, i32, f32, i32, vp, vp, vp]
     lib.dare_unmask_select.restype = i32
     lib.dare_denoise_block.argtypes = ([vp] + [i32] * 7 + [f32] + [vp] * 11 +   # attention operands .. lse
@@ -151,6 +154,31 @@ def dare_lmhead_confidence(ctx: Context, hidden, w, row_tokens=None, mask_id: in
                                        _ptr(pred, torch.int32), _ptr(conf, torch.float32), _stream(stream))
     if rc != 0 and check:
         raise DareError(rc, "dare_lmhead_confidence")
+    return (pred, conf) if check else rc
+
+
+LMHEAD_STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def dare_lmhead_confidence_static(hidden, w, row_tokens=None, mask_id: int = -1, exclude_mask_column: bool = True,
+                                  pred=None, conf=None, stream=None, check: bool = True):
+    """The LM head for callers that may not allocate device memory: no context, fixed scratch inside the library.
+
+    pred and conf should be passed in by such callers (they are only created here as a convenience for tests).
+    Runs on the current device; calls that overlap on the GPU race on the shared scratch.
+    """
+    M, D = hidden.shape
+    V = w.shape[0]
+    if pred is None:
+        pred = torch.empty(M, dtype=torch.int32, device=hidden.device)
+    if conf is None:
+        conf = torch.empty(M, dtype=torch.float32, device=hidden.device)
+    rc = load().dare_lmhead_confidence_static(_ptr(hidden, torch.bfloat16), M, D, _ptr(w, torch.bfloat16), V,
+                                              _ptr(row_tokens, torch.int32), int(mask_id),
+                                              int(bool(exclude_mask_column)), _ptr(pred, torch.int32),
+                                              _ptr(conf, torch.float32), _stream(stream))
+    if rc != 0 and check:
+        raise DareError(rc, "dare_lmhead_confidence_static")
     return (pred, conf) if check else rc
 
 

@@ -10,6 +10,7 @@
 // vocabulary tiles into (token, confidence).  Consecutive tile ids share a W tile (row-tile index runs
 // fastest), so the CTAs that need the same W tile run at the same time and W leaves HBM once.
 #include <math.h>
+#include <mutex>
 
 #include "internal.h"
 #include "ptx.cuh"
@@ -293,3 +294,88 @@ int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M,
 }
 
 }  // namespace dare
+
+// ------------------------------------------------------------------------------------------------
+// Allocation-free variant of the LM-head entry point.
+//
+// Some callers must not allocate device memory at all: code running while a stream is being captured,
+// code inside a framework's allocator callback or under a memory budget that forbids cudaMalloc, and
+// plug-ins loaded into a process whose allocator they do not own.  dare_create allocates its workspace,
+// so those callers cannot have a context.  For them the per-tile (max, sum, argmax) triples of the LM
+// head live in a fixed array inside the library's device image.
+namespace dare {
+namespace {
+
+// Scratch shared by every call of dare_lmhead_confidence_static on a device (8 MiB, resident on every GPU
+// that loads the library until the process exits).
+static __device__ __align__(256) unsigned char g_lm_static_scratch[DARE_LMHEAD_STATIC_SCRATCH_BYTES];
+// Status bits of these calls (only ever OR-ed into; starts at zero when the module is loaded).
+static __device__ uint32_t g_lm_static_status;
+
+struct StaticDeviceState {
+    bool ready = false;
+    void* scratch = nullptr;        // device address of g_lm_static_scratch on this device
+    uint32_t* status = nullptr;     // device address of g_lm_static_status on this device
+    int sm_count = 0;
+    dare_encode_tiled_fn encode = nullptr;
+};
+constexpr int MAX_DEVICES = 64;
+StaticDeviceState g_static_state[MAX_DEVICES];
+std::mutex g_static_mutex;
+
+// One-time set-up for the current device.  In host code the array's name is only a handle; the address a
+// kernel can use has to be asked for, with this device current.
+int static_state_for_current_device(StaticDeviceState** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return DARE_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    StaticDeviceState& st = g_static_state[dev];
+    if (!st.ready) {
+        int major = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return DARE_ERR_CUDA;
+        if (major != 10) return DARE_ERR_UNSUPPORTED;
+        if (cudaDeviceGetAttribute(&st.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return DARE_ERR_CUDA;
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_lm_static_scratch) != cudaSuccess || p == nullptr) return DARE_ERR_CUDA;
+        st.scratch = p;
+        void* ps = nullptr;
+        if (cudaGetSymbolAddress(&ps, g_lm_static_status) != cudaSuccess || ps == nullptr) return DARE_ERR_CUDA;
+        st.status = static_cast<uint32_t*>(ps);
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess || fn == nullptr)
+            return DARE_ERR_CUDA;
+        st.encode = reinterpret_cast<dare_encode_tiled_fn>(fn);
+        st.ready = true;
+    }
+    *out = &st;
+    return DARE_OK;
+}
+
+}  // namespace
+}  // namespace dare
+
+extern "C" int dare_lmhead_confidence_static(const void* hidden, int M, int D, const void* w, int V,
+                                             const int32_t* row_tokens, int32_t mask_id, int exclude_mask_column,
+                                             int32_t* pred, float* conf, void* stream) {
+    if (!hidden || !w || !pred || !conf) return DARE_ERR_NULL;
+    if (M < 1 || D < 8 || D % 8 != 0 || V < 2) return DARE_ERR_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(hidden) & 15u) || (reinterpret_cast<uintptr_t>(w) & 15u)) return DARE_ERR_ALIGN;
+    if (dare::lmhead_workspace_bytes(M, V) > static_cast<size_t>(DARE_LMHEAD_STATIC_SCRATCH_BYTES))
+        return DARE_ERR_WORKSPACE;   // beyond the fixed scratch: use dare_lmhead_confidence with a context
+    dare::StaticDeviceState* st = nullptr;
+    int rc = dare::static_state_for_current_device(&st);
+    if (rc != DARE_OK) return rc;
+    // a context-shaped view of the static state for the shared launcher; nothing here is allocated
+    dare_ctx view;
+    view.device = -1;
+    view.sm_count = st->sm_count;
+    view.workspace = st->scratch;
+    view.workspace_bytes = DARE_LMHEAD_STATIC_SCRATCH_BYTES;
+    view.dev_status = st->status;
+    view.encode_tiled = st->encode;
+    return dare::launch_lmhead(&view, st->scratch, hidden, M, D, w, V, row_tokens, M, 0, mask_id, exclude_mask_column,
+                               pred, conf, static_cast<cudaStream_t>(stream));
+}
+
