@@ -107,6 +107,7 @@ def lm_rows_masked(wl, s_in_block):
 
 def run_ours(args):
     from paper_2604_04215_b200 import binding as dare
+    from paper_2604_04215_b200.dist import reduce_step_stats
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -187,13 +188,7 @@ def run_ours(args):
     committed = int(nc_all[args.warmup:n_total].sum().item())
     if ctx.device_status() != 0:
         raise RuntimeError("device status word is non-zero after the timed region")
-    t_ms = torch.tensor([ms], dtype=torch.float64, device="cuda")
-    tot = torch.tensor([committed], dtype=torch.float64, device="cuda")
-    if world > 1:
-        import torch.distributed as dist
-        dist.all_reduce(t_ms, op=dist.ReduceOp.MAX)
-        dist.all_reduce(tot, op=dist.ReduceOp.SUM)
-    ms_max, committed_all = float(t_ms.item()), float(tot.item())
+    ms_max, committed_all = reduce_step_stats(ms, committed, device="cuda")
     value = committed_all / (ms_max * 1e-3)
 
     # ---- instrumented pass: the same steps issued as the three entry points with events between them, to
@@ -232,7 +227,7 @@ def run_ours(args):
     lm_flops = 2.0 * masked_avg * wl.hidden * wl.vocab          # algorithmic: masked rows only
     achieved = lm_flops / (lm_ms * 1e-3) / 1e12
     peak = peaks["bf16_tflops_sustained"]
-    roofline = {"bound": "tensor", "kernel": "lmhead_partial_kernel(+merge)", "achieved": achieved, "peak": peak,
+    roofline = {"bound": "tensor", "kernel": "lmhead_partial_kernel (+ row compaction and merge kernels)", "achieved": achieved, "peak": peak,
                 "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None, "peak_source": peaks["source"] + " sustained",
                 "executed_tflops": 2.0 * B * L * wl.hidden * wl.vocab / (lm_ms * 1e-3) / 1e12,
                 "ms_per_launch": lm_ms, "masked_rows_avg": masked_avg,
@@ -267,15 +262,10 @@ def run_ours(args):
         torch.cuda.synchronize()
         e2e_tokens += int(nc_h.sum())
     tb = time.perf_counter()
-    e2e_t = torch.tensor([tb - ta], dtype=torch.float64, device="cuda")
-    e2e_n = torch.tensor([e2e_tokens], dtype=torch.float64, device="cuda")
-    if world > 1:
-        import torch.distributed as dist
-        dist.all_reduce(e2e_t, op=dist.ReduceOp.MAX)
-        dist.all_reduce(e2e_n, op=dist.ReduceOp.SUM)
+    e2e_s, e2e_n = reduce_step_stats(tb - ta, e2e_tokens, device="cuda")
     h2d = pool_h[0][0].numel() * 2 + pool_h[0][1].numel() * 2
     d2h = 4 * (B + B + B * L)
-    e2e = {"value": float(e2e_n.item()) / float(e2e_t.item()), "unit": UNIT, "h2d_bytes_per_step": h2d,
+    e2e = {"value": e2e_n / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
            "d2h_bytes_per_step": d2h, "steps": n_e2e}
 
     cpu_baseline = None
@@ -283,7 +273,8 @@ def run_ours(args):
         cpu_baseline = time_oracle(wl, w_h, (k_pre_h, v_pre_h, k_suf_h, v_suf_h), budget_s=20.0)
 
     if rank == 0:
-        attn_launches = 1   # + 1 combine launch when the attention plan splits KV (not in this workload)
+        # per step: attention, LM-head row compaction, LM-head GEMM, LM-head merge, selection
+        attn_launches = 1   # (+ 1 combine launch when the attention plan splits KV: not in this workload)
         out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                "warmup": args.warmup, "ms_per_step": ms_max / args.steps, "higher_is_better": True,
                "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
@@ -292,7 +283,7 @@ def run_ours(args):
                                       f"{'top-k ' + str(wl.k) if wl.mode == I.SELECT_TOPK else 'tau ' + str(wl.threshold)}",
                           "l2": "inputs larger than L2 (W 1.04 GB and KV cache 0.2 GB are re-read every step)",
                           "parallelism": f"dp{world} (independent rollouts per GPU, no collective)"},
-               "clocks": clocks, "e2e": e2e, "gpu_launches": (attn_launches + 3) * args.steps,
+               "clocks": clocks, "e2e": e2e, "gpu_launches": (attn_launches + 4) * args.steps,
                "roofline": roofline, "breakdown": breakdown, "cpu_baseline": cpu_baseline}
         print(json.dumps(out))
     ctx.close()

@@ -106,8 +106,9 @@ int dare_attn_block(dare_ctx* ctx,
  *   row_tokens   int32 [M] or NULL: rows whose token != mask_id are already committed and get
  *                pred = that token, conf = -inf
  *   pred         int32 [M] out      conf  fp32 [M] out
- * Supported: D % 8 == 0, D >= 8; V >= 2; M >= 1.  Needs ctx workspace of 12 * ceil(V/256) *
- * roundup(M,128) bytes.
+ * Only rows that are still masked are evaluated (they are compacted on the device first).
+ * Supported: D % 8 == 0, D >= 8; V >= 2; M >= 1.  Needs ctx workspace of 12 * M * min(#SMs, ceil(V/256))
+ * bytes, plus 2*M*D + 4*M + 2048 bytes when row_tokens is given.
  */
 int dare_lmhead_confidence(dare_ctx* ctx,
                            const void* hidden, int M, int D, const void* w, int V,
@@ -165,7 +166,8 @@ int dare_denoise_block(dare_ctx* ctx,
  *
  * Same arguments, results and arithmetic as dare_lmhead_confidence, without the ctx; it runs on the
  * CURRENT device.  Limits and rules:
- *   - 12 * M * ceil(V/256) must not exceed DARE_LMHEAD_STATIC_SCRATCH_BYTES, else DARE_ERR_WORKSPACE is
+ *   - The scratch the call needs (12 * M * min(#SMs, ceil(V/256)) bytes, plus 2*M*D + 4*M + 2048 bytes when
+ *     row_tokens is given) must not exceed DARE_LMHEAD_STATIC_SCRATCH_BYTES, else DARE_ERR_WORKSPACE is
  *     returned and nothing is launched (use the ctx variant for larger problems).
  *   - The first call on each device looks up the device address of the scratch array and a driver entry
  *     point; make that first call before starting any stream capture.

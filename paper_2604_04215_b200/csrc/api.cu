@@ -50,13 +50,13 @@ int check_attn(const dare_ctx* ctx, int B, int L, int Hq, int Hkv, int d, int pr
     return DARE_OK;
 }
 
-int check_lmhead(const dare_ctx* ctx, const void* hidden, int M, int D, const void* w, int V, int32_t mask_id,
+int check_lmhead(const dare_ctx* ctx, const void* hidden, int M, int D, const void* w, int V, bool with_row_tokens,
                  const void* pred, const void* conf) {
     if (!ctx || !hidden || !w || !pred || !conf) return DARE_ERR_NULL;
     if (M < 1 || D < 8 || D % 8 != 0 || V < 2) return DARE_ERR_SHAPE;
     if (!aligned16(hidden) || !aligned16(w)) return DARE_ERR_ALIGN;
-    (void)mask_id;
-    if (dare::lmhead_workspace_bytes(M, V) > ctx->workspace_bytes) return DARE_ERR_WORKSPACE;
+    if (dare::lmhead_workspace_bytes(M, D, V, ctx->sm_count, with_row_tokens) > ctx->workspace_bytes)
+        return DARE_ERR_WORKSPACE;
     return DARE_OK;
 }
 
@@ -161,7 +161,7 @@ int dare_attn_block(dare_ctx* ctx, int B, int L, int Hq, int Hkv, int d, int pre
 int dare_lmhead_confidence(dare_ctx* ctx, const void* hidden, int M, int D, const void* w, int V,
                            const int32_t* row_tokens, int32_t mask_id, int exclude_mask_column, int32_t* pred,
                            float* conf, void* stream) {
-    int rc = check_lmhead(ctx, hidden, M, D, w, V, mask_id, pred, conf);
+    int rc = check_lmhead(ctx, hidden, M, D, w, V, row_tokens != nullptr, pred, conf);
     if (rc != DARE_OK) return rc;
     return dare::launch_lmhead(ctx, ctx->workspace, hidden, M, D, w, V, row_tokens, M, 0, mask_id, exclude_mask_column,
                                pred, conf, static_cast<cudaStream_t>(stream));
@@ -192,7 +192,7 @@ int dare_denoise_block(dare_ctx* ctx, int B, int L, int Hq, int Hkv, int d, int 
     a.prefix_len = prefix_len; a.suffix_len = suffix_len; a.lse = lse;
     if (static_cast<long long>(B) * L > 0x7fffffffLL) return DARE_ERR_SHAPE;
     const int M = B * L;
-    rc = check_lmhead(ctx, hidden, M, D, w, V, mask_id, pred, conf);
+    rc = check_lmhead(ctx, hidden, M, D, w, V, true, pred, conf);
     if (rc != DARE_OK) return rc;
     rc = check_select(tokens, B, row_stride, block_start, L, pred, conf, mode, threshold, k);
     if (rc != DARE_OK) return rc;

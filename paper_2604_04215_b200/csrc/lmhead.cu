@@ -5,10 +5,15 @@
 //   warp 1      UMMA issuer: 128 x 256 x 16 MMAs into one of two 128 x 256 fp32 accumulators in TMEM
 //   warps 2..5  epilogue: each thread owns one row (one TMEM lane), streams the 256 logits of the tile
 //               through registers and keeps (running max, sum of exp, argmax); no cross-thread traffic
-// The two accumulators let the epilogue of tile i overlap the MMAs of tile i+1.  Each tile writes one
-// (max, sumexp, argmax) triple per row; a small second kernel merges the triples of a row across the
-// vocabulary tiles into (token, confidence).  Consecutive tile ids share a W tile (row-tile index runs
-// fastest), so the CTAs that need the same W tile run at the same time and W leaves HBM once.
+// The two accumulators let the epilogue of tile i overlap the MMAs of tile i+1.
+//
+// Only rows that are still masked need logits.  A first small kernel compacts those rows of X into a dense
+// buffer (and answers the committed rows directly); the GEMM reads the number of live rows from device
+// memory, so the host never synchronises.  Work is cut into items (row tile, vocabulary group): a CTA keeps
+// one row tile for all vocabulary tiles of its group, so every epilogue thread carries its row's running
+// triple in registers across tiles and writes ONE partial per item.  The CTAs of the row tiles of one group
+// walk the same W tiles at the same time, so W leaves HBM once.  A last small kernel merges the (few)
+// partials of a row into (token, confidence) and scatters them to the row's original position.
 #include <math.h>
 #include <mutex>
 
@@ -28,6 +33,7 @@ constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int LM_THREADS = 192;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr float LOG2E = 1.4426950408889634f;
+constexpr int ARG_NONE = 0x7fffffff;
 
 struct LmBarriers {
     uint64_t full[STAGES];
@@ -39,11 +45,75 @@ struct LmBarriers {
 };
 constexpr int LM_SMEM_BYTES = STAGES * STAGE_BYTES + static_cast<int>(sizeof(LmBarriers)) + 1024;
 
+// Number of vocabulary groups for a grid of `grid` CTAs and `m_tiles` row tiles (same formula on the host,
+// in the GEMM and in the merge kernel).
+__host__ __device__ inline int lm_groups(int grid, int m_tiles, int n_tiles) {
+    int g = m_tiles > 0 ? grid / m_tiles : 1;
+    if (g < 1) g = 1;
+    if (g > n_tiles) g = n_tiles;
+    return g;
+}
+
+__device__ __forceinline__ int32_t row_token(const int32_t* row_tokens, int tok_L, int64_t tok_row_stride, int m) {
+    return row_tokens[static_cast<int64_t>(m / tok_L) * tok_row_stride + m % tok_L];
+}
+
+// Compacts the still-masked rows of X into xc (order preserved), records their original indices, counts
+// them, and answers committed rows (pred = their token, conf = -inf).  One warp per row.
+constexpr int CP_ROWS = 8;
+__global__ void __launch_bounds__(CP_ROWS * 32)
+lmhead_compact_kernel(const uint4* __restrict__ x, int M, int D8, const int32_t* __restrict__ row_tokens, int tok_L,
+                      int64_t tok_row_stride, int32_t mask_id, uint4* __restrict__ xc, int32_t* __restrict__ idx,
+                      int32_t* __restrict__ count, int32_t* __restrict__ pred, float* __restrict__ conf) {
+    __shared__ int s_base;
+    __shared__ int s_flag[CP_ROWS];
+    const int row0 = blockIdx.x * CP_ROWS;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) s_base = 0;
+    __syncthreads();
+    int local = 0;
+    for (int m = threadIdx.x; m < row0; m += blockDim.x) local += row_token(row_tokens, tok_L, tok_row_stride, m) == mask_id;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) local += __shfl_xor_sync(0xffffffffu, local, off);
+    if (lane == 0 && local) atomicAdd(&s_base, local);
+    const int row = row0 + warp;
+    int32_t tok = 0;
+    bool masked = false;
+    if (row < M) {
+        tok = row_token(row_tokens, tok_L, tok_row_stride, row);
+        masked = tok == mask_id;
+    }
+    if (lane == 0) s_flag[warp] = masked ? 1 : 0;
+    __syncthreads();
+    int before = s_base, total = s_base;
+    for (int i = 0; i < CP_ROWS; ++i) {
+        if (i < warp) before += s_flag[i];
+        total += s_flag[i];
+    }
+    if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) *count = total;
+    if (row >= M) return;
+    if (!masked) {
+        if (lane == 0) { pred[row] = tok; conf[row] = -INFINITY; }
+        return;
+    }
+    if (lane == 0) idx[before] = row;
+    const uint4* src = x + static_cast<size_t>(row) * D8;
+    uint4* dst = xc + static_cast<size_t>(before) * D8;
+    for (int i = lane; i < D8; i += 32) dst[i] = src[i];
+}
+
 __global__ void __launch_bounds__(LM_THREADS, 1)
 lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
-                      int M, int D, int V, int mask_col, int m_tiles, int n_tiles,
+                      int M, const int32_t* __restrict__ live_rows, int D, int V, int mask_col, int n_tiles,
                       float* __restrict__ part_max, float* __restrict__ part_sum, int32_t* __restrict__ part_arg,
                       uint32_t* __restrict__ dev_status) {
+    const int Mc = live_rows ? *live_rows : M;          // rows that need logits (uniform over the grid)
+    const int m_tiles = (Mc + BM - 1) / BM;
+    if (m_tiles == 0) return;
+    const int groups = lm_groups(gridDim.x, m_tiles, n_tiles);
+    const int n_items = m_tiles * groups;
+    if (static_cast<int>(blockIdx.x) >= n_items) return;
+
     extern __shared__ uint8_t smem_raw[];
     uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     LmBarriers* bars = reinterpret_cast<LmBarriers*>(tiles + STAGES * STAGE_BYTES);
@@ -72,10 +142,9 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = bars->tmem_base;
-
-    const int total_tiles = m_tiles * n_tiles;
     const int num_k = (D + BK - 1) / BK;
 
+    // item w -> row tile w % m_tiles, vocabulary group w / m_tiles; the group's tiles are g, g + groups, ...
     if (warp == 0) {
         if (lane == 0) {
             prefetch_tensormap(&tmap_x);
@@ -83,17 +152,18 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-                const int m_tile = tile % m_tiles;
-                const int n_tile = tile / m_tiles;
-                for (int kb = 0; kb < num_k; ++kb) {
-                    if (!mbar_wait(&bars->empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
-                    uint8_t* a_dst = tiles + stage * STAGE_BYTES;
-                    uint8_t* b_dst = a_dst + A_BYTES;
-                    mbar_arrive_expect_tx(&bars->full[stage], STAGE_BYTES);
-                    tma_load_2d(a_dst, &tmap_x, &bars->full[stage], kb * BK, m_tile * BM);
-                    tma_load_2d(b_dst, &tmap_w, &bars->full[stage], kb * BK, n_tile * BN);
-                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+                const int m_tile = item % m_tiles;
+                for (int n_tile = item / m_tiles; n_tile < n_tiles && ok; n_tile += groups) {
+                    for (int kb = 0; kb < num_k; ++kb) {
+                        if (!mbar_wait(&bars->empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
+                        uint8_t* a_dst = tiles + stage * STAGE_BYTES;
+                        uint8_t* b_dst = a_dst + A_BYTES;
+                        mbar_arrive_expect_tx(&bars->full[stage], STAGE_BYTES);
+                        tma_load_2d(a_dst, &tmap_x, &bars->full[stage], kb * BK, m_tile * BM);
+                        tma_load_2d(b_dst, &tmap_w, &bars->full[stage], kb * BK, n_tile * BN);
+                        if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                    }
                 }
             }
         }
@@ -104,28 +174,30 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
             uint32_t phase = 0;
             int it = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
-                const int acc = it & 1;
-                const uint32_t acc_phase = (it >> 1) & 1;
-                if (!mbar_wait(&bars->tmem_empty[acc], acc_phase ^ 1, abort_flag)) { ok = false; break; }
-                tc_fence_after_sync();
-                const uint32_t d_tmem = tmem_base + acc * BN;
-                for (int kb = 0; kb < num_k; ++kb) {
-                    if (!mbar_wait(&bars->full[stage], phase, abort_flag)) { ok = false; break; }
+            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+                for (int n_tile = item / m_tiles; n_tile < n_tiles && ok; n_tile += groups, ++it) {
+                    const int acc = it & 1;
+                    const uint32_t acc_phase = (it >> 1) & 1;
+                    if (!mbar_wait(&bars->tmem_empty[acc], acc_phase ^ 1, abort_flag)) { ok = false; break; }
                     tc_fence_after_sync();
-                    const uint32_t a_addr = smem_u32(tiles + stage * STAGE_BYTES);
-                    const uint64_t a_desc = umma_desc_sw128_kmajor(a_addr);
-                    const uint64_t b_desc = umma_desc_sw128_kmajor(a_addr + A_BYTES);
+                    const uint32_t d_tmem = tmem_base + acc * BN;
+                    for (int kb = 0; kb < num_k; ++kb) {
+                        if (!mbar_wait(&bars->full[stage], phase, abort_flag)) { ok = false; break; }
+                        tc_fence_after_sync();
+                        const uint32_t a_addr = smem_u32(tiles + stage * STAGE_BYTES);
+                        const uint64_t a_desc = umma_desc_sw128_kmajor(a_addr);
+                        const uint64_t b_desc = umma_desc_sw128_kmajor(a_addr + A_BYTES);
 #pragma unroll
-                    for (int kk = 0; kk < BK / 16; ++kk) {
-                        // 16 bf16 = 32 bytes further along K inside the 128-byte swizzled row: +2 in the
-                        // descriptor's 16-byte address units
-                        umma_bf16(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0);
+                        for (int kk = 0; kk < BK / 16; ++kk) {
+                            // 16 bf16 = 32 bytes further along K inside the 128-byte swizzled row: +2 in the
+                            // descriptor's 16-byte address units
+                            umma_bf16(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0);
+                        }
+                        umma_commit(&bars->empty[stage]);   // frees the stage when these MMAs have read it
+                        if (++stage == STAGES) { stage = 0; phase ^= 1; }
                     }
-                    umma_commit(&bars->empty[stage]);   // frees the stage when these MMAs have read it
-                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                    if (ok) umma_commit(&bars->tmem_full[acc]);
                 }
-                if (ok) umma_commit(&bars->tmem_full[acc]);
             }
         }
     } else {
@@ -134,52 +206,59 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
         const int row_in_tile = lq * 32 + lane;
         int it = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
-            const int m_tile = tile % m_tiles;
-            const int n_tile = tile / m_tiles;
-            const int acc = it & 1;
-            const uint32_t acc_phase = (it >> 1) & 1;
-            if (!mbar_wait(&bars->tmem_full[acc], acc_phase, abort_flag)) { ok = false; break; }
-            tc_fence_after_sync();
-            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(lq * 32) << 16) + acc * BN;
-            const int col0 = n_tile * BN;
+        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+            const int m_tile = item % m_tiles;
+            const int group = item / m_tiles;
             float run_max = -INFINITY;
             float run_sum = 0.f;
-            int run_arg = 0x7fffffff;
+            int run_arg = ARG_NONE;
+            for (int n_tile = group; n_tile < n_tiles && ok; n_tile += groups, ++it) {
+                const int acc = it & 1;
+                const uint32_t acc_phase = (it >> 1) & 1;
+                if (!mbar_wait(&bars->tmem_full[acc], acc_phase, abort_flag)) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t taddr = tmem_base + (static_cast<uint32_t>(lq * 32) << 16) + acc * BN;
+                const int col0 = n_tile * BN;
+                const bool edge = (col0 + BN > V) || (mask_col >= col0 && mask_col < col0 + BN);
 #pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
-                uint32_t v[32];
-                tmem_ld_32cols(taddr + c * 32, v);
-                tmem_ld_wait();
-                const int cbase = col0 + c * 32;
-                float cmax = -INFINITY;
-                int carg = 0x7fffffff;
+                for (int c = 0; c < BN / 32; ++c) {
+                    uint32_t v[32];
+                    tmem_ld_32cols(taddr + c * 32, v);
+                    tmem_ld_wait();
+                    const int cbase = col0 + c * 32;
+                    float cmax = -INFINITY;
+                    int carg = ARG_NONE;
+                    if (edge) {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    float z = __uint_as_float(v[j]);
-                    const int col = cbase + j;
-                    if (col >= V || col == mask_col) z = -INFINITY;
-                    v[j] = __float_as_uint(z);
-                    if (z > cmax) { cmax = z; carg = col; }   // strict '>' keeps the lowest index
-                }
-                if (cmax > -INFINITY) {
-                    if (cmax > run_max) {
-                        run_sum *= fast_exp2((run_max - cmax) * LOG2E);   // exp2(-inf) = 0 on the first chunk
-                        run_max = cmax;
-                        run_arg = carg;
+                        for (int j = 0; j < 32; ++j) {
+                            const int col = cbase + j;
+                            if (col >= V || col == mask_col) v[j] = __float_as_uint(-INFINITY);
+                        }
                     }
-                    const float mb = run_max * LOG2E;
-                    float s = 0.f;
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) s += fast_exp2(fmaf(__uint_as_float(v[j]), LOG2E, -mb));
-                    run_sum += s;
+                    for (int j = 0; j < 32; ++j) {
+                        const float z = __uint_as_float(v[j]);
+                        if (z > cmax) { cmax = z; carg = cbase + j; }   // strict '>' keeps the lowest index
+                    }
+                    if (cmax > -INFINITY) {
+                        if (cmax > run_max) {   // tiles of a group come in ascending order: '>' keeps the lowest id
+                            run_sum *= fast_exp2((run_max - cmax) * LOG2E);   // exp2(-inf) = 0 the first time
+                            run_max = cmax;
+                            run_arg = carg;
+                        }
+                        const float mb = run_max * LOG2E;
+                        float s = 0.f;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) s += fast_exp2(fmaf(__uint_as_float(v[j]), LOG2E, -mb));
+                        run_sum += s;
+                    }
                 }
+                tc_fence_before_sync();
+                mbar_arrive(&bars->tmem_empty[acc]);
             }
-            tc_fence_before_sync();
-            mbar_arrive(&bars->tmem_empty[acc]);
             const int row = m_tile * BM + row_in_tile;
-            if (row < M) {
-                const size_t o = static_cast<size_t>(row) * n_tiles + n_tile;
+            if (ok && row < Mc) {
+                const size_t o = static_cast<size_t>(row) * groups + group;
                 part_max[o] = run_max;
                 part_sum[o] = run_sum;
                 part_arg[o] = run_arg;
@@ -203,25 +282,21 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     }
 }
 
-// One warp per row: fold the per-tile triples into (token, confidence).
+// One warp per live row: fold the row's partial triples (one per vocabulary group) into (token, confidence)
+// and write them at the row's original position.
 __global__ void lmhead_merge_kernel(const float* __restrict__ part_max, const float* __restrict__ part_sum,
-                                    const int32_t* __restrict__ part_arg, int n_tiles, int M,
-                                    const int32_t* __restrict__ row_tokens, int tok_L, int64_t tok_row_stride,
-                                    int32_t mask_id, int32_t* __restrict__ pred, float* __restrict__ conf) {
-    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+                                    const int32_t* __restrict__ part_arg, int grid_gemm, int n_tiles, int M,
+                                    const int32_t* __restrict__ live_rows, const int32_t* __restrict__ idx,
+                                    int32_t* __restrict__ pred, float* __restrict__ conf) {
+    const int c = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
-    if (row >= M) return;
-    if (row_tokens != nullptr) {
-        const int32_t t = row_tokens[static_cast<int64_t>(row / tok_L) * tok_row_stride + row % tok_L];
-        if (t != mask_id) {
-            if (lane == 0) { pred[row] = t; conf[row] = -INFINITY; }
-            return;
-        }
-    }
+    const int Mc = live_rows ? *live_rows : M;
+    if (c >= Mc) return;
+    const int groups = lm_groups(grid_gemm, (Mc + BM - 1) / BM, n_tiles);
     float m = -INFINITY, s = 0.f;
-    int a = 0x7fffffff;
-    const size_t base = static_cast<size_t>(row) * n_tiles;
-    for (int t = lane; t < n_tiles; t += 32) {
+    int a = ARG_NONE;
+    const size_t base = static_cast<size_t>(c) * groups;
+    for (int t = lane; t < groups; t += 32) {
         const float m2 = part_max[base + t];
         const float s2 = part_sum[base + t];
         const int a2 = part_arg[base + t];
@@ -241,54 +316,75 @@ __global__ void lmhead_merge_kernel(const float* __restrict__ part_max, const fl
         }
     }
     if (lane == 0) {
+        const int row = idx ? idx[c] : c;
         pred[row] = a;
         conf[row] = 1.0f / s;   // exp(max - logsumexp) with the sum taken relative to the max
     }
 }
 
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
 }  // namespace
 
-size_t lmhead_workspace_bytes(int M, int V) {
+// Scratch layout: [compacted X: M*D bf16][row indices: M int32][live-row count][partials: 3 x M x groups]
+size_t lmhead_workspace_bytes(int M, int D, int V, int sm_count, bool with_row_tokens) {
     const size_t n_tiles = (static_cast<size_t>(V) + BN - 1) / BN;
-    return 3 * sizeof(float) * n_tiles * static_cast<size_t>(M);
+    size_t groups = static_cast<size_t>(sm_count);
+    if (groups > n_tiles) groups = n_tiles;
+    size_t bytes = 3 * sizeof(float) * groups * static_cast<size_t>(M);
+    if (with_row_tokens)
+        bytes += round_up(static_cast<size_t>(M) * D * 2, 1024) + round_up(static_cast<size_t>(M) * 4 + 4, 1024);
+    return bytes;
 }
 
 int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M, int D, const void* w, int V,
                   const int32_t* row_tokens, int tok_L, int64_t tok_row_stride, int32_t mask_id,
                   int exclude_mask_column, int32_t* pred, float* conf, cudaStream_t stream) {
+    const int n_tiles = (V + BN - 1) / BN;
+    const int m_tiles_max = (M + BM - 1) / BM;
+    int grid = ctx->sm_count;
+    if (grid > m_tiles_max * n_tiles) grid = m_tiles_max * n_tiles;
+
+    uint8_t* cur = static_cast<uint8_t*>(scratch);
+    const void* x_gemm = hidden;
+    int32_t* idx = nullptr;
+    int32_t* live_rows = nullptr;
+    if (row_tokens != nullptr) {
+        void* xc = cur;
+        cur += round_up(static_cast<size_t>(M) * D * 2, 1024);
+        idx = reinterpret_cast<int32_t*>(cur);
+        live_rows = idx + M;
+        cur += round_up(static_cast<size_t>(M) * 4 + 4, 1024);
+        x_gemm = xc;
+        lmhead_compact_kernel<<<(M + CP_ROWS - 1) / CP_ROWS, CP_ROWS * 32, 0, stream>>>(
+            static_cast<const uint4*>(hidden), M, D / 8, row_tokens, tok_L, tok_row_stride, mask_id,
+            static_cast<uint4*>(xc), idx, live_rows, pred, conf);
+        if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
+    }
+    size_t groups_max = static_cast<size_t>(ctx->sm_count);
+    if (groups_max > static_cast<size_t>(n_tiles)) groups_max = n_tiles;
+    const size_t n_part = static_cast<size_t>(M) * groups_max;
+    float* part_max = reinterpret_cast<float*>(cur);
+    float* part_sum = part_max + n_part;
+    int32_t* part_arg = reinterpret_cast<int32_t*>(part_sum + n_part);
+
     CUtensorMap tmap_x, tmap_w;
-    int rc = make_tmap_bf16_2d(ctx, &tmap_x, hidden, static_cast<uint64_t>(M), static_cast<uint64_t>(D), BM, BK);
+    int rc = make_tmap_bf16_2d(ctx, &tmap_x, x_gemm, static_cast<uint64_t>(M), static_cast<uint64_t>(D), BM, BK);
     if (rc != DARE_OK) return rc;
     rc = make_tmap_bf16_2d(ctx, &tmap_w, w, static_cast<uint64_t>(V), static_cast<uint64_t>(D), BN, BK);
     if (rc != DARE_OK) return rc;
 
-    const int m_tiles = (M + BM - 1) / BM;
-    const int n_tiles = (V + BN - 1) / BN;
-    const size_t n_part = static_cast<size_t>(M) * n_tiles;
-    float* part_max = static_cast<float*>(scratch);
-    float* part_sum = part_max + n_part;
-    int32_t* part_arg = reinterpret_cast<int32_t*>(part_sum + n_part);
-
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(lmhead_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, LM_SMEM_BYTES) !=
-            cudaSuccess)
-            return DARE_ERR_CUDA;
-        attr_set = true;
-    }
-    const int total = m_tiles * n_tiles;
-    // a multiple of m_tiles so that the CTAs sharing a W tile always run in the same wave
-    int grid = ctx->sm_count;
-    if (grid > total) grid = total;
-    if (grid >= m_tiles) grid -= grid % m_tiles;
+    if (cudaFuncSetAttribute(lmhead_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, LM_SMEM_BYTES) !=
+        cudaSuccess)
+        return DARE_ERR_CUDA;
     const int mask_col = (exclude_mask_column && mask_id >= 0 && mask_id < V) ? mask_id : -1;
-    lmhead_partial_kernel<<<grid, LM_THREADS, LM_SMEM_BYTES, stream>>>(tmap_x, tmap_w, M, D, V, mask_col, m_tiles,
+    lmhead_partial_kernel<<<grid, LM_THREADS, LM_SMEM_BYTES, stream>>>(tmap_x, tmap_w, M, live_rows, D, V, mask_col,
                                                                        n_tiles, part_max, part_sum, part_arg,
                                                                        ctx->dev_status);
     if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
     const int rows_per_block = 8;
     lmhead_merge_kernel<<<(M + rows_per_block - 1) / rows_per_block, rows_per_block * 32, 0, stream>>>(
-        part_max, part_sum, part_arg, n_tiles, M, row_tokens, tok_L, tok_row_stride, mask_id, pred, conf);
+        part_max, part_sum, part_arg, grid, n_tiles, M, live_rows, idx, pred, conf);
     if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
     return DARE_OK;
 }
@@ -362,11 +458,12 @@ extern "C" int dare_lmhead_confidence_static(const void* hidden, int M, int D, c
     if (!hidden || !w || !pred || !conf) return DARE_ERR_NULL;
     if (M < 1 || D < 8 || D % 8 != 0 || V < 2) return DARE_ERR_SHAPE;
     if ((reinterpret_cast<uintptr_t>(hidden) & 15u) || (reinterpret_cast<uintptr_t>(w) & 15u)) return DARE_ERR_ALIGN;
-    if (dare::lmhead_workspace_bytes(M, V) > static_cast<size_t>(DARE_LMHEAD_STATIC_SCRATCH_BYTES))
-        return DARE_ERR_WORKSPACE;   // beyond the fixed scratch: use dare_lmhead_confidence with a context
     dare::StaticDeviceState* st = nullptr;
     int rc = dare::static_state_for_current_device(&st);
     if (rc != DARE_OK) return rc;
+    if (dare::lmhead_workspace_bytes(M, D, V, st->sm_count, row_tokens != nullptr) >
+        static_cast<size_t>(DARE_LMHEAD_STATIC_SCRATCH_BYTES))
+        return DARE_ERR_WORKSPACE;   // beyond the fixed scratch: use dare_lmhead_confidence with a context
     // a context-shaped view of the static state for the shared launcher; nothing here is allocated
     dare_ctx view;
     view.device = -1;

@@ -56,7 +56,7 @@ def test_static_entry_matches_context_entry_on_two_calls_in_a_row():
 
 
 def test_static_entry_rejects_problems_beyond_its_scratch():
-    M, V = 2048, 126464                      # 12 * 2048 * 494 bytes > 8 MiB
+    M, V = 8192, 126464                      # 12 * 8192 * 148 bytes > 8 MiB
     x = torch.zeros(M, 64, dtype=torch.bfloat16, device="cuda")
     w = torch.zeros(V, 64, dtype=torch.bfloat16, device="cuda")
     rc = dare.dare_lmhead_confidence_static(x, w, None, 0, True, check=False)
