@@ -35,6 +35,9 @@ from paper_2604_04215_b200 import inputs as I  # noqa: E402
 METRIC = "denoised_tokens_per_sec"
 UNIT = "tokens/s"
 NPOOL = 4   # distinct activation sets cycled through the steps
+# dram__bytes_read.sum + dram__bytes_write.sum of one lmhead_partial_kernel launch, from the ncu capture
+# summarised in profiles/lmhead_partial_kernel_llada8b.md (W, 1.036 GB, dominates: it leaves HBM once)
+LMHEAD_TRAFFIC_BYTES = {"llada8b": 1.0497e9}
 
 
 def _peaks():
@@ -98,11 +101,6 @@ class ClockSampler:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unsampled"]}
         return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
                 "samples": len(sm)}
-
-
-def lm_rows_masked(wl, s_in_block):
-    """Masked rows entering step s of a block under top-k: every rollout still has L - k*s masks."""
-    return wl.batch * max(0, wl.block_len - wl.k * s_in_block)
 
 
 def run_ours(args):
@@ -195,6 +193,8 @@ def run_ours(args):
     #      attribute time to the dominant kernel (LM head) for the roofline
     n_inst = min(args.steps, 2 * steps_per_gen)
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(n_inst)]
+    nc_inst = torch.zeros(max(n_inst, 1), B, dtype=torch.int32, device="cuda")
+    nr_inst = torch.zeros(max(n_inst, 1), B, dtype=torch.int32, device="cuda")
     tokens.copy_(tok0)
     torch.cuda.synchronize()
     for t in range(n_inst):
@@ -212,25 +212,32 @@ def run_ours(args):
         ev[t][1].record(stream)
         dare.dare_lmhead_confidence(ctx, x, w, rt, wl.mask_id, True, pred, conf, stream=stream)
         ev[t][2].record(stream)
-        dare.dare_unmask_select(ctx, tokens, bs, L, pred, conf, wl.mask_id, wl.mode, wl.threshold, wl.k, nr, nr,
-                                stream=stream)
+        dare.dare_unmask_select(ctx, tokens, bs, L, pred, conf, wl.mask_id, wl.mode, wl.threshold, wl.k,
+                                nc_inst[t], nr_inst[t], stream=stream)
         ev[t][3].record(stream)
     torch.cuda.synchronize()
     lm_ms = float(np.mean([ev[t][1].elapsed_time(ev[t][2]) for t in range(n_inst)]))
     attn_ms = float(np.mean([ev[t][0].elapsed_time(ev[t][1]) for t in range(n_inst)]))
     sel_ms = float(np.mean([ev[t][2].elapsed_time(ev[t][3]) for t in range(n_inst)]))
-    if wl.mode == I.SELECT_TOPK:
-        masked_avg = float(np.mean([lm_rows_masked(wl, (t % steps_per_gen) % steps_per_block) for t in range(n_inst)]))
-    else:
-        masked_avg = float(B * L)
+    # rows that were still masked when each step began = committed in it + left after it (read back, not assumed)
+    masked = (nc_inst[:n_inst] + nr_inst[:n_inst]).sum(dim=1).cpu().numpy().astype(np.float64)
+    masked_avg = float(masked.mean())
+    executed_rows = float((np.ceil(masked / 128.0) * 128.0).mean())      # the GEMM works on 128-row tiles
     peaks = _peaks()
     lm_flops = 2.0 * masked_avg * wl.hidden * wl.vocab          # algorithmic: masked rows only
     achieved = lm_flops / (lm_ms * 1e-3) / 1e12
     peak = peaks["bf16_tflops_sustained"]
-    roofline = {"bound": "tensor", "kernel": "lmhead_partial_kernel (+ row compaction and merge kernels)", "achieved": achieved, "peak": peak,
-                "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None, "peak_source": peaks["source"] + " sustained",
-                "executed_tflops": 2.0 * B * L * wl.hidden * wl.vocab / (lm_ms * 1e-3) / 1e12,
+    # time the same launches would take at the roofline: per step the slower of the contraction at the measured
+    # tensor peak and one pass over W at the measured HBM bandwidth (few masked rows => the W read bounds it)
+    w_bytes = 2.0 * wl.vocab * wl.hidden
+    ideal_ms = float(np.mean(np.maximum(2.0 * masked * wl.hidden * wl.vocab / (peak * 1e12),
+                                        w_bytes / (peaks["hbm_gbs"] * 1e9)))) * 1e3
+    roofline = {"bound": "tensor", "kernel": "lmhead_partial_kernel (+ row compaction and merge kernels)",
+                "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                "traffic": LMHEAD_TRAFFIC_BYTES.get(wl.name), "peak_source": peaks["source"] + " sustained",
+                "executed_tflops": 2.0 * executed_rows * wl.hidden * wl.vocab / (lm_ms * 1e-3) / 1e12,
                 "ms_per_launch": lm_ms, "masked_rows_avg": masked_avg,
+                "frac_of_tensor_or_hbm_bound_time": ideal_ms / lm_ms,
                 "frac_of_nominal_2250": achieved / 2250.0}
     kv_bytes = 2.0 * 2 * B * wl.n_kv_heads * wl.head_dim * (
         float(np.mean([wl.prompt_len + ((t % steps_per_gen) // steps_per_block) * L + L for t in range(n_inst)])) + wl.suffix_cap)

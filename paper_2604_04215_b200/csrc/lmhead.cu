@@ -394,9 +394,9 @@ int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M,
 // ------------------------------------------------------------------------------------------------
 // Allocation-free variant of the LM-head entry point.
 //
-// Some callers must not allocate device memory at all: code running while a stream is being captured,
-// code inside a framework's allocator callback or under a memory budget that forbids cudaMalloc, and
-// plug-ins loaded into a process whose allocator they do not own.  dare_create allocates its workspace,
+// Some callers must not allocate device memory at all: code inside a framework's allocator callback or
+// under a memory budget that forbids cudaMalloc, and plug-ins loaded into a process whose allocator they
+// do not own.  dare_create allocates its workspace,
 // so those callers cannot have a context.  For them the per-tile (max, sum, argmax) triples of the LM
 // head live in a fixed array inside the library's device image.
 namespace dare {
