@@ -25,6 +25,7 @@ import torch
 # tensor ids (kept stable: they key the random streams)
 TID_Q, TID_KPRE, TID_VPRE, TID_KBLK, TID_VBLK, TID_KSUF, TID_VSUF = 1, 2, 3, 4, 5, 6, 7
 TID_X, TID_W, TID_PLEN, TID_SLEN, TID_PLANT, TID_TOK = 8, 9, 10, 11, 12, 13
+TID_EMB, TID_LAYER0 = 14, 32     # layer l uses ids TID_LAYER0 + 8*l + {0: wqkv, 1: wo, 2: wg, 3: wu, 4: wd}
 
 SELECT_THRESHOLD = 0
 SELECT_TOPK = 1
@@ -235,3 +236,74 @@ def make_step(wl: Workload, step: int = 0, block_index: int = 0, inplace_block: 
         tokens = fresh_tokens(wl)
     return StepInputs(wl, q, k_pre, v_pre, plen, k_blk, v_blk, k_suf, v_suf, slen, x, w, tokens,
                       tokens.shape[1], wl.prompt_len + block_index * wl.block_len, extras)
+
+
+# ---------------------------------------------------------------------------------------------------
+# The end-to-end loop workload: a random-init decoder-shaped stack (RMSNorm, RoPE, SwiGLU, untied LM head).
+
+@dataclass
+class ModelWorkload:
+    """Shape of the end-to-end denoising loop on a small stack of layers."""
+    name: str
+    n_layers: int
+    hidden: int
+    n_q_heads: int
+    n_kv_heads: int
+    head_dim: int
+    ffn: int
+    vocab: int
+    mask_id: int
+    batch: int
+    prompt_len: int
+    gen_len: int
+    block_len: int
+    mode: int
+    threshold: float = 0.9
+    k: int = 1
+    rms_eps: float = 1e-5
+    rope_base: float = 10000.0
+    seed: int = 0
+
+    @property
+    def row_len(self) -> int:
+        return self.prompt_len + self.gen_len
+
+
+MODEL_WORKLOADS = {
+    # the 4-layer LLaDA-shaped loop
+    "llada_loop": ModelWorkload("llada_loop", 4, 4096, 32, 32, 128, 12288, 126464, 126336, 16, 512, 256, 32,
+                                SELECT_THRESHOLD, threshold=0.9),
+    # small cases for element-by-element parity
+    "loop_small": ModelWorkload("loop_small", 2, 256, 4, 4, 64, 768, 4096, 4095, 2, 48, 64, 32,
+                                SELECT_THRESHOLD, threshold=0.9),
+    "loop_small_gqa": ModelWorkload("loop_small_gqa", 3, 512, 4, 2, 128, 1280, 2048, 2000, 3, 40, 32, 16,
+                                    SELECT_TOPK, k=3),
+}
+
+
+def make_model_weights(mw: ModelWorkload):
+    """All weights of the stack, N(0, 0.02) bf16, stored [out features, in features] (K-major).
+
+    Returns dict: embedding [V, D], lm_head [V, D], layers = list of dicts with wqkv [(Hq+2Hkv)d, D] (rows:
+    q heads, k heads, v heads), wo [D, Hq d], wg [F, D], wu [F, D], wd [D, F].
+    """
+    D, F = mw.hidden, mw.ffn
+    nq, nk = mw.n_q_heads * mw.head_dim, mw.n_kv_heads * mw.head_dim
+    layers = []
+    for l in range(mw.n_layers):
+        t = TID_LAYER0 + 8 * l
+        layers.append({"wqkv": normal_bf16(mw.seed, t + 0, (nq + 2 * nk, D), 0.02),
+                       "wo": normal_bf16(mw.seed, t + 1, (D, nq), 0.02),
+                       "wg": normal_bf16(mw.seed, t + 2, (F, D), 0.02),
+                       "wu": normal_bf16(mw.seed, t + 3, (F, D), 0.02),
+                       "wd": normal_bf16(mw.seed, t + 4, (D, F), 0.02)})
+    return {"embedding": normal_bf16(mw.seed, TID_EMB, (mw.vocab, D), 0.02),
+            "lm_head": normal_bf16(mw.seed, TID_W, (mw.vocab, D), 0.02), "layers": layers}
+
+
+def fresh_model_tokens(mw: ModelWorkload) -> torch.Tensor:
+    """Token state [B, prompt + gen]: uniform prompt ids (never the mask id), generation region all <MASK>."""
+    tok = uniform_int(mw.seed, TID_TOK, (mw.batch, mw.row_len), 0, mw.vocab - 2)
+    tok = torch.where(tok >= mw.mask_id, tok + 1, tok).to(torch.int32)
+    tok[:, mw.prompt_len:] = mw.mask_id
+    return tok.contiguous()

@@ -1,0 +1,202 @@
+"""Pins for the oracle of the end-to-end loop (oracle/dare_model_oracle.py), CPU only.
+
+The paper prints no values for this loop, so the oracle is tied down by what the mathematics fixes:
+  * the cache recurrence: the cached loop equals, step by step, a from-scratch forward of the whole sequence
+    under the block-causal visibility rule;
+  * the stack itself: an independently written torch formulation (library attention with a boolean mask,
+    library rms_norm / silu, RoPE as a complex multiplication on re-paired channels);
+  * RoPE: position 0 is the identity, norms are kept, scores depend only on position differences;
+  * RMSNorm: unit root-mean-square; bf16 rounding: torch's own conversion, including ties;
+  * loop counts: every rollout commits exactly G tokens; steps per block = ceil(L / k) under top-k and
+    at most L under the threshold rule; prompt tokens never change; same seed, same tokens.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import dare_model_oracle as MO
+from oracle import dare_oracle as O
+from paper_2604_04215_b200 import inputs as I
+
+
+def _cfg(mw):
+    return MO.ModelConfig(mw.n_layers, mw.hidden, mw.n_q_heads, mw.n_kv_heads, mw.head_dim, mw.ffn, mw.vocab,
+                          mw.mask_id, mw.rms_eps, mw.rope_base)
+
+
+def _weights(mw):
+    w = I.make_model_weights(mw)
+    f = lambda t: t.to(torch.float64).numpy()
+    layers = [MO.LayerWeights(f(l["wqkv"]), f(l["wo"]), f(l["wg"]), f(l["wu"]), f(l["wd"])) for l in w["layers"]]
+    return MO.ModelWeights(f(w["embedding"]), layers, f(w["lm_head"]))
+
+
+def _small(**kw):
+    base = I.MODEL_WORKLOADS["loop_small"]
+    d = dict(base.__dict__)
+    d.update(dict(n_layers=2, hidden=64, n_q_heads=4, n_kv_heads=2, head_dim=16, ffn=96, vocab=128, mask_id=100,
+                  batch=2, prompt_len=5, gen_len=12, block_len=4))
+    d.update(kw)
+    return I.ModelWorkload(**d)
+
+
+def test_bf16_round_is_torch_conversion_including_ties():
+    rng = np.random.default_rng(0)
+    a = np.concatenate([rng.standard_normal(4096) * 10.0 ** rng.integers(-6, 6, 4096),
+                        np.array([1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, -(1.0 + 2.0 ** -8), 0.0, 1e-40, 3.0e38])])
+    want = torch.from_numpy(a).to(torch.float32).to(torch.bfloat16).to(torch.float64).numpy()
+    np.testing.assert_array_equal(MO.bf16_round(a), want)
+    # the two tie cases round to the even mantissa: 1 + 2^-8 -> 1, 1 + 3*2^-8 -> 1 + 2^-6
+    assert MO.bf16_round(np.array([1.0 + 2.0 ** -8]))[0] == 1.0
+    assert MO.bf16_round(np.array([1.0 + 3 * 2.0 ** -8]))[0] == 1.0 + 2.0 ** -6
+
+
+def test_rope_properties():
+    rng = np.random.default_rng(1)
+    T, H, d = 7, 3, 16
+    q, k = rng.standard_normal((T, H, d)), rng.standard_normal((T, H, d))
+    # position 0 is the identity; rotations keep the norm of every (c, c + d/2) pair
+    np.testing.assert_allclose(MO.rope(q, np.zeros(T, dtype=int), 10000.0), q, atol=0)
+    pos = np.array([0, 1, 2, 5, 9, 100, 511])
+    rq = MO.rope(q, pos, 10000.0)
+    np.testing.assert_allclose(rq[..., :8] ** 2 + rq[..., 8:] ** 2, q[..., :8] ** 2 + q[..., 8:] ** 2, rtol=1e-12)
+    # scores depend only on the position difference
+    s1 = np.einsum("thd,shd->hts", MO.rope(q, pos, 10000.0), MO.rope(k, pos, 10000.0))
+    s2 = np.einsum("thd,shd->hts", MO.rope(q, pos + 37, 10000.0), MO.rope(k, pos + 37, 10000.0))
+    np.testing.assert_allclose(s1, s2, atol=1e-10)
+    # a hand-worked pair: d = 2, position 1, base irrelevant (c = 0): rotation by 1 radian
+    out = MO.rope(np.array([[[1.0, 0.0]]]), np.array([1]), 10000.0)
+    np.testing.assert_allclose(out[0, 0], [np.cos(1.0), np.sin(1.0)], atol=1e-15)
+    # channel c turns at base^(-2c/d): d = 4, c = 1 -> 1/100 radian per position
+    out = MO.rope(np.array([[[0.0, 1.0, 0.0, 0.0]]]), np.array([3]), 10000.0)
+    np.testing.assert_allclose(out[0, 0], [0.0, np.cos(0.03), 0.0, np.sin(0.03)], atol=1e-15)
+
+
+def test_rmsnorm_has_unit_rms():
+    rng = np.random.default_rng(2)
+    x = rng.standard_normal((5, 64)) * 7.0
+    y = MO.rmsnorm(x, 0.0)
+    np.testing.assert_allclose(np.sqrt((y * y).mean(axis=-1)), 1.0, rtol=1e-12)
+    np.testing.assert_allclose(MO.rmsnorm(x, 1e-5), x / np.sqrt((x * x).mean(-1, keepdims=True) + 1e-5), rtol=1e-15)
+
+
+def _torch_stack(cfg, wts, tokens_row, seg):
+    """The same architecture written differently, in torch float64: library attention with a boolean mask,
+    library rms_norm and silu, RoPE as multiplication by e^{i angle} of the complex number (x_c, x_{c+d/2})."""
+    F = torch.nn.functional
+    t = lambda a: torch.from_numpy(np.ascontiguousarray(a))
+    T = len(tokens_row)
+    d, Hq, Hkv = cfg.head_dim, cfg.n_q_heads, cfg.n_kv_heads
+    x = t(wts.embedding)[torch.as_tensor(np.asarray(tokens_row), dtype=torch.long)]
+    mask = torch.from_numpy(seg[None, :] <= seg[:, None])
+    inv = torch.tensor(cfg.rope_base, dtype=torch.float64) ** (-torch.arange(0, d, 2, dtype=torch.float64) / d)
+    rot = torch.polar(torch.ones(T, d // 2, dtype=torch.float64), torch.arange(T, dtype=torch.float64)[:, None] * inv)
+
+    def rope(v):   # v [T, H, d]
+        z = torch.complex(v[..., :d // 2], v[..., d // 2:]) * rot[:, None, :]
+        return torch.cat([z.real, z.imag], dim=-1)
+
+    for lw in wts.layers:
+        h = F.rms_norm(x, (cfg.hidden,), eps=cfg.rms_eps)
+        qkv = F.linear(h, t(lw.wqkv))
+        q = rope(qkv[:, :Hq * d].view(T, Hq, d)).transpose(0, 1)
+        k = rope(qkv[:, Hq * d:(Hq + Hkv) * d].view(T, Hkv, d)).transpose(0, 1)
+        v = qkv[:, (Hq + Hkv) * d:].view(T, Hkv, d).transpose(0, 1)
+        k = k.repeat_interleave(Hq // Hkv, dim=0)
+        v = v.repeat_interleave(Hq // Hkv, dim=0)
+        o = F.scaled_dot_product_attention(q[None], k[None], v[None], attn_mask=mask[None, None])[0]
+        x = x + F.linear(o.transpose(0, 1).reshape(T, Hq * d), t(lw.wo))
+        h2 = F.rms_norm(x, (cfg.hidden,), eps=cfg.rms_eps)
+        x = x + F.linear(F.silu(F.linear(h2, t(lw.wg))) * F.linear(h2, t(lw.wu)), t(lw.wd))
+    return F.rms_norm(x, (cfg.hidden,), eps=cfg.rms_eps).numpy()
+
+
+@pytest.mark.parametrize("gqa", [False, True])
+def test_uncached_forward_matches_independent_torch_formulation(gqa):
+    mw = _small(n_kv_heads=2 if gqa else 4)
+    cfg, wts = _cfg(mw), _weights(mw)
+    tok = I.fresh_model_tokens(mw).numpy()
+    tok[:, mw.prompt_len:mw.prompt_len + 6] = 3             # some committed generation tokens
+    seg = MO.segment_ids(mw.prompt_len, mw.gen_len, mw.block_len)
+    got, _ = MO.forward_uncached(cfg, wts, tok[0], seg, rounded=False)
+    want = _torch_stack(cfg, wts, tok[0], seg)
+    np.testing.assert_allclose(got, want, atol=1e-10)
+    # the weights are tiny (sigma 0.02): make sure the check is not vacuous
+    assert np.abs(want).max() > 0.5 and np.abs(got - np.roll(want, 1, axis=0)).max() > 1e-3
+
+
+def test_block_causal_rule():
+    seg = MO.segment_ids(3, 4, 2)
+    np.testing.assert_array_equal(seg, [0, 0, 0, 1, 1, 2, 2])
+    mw = _small()
+    cfg, wts = _cfg(mw), _weights(mw)
+    tok = I.fresh_model_tokens(mw).numpy()[0]
+    seg = MO.segment_ids(mw.prompt_len, mw.gen_len, mw.block_len)
+    base, _ = MO.forward_uncached(cfg, wts, tok, seg, rounded=False)
+    # changing a token of the LAST block leaves every earlier position's output untouched, and changes its own block
+    tok2 = tok.copy()
+    tok2[-1] = 7
+    out2, _ = MO.forward_uncached(cfg, wts, tok2, seg, rounded=False)
+    first_of_last = mw.prompt_len + mw.gen_len - mw.block_len
+    np.testing.assert_array_equal(out2[:first_of_last], base[:first_of_last])
+    assert np.abs(out2[first_of_last:] - base[first_of_last:]).min(axis=1).max() > 0
+    # the prompt is bidirectional: changing its last token changes its first position
+    tok3 = tok.copy()
+    tok3[mw.prompt_len - 1] = (tok3[mw.prompt_len - 1] + 1) % 90
+    out3, _ = MO.forward_uncached(cfg, wts, tok3, seg, rounded=False)
+    assert np.abs(out3[0] - base[0]).max() > 0
+
+
+@pytest.mark.parametrize("rounded", [False, True])
+@pytest.mark.parametrize("mode,k", [(O.SELECT_THRESHOLD, 1), (O.SELECT_TOPK, 3)])
+def test_cached_loop_equals_uncached_forward_step_by_step(rounded, mode, k):
+    mw = _small(batch=2)
+    cfg, wts = _cfg(mw), _weights(mw)
+    tok0 = I.fresh_model_tokens(mw).numpy()
+    seg = MO.segment_ids(mw.prompt_len, mw.gen_len, mw.block_len)
+    L = mw.block_len
+    seen = []
+
+    def on_step(b, n, tok_before, res):
+        start = mw.prompt_len + b * L
+        for r in range(mw.batch):
+            full, _ = MO.forward_uncached(cfg, wts, tok_before[r], seg, rounded)
+            got = res["hidden"][r * L:(r + 1) * L]
+            if rounded:
+                # identical rounding points; a last-bit difference of the two summation orders can move one
+                # bf16 rounding, so allow one bf16 step on O(1) values
+                np.testing.assert_allclose(got, full[start:start + L], atol=2e-2)
+                assert np.abs(got - full[start:start + L]).mean() < 1e-4
+            else:
+                np.testing.assert_allclose(got, full[start:start + L], atol=1e-9)
+            lm = O.lmhead_confidence(full[start:start + L], wts.lm_head, tok_before[r, start:start + L], cfg.mask_id)
+            if not rounded:
+                np.testing.assert_array_equal(lm["pred"], res["lm"]["pred"][r * L:(r + 1) * L])
+        seen.append((b, n))
+
+    tok, steps, cache = MO.generate(cfg, wts, tok0, mw.prompt_len, mw.gen_len, L, mode, 0.9, k, rounded, on_step)
+    assert len(seen) == sum(steps)
+    # counts: every rollout commits all G tokens, nothing of the prompt changes
+    assert (tok[:, mw.prompt_len:] != cfg.mask_id).all()
+    np.testing.assert_array_equal(tok[:, :mw.prompt_len], tok0[:, :mw.prompt_len])
+    if mode == O.SELECT_TOPK:
+        assert steps == [-(-L // k)] * (mw.gen_len // L)
+    else:
+        assert all(1 <= s <= L for s in steps)
+    # after the loop the cache holds the K/V of the final sequence (the refresh forward did its job)
+    for r in range(mw.batch):
+        _, kv = MO.forward_uncached(cfg, wts, tok[r], seg, rounded)
+        for li, (k_full, v_full) in enumerate(kv):
+            tol = 2e-2 if rounded else 1e-9
+            np.testing.assert_allclose(cache[li][0][r], np.transpose(k_full, (1, 0, 2)), atol=tol)
+            np.testing.assert_allclose(cache[li][1][r], np.transpose(v_full, (1, 0, 2)), atol=tol)
+
+
+def test_generate_is_deterministic():
+    mw = _small(batch=1, gen_len=8)
+    cfg, wts = _cfg(mw), _weights(mw)
+    tok0 = I.fresh_model_tokens(mw).numpy()
+    a = MO.generate(cfg, wts, tok0, mw.prompt_len, mw.gen_len, mw.block_len, O.SELECT_THRESHOLD, 0.9, 1)
+    b = MO.generate(cfg, wts, tok0, mw.prompt_len, mw.gen_len, mw.block_len, O.SELECT_THRESHOLD, 0.9, 1)
+    np.testing.assert_array_equal(a[0], b[0])
+    assert a[1] == b[1]
