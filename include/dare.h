@@ -11,6 +11,8 @@
  *                             logits never written to memory
  *     dare_unmask_select      confidence-threshold / per-block top-k commit on the int32 token state
  *     dare_denoise_block      the three above, enqueued back to back
+ *     dare_model_* / dare_generate   the same step with a stack of transformer layers in between, and the
+ *                             whole block-by-block loop
  *
  * Conventions
  *   - Every data pointer is a DEVICE pointer unless the comment says "host".  The caller owns every
@@ -85,7 +87,7 @@ int dare_sm_count(const dare_ctx* ctx);
  *   out          bf16 [B, L, Hq, d]
  *   lse          fp32 [B, Hq, L] or NULL: natural-log sum of exp(scale * score)
  *   scale        softmax scale; 0 => 1/sqrt(d)
- * Supported: d in {64, 128}; Hq % Hkv == 0; L >= 1; L * (Hq/Hkv) <= 1024.
+ * Supported: d in {64, 128}; Hq % Hkv == 0; L >= 1; L * (Hq/Hkv) <= 2^20.
  * Lengths beyond capacity are clamped and flagged in the device status word.
  */
 int dare_attn_block(dare_ctx* ctx,
@@ -152,6 +154,98 @@ int dare_denoise_block(dare_ctx* ctx,
                        int mode, float threshold, int k,
                        int32_t* pred, float* conf,
                        int32_t* n_committed, int32_t* n_remaining, void* stream);
+
+/*
+ * ---------------------------------------------------------------------------------------------------------
+ * End-to-end denoising loop on a decoder-shaped stack (the rollout of Section 3.4 with the layers in between;
+ * Section 2.1: blocks are bidirectional inside and see the prompt and the earlier blocks).  The paper names no
+ * architecture; the stack is pre-norm, without biases: per layer  h = RMSNorm(x);  q, k, v = h Wqkv^T;
+ * RoPE(q, k) at the absolute position (channel c pairs with c + d/2, angle = position * base^(-2c/d));
+ * block attention against the K/V cache;  x += attn Wo^T;  x += (silu(h2 Wg^T) * (h2 Wu^T)) Wd^T with
+ * h2 = RMSNorm(x);  a final RMSNorm feeds the untied LM head.  RMSNorm has unit weight.
+ * bf16 is stored after every RMSNorm, after the QKV projection, after RoPE, after attention, after each
+ * residual addition (rounded once, after the add) and after the SwiGLU product; everything else is fp32.
+ *
+ * All weights are bf16, [out features, in features] row-major, 16-byte aligned, caller-owned DEVICE memory
+ * that must stay valid while the model exists:
+ *   embedding [V, D]; lm_head [V, D]; per layer wqkv [(Hq + 2 Hkv) d, D] (rows: q heads, k heads, v heads),
+ *   wo [D, Hq d], wg [F, D], wu [F, D], wd [D, F].
+ * K/V cache (caller-owned): k_cache and v_cache are bf16 [n_layers, B, Hkv, cache_cap, d]; position p of a
+ * rollout lives at index p.
+ */
+typedef struct dare_model dare_model;
+
+typedef struct {
+    int n_layers, hidden, n_q_heads, n_kv_heads, head_dim, ffn, vocab;
+    int32_t mask_id;
+    float rms_eps;          /* e.g. 1e-5 */
+    float rope_base;        /* e.g. 10000 */
+    int max_positions;      /* largest cache_cap any call will use (size of the RoPE table) */
+    int max_rows;           /* largest B * length one forward processes (B * prompt length for the prefill) */
+    int max_batch;          /* largest B */
+} dare_model_desc;
+
+typedef struct {
+    const void *wqkv, *wo, *wg, *wu, *wd;   /* device pointers */
+} dare_layer_weights;
+
+/* Creates the model object: copies `layers` (HOST array of n_layers entries), allocates the activation
+ * buffers for max_rows rows and builds the RoPE table.  Allocates and synchronises: call at set-up time.
+ * The ctx must outlive the model and serves one stream at a time together with it. */
+int dare_model_create(dare_ctx* ctx, const dare_model_desc* desc, const void* embedding,
+                      const dare_layer_weights* layers, const void* lm_head, dare_model** out);
+int dare_model_destroy(dare_model* model);
+
+/*
+ * Building blocks of the stack, exported so that each can be checked on its own.  All enqueue on `stream`.
+ *
+ * dare_linear:  out[M, N] = epilogue(a[M, K] . w[N, K]^T), bf16 row-major operands, fp32 accumulation.
+ *   epilogue DARE_LINEAR_STORE:    out = acc
+ *            DARE_LINEAR_RESIDUAL: out = residual + acc, rounded once (residual bf16 [M, N]; may be `out`)
+ *            DARE_LINEAR_SWIGLU:   out = silu(a . w^T) * (a . w2^T)   (w, w2 both [N, K])
+ *   Supported: N, K multiples of 8; pointers 16-byte aligned.
+ * dare_rmsnorm: y[m, :] = x[m, :] / sqrt(mean(x[m, :]^2) + eps)   (x, y bf16 [n_rows, D], D % 8 == 0).
+ * dare_rope_kv_write: row m = (b, i) of qkv [B * length, (Hq + 2 Hkv) d] at position start + i:
+ *   q heads rotated -> q_out [B * length, Hq, d]; k heads rotated -> k_cache[b, :, start + i, :];
+ *   v heads copied -> v_cache[b, :, start + i, :]  (caches bf16 [B, Hkv, cache_cap, d], one layer).
+ */
+enum { DARE_LINEAR_STORE = 0, DARE_LINEAR_RESIDUAL = 1, DARE_LINEAR_SWIGLU = 2 };
+int dare_linear(dare_ctx* ctx, int epilogue, const void* a, int M, int K, const void* w, const void* w2, int N,
+                void* out, const void* residual, void* stream);
+int dare_rmsnorm(dare_ctx* ctx, const void* x, int n_rows, int D, float eps, void* y, void* stream);
+int dare_rope_kv_write(dare_model* model, const void* qkv, int B, int length, int start, void* q_out,
+                       void* k_cache, void* v_cache, int cache_cap, void* stream);
+
+/*
+ * The rows [start, start + length) of every rollout through the whole stack: their post-RoPE K/V are
+ * written into the cache at [start, start + length) and they attend to cache[0, start + length).
+ * start = 0, length = prompt length is the prefill; start = a block's first position, length = L is the
+ * refresh of a finished block.  tokens int32 [B, row_stride] (read only).  hidden_out: bf16
+ * [B * length, D] final-RMSNorm hidden states, or NULL.  Enqueues on `stream`, no synchronisation.
+ */
+int dare_model_forward(dare_model* model, const int32_t* tokens, int B, int64_t row_stride, int start, int length,
+                       void* k_cache, void* v_cache, int cache_cap, void* hidden_out, void* stream);
+
+/*
+ * One denoising step of block [block_start, block_start + L): dare_model_forward on the block's rows, the
+ * LM head on the rows that are still masked, the unmask selection in place on `tokens`.
+ * pred int32 [B * L], conf fp32 [B * L] (results of the step), n_committed / n_remaining int32 [B] or NULL.
+ * Enqueues on `stream`, no synchronisation.
+ */
+int dare_model_step(dare_model* model, int32_t* tokens, int B, int64_t row_stride, int block_start, int L,
+                    void* k_cache, void* v_cache, int cache_cap, int mode, float threshold, int k,
+                    int32_t* pred, float* conf, int32_t* n_committed, int32_t* n_remaining, void* stream);
+
+/*
+ * The whole loop: prefill of tokens[:, 0 : prompt_len], then for each block of L positions steps are repeated
+ * until no rollout has a mask left in it (the batch moves block by block), then the block's K/V are refreshed
+ * from the committed tokens and the prefix grows by L.  The host reads the per-step mask counts one step
+ * behind the GPU, so the GPU never waits for it.  steps_per_block: HOST int32 [gen_len / L] or NULL.
+ * n_remaining: device int32 [B] (scratch and last counts).  This call BLOCKS until the loop has finished.
+ */
+int dare_generate(dare_model* model, int32_t* tokens, int B, int64_t row_stride, int prompt_len, int gen_len, int L,
+                  void* k_cache, void* v_cache, int cache_cap, int mode, float threshold, int k,
+                  int32_t* pred, float* conf, int32_t* n_remaining, int32_t* steps_per_block, void* stream);
 
 /*
  * Allocation-free variant of dare_lmhead_confidence.  (The paper has no counterpart for this entry

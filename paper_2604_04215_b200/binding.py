@@ -22,7 +22,8 @@ DEV_WAIT_EXPIRED = 2
 
 EXPORTS = ["dare_create", "dare_destroy", "dare_status_string", "dare_device_status", "dare_sm_count",
            "dare_attn_block", "dare_lmhead_confidence", "dare_unmask_select", "dare_denoise_block",
-           "dare_lmhead_confidence_static"]
+           "dare_lmhead_confidence_static", "dare_model_create", "dare_model_destroy", "dare_model_forward",
+           "dare_model_step", "dare_generate", "dare_linear", "dare_rmsnorm", "dare_rope_kv_write"]
 
 _lib = None
 
@@ -68,8 +69,37 @@ def load():
                                         vp, i64, i32, i32, f32, i32,             # tokens, stride, start, mode, thr, k
                                         vp, vp, vp, vp, vp])                     # pred, conf, n_comm, n_rem, stream
     lib.dare_denoise_block.restype = i32
+    lib.dare_model_create.argtypes = [vp, C.POINTER(ModelDesc), vp, C.POINTER(LayerWeights), vp, C.POINTER(vp)]
+    lib.dare_model_create.restype = i32
+    lib.dare_model_destroy.argtypes = [vp]
+    lib.dare_model_destroy.restype = i32
+    lib.dare_model_forward.argtypes = [vp, vp, i32, i64, i32, i32, vp, vp, i32, vp, vp]
+    lib.dare_model_forward.restype = i32
+    lib.dare_model_step.argtypes = [vp, vp, i32, i64, i32, i32, vp, vp, i32, i32, f32, i32, vp, vp, vp, vp, vp]
+    lib.dare_model_step.restype = i32
+    lib.dare_generate.argtypes = [vp, vp, i32, i64, i32, i32, i32, vp, vp, i32, i32, f32, i32, vp, vp, vp,
+                                  C.POINTER(C.c_int32), vp]
+    lib.dare_generate.restype = i32
+    lib.dare_linear.argtypes = [vp, i32, vp, i32, i32, vp, vp, i32, vp, vp, vp]
+    lib.dare_linear.restype = i32
+    lib.dare_rmsnorm.argtypes = [vp, vp, i32, i32, f32, vp, vp]
+    lib.dare_rmsnorm.restype = i32
+    lib.dare_rope_kv_write.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, i32, vp]
+    lib.dare_rope_kv_write.restype = i32
     _lib = lib
     return lib
+
+
+class ModelDesc(C.Structure):
+    _fields_ = [("n_layers", C.c_int), ("hidden", C.c_int), ("n_q_heads", C.c_int), ("n_kv_heads", C.c_int),
+                ("head_dim", C.c_int), ("ffn", C.c_int), ("vocab", C.c_int), ("mask_id", C.c_int32),
+                ("rms_eps", C.c_float), ("rope_base", C.c_float), ("max_positions", C.c_int),
+                ("max_rows", C.c_int), ("max_batch", C.c_int)]
+
+
+class LayerWeights(C.Structure):
+    _fields_ = [("wqkv", C.c_void_p), ("wo", C.c_void_p), ("wg", C.c_void_p), ("wu", C.c_void_p),
+                ("wd", C.c_void_p)]
 
 
 def _ptr(t: Optional[torch.Tensor], dtype=None):
@@ -216,3 +246,116 @@ def dare_denoise_block(ctx: Context, q, k_pre, v_pre, prefix_len, k_blk, v_blk, 
     if rc != 0 and check:
         raise DareError(rc, "dare_denoise_block")
     return rc
+
+
+LINEAR_STORE, LINEAR_RESIDUAL, LINEAR_SWIGLU = 0, 1, 2
+
+
+def dare_linear(ctx: Context, epilogue: int, a, w, w2=None, residual=None, out=None, stream=None, check: bool = True):
+    M, K = a.shape
+    N = w.shape[0]
+    bf = torch.bfloat16
+    if out is None:
+        out = torch.empty(M, N, dtype=bf, device=a.device)
+    rc = load().dare_linear(ctx.handle, int(epilogue), _ptr(a, bf), M, K, _ptr(w, bf), _ptr(w2, bf), N, _ptr(out, bf),
+                            _ptr(residual, bf), _stream(stream))
+    if rc != 0 and check:
+        raise DareError(rc, "dare_linear")
+    return out if check else rc
+
+
+def dare_rmsnorm(ctx: Context, x, eps: float, y=None, stream=None, check: bool = True):
+    n_rows, D = x.shape
+    if y is None:
+        y = torch.empty_like(x)
+    rc = load().dare_rmsnorm(ctx.handle, _ptr(x, torch.bfloat16), n_rows, D, float(eps), _ptr(y, torch.bfloat16),
+                             _stream(stream))
+    if rc != 0 and check:
+        raise DareError(rc, "dare_rmsnorm")
+    return y if check else rc
+
+
+class Model:
+    """Owns a dare_model: the caller's weight tensors (kept alive here), activation buffers, the RoPE table."""
+
+    def __init__(self, ctx: Context, *, n_layers, hidden, n_q_heads, n_kv_heads, head_dim, ffn, vocab, mask_id,
+                 embedding, layers, lm_head, max_positions, max_rows, max_batch, rms_eps=1e-5, rope_base=10000.0):
+        lib = load()
+        bf = torch.bfloat16
+        self.ctx = ctx
+        self._keep = (embedding, layers, lm_head)
+        self.desc = ModelDesc(n_layers, hidden, n_q_heads, n_kv_heads, head_dim, ffn, vocab, mask_id, rms_eps,
+                              rope_base, max_positions, max_rows, max_batch)
+        arr = (LayerWeights * n_layers)()
+        for i, l in enumerate(layers):
+            arr[i] = LayerWeights(*[_ptr(l[k], bf).value for k in ("wqkv", "wo", "wg", "wu", "wd")])
+        h = C.c_void_p()
+        rc = lib.dare_model_create(ctx.handle, C.byref(self.desc), _ptr(embedding, bf), arr, _ptr(lm_head, bf),
+                                   C.byref(h))
+        if rc != 0:
+            raise DareError(rc, "dare_model_create")
+        self.handle = h
+
+    def close(self):
+        if getattr(self, "handle", None):
+            load().dare_model_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def new_cache(self, batch: int, cap: int, device="cuda"):
+        shp = (self.desc.n_layers, batch, self.desc.n_kv_heads, cap, self.desc.head_dim)
+        return (torch.zeros(shp, dtype=torch.bfloat16, device=device),
+                torch.zeros(shp, dtype=torch.bfloat16, device=device))
+
+
+def dare_rope_kv_write(model: Model, qkv, B: int, length: int, start: int, q_out, k_cache, v_cache, stream=None):
+    bf = torch.bfloat16
+    rc = load().dare_rope_kv_write(model.handle, _ptr(qkv, bf), B, length, start, _ptr(q_out, bf), _ptr(k_cache, bf),
+                                   _ptr(v_cache, bf), k_cache.shape[-2], _stream(stream))
+    if rc != 0:
+        raise DareError(rc, "dare_rope_kv_write")
+
+
+def dare_model_forward(model: Model, tokens, start: int, length: int, k_cache, v_cache, hidden_out=None, stream=None,
+                       check: bool = True):
+    B, row_stride = tokens.shape
+    bf = torch.bfloat16
+    rc = load().dare_model_forward(model.handle, _ptr(tokens, torch.int32), B, row_stride, int(start), int(length),
+                                   _ptr(k_cache, bf), _ptr(v_cache, bf), k_cache.shape[3], _ptr(hidden_out, bf),
+                                   _stream(stream))
+    if rc != 0 and check:
+        raise DareError(rc, "dare_model_forward")
+    return rc
+
+
+def dare_model_step(model: Model, tokens, block_start: int, L: int, k_cache, v_cache, mode: int, threshold: float,
+                    k: int, pred, conf, n_committed=None, n_remaining=None, stream=None, check: bool = True):
+    B, row_stride = tokens.shape
+    bf = torch.bfloat16
+    rc = load().dare_model_step(model.handle, _ptr(tokens, torch.int32), B, row_stride, int(block_start), int(L),
+                                _ptr(k_cache, bf), _ptr(v_cache, bf), k_cache.shape[3], int(mode), float(threshold),
+                                int(k), _ptr(pred, torch.int32), _ptr(conf, torch.float32),
+                                _ptr(n_committed, torch.int32), _ptr(n_remaining, torch.int32), _stream(stream))
+    if rc != 0 and check:
+        raise DareError(rc, "dare_model_step")
+    return rc
+
+
+def dare_generate(model: Model, tokens, prompt_len: int, gen_len: int, L: int, k_cache, v_cache, mode: int,
+                  threshold: float, k: int, pred, conf, n_remaining, stream=None, check: bool = True):
+    """Runs the whole loop (blocks until done); returns the list of denoising steps taken per block."""
+    B, row_stride = tokens.shape
+    bf = torch.bfloat16
+    steps = (C.c_int32 * (gen_len // L))()
+    rc = load().dare_generate(model.handle, _ptr(tokens, torch.int32), B, row_stride, int(prompt_len), int(gen_len),
+                              int(L), _ptr(k_cache, bf), _ptr(v_cache, bf), k_cache.shape[3], int(mode),
+                              float(threshold), int(k), _ptr(pred, torch.int32), _ptr(conf, torch.float32),
+                              _ptr(n_remaining, torch.int32), steps, _stream(stream))
+    if rc != 0 and check:
+        raise DareError(rc, "dare_generate")
+    return list(steps) if check else rc

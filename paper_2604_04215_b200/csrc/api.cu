@@ -34,7 +34,7 @@ int check_attn(const dare_ctx* ctx, int B, int L, int Hq, int Hkv, int d, int pr
     if ((k_suf == nullptr) != (v_suf == nullptr)) return DARE_ERR_NULL;
     if (B < 1 || L < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv != 0) return DARE_ERR_SHAPE;
     if (d != 64 && d != 128) return DARE_ERR_SHAPE;
-    if (static_cast<long long>(L) * (Hq / Hkv) > 1024) return DARE_ERR_SHAPE;
+    if (static_cast<long long>(L) * (Hq / Hkv) > (1 << 20)) return DARE_ERR_SHAPE;
     if (prefix_cap < (k_blk ? 1 : L) || suffix_cap < 0) return DARE_ERR_SHAPE;
     if (k_suf && suffix_cap < 1) return DARE_ERR_SHAPE;
     if (static_cast<long long>(B) * Hkv * prefix_cap > 0x7fffffffLL) return DARE_ERR_SHAPE;
@@ -45,6 +45,7 @@ int check_attn(const dare_ctx* ctx, int B, int L, int Hq, int Hkv, int d, int pr
     a->B = B; a->L = L; a->Hq = Hq; a->Hkv = Hkv; a->d = d; a->prefix_cap = prefix_cap; a->suffix_cap = suffix_cap;
     a->scale = scale; a->q = q; a->k_pre = k_pre; a->v_pre = v_pre; a->k_blk = k_blk; a->v_blk = v_blk;
     a->k_suf = k_suf; a->v_suf = v_suf; a->out = const_cast<void*>(out);
+    a->prefix_len = nullptr; a->prefix_len_uniform = -1; a->suffix_len = nullptr; a->lse = nullptr;
     const int splits = dare::attn_plan_splits(ctx, *a);
     if (dare::attn_workspace_bytes(*a, splits) > ctx->workspace_bytes) return DARE_ERR_WORKSPACE;
     return DARE_OK;

@@ -29,6 +29,7 @@ struct AttnParams {
     int B, L, Hq, Hkv, g, R;      // R = L * g packed query rows per (row, kv head)
     int prefix_cap, suffix_cap;
     int inplace, has_suffix, splits;
+    int uniform_P;                // >= 0: every row's prefix length (used when prefix_len is NULL)
     float scale_log2;
     const __nv_bfloat16* q;
     const int32_t* prefix_len;
@@ -114,7 +115,8 @@ attn_block_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_cons
     __syncthreads();
 
     // lengths (clamped to capacity; a clamp is reported, never trapped on)
-    int P = p.prefix_len ? p.prefix_len[b] : (p.inplace ? p.prefix_cap - p.L : p.prefix_cap);
+    int P = p.prefix_len ? p.prefix_len[b]
+                         : (p.uniform_P >= 0 ? p.uniform_P : (p.inplace ? p.prefix_cap - p.L : p.prefix_cap));
     const int p_max = p.inplace ? p.prefix_cap - p.L : p.prefix_cap;
     int S = p.has_suffix ? (p.suffix_len ? p.suffix_len[b] : p.suffix_cap) : 0;
     if (P < 0 || P > p_max || S < 0 || S > p.suffix_cap) {
@@ -447,6 +449,7 @@ int launch_attn(const dare_ctx* ctx, const AttnArgs& a, cudaStream_t stream) {
     p.prefix_cap = a.prefix_cap; p.suffix_cap = a.k_suf ? a.suffix_cap : 0;
     p.inplace = a.k_blk == nullptr; p.has_suffix = a.k_suf != nullptr && a.suffix_cap > 0;
     p.splits = attn_plan_splits(ctx, a);
+    p.uniform_P = a.prefix_len_uniform;
     const float scale = a.scale != 0.f ? a.scale : 1.0f / sqrtf(static_cast<float>(a.d));
     p.scale_log2 = scale * LOG2E_F;
     p.q = static_cast<const __nv_bfloat16*>(a.q);

@@ -44,6 +44,7 @@ struct AttnArgs {
     const void* q;
     const void *k_pre, *v_pre;
     const int32_t* prefix_len;
+    int prefix_len_uniform;   // used when prefix_len is NULL and this is >= 0 (internal callers)
     const void *k_blk, *v_blk;
     const void *k_suf, *v_suf;
     const int32_t* suffix_len;
@@ -53,5 +54,18 @@ struct AttnArgs {
 int attn_plan_splits(const dare_ctx* ctx, const AttnArgs& a);
 size_t attn_workspace_bytes(const AttnArgs& a, int splits);
 int launch_attn(const dare_ctx* ctx, const AttnArgs& a, cudaStream_t stream);
+
+// ---- layer stack (gemm.cu, layers.cu)
+enum { GEMM_EPI_STORE = 0, GEMM_EPI_RESIDUAL = 1, GEMM_EPI_SWIGLU = 2 };
+// out[M, N] = epilogue(a[M, K] . w[N, K]^T), bf16 row-major, ldo = elements per output row.
+//   STORE: out = acc.  RESIDUAL: out = res + acc (res may be out).  SWIGLU: out = silu(a w^T) * (a w2^T).
+int launch_gemm(const dare_ctx* ctx, int epi, const void* a, int M, int K, const void* w, const void* w2, int N,
+                void* out, const void* res, int ldo, cudaStream_t stream);
+int launch_embed(const void* emb, int D, int V, const int32_t* tokens, int64_t row_stride, int start, int length,
+                 int n_rows, void* x, cudaStream_t stream);
+int launch_rmsnorm(const void* x, int D, int n_rows, float eps, void* y, cudaStream_t stream);
+int launch_rope_table(float* cs, int n_pos, int half, double base, cudaStream_t stream);
+int launch_rope_kv_write(const void* qkv, int n_rows, int Hq, int Hkv, int d, int start, int length, const float* cs,
+                         void* q_out, void* k_cache, void* v_cache, int cap, cudaStream_t stream);
 
 }  // namespace dare

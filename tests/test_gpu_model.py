@@ -1,0 +1,298 @@
+"""GPU parity of the layer stack and of the end-to-end loop against the fp64 oracle (through the C ABI).
+
+Building blocks (projection epilogues, RMSNorm, RoPE + cache write) are compared element by element; the whole
+stack and the loop are compared on small models in full, step by step with teacher forcing (the oracle starts
+every step from the GPU's own token state; selection is checked bit-exactly from the GPU's own confidences).
+The full-size 4-layer LLaDA-shaped case follows one sampled rollout of the batch through the oracle.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import dare_model_oracle as MO
+from oracle import dare_oracle as O
+from paper_2604_04215_b200 import binding as dare
+from paper_2604_04215_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+
+BF16_STEP = 2.0 ** -7          # largest relative distance between neighbouring bf16 values
+# The stack's error is the attention's: its probabilities enter the PV product in bf16 (the attention bars are
+# max-abs 2e-2 and relative-L2 5e-3 on O(1) outputs), and each layer adds one such perturbation to the residual
+# stream.  So per layer: relative-L2 5e-3 and max-abs 4e-2 (two bf16 steps of the largest hidden values, ~4).
+HIDDEN_MAX_ABS_PER_LAYER = 4e-2
+HIDDEN_REL_L2_PER_LAYER = 5e-3
+# log-confidence: 2e-2 for the LM head itself plus 2e-2 per layer for the hidden-state perturbation above (a
+# relative-L2 of 5e-3 per layer on |h| = sqrt(D) against weights of sigma 0.02 moves a logit by ~6e-3 rms per layer)
+LOGCONF_ABS_BASE, LOGCONF_ABS_PER_LAYER = 2e-2, 2e-2
+LOGIT_GAP = 0.05               # tokens must agree wherever the oracle's top-2 logit gap exceeds this
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = dare.Context(0)
+    yield c
+    c.close()
+
+
+def f64(t):
+    return t.to(torch.float64).numpy()
+
+
+def close_bf16(got, ref, steps=1.0, floor=1e-3):
+    """|got - ref| within `steps` bf16 roundings of the reference value (plus a small absolute floor)."""
+    got = got.float().cpu().double().numpy()
+    err = np.abs(got - ref)
+    bound = steps * BF16_STEP * np.abs(ref) + floor
+    assert np.isfinite(got).all()
+    assert (err <= bound).all(), f"max excess {np.max(err - bound)} at {np.unravel_index(np.argmax(err - bound), err.shape)}"
+
+
+@pytest.mark.parametrize("M,K,N", [(300, 200, 520), (512, 1024, 768), (64, 4096, 256), (129, 64, 8)])
+def test_linear_store_and_residual(ctx, M, K, N):
+    a = I.normal_bf16(1, I.TID_X, (M, K))
+    w = I.normal_bf16(1, I.TID_W, (N, K), 0.05)
+    r = I.normal_bf16(1, I.TID_Q, (M, N))
+    ref = f64(a) @ f64(w).T
+    out = dare.dare_linear(ctx, dare.LINEAR_STORE, a.cuda(), w.cuda())
+    torch.cuda.synchronize()
+    close_bf16(out, ref)
+    out = dare.dare_linear(ctx, dare.LINEAR_RESIDUAL, a.cuda(), w.cuda(), residual=r.cuda())
+    torch.cuda.synchronize()
+    close_bf16(out, f64(r) + ref)
+    # in place on the residual stream
+    x = r.cuda().clone()
+    dare.dare_linear(ctx, dare.LINEAR_RESIDUAL, a.cuda(), w.cuda(), residual=x, out=x)
+    torch.cuda.synchronize()
+    assert torch.equal(x, out)
+    assert ctx.device_status() == 0
+
+
+@pytest.mark.parametrize("M,K,F", [(200, 256, 392), (512, 512, 1024), (32, 128, 128)])
+def test_linear_swiglu(ctx, M, K, F):
+    a = I.normal_bf16(2, I.TID_X, (M, K))
+    wg = I.normal_bf16(2, I.TID_W, (F, K), 0.1)
+    wu = I.normal_bf16(2, I.TID_Q, (F, K), 0.1)
+    g, u = f64(a) @ f64(wg).T, f64(a) @ f64(wu).T
+    ref = g / (1.0 + np.exp(-g)) * u
+    out = dare.dare_linear(ctx, dare.LINEAR_SWIGLU, a.cuda(), wg.cuda(), w2=wu.cuda())
+    torch.cuda.synchronize()
+    close_bf16(out, ref, steps=1.0, floor=2e-3)
+    assert ctx.device_status() == 0
+
+
+def test_linear_rejects_bad_arguments(ctx):
+    a = torch.zeros(16, 64, dtype=torch.bfloat16, device="cuda")
+    w = torch.zeros(24, 64, dtype=torch.bfloat16, device="cuda")
+    assert dare.dare_linear(ctx, dare.LINEAR_SWIGLU, a, w, check=False) == -1            # w2 missing
+    assert dare.dare_linear(ctx, dare.LINEAR_RESIDUAL, a, w, check=False) == -1          # residual missing
+    assert dare.dare_linear(ctx, 7, a, w, check=False) == -4
+    w_bad = torch.zeros(20, 64, dtype=torch.bfloat16, device="cuda")                     # N not a multiple of 8
+    assert dare.dare_linear(ctx, dare.LINEAR_STORE, a, w_bad, check=False) == -2
+
+
+@pytest.mark.parametrize("rows,D", [(37, 256), (512, 4096), (3, 8)])
+def test_rmsnorm(ctx, rows, D):
+    x = I.normal_bf16(3, I.TID_X, (rows, D), 3.0)
+    y = dare.dare_rmsnorm(ctx, x.cuda(), 1e-5)
+    torch.cuda.synchronize()
+    close_bf16(y, MO.rmsnorm(f64(x), 1e-5))
+
+
+def _model(ctx, mw, wts_t, max_rows=None):
+    dev = lambda t: t.cuda()
+    layers = [{k: dev(v) for k, v in l.items()} for l in wts_t["layers"]]
+    return dare.Model(ctx, n_layers=mw.n_layers, hidden=mw.hidden, n_q_heads=mw.n_q_heads, n_kv_heads=mw.n_kv_heads,
+                      head_dim=mw.head_dim, ffn=mw.ffn, vocab=mw.vocab, mask_id=mw.mask_id,
+                      embedding=dev(wts_t["embedding"]), layers=layers, lm_head=dev(wts_t["lm_head"]),
+                      max_positions=mw.row_len, max_rows=max_rows or mw.batch * max(mw.prompt_len, mw.block_len),
+                      max_batch=mw.batch, rms_eps=mw.rms_eps, rope_base=mw.rope_base)
+
+
+def _cfg(mw):
+    return MO.ModelConfig(mw.n_layers, mw.hidden, mw.n_q_heads, mw.n_kv_heads, mw.head_dim, mw.ffn, mw.vocab,
+                          mw.mask_id, mw.rms_eps, mw.rope_base)
+
+
+def _oracle_weights(wts_t):
+    layers = [MO.LayerWeights(f64(l["wqkv"]), f64(l["wo"]), f64(l["wg"]), f64(l["wu"]), f64(l["wd"]))
+              for l in wts_t["layers"]]
+    return MO.ModelWeights(f64(wts_t["embedding"]), layers, f64(wts_t["lm_head"]))
+
+
+def test_rope_and_cache_write(ctx):
+    mw = I.MODEL_WORKLOADS["loop_small_gqa"]
+    wts_t = I.make_model_weights(mw)
+    model = _model(ctx, mw, wts_t)
+    B, length, start, cap = 3, 16, 40, mw.row_len
+    Hq, Hkv, d = mw.n_q_heads, mw.n_kv_heads, mw.head_dim
+    qkv = I.normal_bf16(4, I.TID_Q, (B * length, (Hq + 2 * Hkv) * d))
+    q_out = torch.zeros(B * length, Hq, d, dtype=torch.bfloat16, device="cuda")
+    kc = torch.zeros(B, Hkv, cap, d, dtype=torch.bfloat16, device="cuda")
+    vc = torch.zeros_like(kc)
+    dare.dare_rope_kv_write(model, qkv.cuda(), B, length, start, q_out, kc, vc)
+    torch.cuda.synchronize()
+    pos = np.arange(start, start + length)
+    cfg = _cfg(mw)
+    for r in range(B):
+        q, k, v = MO._split_qkv(f64(qkv[r * length:(r + 1) * length]), cfg)
+        close_bf16(q_out[r * length:(r + 1) * length], MO.rope(q, pos, mw.rope_base), floor=2e-3)
+        close_bf16(kc[r, :, start:start + length], np.transpose(MO.rope(k, pos, mw.rope_base), (1, 0, 2)), floor=2e-3)
+        np.testing.assert_array_equal(vc[r, :, start:start + length].float().cpu().numpy(),
+                                      np.transpose(v, (1, 0, 2)).astype(np.float32))
+    # nothing outside the written window was touched
+    assert (kc[:, :, :start] == 0).all() and (kc[:, :, start + length:] == 0).all()
+    model.close()
+
+
+def _check_hidden(got_t, ref, n_layers):
+    got = got_t.float().cpu().double().numpy()
+    assert np.isfinite(got).all()
+    err = np.abs(got - ref).max()
+    rel = np.linalg.norm(got - ref) / np.linalg.norm(ref)
+    assert err <= HIDDEN_MAX_ABS_PER_LAYER * n_layers, f"hidden max-abs {err}"
+    assert rel <= HIDDEN_REL_L2_PER_LAYER * n_layers, f"hidden rel-L2 {rel}"
+    return err, rel
+
+
+def _check_lm(pred_t, conf_t, lm, n_layers):
+    pred, conf = pred_t.cpu().numpy(), conf_t.cpu().numpy().astype(np.float64)
+    live = np.isfinite(lm["conf"])
+    assert (pred[~live] == lm["pred"][~live]).all() and np.isneginf(conf[~live]).all()
+    must = live & (lm["gap_logit"] > LOGIT_GAP)
+    assert (pred[must] == lm["pred"][must]).all()
+    same = live & (pred == lm["pred"])
+    assert np.abs(conf[same] - lm["conf"][same]).max(initial=0) <= 1e-3
+    assert np.abs(np.log(conf[same]) - lm["logconf"][same]).max(initial=0) <= LOGCONF_ABS_BASE + LOGCONF_ABS_PER_LAYER * n_layers
+    assert same.sum() >= 0.8 * live.sum() - 1      # near-ties (logit gap below the bar) may resolve differently
+
+
+@pytest.mark.parametrize("name", ["loop_small", "loop_small_gqa"])
+def test_loop_small_step_by_step_and_generate(ctx, name):
+    mw = I.MODEL_WORKLOADS[name]
+    wts_t = I.make_model_weights(mw)
+    cfg, wts = _cfg(mw), _oracle_weights(wts_t)
+    model = _model(ctx, mw, wts_t)
+    B, L, P, G = mw.batch, mw.block_len, mw.prompt_len, mw.gen_len
+    tok0 = I.fresh_model_tokens(mw)
+    kc, vc = model.new_cache(B, mw.row_len)
+    pred = torch.empty(B * L, dtype=torch.int32, device="cuda")
+    conf = torch.empty(B * L, dtype=torch.float32, device="cuda")
+    nc = torch.zeros(B, dtype=torch.int32, device="cuda")
+    nr = torch.zeros(B, dtype=torch.int32, device="cuda")
+    hid = torch.empty(B * P, mw.hidden, dtype=torch.bfloat16, device="cuda")
+
+    # ---- prefill: hidden states and cache against the oracle
+    tok = tok0.cuda()
+    dare.dare_model_forward(model, tok, 0, P, kc, vc, hidden_out=hid)
+    torch.cuda.synchronize()
+    ocache = MO.new_cache(cfg, B, mw.row_len)
+    ref_h = MO.forward_block_cached(cfg, wts, tok0.numpy(), 0, P, ocache)
+    _check_hidden(hid, ref_h, mw.n_layers)
+    for li in range(mw.n_layers):
+        _check_hidden(kc[li][:, :, :P], ocache[li][0][:, :, :P], li + 1)
+        _check_hidden(vc[li][:, :, :P], ocache[li][1][:, :, :P], li + 1)
+
+    # ---- the loop, step by step, teacher-forced on the GPU's token state
+    steps_manual = []
+    for b in range(G // L):
+        start = P + b * L
+        n = 0
+        while True:
+            pre = tok.cpu().numpy()
+            if not (pre[:, start:start + L] == mw.mask_id).any():
+                break
+            dare.dare_model_step(model, tok, start, L, kc, vc, mw.mode, mw.threshold, mw.k, pred, conf, nc, nr)
+            torch.cuda.synchronize()
+            res = MO.denoise_step_cached(cfg, wts, pre, start, L, ocache, mw.mode, mw.threshold, mw.k)
+            _check_lm(pred, conf, res["lm"], mw.n_layers)
+            want, wnc, wnr = O.unmask_select(pre, start, L, pred.cpu().numpy(), conf.cpu().numpy(), mw.mask_id, mw.mode,
+                                             mw.threshold, mw.k)
+            np.testing.assert_array_equal(tok.cpu().numpy(), want)
+            np.testing.assert_array_equal(nc.cpu().numpy(), wnc)
+            np.testing.assert_array_equal(nr.cpu().numpy(), wnr)
+            n += 1
+            assert n <= L
+        steps_manual.append(n)
+        dare.dare_model_forward(model, tok, start, L, kc, vc)                      # refresh the block's K/V
+        MO.forward_block_cached(cfg, wts, tok.cpu().numpy(), start, L, ocache)
+        torch.cuda.synchronize()
+        for li in range(mw.n_layers):
+            _check_hidden(kc[li][:, :, :start + L], ocache[li][0][:, :, :start + L], li + 1)
+    final_manual = tok.cpu().numpy()
+    assert (final_manual[:, P:] != mw.mask_id).all()
+    np.testing.assert_array_equal(final_manual[:, :P], tok0.numpy()[:, :P])
+    if mw.mode == I.SELECT_TOPK:
+        assert steps_manual == [-(-L // mw.k)] * (G // L)
+    assert ctx.device_status() == 0
+
+    # ---- the one-call loop gives the same tokens, steps and cache as the step-by-step run
+    tok2 = tok0.cuda()
+    kc2, vc2 = model.new_cache(B, mw.row_len)
+    steps = dare.dare_generate(model, tok2, P, G, L, kc2, vc2, mw.mode, mw.threshold, mw.k, pred, conf, nr)
+    np.testing.assert_array_equal(tok2.cpu().numpy(), final_manual)
+    assert steps == steps_manual
+    assert torch.equal(kc2, kc) and torch.equal(vc2, vc)
+    assert ctx.device_status() == 0
+    model.close()
+
+
+class _LazyLayer:
+    """fp64 views of one layer's bf16 weights, converted when touched (the full-size stack would need 7 GB)."""
+
+    def __init__(self, l):
+        self._l = l
+
+    def __getattr__(self, name):
+        return f64(self._l[name])
+
+
+def test_llada_loop_full_size_one_rollout(ctx):
+    """4-layer LLaDA-shaped stack at full size: prefill and the first denoising step of the whole batch on the
+    GPU; one sampled rollout is followed through the oracle (rollouts are independent)."""
+    mw = I.MODEL_WORKLOADS["llada_loop"]
+    wts_t = I.make_model_weights(mw)
+    model = _model(ctx, mw, wts_t)
+    B, L, P = mw.batch, mw.block_len, mw.prompt_len
+    tok0 = I.fresh_model_tokens(mw)
+    tok = tok0.cuda()
+    kc, vc = model.new_cache(B, mw.row_len)
+    pred = torch.empty(B * L, dtype=torch.int32, device="cuda")
+    conf = torch.empty(B * L, dtype=torch.float32, device="cuda")
+    nc = torch.zeros(B, dtype=torch.int32, device="cuda")
+    nr = torch.zeros(B, dtype=torch.int32, device="cuda")
+    hid = torch.empty(B * L, mw.hidden, dtype=torch.bfloat16, device="cuda")
+    dare.dare_model_forward(model, tok, 0, P, kc, vc)
+    dare.dare_model_forward(model, tok, P, L, kc, vc, hidden_out=hid)
+    dare.dare_model_step(model, tok, P, L, kc, vc, mw.mode, mw.threshold, mw.k, pred, conf, nc, nr)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+
+    r = 5
+    cfg = _cfg(mw)
+    wts = MO.ModelWeights(_EmbeddingRows(wts_t["embedding"]), [_LazyLayer(l) for l in wts_t["layers"]], None)
+    ocache = MO.new_cache(cfg, 1, mw.row_len)
+    one = tok0[r:r + 1].numpy()
+    MO.forward_block_cached(cfg, wts, one, 0, P, ocache)
+    ref_h = MO.forward_block_cached(cfg, wts, one, P, L, ocache)
+    print('full-size hidden (max-abs, rel-L2):', _check_hidden(hid[r * L:(r + 1) * L], ref_h, mw.n_layers))
+    for li in range(mw.n_layers):
+        _check_hidden(kc[li][r:r + 1, :, :P + L], ocache[li][0][:, :, :P + L], li + 1)
+    lm = O.lmhead_confidence(ref_h, f64(wts_t["lm_head"]), one[0, P:P + L], mw.mask_id, True)
+    _check_lm(pred[r * L:(r + 1) * L], conf[r * L:(r + 1) * L], lm, mw.n_layers)
+    want, wnc, wnr = O.unmask_select(tok0.numpy(), P, L, pred.cpu().numpy(), conf.cpu().numpy(), mw.mask_id, mw.mode,
+                                     mw.threshold, mw.k)
+    np.testing.assert_array_equal(tok.cpu().numpy(), want)
+    np.testing.assert_array_equal(nc.cpu().numpy(), wnc)
+    assert (wnc >= 1).all()
+    model.close()
+
+
+class _EmbeddingRows:
+    """Row lookup into the bf16 embedding, converted to fp64 per lookup."""
+
+    def __init__(self, e):
+        self._e = e
+
+    def __getitem__(self, idx):
+        return f64(self._e[torch.as_tensor(np.asarray(idx), dtype=torch.long)])
