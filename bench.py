@@ -299,6 +299,191 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def _model_objects(dare, ctx, mw, wts_h):
+    layers = [{k: v.cuda() for k, v in l.items()} for l in wts_h["layers"]]
+    return dare.Model(ctx, n_layers=mw.n_layers, hidden=mw.hidden, n_q_heads=mw.n_q_heads, n_kv_heads=mw.n_kv_heads,
+                      head_dim=mw.head_dim, ffn=mw.ffn, vocab=mw.vocab, mask_id=mw.mask_id,
+                      embedding=wts_h["embedding"].cuda(), layers=layers, lm_head=wts_h["lm_head"].cuda(),
+                      max_positions=mw.row_len, max_rows=mw.batch * max(mw.prompt_len, mw.block_len),
+                      max_batch=mw.batch, rms_eps=mw.rms_eps, rope_base=mw.rope_base)
+
+
+def run_model(args):
+    """The end-to-end loop workload: prefill + block-by-block denoising on the 4-layer stack (dare_generate).
+    --steps counts denoising steps; whole generations are timed (steps / steps-per-generation, at least one)."""
+    from paper_2604_04215_b200 import binding as dare
+    from paper_2604_04215_b200.dist import reduce_step_stats
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback for the product path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    mw = I.MODEL_WORKLOADS[args.workload]
+    wts_h = I.make_model_weights(mw)                                   # same weights on every rank
+    mw_rank = I.ModelWorkload(**{**mw.__dict__, "seed": rank})         # its own prompts
+    ctx = dare.Context(local)
+    model = _model_objects(dare, ctx, mw, wts_h)
+    B, L, P, G = mw.batch, mw.block_len, mw.prompt_len, mw.gen_len
+    tok0_h = I.fresh_model_tokens(mw_rank).pin_memory()
+    tok0 = tok0_h.cuda()
+    tok = tok0.clone()
+    kc, vc = model.new_cache(B, mw.row_len)
+    pred = torch.empty(B * L, dtype=torch.int32, device="cuda")
+    conf = torch.empty(B * L, dtype=torch.float32, device="cuda")
+    nr = torch.zeros(B, dtype=torch.int32, device="cuda")
+    stream = torch.cuda.current_stream()
+    max_steps_per_gen = (G // L) * (L if mw.mode == I.SELECT_THRESHOLD else -(-L // mw.k))
+    n_gen = max(1, int(round(args.steps / max_steps_per_gen)))
+    n_warm = max(1, int(round(args.warmup / max_steps_per_gen))) if args.warmup > 0 else 0
+
+    def generation(src):
+        tok.copy_(src, non_blocking=True)
+        return dare.dare_generate(model, tok, P, G, L, kc, vc, mw.mode, mw.threshold, mw.k, pred, conf, nr,
+                                  stream=stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(n_warm):
+        generation(tok0)
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    w0 = time.time()
+    e0.record(stream)
+    steps_taken, committed = 0, 0
+    for _ in range(n_gen):
+        steps_taken += sum(generation(tok0))
+        committed += B * G
+    e1.record(stream)
+    barrier()
+    w1 = time.time()
+    clocks = sampler.stop(w0, w1) if rank == 0 else None
+    ms = e0.elapsed_time(e1)
+    if not bool((tok[:, P:] != mw.mask_id).all()) or ctx.device_status() != 0:
+        raise RuntimeError("the loop left masks behind or the device status word is non-zero")
+    ms_max, committed_all = reduce_step_stats(ms, committed, device="cuda")
+    value = committed_all / (ms_max * 1e-3)
+
+    # ---- the projections of one layer at the step's row count, timed one by one for the roofline
+    M = B * L
+    D, F = mw.hidden, mw.ffn
+    nq, nkv = mw.n_q_heads * mw.head_dim, mw.n_kv_heads * mw.head_dim
+    lw = model._keep[1][0]
+    a_d = I.normal_bf16(1, I.TID_X, (M, D)).cuda()
+    a_f = I.normal_bf16(1, I.TID_Q, (M, F)).cuda()
+    a_q = I.normal_bf16(1, I.TID_KBLK, (M, nq)).cuda()
+    x_res = I.normal_bf16(1, I.TID_VBLK, (M, D)).cuda()
+    o_qkv = torch.empty(M, nq + 2 * nkv, dtype=torch.bfloat16, device="cuda")
+    o_act = torch.empty(M, F, dtype=torch.bfloat16, device="cuda")
+    cases = [("qkv", lambda: dare.dare_linear(ctx, dare.LINEAR_STORE, a_d, lw["wqkv"], out=o_qkv), 2.0 * M * D * (nq + 2 * nkv)),
+             ("attn_out", lambda: dare.dare_linear(ctx, dare.LINEAR_RESIDUAL, a_q, lw["wo"], residual=x_res, out=x_res), 2.0 * M * nq * D),
+             ("gate_up_swiglu", lambda: dare.dare_linear(ctx, dare.LINEAR_SWIGLU, a_d, lw["wg"], w2=lw["wu"], out=o_act), 4.0 * M * D * F),
+             ("down", lambda: dare.dare_linear(ctx, dare.LINEAR_RESIDUAL, a_f, lw["wd"], residual=x_res, out=x_res), 2.0 * M * F * D)]
+    reps = 20
+    per = {}
+    tot_ms, tot_flop = 0.0, 0.0
+    for name, fn, flop in cases:
+        for _ in range(3):
+            fn()
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+        evs[0].record(stream)
+        for i in range(reps):
+            # repeated on the same weight matrix: the smallest one (attn_out, 34 MB) can stay in L2 between
+            # repeats, which flatters only that projection; the others exceed what L2 keeps
+            fn()
+            evs[i + 1].record(stream)
+        torch.cuda.synchronize()
+        t = float(np.mean([evs[i].elapsed_time(evs[i + 1]) for i in range(reps)]))
+        per[name] = {"ms": t, "tflops": flop / (t * 1e-3) / 1e12}
+        tot_ms += t
+        tot_flop += flop
+    peaks = _peaks()
+    peak = peaks["bf16_tflops_sustained"]
+    achieved = tot_flop / (tot_ms * 1e-3) / 1e12
+    roofline = {"bound": "tensor", "kernel": "gemm_bf16_kernel (the four projections of one layer at M = B*L rows)",
+                "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                "peak_source": peaks["source"] + " sustained", "per_projection": per,
+                "frac_of_nominal_2250": achieved / 2250.0}
+
+    # ---- end to end: prompts come from pinned host memory, the generated tokens go back to the host
+    out_h = torch.empty_like(tok0_h).pin_memory()
+    barrier()
+    ta = time.perf_counter()
+    e2e_tokens = 0
+    for _ in range(n_gen):
+        generation(tok0_h)
+        out_h.copy_(tok, non_blocking=True)
+        torch.cuda.synchronize()
+        e2e_tokens += int((out_h[:, P:] != mw.mask_id).sum())
+    tb = time.perf_counter()
+    e2e_s, e2e_n = reduce_step_stats(tb - ta, e2e_tokens, device="cuda")
+    e2e = {"value": e2e_n / e2e_s, "unit": UNIT, "h2d_bytes_per_step": tok0_h.numel() * 4 / max_steps_per_gen,
+           "d2h_bytes_per_step": out_h.numel() * 4 / max_steps_per_gen, "generations": n_gen}
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu_baseline = time_model_oracle(mw, wts_h, budget_s=20.0)
+    if rank == 0:
+        per_fwd = 2 + 8 * mw.n_layers                   # embedding, final norm, 8 launches per layer
+        launches = n_gen * (per_fwd + (steps_taken // n_gen + G // L) * (per_fwd + 4))
+        out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps_taken, "warmup": args.warmup,
+               "ms_per_step": ms_max / max(steps_taken, 1), "higher_is_better": True, "scaling": "weak",
+               "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+               "config": {"workload": f"{mw.name}: {mw.n_layers} layers D{D} Hq{mw.n_q_heads}/Hkv{mw.n_kv_heads} "
+                                      f"d{mw.head_dim} F{F} V{mw.vocab} B{B} prompt{P}+gen{G} L{L} tau {mw.threshold}",
+                          "generations": n_gen, "ms_per_generation": ms_max / n_gen,
+                          "l2": "inputs larger than L2 (2.8 GB of weights are re-read every step)",
+                          "parallelism": f"dp{world} (independent rollouts per GPU, no collective)"},
+               "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
+               "cpu_baseline": cpu_baseline}
+        print(json.dumps(out))
+    model.close()
+    ctx.close()
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def time_model_oracle(mw, wts_h, budget_s=20.0, max_steps=8):
+    """Times the loop oracle, as it stands, on a bounded sample: denoising steps of ONE rollout right after its
+    prefill (the prefill itself is not timed)."""
+    from oracle import dare_model_oracle as MO
+    f = lambda t: t.to(torch.float64).numpy()
+    cfg = MO.ModelConfig(mw.n_layers, mw.hidden, mw.n_q_heads, mw.n_kv_heads, mw.head_dim, mw.ffn, mw.vocab,
+                         mw.mask_id, mw.rms_eps, mw.rope_base)
+    layers = [MO.LayerWeights(f(l["wqkv"]), f(l["wo"]), f(l["wg"]), f(l["wu"]), f(l["wd"])) for l in wts_h["layers"]]
+    wts = MO.ModelWeights(f(wts_h["embedding"]), layers, f(wts_h["lm_head"]))
+    one = I.ModelWorkload(**{**mw.__dict__, "batch": 1})
+    tok = I.fresh_model_tokens(one).numpy()
+    cache = MO.new_cache(cfg, 1, mw.row_len)
+    MO.forward_block_cached(cfg, wts, tok, 0, mw.prompt_len, cache)
+    committed, steps = 0, 0
+    t0 = time.perf_counter()
+    while steps < max_steps and (time.perf_counter() - t0 < budget_s or steps == 0):
+        res = MO.denoise_step_cached(cfg, wts, tok, mw.prompt_len, mw.block_len, cache, mw.mode, mw.threshold, mw.k)
+        committed += int(res["n_committed"].sum())
+        tok = res["tokens"]
+        steps += 1
+    dt = time.perf_counter() - t0
+    return {"value": committed / dt, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
+            "sample": f"{steps} denoising steps of 1 rollout out of {mw.batch} (all layers, full vocabulary) after its "
+                      f"prefill, {dt:.1f} s; tokens/s of that single rollout, not scaled",
+            "seconds_per_step_one_rollout": dt / steps}
+
+
 def time_oracle(wl, w_h, caches_h, budget_s=20.0, max_steps=64):
     """Times the oracle, as it stands, on a bounded sample: ONE rollout (of the batch) per step."""
     from oracle import dare_oracle as O
@@ -332,6 +517,19 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
+    if args.workload in I.MODEL_WORKLOADS:
+        mw = I.MODEL_WORKLOADS[args.workload]
+        res = time_model_oracle(mw, I.make_model_weights(mw), budget_s=1e9, max_steps=max(1, min(args.steps, 8)))
+        print(json.dumps({"impl": "reference", "metric": METRIC, "value": res["value"], "unit": UNIT, "n_gpus": args.gpus,
+                          "steps": max(1, min(args.steps, 8)), "warmup": 0,
+                          "ms_per_step": res["seconds_per_step_one_rollout"] * 1e3, "higher_is_better": True,
+                          "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+                          "config": {"workload": f"{mw.name} (bounded sample: one rollout, steps after its prefill)"},
+                          "cpu_baseline": {"value": res["value"], "unit": UNIT, "cores": res["cores"], "kind": "oracle",
+                                           "sample": res["sample"]},
+                          "e2e": {"value": res["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                          "gpu_launches": 0}))
+        return
     wl = I.WORKLOADS[args.workload]
     w_h = I.normal_bf16(0, I.TID_W, (wl.vocab, wl.hidden), 0.02)
     caches = I.make_caches(I.scaled(wl, batch=1))
@@ -357,11 +555,13 @@ def main():
     ap.add_argument("--steps", type=int, default=1536)
     ap.add_argument("--warmup", type=int, default=32)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="llada8b", choices=sorted(I.WORKLOADS))
+    ap.add_argument("--workload", default="llada8b", choices=sorted(I.WORKLOADS) + sorted(I.MODEL_WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload in I.MODEL_WORKLOADS:
+        run_model(args)
     else:
         run_ours(args)
 
