@@ -1,16 +1,22 @@
 // Dense bf16 projections of the layer stack on the tcgen05 tensor cores: out = epilogue(A W^T).
 //
-// A [M, K] activations and W [N, K] weights are both K-major bf16, so one pipeline serves every projection:
-//   warp 0      TMA producer: A tile [128 x 64] and W tile [BN x 64] per stage (128-byte swizzle)
-//   warp 1      UMMA issuer: 128 x BN x 16 MMAs into one of two fp32 accumulators in TMEM
-//   warps 2..5  epilogue: one TMEM lane = one output row per thread, 32 columns at a time
-// Two accumulators let the epilogue of one tile overlap the MMAs of the next.  CTAs are persistent and walk
-// the tiles with the row-tile index fastest, so the CTAs that share a weight tile run at the same time and the
-// weights leave HBM once.
+// A [M, K] activations and W [N, K] weights are both K-major bf16.  One CTA computes one output tile of up to
+// two 128-row tiles by `bn` columns over a range of K:
+//   warp 0      TMA producer: one or two A tiles [128 x 64] and a W tile [bn x 64] per stage (128-byte swizzle)
+//   warp 1      UMMA issuer: 128 x bn x 16 MMAs, one fp32 accumulator in TMEM per row tile
+//   warps 2..9  epilogue: one TMEM lane = one output row per thread, 8 columns at a time
+// The tile shape is chosen per problem on the host (gemm_plan): at the few hundred rows of a denoising step a
+// projection has too few 128 x 256 tiles to fill the SMs evenly, so the column width bn (any multiple of 16)
+// and, for long K, a split of K are picked so that the CTAs make whole waves; two row tiles per CTA share
+// each W tile, which keeps the shared-memory and L2 traffic per flop low.  CTAs are numbered with the row index
+// fastest, so the CTAs that share a weight tile run at the same time and the weights leave HBM once.
 // Epilogues: plain bf16 store (QKV projection); residual add, rounded once after the add (attention output
-// and feed-forward down projections, in place on the residual stream); SwiGLU, where a 256-column tile holds
-// 128 gate columns and the matching 128 up columns (two TMA loads, one per matrix) and silu(g) * u is formed
-// in registers, so the 2F-wide intermediate never reaches memory.
+// and feed-forward down projections, in place on the residual stream); SwiGLU, where a tile holds w gate
+// columns and the matching w up columns (two TMA loads, one per matrix) and silu(g) * u is formed in
+// registers, so the 2F-wide intermediate never reaches memory.
+// Split K: every CTA of an output tile writes its fp32 partial to the workspace and counts itself in; the
+// one that arrives last adds the partials in split order (so the result does not depend on who was last),
+// applies the epilogue and resets the counter.
 #include <math.h>
 
 #include "internal.h"
@@ -21,80 +27,109 @@ namespace {
 
 constexpr int GM = 128;
 constexpr int GK = 64;
-constexpr int GEMM_THREADS = 192;
+constexpr int GEMM_THREADS = 320;
 constexpr int A_TILE_BYTES = GM * GK * 2;
+constexpr int MAX_STAGES = 8;
+constexpr int RING_BYTES = 226 * 1024;      // shared memory for the operand ring (the CTA has 227 KB)
+constexpr int EPI_THREADS = 256;
+constexpr uint32_t EPI_BARRIER = 1;
+constexpr int MAX_SPLITS = 3;
 
-template <int BN>
-struct GemmShape {
-    static constexpr int STAGES = BN == 256 ? 4 : 6;
-    static constexpr int B_TILE_BYTES = BN * GK * 2;
-    static constexpr int STAGE_BYTES = A_TILE_BYTES + B_TILE_BYTES;
-    static constexpr uint32_t TMEM_COLS = 2 * BN;
-};
-
-template <int STAGES>
 struct GemmBarriers {
-    uint64_t full[STAGES];
-    uint64_t empty[STAGES];
-    uint64_t tmem_full[2];
-    uint64_t tmem_empty[2];
+    uint64_t full[MAX_STAGES];
+    uint64_t empty[MAX_STAGES];
+    uint64_t tmem_full;
     uint32_t tmem_base;
     uint32_t abort_flag;
+    uint32_t is_last;
+};
+constexpr int GEMM_SMEM_BYTES = RING_BYTES - 1024;   // dynamic request; the ring starts at the next 1 KB boundary
+
+struct GemmPlan {
+    int nsub;        // row tiles per CTA (1 or 2)
+    int bn;          // MMA N: columns of W per tile (SwiGLU: w gate rows + w up rows)
+    int wcols;       // output columns per tile (bn, or bn / 2 for SwiGLU)
+    int splits;      // CTAs along K per output tile
+    int stages;
+    int m_items, n_tiles;
+    uint32_t tmem_cols;
 };
 
-template <int BN>
-constexpr int gemm_smem_bytes() {
-    return GemmShape<BN>::STAGES * GemmShape<BN>::STAGE_BYTES +
-           static_cast<int>(sizeof(GemmBarriers<GemmShape<BN>::STAGES>)) + 1024;
-}
+struct GemmArgs {
+    int M, N, K, ldo;
+    GemmPlan p;
+    __nv_bfloat16* out;
+    const __nv_bfloat16* res;
+    float* partial;            // [tile][split][bn / 8][nsub * 128][8] fp32, used when splits > 1
+    int32_t* counters;         // one per output tile, zero between launches
+    uint32_t* dev_status;
+};
 
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
-// N = rows of W covered by the output (EPI_SWIGLU: rows of each of the two matrices); n_cols_per_tile is BN,
-// or 128 for EPI_SWIGLU.  `res` may alias `out` (every element is read and written by the same thread).
-template <int BN, int EPI>
+// Applies the epilogue to 8 accumulated columns of one row and stores them.  `res` may alias `out`.
+template <int EPI>
+__device__ __forceinline__ void store_group(const float (&f)[8], const float (&u)[8], __nv_bfloat16* out,
+                                            const __nv_bfloat16* res, size_t off) {
+    float r[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) r[j] = f[j];
+    if (EPI == GEMM_EPI_RESIDUAL) {
+        const uint4 x = *reinterpret_cast<const uint4*>(res + off);
+        r[0] += bf16_lo(x.x); r[1] += bf16_hi(x.x); r[2] += bf16_lo(x.y); r[3] += bf16_hi(x.y);
+        r[4] += bf16_lo(x.z); r[5] += bf16_hi(x.z); r[6] += bf16_lo(x.w); r[7] += bf16_hi(x.w);
+    } else if (EPI == GEMM_EPI_SWIGLU) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) r[j] = __fdividef(f[j], 1.0f + __expf(-f[j])) * u[j];   // silu(g) * u
+    }
+    uint4 o;
+    o.x = pack_bf16(r[0], r[1]); o.y = pack_bf16(r[2], r[3]);
+    o.z = pack_bf16(r[4], r[5]); o.w = pack_bf16(r[6], r[7]);
+    *reinterpret_cast<uint4*>(out + off) = o;
+}
+
+template <int EPI>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                 const __grid_constant__ CUtensorMap tmap_b2, int M, int N, int K, __nv_bfloat16* out,
-                 const __nv_bfloat16* res, int ldo, uint32_t* __restrict__ dev_status) {
-    using S = GemmShape<BN>;
-    constexpr int STAGES = S::STAGES;
-    constexpr int OUT_COLS = EPI == GEMM_EPI_SWIGLU ? BN / 2 : BN;   // output columns per tile
-    static_assert(EPI != GEMM_EPI_SWIGLU || BN == 256, "the SwiGLU tile pairs 128 gate with 128 up columns");
+                 const __grid_constant__ CUtensorMap tmap_b2, const GemmArgs g) {
+    const GemmPlan& p = g.p;
+    const int stage_bytes = p.nsub * A_TILE_BYTES + p.bn * (GK * 2);
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    GemmBarriers<STAGES>* bars = reinterpret_cast<GemmBarriers<STAGES>*>(tiles + STAGES * S::STAGE_BYTES);
+    GemmBarriers* bars = reinterpret_cast<GemmBarriers*>(tiles + p.stages * stage_bytes);
     volatile uint32_t* abort_flag = &bars->abort_flag;
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int m_tiles = (M + GM - 1) / GM;
-    const int n_tiles = (N + OUT_COLS - 1) / OUT_COLS;
-    const int n_work = m_tiles * n_tiles;
-    const int num_k = (K + GK - 1) / GK;
+    // CTA -> (row item, K split, column tile), row item fastest
+    const int m_item = blockIdx.x % p.m_items;
+    const int split = (blockIdx.x / p.m_items) % p.splits;
+    const int n_tile = blockIdx.x / (p.m_items * p.splits);
+    const int nk = (g.K + GK - 1) / GK;
+    const int kb_begin = static_cast<int>(static_cast<long long>(nk) * split / p.splits);
+    const int kb_end = static_cast<int>(static_cast<long long>(nk) * (split + 1) / p.splits);
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) {
+        for (int s = 0; s < p.stages; ++s) {
             mbar_init(&bars->full[s], 1);
             mbar_init(&bars->empty[s], 1);
         }
-        for (int a = 0; a < 2; ++a) {
-            mbar_init(&bars->tmem_full[a], 1);
-            mbar_init(&bars->tmem_empty[a], 128);
-        }
+        mbar_init(&bars->tmem_full, 1);
         bars->abort_flag = 0;
+        bars->is_last = 0;
         fence_barrier_init();
     }
     if (warp == 1) {
-        tmem_alloc(&bars->tmem_base, S::TMEM_COLS);
+        tmem_alloc(&bars->tmem_base, p.tmem_cols);
         tmem_relinquish();
     }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = bars->tmem_base;
+    const int acc_stride = p.nsub == 2 ? 256 : 0;   // accumulator of row tile s starts at column s * 256
 
     if (warp == 0) {
         if (lane == 0) {
@@ -103,108 +138,170 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             if (EPI == GEMM_EPI_SWIGLU) prefetch_tensormap(&tmap_b2);
             int stage = 0;
             uint32_t phase = 0;
-            bool ok = true;
-            for (int t = blockIdx.x; t < n_work && ok; t += gridDim.x) {
-                const int m_tile = t % m_tiles, n_tile = t / m_tiles;
-                for (int kb = 0; kb < num_k; ++kb) {
-                    if (!mbar_wait(&bars->empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
-                    uint8_t* a_dst = tiles + stage * S::STAGE_BYTES;
-                    uint8_t* b_dst = a_dst + A_TILE_BYTES;
-                    mbar_arrive_expect_tx(&bars->full[stage], S::STAGE_BYTES);
-                    tma_load_2d(a_dst, &tmap_a, &bars->full[stage], kb * GK, m_tile * GM);
-                    if (EPI == GEMM_EPI_SWIGLU) {
-                        tma_load_2d(b_dst, &tmap_b, &bars->full[stage], kb * GK, n_tile * 128);
-                        tma_load_2d(b_dst + 128 * GK * 2, &tmap_b2, &bars->full[stage], kb * GK, n_tile * 128);
-                    } else {
-                        tma_load_2d(b_dst, &tmap_b, &bars->full[stage], kb * GK, n_tile * BN);
-                    }
-                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+            for (int kb = kb_begin; kb < kb_end; ++kb) {
+                if (!mbar_wait(&bars->empty[stage], phase ^ 1, abort_flag)) break;
+                uint8_t* a_dst = tiles + stage * stage_bytes;
+                uint8_t* b_dst = a_dst + p.nsub * A_TILE_BYTES;
+                mbar_arrive_expect_tx(&bars->full[stage], stage_bytes);
+                for (int s = 0; s < p.nsub; ++s)
+                    tma_load_2d(a_dst + s * A_TILE_BYTES, &tmap_a, &bars->full[stage], kb * GK, (m_item * p.nsub + s) * GM);
+                if (EPI == GEMM_EPI_SWIGLU) {
+                    tma_load_2d(b_dst, &tmap_b, &bars->full[stage], kb * GK, n_tile * p.wcols);
+                    tma_load_2d(b_dst + p.wcols * (GK * 2), &tmap_b2, &bars->full[stage], kb * GK, n_tile * p.wcols);
+                } else {
+                    tma_load_2d(b_dst, &tmap_b, &bars->full[stage], kb * GK, n_tile * p.bn);
                 }
+                if (++stage == p.stages) { stage = 0; phase ^= 1; }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc = umma_idesc_bf16(GM, BN);
+            const uint32_t idesc = umma_idesc_bf16(GM, p.bn);
             int stage = 0;
             uint32_t phase = 0;
-            int it = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < n_work && ok; t += gridDim.x, ++it) {
-                const int acc = it & 1;
-                const uint32_t acc_phase = (it >> 1) & 1;
-                if (!mbar_wait(&bars->tmem_empty[acc], acc_phase ^ 1, abort_flag)) { ok = false; break; }
+            for (int kb = kb_begin; kb < kb_end; ++kb) {
+                if (!mbar_wait(&bars->full[stage], phase, abort_flag)) { ok = false; break; }
                 tc_fence_after_sync();
-                const uint32_t d_tmem = tmem_base + acc * BN;
-                for (int kb = 0; kb < num_k; ++kb) {
-                    if (!mbar_wait(&bars->full[stage], phase, abort_flag)) { ok = false; break; }
-                    tc_fence_after_sync();
-                    const uint32_t a_addr = smem_u32(tiles + stage * S::STAGE_BYTES);
-                    const uint64_t a_desc = umma_desc_sw128_kmajor(a_addr);
-                    const uint64_t b_desc = umma_desc_sw128_kmajor(a_addr + A_TILE_BYTES);
+                const uint32_t a_addr = smem_u32(tiles + stage * stage_bytes);
+                const uint64_t b_desc = umma_desc_sw128_kmajor(a_addr + p.nsub * A_TILE_BYTES);
+                for (int s = 0; s < p.nsub; ++s) {
+                    const uint64_t a_desc = umma_desc_sw128_kmajor(a_addr + s * A_TILE_BYTES);
 #pragma unroll
                     for (int kk = 0; kk < GK / 16; ++kk)   // +32 bytes along K per step = +2 descriptor units
-                        umma_bf16(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0);
-                    umma_commit(&bars->empty[stage]);
-                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                        umma_bf16(tmem_base + s * acc_stride, a_desc + 2 * kk, b_desc + 2 * kk, idesc,
+                                  (kb > kb_begin) || kk != 0);
                 }
-                if (ok) umma_commit(&bars->tmem_full[acc]);
+                umma_commit(&bars->empty[stage]);
+                if (++stage == p.stages) { stage = 0; phase ^= 1; }
             }
+            if (ok) umma_commit(&bars->tmem_full);
         }
     } else {
-        const int lq = warp & 3;   // warp w may touch TMEM lanes [32 * (w % 4), +32)
-        int it = 0;
-        bool ok = true;
-        for (int t = blockIdx.x; t < n_work && ok; t += gridDim.x, ++it) {
-            const int m_tile = t % m_tiles, n_tile = t / m_tiles;
-            const int acc = it & 1;
-            const uint32_t acc_phase = (it >> 1) & 1;
-            if (!mbar_wait(&bars->tmem_full[acc], acc_phase, abort_flag)) { ok = false; break; }
-            tc_fence_after_sync();
-            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(lq * 32) << 16) + acc * BN;
-            const int row = m_tile * GM + lq * 32 + lane;
-            const size_t row_off = static_cast<size_t>(row) * ldo;
-#pragma unroll 1
-            for (int c = 0; c < OUT_COLS / 32; ++c) {
-                uint32_t v[32];
-                const int col0 = n_tile * OUT_COLS + c * 32;
-                if (EPI == GEMM_EPI_SWIGLU) {
-                    uint32_t u[32];
-                    tmem_ld_32cols(taddr + c * 32, v);
-                    tmem_ld_32cols(taddr + 128 + c * 32, u);
+        // epilogue: warp w may touch TMEM lanes [32 * (w % 4), +32); warps 2..5 are set 0, warps 6..9 set 1.
+        // Two row tiles: set s owns row tile s.  One row tile: the sets share it, alternating 8-column groups.
+        const int lq = warp & 3;
+        const int set = (warp - 2) >> 2;
+        const int rt = p.nsub == 2 ? set : 0;
+        const int g_first = p.nsub == 2 ? 0 : set, g_step = p.nsub == 2 ? 1 : 2;
+        const int n_groups = p.wcols / 8;
+        const int row_local = rt * GM + lq * 32 + lane;
+        const int row = m_item * p.nsub * GM + row_local;
+        const bool row_ok = row < g.M;
+        const size_t row_off = static_cast<size_t>(row) * g.ldo;
+        const int col_base = n_tile * p.wcols;
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(lq * 32) << 16) + rt * acc_stride;
+        const int tile_id = m_item + p.m_items * n_tile;
+        const int tile_rows = p.nsub * GM;
+        bool ok = mbar_wait(&bars->tmem_full, 0, abort_flag);
+        tc_fence_after_sync();
+        bool finish = ok;
+        if (p.splits > 1) {
+            // (EPI_SWIGLU never splits K: the partial below holds plain accumulator columns)
+            if (ok) {
+                // layout [tile][split][column group][row][8]: a warp's 32 rows of one group are 1 KB in a row
+                float* mine = g.partial + (static_cast<size_t>(tile_id) * p.splits + split) * tile_rows * p.bn + row_local * 8;
+                for (int gi = g_first; gi < n_groups; gi += g_step) {
+                    uint32_t v[8];
+                    tmem_ld_8cols(taddr + gi * 8, v);
                     tmem_ld_wait();
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const float g = __uint_as_float(v[j]);
-                        const float s = __fdividef(g, 1.0f + __expf(-g));      // silu(g)
-                        v[j] = __float_as_uint(s * __uint_as_float(u[j]));
+                    if (row_ok && col_base + gi * 8 < g.N) {
+                        float* dst = mine + static_cast<size_t>(gi) * tile_rows * 8;
+                        *reinterpret_cast<uint4*>(dst) = make_uint4(v[0], v[1], v[2], v[3]);
+                        *reinterpret_cast<uint4*>(dst + 4) = make_uint4(v[4], v[5], v[6], v[7]);
                     }
-                } else {
-                    tmem_ld_32cols(taddr + c * 32, v);
-                    tmem_ld_wait();
                 }
-                if (row < M) {
+                __threadfence();
+            }
+            named_barrier_sync(EPI_BARRIER, EPI_THREADS);
+            if (warp == 2 && lane == 0) {
+                uint32_t last = 0;
+                if (!*abort_flag) {
+                    const int old = atomicAdd(g.counters + tile_id, 1);
+                    if (old == p.splits - 1) {
+                        last = 1;
+                        atomicExch(g.counters + tile_id, 0);   // ready for the next launch
+                    }
+                    __threadfence();
+                }
+                bars->is_last = last;
+            }
+            named_barrier_sync(EPI_BARRIER, EPI_THREADS);
+            finish = ok && *reinterpret_cast<volatile uint32_t*>(&bars->is_last) != 0;
+        }
+        if (finish && p.splits > 1) {
+            // last CTA of the tile: add the partials in split order (this CTA's own values take their place in
+            // it, so the sum does not depend on who came last).  The other CTAs' partials are fetched four column
+            // groups at a time so that the loads overlap.
+            constexpr int BATCH = 4;
+            const float* base = g.partial + static_cast<size_t>(tile_id) * p.splits * tile_rows * p.bn + row_local * 8;
+            for (int gb = g_first; gb < n_groups; gb += BATCH * g_step) {
+                float4 oth[BATCH][MAX_SPLITS][2];
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const int col = col0 + q * 8;
-                        if (col < N) {    // N is a multiple of 8: a group of 8 columns is inside or outside
-                            float f[8];
+                for (int b = 0; b < BATCH; ++b) {
+                    const int gi = gb + b * g_step;
+                    const bool live = gi < n_groups && row_ok && col_base + gi * 8 < g.N;
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) f[j] = __uint_as_float(v[q * 8 + j]);
-                            if (EPI == GEMM_EPI_RESIDUAL) {
-                                const uint4 r = *reinterpret_cast<const uint4*>(res + row_off + col);
-                                f[0] += bf16_lo(r.x); f[1] += bf16_hi(r.x); f[2] += bf16_lo(r.y); f[3] += bf16_hi(r.y);
-                                f[4] += bf16_lo(r.z); f[5] += bf16_hi(r.z); f[6] += bf16_lo(r.w); f[7] += bf16_hi(r.w);
-                            }
-                            uint4 o;
-                            o.x = pack_bf16(f[0], f[1]); o.y = pack_bf16(f[2], f[3]);
-                            o.z = pack_bf16(f[4], f[5]); o.w = pack_bf16(f[6], f[7]);
-                            *reinterpret_cast<uint4*>(out + row_off + col) = o;
+                    for (int s = 0; s < MAX_SPLITS; ++s) {           // slot s = split s (this CTA's own slot stays empty)
+                        if (live && s < p.splits && s != split) {
+                            const float* q = base + static_cast<size_t>(s) * tile_rows * p.bn +
+                                             static_cast<size_t>(gi) * tile_rows * 8;
+                            oth[b][s][0] = ld_global_cg_f4(q);
+                            oth[b][s][1] = ld_global_cg_f4(q + 4);
+                        } else {
+                            oth[b][s][0] = oth[b][s][1] = make_float4(0.f, 0.f, 0.f, 0.f);
                         }
                     }
                 }
+#pragma unroll
+                for (int b = 0; b < BATCH; ++b) {
+                    const int gi = gb + b * g_step;
+                    if (gi >= n_groups) break;
+                    uint32_t v[8];
+                    tmem_ld_8cols(taddr + gi * 8, v);
+                    tmem_ld_wait();
+                    const int col = col_base + gi * 8;
+                    if (row_ok && col < g.N) {
+                        float acc[8], u[8];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) { acc[j] = 0.f; u[j] = 0.f; }
+#pragma unroll
+                        for (int s = 0; s < MAX_SPLITS; ++s) {
+                            if (s == split) {
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) acc[j] += __uint_as_float(v[j]);
+                            } else if (s < p.splits) {
+                                const float4 a = oth[b][s][0], c = oth[b][s][1];
+                                acc[0] += a.x; acc[1] += a.y; acc[2] += a.z; acc[3] += a.w;
+                                acc[4] += c.x; acc[5] += c.y; acc[6] += c.z; acc[7] += c.w;
+                            }
+                        }
+                        store_group<EPI>(acc, u, g.out, g.res, row_off + col);
+                    }
+                }
             }
-            tc_fence_before_sync();
-            mbar_arrive(&bars->tmem_empty[acc]);
+        } else if (finish) {
+            for (int gi = g_first; gi < n_groups; gi += g_step) {
+                uint32_t v[8];
+                float f[8], u[8];
+                tmem_ld_8cols(taddr + gi * 8, v);
+                if (EPI == GEMM_EPI_SWIGLU) {
+                    uint32_t w[8];
+                    tmem_ld_8cols(taddr + p.wcols + gi * 8, w);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) u[j] = __uint_as_float(w[j]);
+                } else {
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) u[j] = 0.f;
+                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j) f[j] = __uint_as_float(v[j]);
+                const int col = col_base + gi * 8;
+                if (row_ok && col < g.N)      // N is a multiple of 8: a group of 8 columns is inside or outside
+                    store_group<EPI>(f, u, g.out, g.res, row_off + col);
+            }
         }
     }
 
@@ -214,25 +311,71 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     if (*abort_flag) {
         const long long t0 = clock64();
         while (clock64() - t0 < 2000000LL) {}   // let copies in flight land before the shared memory goes away
-        if (threadIdx.x == 0) atomicOr(dev_status, DEV_WAIT_EXPIRED);
+        if (threadIdx.x == 0) atomicOr(g.dev_status, DEV_WAIT_EXPIRED);
         __syncthreads();
     }
     if (warp == 1) {
         tc_fence_after_sync();
-        tmem_dealloc(tmem_base, S::TMEM_COLS);
+        tmem_dealloc(tmem_base, p.tmem_cols);
     }
 }
 
-template <int BN, int EPI>
-int launch_one(const dare_ctx* ctx, const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tb2, int M, int N,
-               int K, void* out, const void* res, int ldo, int tiles, cudaStream_t stream) {
-    constexpr int SMEM = gemm_smem_bytes<BN>();
-    if (cudaFuncSetAttribute(gemm_bf16_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
+// Picks the tile shape by a small cost model: a CTA's time is the longer of its MMA issue time (bn / 2 cycles
+// per 128 x bn x 16 MMA) and its operand traffic at ~90 bytes per cycle, plus prologue and epilogue; the launch
+// takes ceil(CTAs / SMs) rounds of it.
+GemmPlan gemm_plan(int epi, int M, int N, int K, int sm_count, size_t workspace_bytes) {
+    const int nk = (K + GK - 1) / GK;
+    const int m_tiles = (M + GM - 1) / GM;
+    const int ring = GEMM_SMEM_BYTES - 1024 - 256;
+    GemmPlan best{};
+    double best_cost = 1e300;
+    for (int nsub = 1; nsub <= (m_tiles >= 2 ? 2 : 1); ++nsub) {
+        const int m_items = (m_tiles + nsub - 1) / nsub;
+        for (int bn = 256; bn >= 32; bn -= 16) {
+            const int wcols = epi == GEMM_EPI_SWIGLU ? bn / 2 : bn;
+            if (wcols > ((N + 7) / 8) * 8 + 15 && bn > 32) continue;          // wider than the whole output
+            const int n_tiles = (N + wcols - 1) / wcols;
+            const int stage_bytes = nsub * A_TILE_BYTES + bn * GK * 2;
+            int stages = ring / stage_bytes;
+            if (stages > MAX_STAGES) stages = MAX_STAGES;
+            if (stages < 2) continue;
+            for (int splits = 1; splits <= MAX_SPLITS; ++splits) {
+                if (splits > 1) {
+                    if (epi == GEMM_EPI_SWIGLU || nk < 8 * splits) break;
+                    const long long tiles = static_cast<long long>(m_items) * n_tiles;
+                    if (tiles > DARE_TILE_COUNTERS) break;
+                    if (static_cast<size_t>(tiles) * splits * nsub * GM * bn * sizeof(float) > workspace_bytes) break;
+                }
+                const long long ctas = static_cast<long long>(m_items) * n_tiles * splits;
+                const long long rounds = (ctas + sm_count - 1) / sm_count;
+                const double kb = static_cast<double>((nk + splits - 1) / splits);
+                const double mma = kb * nsub * 4 * (bn / 2.0);
+                const double ld = kb * stage_bytes / 90.0;
+                const double epilogue = wcols * 14.0 * (splits > 1 ? 1.0 + splits : 1.0);
+                const double cost = rounds * ((mma > ld ? mma : ld) + 2500.0 + epilogue);
+                if (cost < best_cost) {
+                    best_cost = cost;
+                    best.nsub = nsub; best.bn = bn; best.wcols = wcols; best.splits = splits; best.stages = stages;
+                    best.m_items = m_items; best.n_tiles = n_tiles;
+                    uint32_t cols = 32;
+                    while (cols < static_cast<uint32_t>(nsub == 2 ? 256 + bn : bn)) cols <<= 1;
+                    best.tmem_cols = cols;
+                }
+            }
+        }
+    }
+    return best;
+}
+
+template <int EPI>
+int launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tb2, const GemmArgs& g,
+               cudaStream_t stream) {
+    if (cudaFuncSetAttribute(gemm_bf16_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_BYTES) !=
+        cudaSuccess)
         return DARE_ERR_CUDA;
-    const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
-    gemm_bf16_kernel<BN, EPI><<<grid, GEMM_THREADS, SMEM, stream>>>(ta, tb, tb2, M, N, K, static_cast<__nv_bfloat16*>(out),
-                                                                    static_cast<const __nv_bfloat16*>(res), ldo,
-                                                                    ctx->dev_status);
+    const long long ctas = static_cast<long long>(g.p.m_items) * g.p.n_tiles * g.p.splits;
+    if (ctas > 0x7fffffffLL) return DARE_ERR_SHAPE;
+    gemm_bf16_kernel<EPI><<<static_cast<unsigned>(ctas), GEMM_THREADS, GEMM_SMEM_BYTES, stream>>>(ta, tb, tb2, g);
     return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
 }
 
@@ -241,30 +384,29 @@ int launch_one(const dare_ctx* ctx, const CUtensorMap& ta, const CUtensorMap& tb
 int launch_gemm(const dare_ctx* ctx, int epi, const void* a, int M, int K, const void* w, const void* w2, int N,
                 void* out, const void* res, int ldo, cudaStream_t stream) {
     if (M < 1 || N < 8 || K < 8 || (N % 8) || (K % 8) || (ldo % 8)) return DARE_ERR_SHAPE;
-    const int m_tiles = (M + GM - 1) / GM;
+    if (epi < GEMM_EPI_STORE || epi > GEMM_EPI_SWIGLU) return DARE_ERR_RANGE;
+    GemmArgs g;
+    g.M = M; g.N = N; g.K = K; g.ldo = ldo;
+    g.p = gemm_plan(epi, M, N, K, ctx->sm_count, ctx->tile_counters ? ctx->workspace_bytes : 0);
+    if (g.p.bn == 0) return DARE_ERR_SHAPE;
+    g.out = static_cast<__nv_bfloat16*>(out);
+    g.res = static_cast<const __nv_bfloat16*>(res);
+    g.partial = static_cast<float*>(ctx->workspace);
+    g.counters = ctx->tile_counters;
+    g.dev_status = ctx->dev_status;
     CUtensorMap ta, tb, tb2;
     int rc = make_tmap_bf16_2d(ctx, &ta, a, static_cast<uint64_t>(M), static_cast<uint64_t>(K), GM, GK);
     if (rc != DARE_OK) return rc;
-    if (epi == GEMM_EPI_SWIGLU) {
-        rc = make_tmap_bf16_2d(ctx, &tb, w, static_cast<uint64_t>(N), static_cast<uint64_t>(K), 128, GK);
-        if (rc == DARE_OK) rc = make_tmap_bf16_2d(ctx, &tb2, w2, static_cast<uint64_t>(N), static_cast<uint64_t>(K), 128, GK);
-        if (rc != DARE_OK) return rc;
-        return launch_one<256, GEMM_EPI_SWIGLU>(ctx, ta, tb, tb2, M, N, K, out, res, ldo, m_tiles * ((N + 127) / 128), stream);
-    }
-    // tile width by the number of waves it takes: a 256-wide tile costs two 128-wide ones
-    const long long t256 = static_cast<long long>(m_tiles) * ((N + 255) / 256);
-    const long long t128 = static_cast<long long>(m_tiles) * ((N + 127) / 128);
-    const long long sms = ctx->sm_count;
-    const bool wide = 2 * ((t256 + sms - 1) / sms) <= (t128 + sms - 1) / sms;
-    rc = make_tmap_bf16_2d(ctx, &tb, w, static_cast<uint64_t>(N), static_cast<uint64_t>(K), wide ? 256 : 128, GK);
+    const uint32_t box_rows = static_cast<uint32_t>(epi == GEMM_EPI_SWIGLU ? g.p.wcols : g.p.bn);
+    rc = make_tmap_bf16_2d(ctx, &tb, w, static_cast<uint64_t>(N), static_cast<uint64_t>(K), box_rows, GK);
     if (rc != DARE_OK) return rc;
-    if (epi == GEMM_EPI_STORE)
-        return wide ? launch_one<256, GEMM_EPI_STORE>(ctx, ta, tb, tb, M, N, K, out, res, ldo, static_cast<int>(t256), stream)
-                    : launch_one<128, GEMM_EPI_STORE>(ctx, ta, tb, tb, M, N, K, out, res, ldo, static_cast<int>(t128), stream);
-    if (epi == GEMM_EPI_RESIDUAL)
-        return wide ? launch_one<256, GEMM_EPI_RESIDUAL>(ctx, ta, tb, tb, M, N, K, out, res, ldo, static_cast<int>(t256), stream)
-                    : launch_one<128, GEMM_EPI_RESIDUAL>(ctx, ta, tb, tb, M, N, K, out, res, ldo, static_cast<int>(t128), stream);
-    return DARE_ERR_RANGE;
+    if (epi == GEMM_EPI_SWIGLU) {
+        rc = make_tmap_bf16_2d(ctx, &tb2, w2, static_cast<uint64_t>(N), static_cast<uint64_t>(K), box_rows, GK);
+        if (rc != DARE_OK) return rc;
+        return launch_one<GEMM_EPI_SWIGLU>(ta, tb, tb2, g, stream);
+    }
+    return epi == GEMM_EPI_STORE ? launch_one<GEMM_EPI_STORE>(ta, tb, tb, g, stream)
+                                 : launch_one<GEMM_EPI_RESIDUAL>(ta, tb, tb, g, stream);
 }
 
 }  // namespace dare

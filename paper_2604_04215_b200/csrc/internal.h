@@ -8,6 +8,8 @@
 
 #include "../../include/dare.h"
 
+#define DARE_TILE_COUNTERS 4096
+
 typedef CUresult (*dare_encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                          const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
                                          CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
@@ -19,6 +21,7 @@ struct dare_ctx {
     void* workspace;
     size_t workspace_bytes;
     uint32_t* dev_status;   // device word, bits DARE_DEV_*
+    int32_t* tile_counters; // DARE_TILE_COUNTERS zero-initialised words; split-K tiles count arrivals and reset them
     dare_encode_tiled_fn encode_tiled;
 };
 

@@ -48,7 +48,11 @@ def close_bf16(got, ref, steps=1.0, floor=1e-3):
     assert (err <= bound).all(), f"max excess {np.max(err - bound)} at {np.unravel_index(np.argmax(err - bound), err.shape)}"
 
 
-@pytest.mark.parametrize("M,K,N", [(300, 200, 520), (512, 1024, 768), (64, 4096, 256), (129, 64, 8)])
+@pytest.mark.parametrize("M,K,N", [(300, 200, 520), (512, 1024, 768), (64, 4096, 256), (129, 64, 8),
+                                   (512, 4096, 12288),     # two row tiles per CTA, 176-column tiles
+                                   (500, 12288, 4096),     # K split three ways, ragged last row tile
+                                   (512, 4096, 4096),      # K split two ways
+                                   (1100, 512, 1000)])     # many row items, odd number of row tiles
 def test_linear_store_and_residual(ctx, M, K, N):
     a = I.normal_bf16(1, I.TID_X, (M, K))
     w = I.normal_bf16(1, I.TID_W, (N, K), 0.05)
@@ -68,7 +72,7 @@ def test_linear_store_and_residual(ctx, M, K, N):
     assert ctx.device_status() == 0
 
 
-@pytest.mark.parametrize("M,K,F", [(200, 256, 392), (512, 512, 1024), (32, 128, 128)])
+@pytest.mark.parametrize("M,K,F", [(200, 256, 392), (512, 512, 1024), (32, 128, 128), (512, 4096, 12288)])
 def test_linear_swiglu(ctx, M, K, F):
     a = I.normal_bf16(2, I.TID_X, (M, K))
     wg = I.normal_bf16(2, I.TID_W, (F, K), 0.1)
