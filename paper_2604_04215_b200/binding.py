@@ -23,7 +23,7 @@ DEV_WAIT_EXPIRED = 2
 EXPORTS = ["dare_create", "dare_destroy", "dare_status_string", "dare_device_status", "dare_sm_count",
            "dare_attn_block", "dare_lmhead_confidence", "dare_unmask_select", "dare_denoise_block",
            "dare_lmhead_confidence_static", "dare_model_create", "dare_model_destroy", "dare_model_forward",
-           "dare_model_step", "dare_generate", "dare_linear", "dare_rmsnorm", "dare_rope_kv_write"]
+           "dare_model_step", "dare_generate", "dare_linear", "dare_linear_plan", "dare_rmsnorm", "dare_rope_kv_write"]
 
 _lib = None
 
@@ -82,6 +82,8 @@ def load():
     lib.dare_generate.restype = i32
     lib.dare_linear.argtypes = [vp, i32, vp, i32, i32, vp, vp, i32, vp, vp, vp]
     lib.dare_linear.restype = i32
+    lib.dare_linear_plan.argtypes = [vp, i32, i32, i32, i32, C.POINTER(C.c_int)]
+    lib.dare_linear_plan.restype = i32
     lib.dare_rmsnorm.argtypes = [vp, vp, i32, i32, f32, vp, vp]
     lib.dare_rmsnorm.restype = i32
     lib.dare_rope_kv_write.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, i32, vp]
@@ -262,6 +264,16 @@ def dare_linear(ctx: Context, epilogue: int, a, w, w2=None, residual=None, out=N
     if rc != 0 and check:
         raise DareError(rc, "dare_linear")
     return out if check else rc
+
+
+def dare_linear_plan(ctx: Context, epilogue: int, M: int, K: int, N: int):
+    """The launch shape dare_linear would use: dict of the eight plan numbers."""
+    out = (C.c_int * 8)()
+    rc = load().dare_linear_plan(ctx.handle, int(epilogue), int(M), int(K), int(N), out)
+    if rc != 0:
+        raise DareError(rc, "dare_linear_plan")
+    keys = ("row_tiles", "w_rows", "out_cols", "k_splits", "stages", "row_items", "col_tiles", "resident_clusters")
+    return dict(zip(keys, list(out)))
 
 
 def dare_rmsnorm(ctx: Context, x, eps: float, y=None, stream=None, check: bool = True):

@@ -92,7 +92,6 @@ int dare_create(dare_ctx** out, int device, size_t workspace_bytes) {
     ctx->workspace_bytes = workspace_bytes ? workspace_bytes : (size_t(256) << 20);
     ctx->workspace = nullptr;
     ctx->dev_status = nullptr;
-    ctx->tile_counters = nullptr;
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
@@ -103,12 +102,9 @@ int dare_create(dare_ctx** out, int device, size_t workspace_bytes) {
     ctx->encode_tiled = reinterpret_cast<dare_encode_tiled_fn>(fn);
     if (cudaMalloc(&ctx->workspace, ctx->workspace_bytes) != cudaSuccess ||
         cudaMalloc(reinterpret_cast<void**>(&ctx->dev_status), sizeof(uint32_t)) != cudaSuccess ||
-        cudaMemset(ctx->dev_status, 0, sizeof(uint32_t)) != cudaSuccess ||
-        cudaMalloc(reinterpret_cast<void**>(&ctx->tile_counters), sizeof(int32_t) * DARE_TILE_COUNTERS) != cudaSuccess ||
-        cudaMemset(ctx->tile_counters, 0, sizeof(int32_t) * DARE_TILE_COUNTERS) != cudaSuccess) {
+        cudaMemset(ctx->dev_status, 0, sizeof(uint32_t)) != cudaSuccess) {
         if (ctx->workspace) cudaFree(ctx->workspace);
         if (ctx->dev_status) cudaFree(ctx->dev_status);
-        if (ctx->tile_counters) cudaFree(ctx->tile_counters);
         delete ctx;
         return DARE_ERR_CUDA;
     }
@@ -121,7 +117,6 @@ int dare_destroy(dare_ctx* ctx) {
     cudaSetDevice(ctx->device);
     cudaFree(ctx->workspace);
     cudaFree(ctx->dev_status);
-    cudaFree(ctx->tile_counters);
     delete ctx;
     return DARE_OK;
 }
@@ -146,8 +141,6 @@ int dare_device_status(dare_ctx* ctx, void* stream, uint32_t* host_out) {
     if (cudaMemcpyAsync(host_out, ctx->dev_status, sizeof(uint32_t), cudaMemcpyDeviceToHost, s) != cudaSuccess)
         return DARE_ERR_CUDA;
     if (cudaMemsetAsync(ctx->dev_status, 0, sizeof(uint32_t), s) != cudaSuccess) return DARE_ERR_CUDA;
-    // a kernel that gave up on a wait may have left split-K arrival counts behind
-    if (cudaMemsetAsync(ctx->tile_counters, 0, sizeof(int32_t) * DARE_TILE_COUNTERS, s) != cudaSuccess) return DARE_ERR_CUDA;
     if (cudaStreamSynchronize(s) != cudaSuccess) return DARE_ERR_CUDA;
     return DARE_OK;
 }

@@ -14,9 +14,10 @@
 // and feed-forward down projections, in place on the residual stream); SwiGLU, where a tile holds w gate
 // columns and the matching w up columns (two TMA loads, one per matrix) and silu(g) * u is formed in
 // registers, so the 2F-wide intermediate never reaches memory.
-// Split K: every CTA of an output tile writes its fp32 partial to the workspace and counts itself in; the
-// one that arrives last adds the partials in split order (so the result does not depend on who was last),
-// applies the epilogue and resets the counter.
+// Split K: the CTAs that share an output tile form a thread-block cluster.  After the main loop each CTA
+// sends, through distributed shared memory, the accumulator column groups it does not own into the idle
+// operand ring of the CTA that owns them; every CTA then adds the partials of its own groups in split order
+// and applies the epilogue, so all CTAs of the cluster share the output work and nothing goes through HBM.
 #include <math.h>
 
 #include "internal.h"
@@ -31,9 +32,8 @@ constexpr int GEMM_THREADS = 320;
 constexpr int A_TILE_BYTES = GM * GK * 2;
 constexpr int MAX_STAGES = 8;
 constexpr int RING_BYTES = 226 * 1024;      // shared memory for the operand ring (the CTA has 227 KB)
-constexpr int EPI_THREADS = 256;
-constexpr uint32_t EPI_BARRIER = 1;
-constexpr int MAX_SPLITS = 3;
+constexpr int MAX_SPLITS = 2;                // CTAs along K per output tile (pairs are always co-resident)
+constexpr int L2_AHEAD = 8;                 // pipeline steps between the L2 prefetch of a W tile and its load
 
 struct GemmBarriers {
     uint64_t full[MAX_STAGES];
@@ -41,7 +41,6 @@ struct GemmBarriers {
     uint64_t tmem_full;
     uint32_t tmem_base;
     uint32_t abort_flag;
-    uint32_t is_last;
 };
 constexpr int GEMM_SMEM_BYTES = RING_BYTES - 1024;   // dynamic request; the ring starts at the next 1 KB boundary
 
@@ -60,8 +59,6 @@ struct GemmArgs {
     GemmPlan p;
     __nv_bfloat16* out;
     const __nv_bfloat16* res;
-    float* partial;            // [tile][split][bn / 8][nsub * 128][8] fp32, used when splits > 1
-    int32_t* counters;         // one per output tile, zero between launches
     uint32_t* dev_status;
 };
 
@@ -103,9 +100,9 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    // CTA -> (row item, K split, column tile), row item fastest
-    const int m_item = blockIdx.x % p.m_items;
-    const int split = (blockIdx.x / p.m_items) % p.splits;
+    // CTA -> (K split, row item, column tile): the splits of one output tile form a cluster, row items next
+    const int split = p.splits > 1 ? static_cast<int>(cluster_cta_rank()) : 0;
+    const int m_item = (blockIdx.x / p.splits) % p.m_items;
     const int n_tile = blockIdx.x / (p.m_items * p.splits);
     const int nk = (g.K + GK - 1) / GK;
     const int kb_begin = static_cast<int>(static_cast<long long>(nk) * split / p.splits);
@@ -118,7 +115,6 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         }
         mbar_init(&bars->tmem_full, 1);
         bars->abort_flag = 0;
-        bars->is_last = 0;
         fence_barrier_init();
     }
     if (warp == 1) {
@@ -138,7 +134,16 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             if (EPI == GEMM_EPI_SWIGLU) prefetch_tensormap(&tmap_b2);
             int stage = 0;
             uint32_t phase = 0;
+            // the weights come from HBM: ask L2 for them L2_AHEAD steps before the load that needs them
+            for (int kb = kb_begin; kb < kb_end && kb < kb_begin + L2_AHEAD; ++kb) {
+                tma_prefetch_l2_2d(&tmap_b, kb * GK, n_tile * (EPI == GEMM_EPI_SWIGLU ? p.wcols : p.bn));
+                if (EPI == GEMM_EPI_SWIGLU) tma_prefetch_l2_2d(&tmap_b2, kb * GK, n_tile * p.wcols);
+            }
             for (int kb = kb_begin; kb < kb_end; ++kb) {
+                if (kb + L2_AHEAD < kb_end) {
+                    tma_prefetch_l2_2d(&tmap_b, (kb + L2_AHEAD) * GK, n_tile * (EPI == GEMM_EPI_SWIGLU ? p.wcols : p.bn));
+                    if (EPI == GEMM_EPI_SWIGLU) tma_prefetch_l2_2d(&tmap_b2, (kb + L2_AHEAD) * GK, n_tile * p.wcols);
+                }
                 if (!mbar_wait(&bars->empty[stage], phase ^ 1, abort_flag)) break;
                 uint8_t* a_dst = tiles + stage * stage_bytes;
                 uint8_t* b_dst = a_dst + p.nsub * A_TILE_BYTES;
@@ -177,131 +182,94 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             }
             if (ok) umma_commit(&bars->tmem_full);
         }
-    } else {
-        // epilogue: warp w may touch TMEM lanes [32 * (w % 4), +32); warps 2..5 are set 0, warps 6..9 set 1.
-        // Two row tiles: set s owns row tile s.  One row tile: the sets share it, alternating 8-column groups.
-        const int lq = warp & 3;
-        const int set = (warp - 2) >> 2;
-        const int rt = p.nsub == 2 ? set : 0;
-        const int g_first = p.nsub == 2 ? 0 : set, g_step = p.nsub == 2 ? 1 : 2;
-        const int n_groups = p.wcols / 8;
-        const int row_local = rt * GM + lq * 32 + lane;
-        const int row = m_item * p.nsub * GM + row_local;
-        const bool row_ok = row < g.M;
-        const size_t row_off = static_cast<size_t>(row) * g.ldo;
-        const int col_base = n_tile * p.wcols;
-        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(lq * 32) << 16) + rt * acc_stride;
-        const int tile_id = m_item + p.m_items * n_tile;
-        const int tile_rows = p.nsub * GM;
-        bool ok = mbar_wait(&bars->tmem_full, 0, abort_flag);
+    }
+
+    // ---- epilogue (warps 2..9).  Warp w may touch TMEM lanes [32 * (w % 4), +32); warps 2..5 are set 0, warps
+    // 6..9 set 1.  Two row tiles: set s owns row tile s.  One row tile: the sets share it, alternating 8-column
+    // groups.  With a K split the CTAs of the cluster first hand each other the column groups they do not own.
+    const bool epi_warp = warp >= 2;
+    const int lq = warp & 3;
+    const int set = epi_warp ? (warp - 2) >> 2 : 0;
+    const int rt = p.nsub == 2 ? set : 0;
+    const int g_first = p.nsub == 2 ? 0 : set, g_step = p.nsub == 2 ? 1 : 2;
+    const int n_groups = p.wcols / 8;
+    const int tile_rows = p.nsub * GM;
+    const int row_local = rt * GM + lq * 32 + lane;
+    const int row = m_item * tile_rows + row_local;
+    const bool row_ok = row < g.M;
+    const size_t row_off = static_cast<size_t>(row) * g.ldo;
+    const int col_base = n_tile * p.wcols;
+    const uint32_t taddr = tmem_base + (static_cast<uint32_t>(lq * 32) << 16) + rt * acc_stride;
+    if (epi_warp) {
+        mbar_wait(&bars->tmem_full, 0, abort_flag);     // (a wait that gave up leaves the abort flag set)
         tc_fence_after_sync();
-        bool finish = ok;
-        if (p.splits > 1) {
-            // (EPI_SWIGLU never splits K: the partial below holds plain accumulator columns)
-            if (ok) {
-                // layout [tile][split][column group][row][8]: a warp's 32 rows of one group are 1 KB in a row
-                float* mine = g.partial + (static_cast<size_t>(tile_id) * p.splits + split) * tile_rows * p.bn + row_local * 8;
-                for (int gi = g_first; gi < n_groups; gi += g_step) {
-                    uint32_t v[8];
-                    tmem_ld_8cols(taddr + gi * 8, v);
-                    tmem_ld_wait();
-                    if (row_ok && col_base + gi * 8 < g.N) {
-                        float* dst = mine + static_cast<size_t>(gi) * tile_rows * 8;
-                        *reinterpret_cast<uint4*>(dst) = make_uint4(v[0], v[1], v[2], v[3]);
-                        *reinterpret_cast<uint4*>(dst + 4) = make_uint4(v[4], v[5], v[6], v[7]);
-                    }
-                }
-                __threadfence();
-            }
-            named_barrier_sync(EPI_BARRIER, EPI_THREADS);
-            if (warp == 2 && lane == 0) {
-                uint32_t last = 0;
-                if (!*abort_flag) {
-                    const int old = atomicAdd(g.counters + tile_id, 1);
-                    if (old == p.splits - 1) {
-                        last = 1;
-                        atomicExch(g.counters + tile_id, 0);   // ready for the next launch
-                    }
-                    __threadfence();
-                }
-                bars->is_last = last;
-            }
-            named_barrier_sync(EPI_BARRIER, EPI_THREADS);
-            finish = ok && *reinterpret_cast<volatile uint32_t*>(&bars->is_last) != 0;
-        }
-        if (finish && p.splits > 1) {
-            // last CTA of the tile: add the partials in split order (this CTA's own values take their place in
-            // it, so the sum does not depend on who came last).  The other CTAs' partials are fetched four column
-            // groups at a time so that the loads overlap.
-            constexpr int BATCH = 4;
-            const float* base = g.partial + static_cast<size_t>(tile_id) * p.splits * tile_rows * p.bn + row_local * 8;
-            for (int gb = g_first; gb < n_groups; gb += BATCH * g_step) {
-                float4 oth[BATCH][MAX_SPLITS][2];
-#pragma unroll
-                for (int b = 0; b < BATCH; ++b) {
-                    const int gi = gb + b * g_step;
-                    const bool live = gi < n_groups && row_ok && col_base + gi * 8 < g.N;
-#pragma unroll
-                    for (int s = 0; s < MAX_SPLITS; ++s) {           // slot s = split s (this CTA's own slot stays empty)
-                        if (live && s < p.splits && s != split) {
-                            const float* q = base + static_cast<size_t>(s) * tile_rows * p.bn +
-                                             static_cast<size_t>(gi) * tile_rows * 8;
-                            oth[b][s][0] = ld_global_cg_f4(q);
-                            oth[b][s][1] = ld_global_cg_f4(q + 4);
-                        } else {
-                            oth[b][s][0] = oth[b][s][1] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        }
-                    }
-                }
-#pragma unroll
-                for (int b = 0; b < BATCH; ++b) {
-                    const int gi = gb + b * g_step;
-                    if (gi >= n_groups) break;
-                    uint32_t v[8];
-                    tmem_ld_8cols(taddr + gi * 8, v);
-                    tmem_ld_wait();
-                    const int col = col_base + gi * 8;
-                    if (row_ok && col < g.N) {
-                        float acc[8], u[8];
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) { acc[j] = 0.f; u[j] = 0.f; }
-#pragma unroll
-                        for (int s = 0; s < MAX_SPLITS; ++s) {
-                            if (s == split) {
-#pragma unroll
-                                for (int j = 0; j < 8; ++j) acc[j] += __uint_as_float(v[j]);
-                            } else if (s < p.splits) {
-                                const float4 a = oth[b][s][0], c = oth[b][s][1];
-                                acc[0] += a.x; acc[1] += a.y; acc[2] += a.z; acc[3] += a.w;
-                                acc[4] += c.x; acc[5] += c.y; acc[6] += c.z; acc[7] += c.w;
-                            }
-                        }
-                        store_group<EPI>(acc, u, g.out, g.res, row_off + col);
-                    }
-                }
-            }
-        } else if (finish) {
+    }
+    __syncwarp();
+    if (p.splits > 1) {
+        // Group gi belongs to the CTA of rank gi % splits.  Receiver layout in the (now idle) operand ring:
+        // [slot of the sending split, ascending, own split left out][gi / splits][row][8 floats].
+        const int per_owner = (n_groups + p.splits - 1) / p.splits;
+        cluster_sync_all();                              // every CTA of the cluster is done with its ring
+        if (epi_warp) {
+            const uint32_t ring = smem_u32(tiles);
             for (int gi = g_first; gi < n_groups; gi += g_step) {
+                const int owner = gi % p.splits;
+                if (owner == split) continue;
                 uint32_t v[8];
-                float f[8], u[8];
                 tmem_ld_8cols(taddr + gi * 8, v);
-                if (EPI == GEMM_EPI_SWIGLU) {
-                    uint32_t w[8];
-                    tmem_ld_8cols(taddr + p.wcols + gi * 8, w);
-                    tmem_ld_wait();
+                tmem_ld_wait();
+                const int slot = split < owner ? split : split - 1;
+                const uint32_t local = ring + ((static_cast<uint32_t>(slot * per_owner + gi / p.splits) * tile_rows + row_local) << 5);
+                const uint32_t remote = cluster_map_shared(local, static_cast<uint32_t>(owner));
+                st_shared_cluster_v4(remote, v[0], v[1], v[2], v[3]);
+                st_shared_cluster_v4(remote + 16, v[4], v[5], v[6], v[7]);
+            }
+        }
+        cluster_sync_all();                              // the partials of the groups this CTA owns have arrived
+    }
+    if (epi_warp && !*abort_flag) {
+        for (int gi = g_first; gi < n_groups; gi += g_step) {
+            if (p.splits > 1 && gi % p.splits != split) continue;
+            uint32_t v[8];
+            float f[8], u[8];
+            tmem_ld_8cols(taddr + gi * 8, v);
+            if (EPI == GEMM_EPI_SWIGLU) {
+                uint32_t w[8];
+                tmem_ld_8cols(taddr + p.wcols + gi * 8, w);
+                tmem_ld_wait();
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) u[j] = __uint_as_float(w[j]);
-                } else {
-                    tmem_ld_wait();
+                for (int j = 0; j < 8; ++j) u[j] = __uint_as_float(w[j]);
+            } else {
+                tmem_ld_wait();
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) u[j] = 0.f;
+                for (int j = 0; j < 8; ++j) u[j] = 0.f;
+            }
+            if (p.splits > 1) {
+                // add the partials in split order; this CTA's own values take their place in it
+                const int per_owner = (n_groups + p.splits - 1) / p.splits;
+                const float* base = reinterpret_cast<const float*>(tiles) +
+                                    (static_cast<size_t>(gi / p.splits) * tile_rows + row_local) * 8;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) f[j] = 0.f;
+                for (int s = 0; s < p.splits; ++s) {
+                    if (s == split) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) f[j] += __uint_as_float(v[j]);
+                    } else {
+                        const int slot = s < split ? s : s - 1;
+                        const float4* q = reinterpret_cast<const float4*>(base + static_cast<size_t>(slot) * per_owner * tile_rows * 8);
+                        const float4 a = q[0], c = q[1];
+                        f[0] += a.x; f[1] += a.y; f[2] += a.z; f[3] += a.w;
+                        f[4] += c.x; f[5] += c.y; f[6] += c.z; f[7] += c.w;
+                    }
                 }
+            } else {
 #pragma unroll
                 for (int j = 0; j < 8; ++j) f[j] = __uint_as_float(v[j]);
-                const int col = col_base + gi * 8;
-                if (row_ok && col < g.N)      // N is a multiple of 8: a group of 8 columns is inside or outside
-                    store_group<EPI>(f, u, g.out, g.res, row_off + col);
             }
+            const int col = col_base + gi * 8;
+            if (row_ok && col < g.N)          // N is a multiple of 8: a group of 8 columns is inside or outside
+                store_group<EPI>(f, u, g.out, g.res, row_off + col);
         }
     }
 
@@ -320,10 +288,53 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     }
 }
 
+template <int EPI>
+int launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tb2, const GemmArgs& g,
+               cudaStream_t stream, int* max_clusters_query) {
+    if (cudaFuncSetAttribute(gemm_bf16_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_BYTES) !=
+        cudaSuccess)
+        return DARE_ERR_CUDA;
+    const long long ctas = static_cast<long long>(g.p.m_items) * g.p.n_tiles * g.p.splits;
+    if (ctas > 0x7fffffffLL) return DARE_ERR_SHAPE;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(ctas), 1, 1);
+    cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = GEMM_SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = static_cast<unsigned>(g.p.splits);
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    if (max_clusters_query) {     // how many clusters of this size the device runs at once (plan input)
+        cfg.gridDim = dim3(static_cast<unsigned>(g.p.splits) * 1024u, 1, 1);
+        return cudaOccupancyMaxActiveClusters(max_clusters_query, gemm_bf16_kernel<EPI>, &cfg) == cudaSuccess
+                   ? DARE_OK : DARE_ERR_CUDA;
+    }
+    return cudaLaunchKernelEx(&cfg, gemm_bf16_kernel<EPI>, ta, tb, tb2, g) == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
+}
+
+// Clusters of `splits` CTAs of this kernel that can be resident at once (cached; 0 = such clusters cannot run).
+int max_active_clusters(int splits) {
+    static int cache[MAX_SPLITS + 1] = {-1, -1, -1};
+    if (cache[splits] < 0) {
+        GemmArgs g{};
+        g.p.m_items = g.p.n_tiles = 1;
+        g.p.splits = splits;
+        CUtensorMap dummy{};
+        int n = 0;
+        if (launch_one<GEMM_EPI_STORE>(dummy, dummy, dummy, g, nullptr, &n) != DARE_OK) n = 0;
+        cache[splits] = n;
+    }
+    return cache[splits];
+}
+
 // Picks the tile shape by a small cost model: a CTA's time is the longer of its MMA issue time (bn / 2 cycles
-// per 128 x bn x 16 MMA) and its operand traffic at ~90 bytes per cycle, plus prologue and epilogue; the launch
-// takes ceil(CTAs / SMs) rounds of it.
-GemmPlan gemm_plan(int epi, int M, int N, int K, int sm_count, size_t workspace_bytes) {
+// per 128 x bn x 16 MMA) and its operand traffic at ~55 bytes per cycle (what L2 delivers per SM when every SM streams), plus prologue and epilogue; the launch
+// takes as many rounds of it as the CTAs (or clusters, with a K split) need on the device.
+GemmPlan gemm_plan(int epi, int M, int N, int K, int sm_count) {
     const int nk = (K + GK - 1) / GK;
     const int m_tiles = (M + GM - 1) / GM;
     const int ring = GEMM_SMEM_BYTES - 1024 - 256;
@@ -340,18 +351,23 @@ GemmPlan gemm_plan(int epi, int M, int N, int K, int sm_count, size_t workspace_
             if (stages > MAX_STAGES) stages = MAX_STAGES;
             if (stages < 2) continue;
             for (int splits = 1; splits <= MAX_SPLITS; ++splits) {
+                const long long tiles = static_cast<long long>(m_items) * n_tiles;
+                long long rounds;
                 if (splits > 1) {
                     if (epi == GEMM_EPI_SWIGLU || nk < 8 * splits) break;
-                    const long long tiles = static_cast<long long>(m_items) * n_tiles;
-                    if (tiles > DARE_TILE_COUNTERS) break;
-                    if (static_cast<size_t>(tiles) * splits * nsub * GM * bn * sizeof(float) > workspace_bytes) break;
+                    const int per_owner = (wcols / 8 + splits - 1) / splits;
+                    if (static_cast<long long>(splits - 1) * per_owner * nsub * GM * 32 > static_cast<long long>(stages) * stage_bytes)
+                        continue;                                              // partials must fit the idle ring
+                    const int resident = max_active_clusters(splits);
+                    if (resident < 1) continue;
+                    rounds = (tiles + resident - 1) / resident;
+                } else {
+                    rounds = (tiles + sm_count - 1) / sm_count;
                 }
-                const long long ctas = static_cast<long long>(m_items) * n_tiles * splits;
-                const long long rounds = (ctas + sm_count - 1) / sm_count;
                 const double kb = static_cast<double>((nk + splits - 1) / splits);
                 const double mma = kb * nsub * 4 * (bn / 2.0);
-                const double ld = kb * stage_bytes / 90.0;
-                const double epilogue = wcols * 14.0 * (splits > 1 ? 1.0 + splits : 1.0);
+                const double ld = kb * stage_bytes / 55.0;
+                const double epilogue = wcols * 14.0 + (splits > 1 ? 9000.0 : 0.0);   // two cluster barriers and the exchange
                 const double cost = rounds * ((mma > ld ? mma : ld) + 2500.0 + epilogue);
                 if (cost < best_cost) {
                     best_cost = cost;
@@ -367,19 +383,14 @@ GemmPlan gemm_plan(int epi, int M, int N, int K, int sm_count, size_t workspace_
     return best;
 }
 
-template <int EPI>
-int launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tb2, const GemmArgs& g,
-               cudaStream_t stream) {
-    if (cudaFuncSetAttribute(gemm_bf16_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_BYTES) !=
-        cudaSuccess)
-        return DARE_ERR_CUDA;
-    const long long ctas = static_cast<long long>(g.p.m_items) * g.p.n_tiles * g.p.splits;
-    if (ctas > 0x7fffffffLL) return DARE_ERR_SHAPE;
-    gemm_bf16_kernel<EPI><<<static_cast<unsigned>(ctas), GEMM_THREADS, GEMM_SMEM_BYTES, stream>>>(ta, tb, tb2, g);
-    return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
-}
-
 }  // namespace
+
+int gemm_plan_describe(const dare_ctx* ctx, int epi, int M, int N, int K, int* out) {
+    const GemmPlan p = gemm_plan(epi, M, N, K, ctx->sm_count);
+    out[0] = p.nsub; out[1] = p.bn; out[2] = p.wcols; out[3] = p.splits; out[4] = p.stages;
+    out[5] = p.m_items; out[6] = p.n_tiles; out[7] = p.splits > 1 ? max_active_clusters(p.splits) : 0;
+    return p.bn ? DARE_OK : DARE_ERR_SHAPE;
+}
 
 int launch_gemm(const dare_ctx* ctx, int epi, const void* a, int M, int K, const void* w, const void* w2, int N,
                 void* out, const void* res, int ldo, cudaStream_t stream) {
@@ -387,12 +398,10 @@ int launch_gemm(const dare_ctx* ctx, int epi, const void* a, int M, int K, const
     if (epi < GEMM_EPI_STORE || epi > GEMM_EPI_SWIGLU) return DARE_ERR_RANGE;
     GemmArgs g;
     g.M = M; g.N = N; g.K = K; g.ldo = ldo;
-    g.p = gemm_plan(epi, M, N, K, ctx->sm_count, ctx->tile_counters ? ctx->workspace_bytes : 0);
+    g.p = gemm_plan(epi, M, N, K, ctx->sm_count);
     if (g.p.bn == 0) return DARE_ERR_SHAPE;
     g.out = static_cast<__nv_bfloat16*>(out);
     g.res = static_cast<const __nv_bfloat16*>(res);
-    g.partial = static_cast<float*>(ctx->workspace);
-    g.counters = ctx->tile_counters;
     g.dev_status = ctx->dev_status;
     CUtensorMap ta, tb, tb2;
     int rc = make_tmap_bf16_2d(ctx, &ta, a, static_cast<uint64_t>(M), static_cast<uint64_t>(K), GM, GK);
@@ -403,10 +412,10 @@ int launch_gemm(const dare_ctx* ctx, int epi, const void* a, int M, int K, const
     if (epi == GEMM_EPI_SWIGLU) {
         rc = make_tmap_bf16_2d(ctx, &tb2, w2, static_cast<uint64_t>(N), static_cast<uint64_t>(K), box_rows, GK);
         if (rc != DARE_OK) return rc;
-        return launch_one<GEMM_EPI_SWIGLU>(ta, tb, tb2, g, stream);
+        return launch_one<GEMM_EPI_SWIGLU>(ta, tb, tb2, g, stream, nullptr);
     }
-    return epi == GEMM_EPI_STORE ? launch_one<GEMM_EPI_STORE>(ta, tb, tb, g, stream)
-                                 : launch_one<GEMM_EPI_RESIDUAL>(ta, tb, tb, g, stream);
+    return epi == GEMM_EPI_STORE ? launch_one<GEMM_EPI_STORE>(ta, tb, tb, g, stream, nullptr)
+                                 : launch_one<GEMM_EPI_RESIDUAL>(ta, tb, tb, g, stream, nullptr);
 }
 
 }  // namespace dare

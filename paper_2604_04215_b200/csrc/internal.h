@@ -8,8 +8,6 @@
 
 #include "../../include/dare.h"
 
-#define DARE_TILE_COUNTERS 4096
-
 typedef CUresult (*dare_encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                          const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
                                          CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
@@ -21,7 +19,6 @@ struct dare_ctx {
     void* workspace;
     size_t workspace_bytes;
     uint32_t* dev_status;   // device word, bits DARE_DEV_*
-    int32_t* tile_counters; // DARE_TILE_COUNTERS zero-initialised words; split-K tiles count arrivals and reset them
     dare_encode_tiled_fn encode_tiled;
 };
 
@@ -64,6 +61,8 @@ enum { GEMM_EPI_STORE = 0, GEMM_EPI_RESIDUAL = 1, GEMM_EPI_SWIGLU = 2 };
 //   STORE: out = acc.  RESIDUAL: out = res + acc (res may be out).  SWIGLU: out = silu(a w^T) * (a w2^T).
 int launch_gemm(const dare_ctx* ctx, int epi, const void* a, int M, int K, const void* w, const void* w2, int N,
                 void* out, const void* res, int ldo, cudaStream_t stream);
+// out[8] = {row tiles per CTA, bn, output columns per tile, K splits, stages, row items, column tiles, resident clusters}
+int gemm_plan_describe(const dare_ctx* ctx, int epi, int M, int N, int K, int* out);
 int launch_embed(const void* emb, int D, int V, const int32_t* tokens, int64_t row_stride, int start, int length,
                  int n_rows, void* x, cudaStream_t stream);
 int launch_rmsnorm(const void* x, int D, int n_rows, float eps, void* y, cudaStream_t stream);

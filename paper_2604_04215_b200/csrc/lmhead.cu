@@ -471,7 +471,6 @@ extern "C" int dare_lmhead_confidence_static(const void* hidden, int M, int D, c
     view.workspace = st->scratch;
     view.workspace_bytes = DARE_LMHEAD_STATIC_SCRATCH_BYTES;
     view.dev_status = st->status;
-    view.tile_counters = nullptr;
     view.encode_tiled = st->encode;
     return dare::launch_lmhead(&view, st->scratch, hidden, M, D, w, V, row_tokens, M, 0, mask_id, exclude_mask_column,
                                pred, conf, static_cast<cudaStream_t>(stream));

@@ -179,6 +179,13 @@ int dare_linear(dare_ctx* ctx, int epilogue, const void* a, int M, int K, const 
     return dare::launch_gemm(ctx, epilogue, a, M, K, w, w2, N, out, residual, N, static_cast<cudaStream_t>(stream));
 }
 
+int dare_linear_plan(dare_ctx* ctx, int epilogue, int M, int K, int N, int* plan_out) {
+    if (!ctx || !plan_out) return DARE_ERR_NULL;
+    if (M < 1 || N < 8 || K < 8 || (N % 8) || (K % 8)) return DARE_ERR_SHAPE;
+    if (epilogue < DARE_LINEAR_STORE || epilogue > DARE_LINEAR_SWIGLU) return DARE_ERR_RANGE;
+    return dare::gemm_plan_describe(ctx, epilogue, M, N, K, plan_out);
+}
+
 int dare_rmsnorm(dare_ctx* ctx, const void* x, int n_rows, int D, float eps, void* y, void* stream) {
     if (!ctx || !x || !y) return DARE_ERR_NULL;
     if (n_rows < 1 || D < 8 || D % 8) return DARE_ERR_SHAPE;
