@@ -24,6 +24,8 @@ struct dare_model {
     int32_t* host_counts;          // pinned: n_remaining of two steps in flight, [2][max_batch]
     int max_batch;
     cudaEvent_t ev[2];
+    cudaStream_t work;             // the loop runs here: a block's step is captured once into a CUDA graph
+    cudaEvent_t ev_in, ev_out;     // order the work stream after / before the caller's stream
 };
 
 namespace {
@@ -129,6 +131,7 @@ int dare_model_create(dare_ctx* ctx, const dare_model_desc* desc, const void* em
     m->layers = new (std::nothrow) dare_layer_weights[c.n_layers];
     m->rope_cs = nullptr; m->x = m->h = m->qkv = m->q = m->attn = m->act = nullptr; m->host_counts = nullptr;
     m->ev[0] = m->ev[1] = nullptr;
+    m->work = nullptr; m->ev_in = m->ev_out = nullptr;
     bool ok = m->layers != nullptr;
     if (ok) for (int l = 0; l < c.n_layers; ++l) m->layers[l] = layers[l];
     const size_t rows = static_cast<size_t>(c.max_rows);
@@ -143,6 +146,9 @@ int dare_model_create(dare_ctx* ctx, const dare_model_desc* desc, const void* em
     ok = ok && cudaMallocHost(reinterpret_cast<void**>(&m->host_counts), sizeof(int32_t) * 2 * c.max_batch) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&m->ev[0], cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&m->ev[1], cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&m->ev_in, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&m->ev_out, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&m->work, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && dare::launch_rope_table(m->rope_cs, c.max_positions, c.head_dim / 2, static_cast<double>(c.rope_base),
                                        nullptr) == DARE_OK;
     ok = ok && cudaDeviceSynchronize() == cudaSuccess;
@@ -162,6 +168,9 @@ int dare_model_destroy(dare_model* m) {
     if (m->host_counts) cudaFreeHost(m->host_counts);
     if (m->ev[0]) cudaEventDestroy(m->ev[0]);
     if (m->ev[1]) cudaEventDestroy(m->ev[1]);
+    if (m->ev_in) cudaEventDestroy(m->ev_in);
+    if (m->ev_out) cudaEventDestroy(m->ev_out);
+    if (m->work) cudaStreamDestroy(m->work);
     delete[] m->layers;
     delete m;
     return DARE_OK;
@@ -235,38 +244,72 @@ int dare_generate(dare_model* m, int32_t* tokens, int B, int64_t row_stride, int
     if (rc == DARE_OK) rc = check_rows(m, tokens, B, row_stride, prompt_len + gen_len - L, L, k_cache, v_cache, cache_cap);
     if (rc == DARE_OK) rc = check_step(m, B, L, mode, threshold, k, pred, conf);
     if (rc != DARE_OK) return rc;
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // The loop runs on the model's own stream, ordered after the caller's stream at entry and before it at
+    // exit: a block's denoising step (about forty launches with fixed arguments) is captured once into a CUDA
+    // graph and replayed, which the caller's stream (possibly the legacy default stream) may not allow.
+    cudaStream_t user = static_cast<cudaStream_t>(stream);
+    cudaStream_t s = m->work;
+    if (cudaEventRecord(m->ev_in, user) != cudaSuccess || cudaStreamWaitEvent(s, m->ev_in, 0) != cudaSuccess)
+        return DARE_ERR_CUDA;
     rc = forward_rows(m, tokens, B, row_stride, 0, prompt_len, k_cache, v_cache, cache_cap, nullptr, s);
     if (rc != DARE_OK) return rc;
     // A step whose block holds no mask any more does exactly what the refresh forward must do (the LM head
     // finds no live row, the selection changes nothing, the stack rewrites the block's K/V from the committed
     // tokens).  So step t + 1 is enqueued before step t's counts are read: when step t turns out to have
     // finished the block, step t + 1 was the refresh, and the GPU never waits for the host.
-    for (int b = 0; b < gen_len / L; ++b) {
+    cudaGraph_t old_graph = nullptr;         // the previous block's graph: destroyed once its launches are known done
+    cudaGraphExec_t old_exec = nullptr;
+    for (int b = 0; b < gen_len / L && rc == DARE_OK; ++b) {
         const int start = prompt_len + b * L;
+        cudaGraph_t graph = nullptr;
+        cudaGraphExec_t exec = nullptr;
+        if (cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal) != cudaSuccess) return DARE_ERR_CUDA;
+        rc = step_rows(m, tokens, B, row_stride, start, L, k_cache, v_cache, cache_cap, mode, threshold, k, pred, conf,
+                       nullptr, n_remaining, s);
+        const cudaError_t end = cudaStreamEndCapture(s, &graph);      // always ends the capture, also after an error
+        if (rc == DARE_OK && (end != cudaSuccess || graph == nullptr)) rc = DARE_ERR_CUDA;
+        if (rc == DARE_OK && cudaGraphInstantiate(&exec, graph, 0) != cudaSuccess) rc = DARE_ERR_CUDA;
         int issued = 0, taken = -1;
-        while (taken < 0) {
-            if (issued > L + 1) return DARE_ERR_CUDA;   // cannot happen: every step commits at least one token per row
+        while (rc == DARE_OK && taken < 0) {
+            if (issued > L + 1) { rc = DARE_ERR_CUDA; break; }   // cannot happen: every step commits a token per row
             const int slot = issued & 1;
-            rc = step_rows(m, tokens, B, row_stride, start, L, k_cache, v_cache, cache_cap, mode, threshold, k, pred,
-                           conf, nullptr, n_remaining, s);
-            if (rc != DARE_OK) return rc;
-            if (cudaMemcpyAsync(m->host_counts + slot * m->max_batch, n_remaining, sizeof(int32_t) * B,
+            if (cudaGraphLaunch(exec, s) != cudaSuccess ||
+                cudaMemcpyAsync(m->host_counts + slot * m->max_batch, n_remaining, sizeof(int32_t) * B,
                                 cudaMemcpyDeviceToHost, s) != cudaSuccess ||
-                cudaEventRecord(m->ev[slot], s) != cudaSuccess)
-                return DARE_ERR_CUDA;
+                cudaEventRecord(m->ev[slot], s) != cudaSuccess) {
+                rc = DARE_ERR_CUDA;
+                break;
+            }
             ++issued;
             if (issued >= 2) {
                 const int prev = (issued - 2) & 1;
-                if (cudaEventSynchronize(m->ev[prev]) != cudaSuccess) return DARE_ERR_CUDA;
+                if (cudaEventSynchronize(m->ev[prev]) != cudaSuccess) { rc = DARE_ERR_CUDA; break; }
+                if (old_exec) {      // a step of this block has finished, so every launch of the previous block has
+                    cudaGraphExecDestroy(old_exec);
+                    cudaGraphDestroy(old_graph);
+                    old_exec = nullptr; old_graph = nullptr;
+                }
                 bool done = true;
                 for (int r = 0; r < B; ++r) done = done && m->host_counts[prev * m->max_batch + r] == 0;
                 if (done) taken = issued - 1;   // steps 0 .. issued-2 denoised; the last one issued was the refresh
             }
         }
-        if (steps_per_block) steps_per_block[b] = taken;
+        if (rc == DARE_OK && steps_per_block) steps_per_block[b] = taken;
+        if (old_exec) {      // (only if this block issued fewer than two steps or failed)
+            cudaStreamSynchronize(s);
+            cudaGraphExecDestroy(old_exec);
+            cudaGraphDestroy(old_graph);
+        }
+        old_exec = exec;
+        old_graph = graph;
     }
-    return cudaStreamSynchronize(s) == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
+    const bool synced = cudaStreamSynchronize(s) == cudaSuccess;
+    if (old_exec) cudaGraphExecDestroy(old_exec);
+    if (old_graph) cudaGraphDestroy(old_graph);
+    if (rc != DARE_OK) return rc;
+    if (!synced || cudaEventRecord(m->ev_out, s) != cudaSuccess || cudaStreamWaitEvent(user, m->ev_out, 0) != cudaSuccess)
+        return DARE_ERR_CUDA;
+    return DARE_OK;
 }
 
 }  // extern "C"
