@@ -117,6 +117,8 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     wl = I.scaled(I.WORKLOADS[args.workload], seed=rank)
+    if args.batch:
+        wl = I.scaled(wl, batch=args.batch)      # smaller copies of a workload (profiler captures)
     ctx = dare.Context(local)
     B, L = wl.batch, wl.block_len
     steps_per_block = -(-L // wl.k) if wl.mode == I.SELECT_TOPK else L
@@ -557,6 +559,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llada8b", choices=sorted(I.WORKLOADS) + sorted(I.MODEL_WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (0 = as defined)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
