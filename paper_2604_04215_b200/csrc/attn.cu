@@ -371,6 +371,358 @@ attn_block_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_cons
     }
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// tcgen05 path: used when the query rows that share a KV head fill 128-row tensor-core tiles well (GQA
+// groups, long blocks such as the prefill).  One CTA per (one or two tiles of packed query rows, rollout x
+// KV head); the two query tiles share every K/V tile:
+//   warp 0        TMA producer: 64-key K and V tiles through a shared-memory ring (as above)
+//   warp 1        UMMA issuer:  S = Q K^T (128 x 64, K-major operands) into one of two TMEM buffers per query
+//                 tile, then O += P V (128 x D; V is the MN-major operand, straight from the TMA tile),
+//                 accumulated in TMEM over the whole key range
+//   warps 2..5    softmax of query tile 0 (warps 6..9: tile 1): one TMEM lane = one query row per thread;
+//                 reads S, keeps the row's reference max and sum, writes P as a bf16 K-major tile into
+//                 shared memory for the second MMA
+// O stays in TMEM, so it cannot be rescaled for free when a row's max grows.  The exponentials are therefore
+// taken relative to a reference max that is only moved when the true max has run more than 2^8 ahead of it;
+// then (rarely, mostly in the first tiles) the warp waits for the MMAs in flight, multiplies its rows of O by
+// the correction factor in place and moves the reference.  The sum uses the same reference, so O / l is exact.
+// A tile holds floor(128 / g) block positions x g heads so that a position's heads never straddle two tiles.
+constexpr int TC_KT = 64;                 // keys per tile
+constexpr float TC_RESCALE_GAP = 8.0f;    // log2 units the true max may run ahead of the reference
+
+template <int D, int QT>
+struct TcShape {
+    static constexpr int Q_BYTES = 128 * D * 2;                        // per query tile
+    static constexpr int KV_STAGE = 2 * TC_KT * D * 2;                 // K tile + V tile
+    static constexpr int P_BYTES = 128 * TC_KT * 2;                    // per query tile and buffer
+    static constexpr int FIXED = QT * Q_BYTES + QT * 2 * P_BYTES;
+    static constexpr int STAGES = (226 * 1024 - 2048 - FIXED) / KV_STAGE > 6 ? 6 : (226 * 1024 - 2048 - FIXED) / KV_STAGE;
+    static constexpr int SMEM = FIXED + STAGES * KV_STAGE + 1024 + 512;
+    static constexpr int THREADS = (2 + 4 * QT) * 32;
+    static constexpr uint32_t TMEM_COLS = QT * 256;                    // per query tile: S 2 x 64 columns, O D columns
+    static_assert(STAGES >= 2, "K/V ring too small");
+};
+
+template <int STAGES, int QT>
+struct TcBarriers {
+    uint64_t full[STAGES];
+    uint64_t empty[STAGES];
+    uint64_t q_ready;
+    uint64_t s_full[QT][2], s_free[QT][2], p_full[QT][2], o_done[QT][2];
+    uint32_t tmem_base;
+    uint32_t abort_flag;
+};
+
+template <int D, int QT>
+__global__ void __launch_bounds__(TcShape<D, QT>::THREADS, 1)
+attn_block_tc_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_constant__ CUtensorMap tm_vpre,
+                     const __grid_constant__ CUtensorMap tm_kblk, const __grid_constant__ CUtensorMap tm_vblk,
+                     const __grid_constant__ CUtensorMap tm_ksuf, const __grid_constant__ CUtensorMap tm_vsuf,
+                     const AttnParams p) {
+    using S = TcShape<D, QT>;
+    constexpr int STAGES = S::STAGES;
+    constexpr int NHALF = D / 64;
+    constexpr int HALF_K = TC_KT * 128;            // one 64-column half of a K or V tile: 64 rows x 128 bytes
+    constexpr int KV_BYTES = TC_KT * D * 2;
+    constexpr int HALF_Q = 128 * 128;              // one 64-column half of a Q tile: 128 rows x 128 bytes
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* q_s = base;                                   // [QT][Q_BYTES]
+    uint8_t* p_s = q_s + QT * S::Q_BYTES;                  // [QT][2][P_BYTES]
+    uint8_t* kv_s = p_s + QT * 2 * S::P_BYTES;             // [STAGES][KV_STAGE]
+    TcBarriers<STAGES, QT>* bars = reinterpret_cast<TcBarriers<STAGES, QT>*>(kv_s + STAGES * S::KV_STAGE);
+    volatile uint32_t* abort_flag = &bars->abort_flag;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int unit = blockIdx.y;
+    const int b = unit / p.Hkv;
+    const int kvh = unit % p.Hkv;
+    const int pos_per_tile = 128 / p.g;            // block positions per query tile
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(&bars->full[s], 1);
+            mbar_init(&bars->empty[s], 1);
+        }
+        mbar_init(&bars->q_ready, 128 * QT);
+        for (int j = 0; j < QT; ++j)
+            for (int i = 0; i < 2; ++i) {
+                mbar_init(&bars->s_full[j][i], 1);
+                mbar_init(&bars->s_free[j][i], 128);
+                mbar_init(&bars->p_full[j][i], 128);
+                mbar_init(&bars->o_done[j][i], 1);
+            }
+        bars->abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(&bars->tmem_base, S::TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = bars->tmem_base;    // query tile j: S buffers at columns j*256 + {0, 64}, O at j*256 + 128
+
+    // lengths and tiles of this unit (same bookkeeping as the warp-level kernel)
+    int P = p.prefix_len ? p.prefix_len[b]
+                         : (p.uniform_P >= 0 ? p.uniform_P : (p.inplace ? p.prefix_cap - p.L : p.prefix_cap));
+    const int p_max = p.inplace ? p.prefix_cap - p.L : p.prefix_cap;
+    int Sx = p.has_suffix ? (p.suffix_len ? p.suffix_len[b] : p.suffix_cap) : 0;
+    if (P < 0 || P > p_max || Sx < 0 || Sx > p.suffix_cap) {
+        P = max(0, min(P, p_max));
+        Sx = max(0, min(Sx, p.suffix_cap));
+        if (threadIdx.x == 0) atomicOr(p.dev_status, DEV_LEN_CLAMPED);
+    }
+    const int len_pre = p.inplace ? P + p.L : P;
+    const int len_blk = p.inplace ? 0 : p.L;
+    const int n_pre = (len_pre + TC_KT - 1) / TC_KT;
+    const int n_blk = (len_blk + TC_KT - 1) / TC_KT;
+    const int n_suf = (Sx + TC_KT - 1) / TC_KT;
+    const int n_tiles = n_pre + n_blk + n_suf;
+    const int base_pre = unit * p.prefix_cap;
+    const int base_blk = unit * p.L;
+    const int base_suf = unit * p.suffix_cap;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            prefetch_tensormap(&tm_kpre);
+            prefetch_tensormap(&tm_vpre);
+            int stage = 0;
+            uint32_t phase = 0;
+            for (int t = 0; t < n_tiles; ++t) {
+                const TileInfo ti = tile_info(t, n_pre, n_blk, len_pre, len_blk, Sx, base_pre, base_blk, base_suf);
+                const CUtensorMap* mk = ti.seg == 0 ? &tm_kpre : (ti.seg == 1 ? &tm_kblk : &tm_ksuf);
+                const CUtensorMap* mv = ti.seg == 0 ? &tm_vpre : (ti.seg == 1 ? &tm_vblk : &tm_vsuf);
+                if (!mbar_wait(&bars->empty[stage], phase ^ 1, abort_flag)) break;
+                uint8_t* kdst = kv_s + stage * S::KV_STAGE;
+                uint8_t* vdst = kdst + KV_BYTES;
+                mbar_arrive_expect_tx(&bars->full[stage], 2 * KV_BYTES);
+#pragma unroll
+                for (int h = 0; h < NHALF; ++h) {
+                    tma_load_2d(kdst + h * HALF_K, mk, &bars->full[stage], h * 64, ti.row0);
+                    tma_load_2d(vdst + h * HALF_K, mv, &bars->full[stage], h * 64, ti.row0);
+                }
+                if (++stage == STAGES) { stage = 0; phase ^= 1; }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc_s = umma_idesc_bf16(128, TC_KT);
+            constexpr uint32_t idesc_o = umma_idesc_bf16(128, D) | UMMA_B_MN_MAJOR;
+            const uint32_t q_addr = smem_u32(q_s), kv_addr = smem_u32(kv_s), p_addr = smem_u32(p_s);
+            bool ok = mbar_wait(&bars->q_ready, 0, abort_flag);
+            // S_j(t) = Q_j K_t^T into S buffer t & 1 of query tile j once its softmax warps have read what it held
+            auto issue_s = [&](int t) -> bool {
+                const int stage = t % STAGES, buf = t & 1;
+                if (!mbar_wait(&bars->full[stage], (t / STAGES) & 1, abort_flag)) return false;
+                const uint32_t k_addr = kv_addr + stage * S::KV_STAGE;
+#pragma unroll
+                for (int j = 0; j < QT; ++j) {
+                    if (!mbar_wait(&bars->s_free[j][buf], ((t >> 1) & 1) ^ 1, abort_flag)) return false;
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        const uint64_t a_desc = umma_desc_sw128_kmajor(q_addr + j * S::Q_BYTES + (kk >> 2) * HALF_Q) + 2 * (kk & 3);
+                        const uint64_t b_desc = umma_desc_sw128_kmajor(k_addr + (kk >> 2) * HALF_K) + 2 * (kk & 3);
+                        umma_bf16(tmem_base + j * 256 + buf * TC_KT, a_desc, b_desc, idesc_s, kk != 0);
+                    }
+                    umma_commit(&bars->s_full[j][buf]);
+                }
+                return true;
+            };
+            if (ok && n_tiles > 0) ok = issue_s(0);
+            for (int t = 0; t < n_tiles && ok; ++t) {
+                if (t + 1 < n_tiles && !issue_s(t + 1)) { ok = false; break; }
+                const int stage = t % STAGES, buf = t & 1;
+                const uint32_t v_addr = kv_addr + stage * S::KV_STAGE + KV_BYTES;
+#pragma unroll
+                for (int j = 0; j < QT; ++j) {
+                    if (!mbar_wait(&bars->p_full[j][buf], (t >> 1) & 1, abort_flag)) { ok = false; break; }
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int kk = 0; kk < TC_KT / 16; ++kk) {
+                        // A: 16 keys further along the 128-byte row of P; B: 16 key rows (2 KB) further down the V
+                        // tile, the second 64 head-dim columns one half tile (HALF_K bytes) away
+                        const uint64_t a_desc = umma_desc_sw128_kmajor(p_addr + (j * 2 + buf) * S::P_BYTES) + 2 * kk;
+                        const uint64_t b_desc = umma_desc_sw128_mnmajor(v_addr + kk * 2048, HALF_K);
+                        umma_bf16(tmem_base + j * 256 + 128, a_desc, b_desc, idesc_o, (t | kk) != 0);
+                    }
+                    umma_commit(&bars->o_done[j][buf]);    // P buffer free again; O holds tiles 0..t
+                }
+                if (!ok) break;
+                umma_commit(&bars->empty[stage]);          // K and V of this tile have been read
+            }
+        }
+    } else {
+        // ---------------- softmax warps: set j = query tile, thread = packed query row r of that tile = TMEM lane r
+        const int j = (warp - 2) >> 2;
+        const int r = (warp & 3) * 32 + lane;          // warp w may touch TMEM lanes [32 * (w % 4), +32)
+        const int rows_in_tile = pos_per_tile * p.g;
+        const int i = (blockIdx.x * QT + j) * pos_per_tile + r / p.g;   // block position
+        const int h = kvh * p.g + r % p.g;                              // query head
+        const bool live = r < rows_in_tile && i < p.L;
+        const size_t qrow = ((static_cast<size_t>(b) * p.L + (live ? i : 0)) * p.Hq + (live ? h : 0)) * D;
+        // Q row -> shared memory, K-major with the 128-byte swizzle (16-byte chunk c of row r sits at c ^ (r & 7))
+        {
+            const uint4* src = reinterpret_cast<const uint4*>(p.q + qrow);
+            uint8_t* qt = q_s + j * S::Q_BYTES;
+#pragma unroll
+            for (int c = 0; c < D / 8; ++c) {
+                const uint4 v = live ? src[c] : make_uint4(0, 0, 0, 0);
+                *reinterpret_cast<uint4*>(qt + (c >> 3) * HALF_Q + r * 128 + (((c & 7) ^ (r & 7)) << 4)) = v;
+            }
+            fence_proxy_async_smem();
+            mbar_arrive(&bars->q_ready);
+        }
+        float m_ref = -INFINITY, l = 0.f;              // reference max (log2 domain) and sum of exp2(s - m_ref)
+        const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
+        const uint32_t tm_s = tmem_base + j * 256 + lane_off;
+        const uint32_t tm_o = tmem_base + j * 256 + 128 + lane_off;
+        bool ok = true;
+        for (int t = 0; t < n_tiles; ++t) {
+            const TileInfo ti = tile_info(t, n_pre, n_blk, len_pre, len_blk, Sx, base_pre, base_blk, base_suf);
+            const int buf = t & 1, stage = t % STAGES;
+            if (!mbar_wait(&bars->s_full[j][buf], (t >> 1) & 1, abort_flag)) { ok = false; break; }
+            tc_fence_after_sync();
+            uint32_t sv[TC_KT];
+            {
+                uint32_t (&lo)[32] = *reinterpret_cast<uint32_t (*)[32]>(&sv[0]);
+                uint32_t (&hi)[32] = *reinterpret_cast<uint32_t (*)[32]>(&sv[32]);
+                tmem_ld_32cols(tm_s + buf * TC_KT, lo);
+                tmem_ld_32cols(tm_s + buf * TC_KT + 32, hi);
+                tmem_ld_wait();
+            }
+            tc_fence_before_sync();
+            mbar_arrive(&bars->s_free[j][buf]);
+            // scores -> log2 domain, keys past the segment's end masked out, tile max
+            float tmax = -INFINITY;
+#pragma unroll
+            for (int c = 0; c < TC_KT; ++c) {
+                float sc = __uint_as_float(sv[c]) * p.scale_log2;
+                if (c >= ti.valid) sc = -INFINITY;
+                sv[c] = __float_as_uint(sc);
+                tmax = fmaxf(tmax, sc);
+            }
+            // move the reference only when the true max has run away from it (decided per warp, so that the
+            // TMEM loads and stores below are executed by whole warps)
+            const bool move = __any_sync(0xffffffffu, tmax > m_ref + TC_RESCALE_GAP);
+            float factor = 1.f;
+            if (move) {
+                const float m_new = fmaxf(m_ref, tmax);         // finite: every tile has at least one key
+                factor = fast_exp2(m_ref - m_new);              // exp2(-inf) = 0 on the first tile
+                m_ref = m_new;
+                l *= factor;
+            }
+            float psum = 0.f;
+            if (t >= 2) {   // P buffer `buf` was read by the second MMA of tile t - 2
+                if (!mbar_wait(&bars->o_done[j][buf], ((t >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
+            }
+            uint8_t* prow = p_s + (j * 2 + buf) * S::P_BYTES + r * 128;
+#pragma unroll
+            for (int c = 0; c < TC_KT / 8; ++c) {
+                float e[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    e[k] = fast_exp2(__uint_as_float(sv[c * 8 + k]) - m_ref);
+                    psum += e[k];
+                }
+                uint4 o;
+                o.x = pack_bf16(e[0], e[1]); o.y = pack_bf16(e[2], e[3]);
+                o.z = pack_bf16(e[4], e[5]); o.w = pack_bf16(e[6], e[7]);
+                *reinterpret_cast<uint4*>(prow + ((c ^ (r & 7)) << 4)) = o;
+            }
+            l += psum;
+            if (move && t >= 1) {
+                // every MMA that adds to O must have landed before O is rescaled in place: tile t - 1 is the last
+                if (!mbar_wait(&bars->o_done[j][(t - 1) & 1], ((t - 1) >> 1) & 1, abort_flag)) { ok = false; break; }
+                tc_fence_after_sync();
+#pragma unroll
+                for (int c = 0; c < D / 32; ++c) {
+                    uint32_t ov[32];
+                    tmem_ld_32cols(tm_o + c * 32, ov);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int k = 0; k < 32; ++k) ov[k] = __float_as_uint(__uint_as_float(ov[k]) * factor);
+                    tmem_st_32cols(tm_o + c * 32, ov);
+                }
+                tmem_st_wait();
+                tc_fence_before_sync();
+            }
+            if (ti.valid < TC_KT) {
+                // V rows past the segment's end hold whatever lies behind it in memory: zero them so that
+                // probability 0 times garbage cannot make a NaN (thread r clears 16-byte pieces of those rows;
+                // both query tiles' warps do it, each before it releases its own second MMA)
+                uint8_t* vt = kv_s + stage * S::KV_STAGE + KV_BYTES;
+                const int n_bad = (TC_KT - ti.valid) * 8;       // 16-byte pieces per 64-column half
+                for (int h2 = 0; h2 < NHALF; ++h2)
+                    for (int q = r; q < n_bad; q += 128)
+                        *reinterpret_cast<uint4*>(vt + h2 * HALF_K + ti.valid * 128 + q * 16) = make_uint4(0, 0, 0, 0);
+            }
+            fence_proxy_async_smem();
+            mbar_arrive(&bars->p_full[j][buf]);
+        }
+        if (ok && n_tiles > 0) ok = mbar_wait(&bars->o_done[j][(n_tiles - 1) & 1], ((n_tiles - 1) >> 1) & 1, abort_flag);
+        tc_fence_after_sync();
+        const float inv = l > 0.f ? 1.f / l : 0.f;
+        __nv_bfloat16* dst = p.out + qrow;
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+            uint32_t ov[32];
+            tmem_ld_32cols(tm_o + c * 32, ov);          // (whole warp, also for rows that are not stored)
+            tmem_ld_wait();
+            if (ok && live) {
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    uint4 o;
+                    o.x = pack_bf16(__uint_as_float(ov[k * 8 + 0]) * inv, __uint_as_float(ov[k * 8 + 1]) * inv);
+                    o.y = pack_bf16(__uint_as_float(ov[k * 8 + 2]) * inv, __uint_as_float(ov[k * 8 + 3]) * inv);
+                    o.z = pack_bf16(__uint_as_float(ov[k * 8 + 4]) * inv, __uint_as_float(ov[k * 8 + 5]) * inv);
+                    o.w = pack_bf16(__uint_as_float(ov[k * 8 + 6]) * inv, __uint_as_float(ov[k * 8 + 7]) * inv);
+                    reinterpret_cast<uint4*>(dst)[c * 4 + k] = o;
+                }
+            }
+        }
+        if (ok && live && p.lse != nullptr)
+            p.lse[(static_cast<size_t>(b) * p.Hq + h) * p.L + i] = l > 0.f ? (m_ref + log2f(l)) * LN2_F : -INFINITY;
+    }
+
+    // teardown
+    tc_fence_before_sync();
+    __syncthreads();
+    if (*abort_flag) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) {}
+        if (threadIdx.x == 0) atomicOr(p.dev_status, DEV_WAIT_EXPIRED);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, S::TMEM_COLS);
+    }
+}
+
+template <int D, int QT>
+int launch_tc(const CUtensorMap* tm, const AttnParams& p, int q_tiles, cudaStream_t stream) {
+    constexpr int SMEM = TcShape<D, QT>::SMEM;
+    if (cudaFuncSetAttribute(attn_block_tc_kernel<D, QT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
+        return DARE_ERR_CUDA;
+    dim3 grid((q_tiles + QT - 1) / QT, p.B * p.Hkv, 1);
+    attn_block_tc_kernel<D, QT><<<grid, TcShape<D, QT>::THREADS, SMEM, stream>>>(tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], p);
+    return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
+}
+
+// The tensor-core tile is worth it when a tile's 128 rows are mostly real query rows.
+bool use_tc_path(const AttnArgs& a) {
+    const int g = a.Hq / a.Hkv;
+    if (g > 128) return false;
+    const int pos_per_tile = 128 / g;
+    const int rows = (a.L < pos_per_tile ? a.L : pos_per_tile) * g;
+    return rows >= 96;
+}
+
 // Combine KV-split partials: out = sum_s w_s o_s / sum_s w_s with w_s = exp(lse_s - max lse).
 template <int D>
 __global__ void attn_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_lse, int splits,
@@ -419,6 +771,7 @@ int pick_warps(int R) { return R <= 16 ? 1 : (R <= 32 ? 2 : 4); }
 }  // namespace
 
 int attn_plan_splits(const dare_ctx* ctx, const AttnArgs& a) {
+    if (use_tc_path(a)) return 1;
     const int g = a.Hq / a.Hkv;
     const int R = a.L * g;
     const int nw = pick_warps(R);
@@ -480,6 +833,15 @@ int launch_attn(const dare_ctx* ctx, const AttnArgs& a, cudaStream_t stream) {
         tm[4] = tm[0]; tm[5] = tm[1];
     }
 
+    if (use_tc_path(a)) {
+        // two query tiles per CTA halve the K/V traffic, but only pay when the CTAs still fill the SMs
+        const int pos_per_tile = 128 / p.g;
+        const int q_tiles = (p.L + pos_per_tile - 1) / pos_per_tile;
+        const long long pairs = static_cast<long long>((q_tiles + 1) / 2) * p.B * p.Hkv;
+        if (q_tiles >= 2 && 4 * pairs >= 3LL * ctx->sm_count)
+            return a.d == 128 ? launch_tc<128, 2>(tm, p, q_tiles, stream) : launch_tc<64, 2>(tm, p, q_tiles, stream);
+        return a.d == 128 ? launch_tc<128, 1>(tm, p, q_tiles, stream) : launch_tc<64, 1>(tm, p, q_tiles, stream);
+    }
     const int nw = pick_warps(p.R);
     const int chunks = (p.R + nw * 16 - 1) / (nw * 16);
     if (a.d == 128) {

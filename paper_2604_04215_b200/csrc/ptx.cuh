@@ -196,6 +196,19 @@ __device__ __forceinline__ float4 ld_global_cg_f4(const float* p) {
     asm volatile("ld.global.cg.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
     return v;
 }
+// Store 32 consecutive fp32 columns of this thread's TMEM lane.  Whole warp.
+__device__ __forceinline__ void tmem_st_32cols(uint32_t taddr, const uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
+          "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]),
+          "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]),
+          "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor for a K-major bf16 operand tile stored as 128-byte rows with the
@@ -212,6 +225,19 @@ __device__ __forceinline__ uint64_t umma_desc_sw128_kmajor(uint32_t smem_addr) {
     desc |= static_cast<uint64_t>(2) << 61;
     return desc;
 }
+// Shared-memory matrix descriptor for an MN-major bf16 operand (the MN index is contiguous in memory): rows of
+// 64 MN-elements (128 bytes, 128-byte swizzle) are one step along K each; groups of 8 K-rows are 1024 bytes
+// apart (stride byte offset); the next 64 MN-elements start `lbo_bytes` further (leading byte offset).
+__device__ __forceinline__ uint64_t umma_desc_sw128_mnmajor(uint32_t smem_addr, uint32_t lbo_bytes) {
+    uint64_t desc = 0;
+    desc |= static_cast<uint64_t>((smem_addr & 0x3FFFF) >> 4);
+    desc |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFF) << 16;
+    desc |= static_cast<uint64_t>(1024 >> 4) << 32;
+    desc |= static_cast<uint64_t>(1) << 46;
+    desc |= static_cast<uint64_t>(2) << 61;
+    return desc;
+}
+constexpr uint32_t UMMA_B_MN_MAJOR = 1u << 16;   // instruction-descriptor bit: B operand is MN-major
 // Instruction descriptor, kind::f16: bf16 x bf16 -> fp32, both operands K-major, dense.
 // [4,6) D format (1 = f32), [7,10) A format (1 = bf16), [10,13) B format (1 = bf16), [15] A major,
 // [16] B major (0 = K), [17,23) N >> 3, [24,29) M >> 4.

@@ -153,14 +153,22 @@ def _attn_case(ctx, B, L, Hq, Hkv, d, P, S=0, ragged=False, inplace=False, seed=
     (1, 5, 6, 3, 64, 0 + 16, 7, True, False),    # odd sizes everywhere
     (4, 32, 2, 1, 64, 2048, 0, False, False),    # long prefix, few units: KV splits + combine
     (1, 1, 1, 1, 64, 16, 0, False, True),        # a single query
+    # shapes that fill a 128-row tensor-core tile (tcgen05 path)
+    (2, 128, 4, 4, 64, 100, 0, False, False),    # one full tile per head, head_dim 64, ragged prefix tile
+    (2, 40, 8, 2, 128, 300, 70, True, False),    # GQA group of 4: 32 positions per tile, two tiles, dual cache, ragged
+    (2, 100, 6, 2, 128, 0 + 8, 0, False, True),  # group of 3: 42 positions x 3 heads = 126 rows per tile, in place
+    (1, 300, 2, 2, 64, 64, 0, False, True),      # prefill-like: three tiles of 128 rows, block in place
+    (60, 256, 2, 2, 128, 200, 0, False, False),  # enough units for two query tiles per CTA (and a third, single one)
+    (30, 130, 4, 4, 64, 70, 20, True, False),    # two query tiles per CTA, head_dim 64, second tile nearly empty
 ])
 def test_attention_matches_oracle(ctx, B, L, Hq, Hkv, d, P, S, ragged, inplace):
     _attn_case(ctx, B, L, Hq, Hkv, d, P, S, ragged, inplace, seed=B + L + P)
 
 
-def test_attention_zero_prefix_and_garbage_behind_lengths(ctx):
-    """prefix_len = 0 for some rows, and NaNs planted behind every valid length must not leak in."""
-    B, L, H, d, P, S = 3, 8, 2, 64, 96, 40
+@pytest.mark.parametrize("L", [8, 128])
+def test_attention_zero_prefix_and_garbage_behind_lengths(ctx, L):
+    """prefix_len = 0 for some rows, and NaNs planted behind every valid length must not leak in (both kernels)."""
+    B, H, d, P, S = 3, 2, 64, 96, 40
     wl = I.scaled(I.WORKLOADS["tiny"], batch=B, block_len=L, n_q_heads=H, n_kv_heads=H, head_dim=d, prompt_len=P,
                   gen_len=L, suffix_cap=S, seed=9)
     k_pre, v_pre, k_suf, v_suf = I.make_caches(wl)
