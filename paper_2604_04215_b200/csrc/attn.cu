@@ -512,23 +512,26 @@ attn_block_tc_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_c
         if (lane == 0) {
             constexpr uint32_t idesc_s = umma_idesc_bf16(128, TC_KT);
             constexpr uint32_t idesc_o = umma_idesc_bf16(128, D) | UMMA_B_MN_MAJOR;
-            const uint32_t q_addr = smem_u32(q_s), kv_addr = smem_u32(kv_s), p_addr = smem_u32(p_s);
+            // descriptor lower words (address >> 4 [| leading byte offset]); the upper word is a constant
+            const uint32_t q_lo = smem_u32(q_s) >> 4, kv_lo = smem_u32(kv_s) >> 4, p_lo = smem_u32(p_s) >> 4;
+            const uint32_t v_lbo = static_cast<uint32_t>(HALF_K >> 4) << 16;   // second 64 head-dim columns: one half tile on
             bool ok = mbar_wait(&bars->q_ready, 0, abort_flag);
             // S_j(t) = Q_j K_t^T into S buffer t & 1 of query tile j once its softmax warps have read what it held
             auto issue_s = [&](int t) -> bool {
                 const int stage = t % STAGES, buf = t & 1;
                 if (!mbar_wait(&bars->full[stage], (t / STAGES) & 1, abort_flag)) return false;
-                const uint32_t k_addr = kv_addr + stage * S::KV_STAGE;
+                const uint32_t k_lo = kv_lo + stage * (S::KV_STAGE >> 4);
 #pragma unroll
                 for (int j = 0; j < QT; ++j) {
                     if (!mbar_wait(&bars->s_free[j][buf], ((t >> 1) & 1) ^ 1, abort_flag)) return false;
                     tc_fence_after_sync();
 #pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk) {
-                        const uint64_t a_desc = umma_desc_sw128_kmajor(q_addr + j * S::Q_BYTES + (kk >> 2) * HALF_Q) + 2 * (kk & 3);
-                        const uint64_t b_desc = umma_desc_sw128_kmajor(k_addr + (kk >> 2) * HALF_K) + 2 * (kk & 3);
-                        umma_bf16(tmem_base + j * 256 + buf * TC_KT, a_desc, b_desc, idesc_s, kk != 0);
-                    }
+                    const uint32_t qa = q_lo + j * (S::Q_BYTES >> 4), sd = tmem_base + j * 256 + buf * TC_KT;
+                    umma_bf16_lo<false>(sd, qa, k_lo, idesc_s);
+#pragma unroll
+                    for (int kk = 1; kk < D / 16; ++kk)     // 16 channels = 32 bytes along the swizzled row: +2
+                        umma_bf16_lo<true>(sd, qa + (kk >> 2) * (HALF_Q >> 4) + 2 * (kk & 3),
+                                           k_lo + (kk >> 2) * (HALF_K >> 4) + 2 * (kk & 3), idesc_s);
                     umma_commit(&bars->s_full[j][buf]);
                 }
                 return true;
@@ -537,19 +540,19 @@ attn_block_tc_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_c
             for (int t = 0; t < n_tiles && ok; ++t) {
                 if (t + 1 < n_tiles && !issue_s(t + 1)) { ok = false; break; }
                 const int stage = t % STAGES, buf = t & 1;
-                const uint32_t v_addr = kv_addr + stage * S::KV_STAGE + KV_BYTES;
+                const uint32_t v_lo = (kv_lo + stage * (S::KV_STAGE >> 4) + (KV_BYTES >> 4)) | v_lbo;
 #pragma unroll
                 for (int j = 0; j < QT; ++j) {
                     if (!mbar_wait(&bars->p_full[j][buf], (t >> 1) & 1, abort_flag)) { ok = false; break; }
                     tc_fence_after_sync();
 #pragma unroll
-                    for (int kk = 0; kk < TC_KT / 16; ++kk) {
-                        // A: 16 keys further along the 128-byte row of P; B: 16 key rows (2 KB) further down the V
-                        // tile, the second 64 head-dim columns one half tile (HALF_K bytes) away
-                        const uint64_t a_desc = umma_desc_sw128_kmajor(p_addr + (j * 2 + buf) * S::P_BYTES) + 2 * kk;
-                        const uint64_t b_desc = umma_desc_sw128_mnmajor(v_addr + kk * 2048, HALF_K);
-                        umma_bf16(tmem_base + j * 256 + 128, a_desc, b_desc, idesc_o, (t | kk) != 0);
-                    }
+                    // A: 16 keys further along the 128-byte row of P (+2); B: 16 key rows (2 KB) further down V
+                    const uint32_t pa = p_lo + (j * 2 + buf) * (S::P_BYTES >> 4), od = tmem_base + j * 256 + 128;
+                    if (t == 0) umma_bf16_lo<false>(od, pa, v_lo, idesc_o);
+                    else umma_bf16_lo<true>(od, pa, v_lo, idesc_o);
+#pragma unroll
+                    for (int kk = 1; kk < TC_KT / 16; ++kk)
+                        umma_bf16_lo<true>(od, pa + 2 * kk, v_lo + kk * (2048 >> 4), idesc_o);
                     umma_commit(&bars->o_done[j][buf]);    // P buffer free again; O holds tiles 0..t
                 }
                 if (!ok) break;

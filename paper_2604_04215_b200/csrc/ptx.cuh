@@ -237,6 +237,30 @@ __device__ __forceinline__ uint64_t umma_desc_sw128_mnmajor(uint32_t smem_addr, 
     desc |= static_cast<uint64_t>(2) << 61;
     return desc;
 }
+// The same descriptors assembled from parts, for loops in which one thread issues many short MMAs and the
+// 64-bit field arithmetic above would dominate: the upper word is a constant (stride byte offset 1024, version
+// 1, 128-byte swizzle), the lower word is (address >> 4) | (leading byte offset >> 4) << 16.  Shared-memory
+// addresses are below 2^18, so adding a byte offset >> 4 to the lower word never carries out of the address field.
+constexpr uint32_t UMMA_DESC_HI_SW128 = (1024u >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint64_t umma_desc_pack(uint32_t lo) {
+    return (static_cast<uint64_t>(UMMA_DESC_HI_SW128) << 32) | lo;
+}
+// MMA issue with the descriptors given as lower words (upper word = UMMA_DESC_HI_SW128) and the accumulate flag
+// as a compile-time constant: the fewest instructions per MMA for the one issuing thread.
+template <bool ACCUMULATE>
+__device__ __forceinline__ void umma_bf16_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        ".reg .b64 da, db;\n"
+        "setp.ne.b32 p, %5, 0;\n"
+        "mov.b64 da, {%1, %4};\n"
+        "mov.b64 db, {%2, %4};\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n"
+        "}\n" ::"r"(d_tmem),
+        "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(UMMA_DESC_HI_SW128), "n"(ACCUMULATE ? 1 : 0)
+        : "memory");
+}
 constexpr uint32_t UMMA_B_MN_MAJOR = 1u << 16;   // instruction-descriptor bit: B operand is MN-major
 // Instruction descriptor, kind::f16: bf16 x bf16 -> fp32, both operands K-major, dense.
 // [4,6) D format (1 = f32), [7,10) A format (1 = bf16), [10,13) B format (1 = bf16), [15] A major,
