@@ -1,0 +1,106 @@
+"""Pins for the oracle of the stochastic rollout epilogue (oracle/dare_sampling_oracle.py), CPU only.
+
+  * the counter-based generator against the known-answer vectors published with its reference implementation
+    (tests/golden/philox4x32_10_kat.txt);
+  * the uniforms: inside (0, 1), exact in float32, flat histogram, different for different (seed, row, step);
+  * the Gumbel transform: closed-form values, mean = Euler's constant, variance = pi^2 / 6;
+  * the sampling law (Gumbel-max): token frequencies follow softmax(z / T), checked on a small vocabulary;
+  * limits: T -> 0 gives the greedy head's token; the confidence is the temperature-1 probability of the token;
+    committed rows are skipped; the mask column is never sampled.
+"""
+import os
+
+import numpy as np
+
+from oracle import dare_oracle as O
+from oracle import dare_sampling_oracle as SO
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "philox4x32_10_kat.txt")
+
+
+def test_philox_known_answers():
+    n = 0
+    for line in open(GOLDEN):
+        line = line.split("#")[0].strip()
+        if not line:
+            continue
+        w = [int(t, 16) for t in line.split()]
+        ctr, key, want = w[0:4], w[4:6], w[6:10]
+        got = SO.philox4x32_10(np.array(ctr, dtype=np.uint32), np.array(key, dtype=np.uint32))
+        assert [int(v) for v in got] == want
+        n += 1
+    assert n == 3
+
+
+def test_philox_is_a_bijection_of_the_counter_and_vectorises():
+    ctr = np.zeros((1000, 4), dtype=np.uint32)
+    ctr[:, 0] = np.arange(1000)
+    out = SO.philox4x32_10(ctr, np.array([7, 9], dtype=np.uint32))
+    assert len({tuple(r) for r in out.tolist()}) == 1000
+    one = SO.philox4x32_10(np.array([17, 0, 0, 0], dtype=np.uint32), np.array([7, 9], dtype=np.uint32))
+    np.testing.assert_array_equal(out[17], one)
+
+
+def test_uniforms_are_exact_float32_in_the_open_interval():
+    u = SO.uniforms(seed=0x1234_5678_9ABC_DEF0, row=3, step=5, V=100003)
+    assert u.shape == (100003,)
+    assert u.min() > 0.0 and u.max() < 1.0
+    np.testing.assert_array_equal(u.astype(np.float32).astype(np.float64), u)
+    np.testing.assert_array_equal((u * 2 ** 24) % 2, 1.0)                 # odd multiples of 2^-24
+    hist, _ = np.histogram(u, bins=20, range=(0, 1))
+    assert np.abs(hist / len(u) - 0.05).max() < 0.004
+    assert abs(u.mean() - 0.5) < 0.004
+    # a different row, step or seed gives a different stream; the same triple the same one
+    base = SO.uniforms(1, 2, 3, 64)
+    np.testing.assert_array_equal(base, SO.uniforms(1, 2, 3, 64))
+    for other in (SO.uniforms(2, 2, 3, 64), SO.uniforms(1, 3, 3, 64), SO.uniforms(1, 2, 4, 64),
+                  SO.uniforms(1 + (1 << 32), 2, 3, 64)):
+        assert (other != base).mean() > 0.9
+    # element v is word v % 4 of block v // 4: a longer request extends a shorter one
+    np.testing.assert_array_equal(SO.uniforms(1, 2, 3, 70)[:64], base)
+
+
+def test_gumbel_closed_forms_and_moments():
+    np.testing.assert_allclose(SO.gumbel(np.array([np.exp(-1.0)])), [0.0], atol=1e-15)
+    np.testing.assert_allclose(SO.gumbel(np.array([np.exp(-np.e)])), [-1.0], atol=1e-15)
+    g = SO.gumbel(SO.uniforms(11, 0, 0, 400000))
+    assert abs(g.mean() - 0.5772156649) < 0.01
+    assert abs(g.var() - np.pi ** 2 / 6) < 0.03
+
+
+def test_sampling_law_follows_softmax_of_scaled_logits():
+    rng = np.random.default_rng(0)
+    V, D, T = 12, 8, 0.7
+    w = rng.standard_normal((V, D))
+    x = np.tile(rng.standard_normal((1, D)), (4000, 1))                   # the same row 4000 times: rows differ in noise only
+    mask_id = 5
+    res = SO.lmhead_sample(x, w, None, mask_id, True, T, seed=99, step=1)
+    z = w @ x[0]
+    z[mask_id] = -np.inf
+    p = np.exp(z / T - (z / T)[np.isfinite(z)].max())
+    p /= p.sum()
+    freq = np.bincount(res["pred"], minlength=V) / len(x)
+    assert freq[mask_id] == 0
+    assert np.abs(freq - p).max() < 4.0 * np.sqrt(0.25 / len(x))          # 4 sigma of a binomial proportion
+    # confidence = temperature-1 probability of the sampled token
+    p1 = np.exp(z - z[np.isfinite(z)].max())
+    p1 /= p1.sum()
+    np.testing.assert_allclose(res["conf"], p1[res["pred"]], rtol=1e-12)
+
+
+def test_low_temperature_recovers_the_greedy_head_and_rows_are_skipped():
+    rng = np.random.default_rng(1)
+    M, V, D = 9, 200, 16
+    x, w = rng.standard_normal((M, D)), rng.standard_normal((V, D))
+    row_tokens = np.full(M, 150)
+    row_tokens[[2, 6]] = 17                                                 # committed rows
+    greedy = O.lmhead_confidence(x, w, row_tokens, 150, True)
+    res = SO.lmhead_sample(x, w, row_tokens, 150, True, temperature=1e-6, seed=5, step=0)
+    np.testing.assert_array_equal(res["pred"], greedy["pred"])
+    np.testing.assert_allclose(res["conf"][np.isfinite(res["conf"])], greedy["conf"][np.isfinite(greedy["conf"])], rtol=1e-12)
+    assert np.isneginf(res["conf"][[2, 6]]).all() and (res["pred"][[2, 6]] == 17).all()
+    # at T = 1 the samples differ from the greedy tokens somewhere, and change with the step
+    a = SO.lmhead_sample(x, w, None, 150, True, 1.0, seed=5, step=0)["pred"]
+    b = SO.lmhead_sample(x, w, None, 150, True, 1.0, seed=5, step=1)["pred"]
+    assert (a != greedy["pred"]).any() and (a != b).any()
+    assert (a != 150).all() and (b != 150).all()
