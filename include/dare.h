@@ -118,6 +118,24 @@ int dare_lmhead_confidence(dare_ctx* ctx,
                            int32_t* pred, float* conf, void* stream);
 
 /*
+ * Stochastic variant of dare_lmhead_confidence for rollouts that must differ from one another (Section 4.2:
+ * several rollouts per prompt).  Per masked row, with z the logits as above:
+ *     y_v = z_v / temperature + g_v,   g_v = -ln(-ln u_v),   pred = lowest index attaining max_v y_v
+ *     conf = softmax(z)[pred] = exp(z_pred - logsumexp z)          (probability at temperature 1)
+ * so pred is a sample of softmax(z / temperature) (Gumbel-max).  The uniforms come from the counter-based
+ * generator Philox4x32 with 10 rounds (Salmon et al., SC 2011), key = (seed low word, seed high word), counter =
+ * (v / 4, m, step, 0x44415245) where m is the row's index in `hidden`; element v uses output word v % 4, whose top
+ * 23 bits k give u_v = (2 k + 1) / 2^24.  The same (seed, step) reproduces the same tokens; callers advance `step`
+ * from one denoising step to the next.  Other arguments, skipped rows and limits as dare_lmhead_confidence;
+ * temperature > 0; the workspace need is 20 instead of 12 bytes per (row, vocabulary group).
+ */
+int dare_lmhead_sample(dare_ctx* ctx,
+                       const void* hidden, int M, int D, const void* w, int V,
+                       const int32_t* row_tokens, int32_t mask_id, int exclude_mask_column,
+                       float temperature, uint64_t seed, uint32_t step,
+                       int32_t* pred, float* conf, void* stream);
+
+/*
  * Parallel unmask selection, in place on the token state (Section 3.4, "partially fixed states";
  * Section 4.2: block length 32, two tokens per step).  Per row, U = block positions whose token is
  * mask_id.  THRESHOLD: commit every i in U with conf > threshold, or the single most confident one

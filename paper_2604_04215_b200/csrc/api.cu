@@ -52,11 +52,11 @@ int check_attn(const dare_ctx* ctx, int B, int L, int Hq, int Hkv, int d, int pr
 }
 
 int check_lmhead(const dare_ctx* ctx, const void* hidden, int M, int D, const void* w, int V, bool with_row_tokens,
-                 const void* pred, const void* conf) {
+                 const void* pred, const void* conf, bool sampling = false) {
     if (!ctx || !hidden || !w || !pred || !conf) return DARE_ERR_NULL;
     if (M < 1 || D < 8 || D % 8 != 0 || V < 2) return DARE_ERR_SHAPE;
     if (!aligned16(hidden) || !aligned16(w)) return DARE_ERR_ALIGN;
-    if (dare::lmhead_workspace_bytes(M, D, V, ctx->sm_count, with_row_tokens) > ctx->workspace_bytes)
+    if (dare::lmhead_workspace_bytes(M, D, V, ctx->sm_count, with_row_tokens, sampling) > ctx->workspace_bytes)
         return DARE_ERR_WORKSPACE;
     return DARE_OK;
 }
@@ -165,7 +165,18 @@ int dare_lmhead_confidence(dare_ctx* ctx, const void* hidden, int M, int D, cons
     int rc = check_lmhead(ctx, hidden, M, D, w, V, row_tokens != nullptr, pred, conf);
     if (rc != DARE_OK) return rc;
     return dare::launch_lmhead(ctx, ctx->workspace, hidden, M, D, w, V, row_tokens, M, 0, mask_id, exclude_mask_column,
-                               pred, conf, static_cast<cudaStream_t>(stream));
+                               pred, conf, static_cast<cudaStream_t>(stream), nullptr);
+}
+
+int dare_lmhead_sample(dare_ctx* ctx, const void* hidden, int M, int D, const void* w, int V, const int32_t* row_tokens,
+                       int32_t mask_id, int exclude_mask_column, float temperature, uint64_t seed, uint32_t step,
+                       int32_t* pred, float* conf, void* stream) {
+    int rc = check_lmhead(ctx, hidden, M, D, w, V, row_tokens != nullptr, pred, conf, true);
+    if (rc != DARE_OK) return rc;
+    if (!(temperature > 0.f) || isinf(temperature)) return DARE_ERR_RANGE;
+    const dare::LmSampleArgs smp = {temperature, seed, step};
+    return dare::launch_lmhead(ctx, ctx->workspace, hidden, M, D, w, V, row_tokens, M, 0, mask_id, exclude_mask_column,
+                               pred, conf, static_cast<cudaStream_t>(stream), &smp);
 }
 
 int dare_unmask_select(dare_ctx* ctx, int32_t* tokens, int B, int64_t row_stride, int block_start, int L,
@@ -203,7 +214,7 @@ int dare_denoise_block(dare_ctx* ctx, int B, int L, int Hq, int Hkv, int d, int 
     // The LM head reads each row's current token straight from the token state: row m = (r, i) lives at
     // tokens[r * row_stride + block_start + i].
     rc = dare::launch_lmhead(ctx, ctx->workspace, hidden, M, D, w, V, tokens + block_start, L, row_stride, mask_id,
-                             exclude_mask_column, pred, conf, s);
+                             exclude_mask_column, pred, conf, s, nullptr);
     if (rc != DARE_OK) return rc;
     return dare::launch_unmask_select(tokens, B, row_stride, block_start, L, pred, conf, mask_id, mode, threshold, k,
                                       n_committed, n_remaining, s);

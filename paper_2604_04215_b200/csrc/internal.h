@@ -32,11 +32,13 @@ int launch_unmask_select(int32_t* tokens, int B, int64_t row_stride, int block_s
                          const float* conf, int32_t mask_id, int mode, float threshold, int k, int32_t* n_committed,
                          int32_t* n_remaining, cudaStream_t stream);
 
-size_t lmhead_workspace_bytes(int M, int D, int V, int sm_count, bool with_row_tokens);
+// Sampling epilogue of the LM head (NULL = greedy): temperature, 64-bit seed and step counter of the generator.
+struct LmSampleArgs { float temperature; uint64_t seed; uint32_t step; };
+size_t lmhead_workspace_bytes(int M, int D, int V, int sm_count, bool with_row_tokens, bool sampling);
 // Token of LM-head row m (to skip committed rows) = row_tokens[(m / tok_L) * tok_row_stride + m % tok_L].
 int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M, int D, const void* w, int V,
                   const int32_t* row_tokens, int tok_L, int64_t tok_row_stride, int32_t mask_id, int exclude_mask_column, int32_t* pred, float* conf,
-                  cudaStream_t stream);
+                  cudaStream_t stream, const LmSampleArgs* sample);
 
 struct AttnArgs {
     int B, L, Hq, Hkv, d, prefix_cap, suffix_cap;

@@ -102,11 +102,39 @@ lmhead_compact_kernel(const uint4* __restrict__ x, int M, int D8, const int32_t*
     for (int i = lane; i < D8; i += 32) dst[i] = src[i];
 }
 
+// Sampling epilogue (temperature + Gumbel-max): token = argmax_v (z_v / T + g_v), g_v = -ln(-ln u_v), with u_v from
+// the counter-based generator Philox4x32-10 (Salmon et al., SC 2011) keyed by the seed, counter = (v / 4, row,
+// step, tag); element v takes output word v % 4, whose top 23 bits k give u = (2 k + 1) / 2^24 (exact in fp32).
+struct LmSampling {
+    float inv_temperature;
+    uint32_t seed_lo, seed_hi, step;
+    const int32_t* row_index;      // original row of compacted row c (NULL: identity): keys the generator
+    float* part_y;                 // per partial: best perturbed score and the raw logit there
+    float* part_zb;
+};
+
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1) {
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint32_t hi0 = __umulhi(0xD2511F53u, c.x), lo0 = 0xD2511F53u * c.x;
+        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c.z), lo1 = 0xCD9E8D57u * c.z;
+        c = make_uint4(hi1 ^ c.y ^ k0, lo1, hi0 ^ c.w ^ k1, lo0);
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    return c;
+}
+__device__ __forceinline__ float gumbel_from_word(uint32_t w) {
+    const float u = static_cast<float>(((w >> 9) << 1) | 1u) * 5.9604644775390625e-08f;   // (2 k + 1) / 2^24, exact
+    return -logf(-logf(u));
+}
+
+template <bool SAMPLE>
 __global__ void __launch_bounds__(LM_THREADS, 1)
 lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                       int M, const int32_t* __restrict__ live_rows, int D, int V, int mask_col, int n_tiles,
                       float* __restrict__ part_max, float* __restrict__ part_sum, int32_t* __restrict__ part_arg,
-                      uint32_t* __restrict__ dev_status) {
+                      uint32_t* __restrict__ dev_status, const LmSampling smp) {
     const int Mc = live_rows ? *live_rows : M;          // rows that need logits (uniform over the grid)
     const int m_tiles = (Mc + BM - 1) / BM;
     if (m_tiles == 0) return;
@@ -212,6 +240,12 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
             float run_max = -INFINITY;
             float run_sum = 0.f;
             int run_arg = ARG_NONE;
+            float best_y = -INFINITY, best_z = -INFINITY;       // SAMPLE: best perturbed score, raw logit there
+            uint32_t rng_row = 0;
+            if (SAMPLE) {
+                const int row_c = m_tile * BM + row_in_tile;
+                rng_row = static_cast<uint32_t>(row_c < Mc && smp.row_index ? smp.row_index[row_c] : row_c);
+            }
             for (int n_tile = group; n_tile < n_tiles && ok; n_tile += groups, ++it) {
                 const int acc = it & 1;
                 const uint32_t acc_phase = (it >> 1) & 1;
@@ -240,11 +274,25 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
                         const float z = __uint_as_float(v[j]);
                         if (z > cmax) { cmax = z; carg = cbase + j; }   // strict '>' keeps the lowest index
                     }
+                    if (SAMPLE) {
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) {
+                            const uint4 w4 = philox4x32_10(make_uint4(static_cast<uint32_t>(cbase >> 2) + q, rng_row, smp.step,
+                                                                      0x44415245u), smp.seed_lo, smp.seed_hi);
+                            const uint32_t ww[4] = {w4.x, w4.y, w4.z, w4.w};
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const float z = __uint_as_float(v[q * 4 + e]);
+                                const float y = fmaf(z, smp.inv_temperature, gumbel_from_word(ww[e]));
+                                if (y > best_y) { best_y = y; best_z = z; run_arg = cbase + q * 4 + e; }   // ascending columns
+                            }
+                        }
+                    }
                     if (cmax > -INFINITY) {
                         if (cmax > run_max) {   // tiles of a group come in ascending order: '>' keeps the lowest id
                             run_sum *= fast_exp2((run_max - cmax) * LOG2E);   // exp2(-inf) = 0 the first time
                             run_max = cmax;
-                            run_arg = carg;
+                            if (!SAMPLE) run_arg = carg;
                         }
                         const float mb = run_max * LOG2E;
                         float s = 0.f;
@@ -262,6 +310,7 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
                 part_max[o] = run_max;
                 part_sum[o] = run_sum;
                 part_arg[o] = run_arg;
+                if (SAMPLE) { smp.part_y[o] = best_y; smp.part_zb[o] = best_z; }
             }
         }
     }
@@ -322,16 +371,61 @@ __global__ void lmhead_merge_kernel(const float* __restrict__ part_max, const fl
     }
 }
 
+// The same fold for the sampling epilogue: log-sum-exp of the raw logits from (max, sum); the sampled token is the
+// partial with the best perturbed score (lowest token id on ties); confidence = exp(z_token - logsumexp z).
+__global__ void lmhead_merge_sample_kernel(const float* __restrict__ part_max, const float* __restrict__ part_sum,
+                                           const int32_t* __restrict__ part_arg, const float* __restrict__ part_y,
+                                           const float* __restrict__ part_zb, int grid_gemm, int n_tiles, int M,
+                                           const int32_t* __restrict__ live_rows, const int32_t* __restrict__ idx,
+                                           int32_t* __restrict__ pred, float* __restrict__ conf) {
+    const int c = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    const int Mc = live_rows ? *live_rows : M;
+    if (c >= Mc) return;
+    const int groups = lm_groups(grid_gemm, (Mc + BM - 1) / BM, n_tiles);
+    float m = -INFINITY, s = 0.f, y = -INFINITY, zb = -INFINITY;
+    int a = ARG_NONE;
+    const size_t base = static_cast<size_t>(c) * groups;
+    for (int t = lane; t < groups; t += 32) {
+        const float m2 = part_max[base + t], s2 = part_sum[base + t];
+        if (m2 > -INFINITY) {
+            if (m2 > m) { s = s * exp2f((m - m2) * LOG2E) + s2; m = m2; }
+            else s += s2 * exp2f((m2 - m) * LOG2E);
+        }
+        const float y2 = part_y[base + t];
+        const int a2 = part_arg[base + t];
+        if (y2 > y || (y2 == y && a2 < a)) { y = y2; a = a2; zb = part_zb[base + t]; }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const float m2 = __shfl_xor_sync(0xffffffffu, m, off);
+        const float s2 = __shfl_xor_sync(0xffffffffu, s, off);
+        const float y2 = __shfl_xor_sync(0xffffffffu, y, off);
+        const float z2 = __shfl_xor_sync(0xffffffffu, zb, off);
+        const int a2 = __shfl_xor_sync(0xffffffffu, a, off);
+        if (m2 > -INFINITY) {
+            if (m2 > m) { s = s * exp2f((m - m2) * LOG2E) + s2; m = m2; }
+            else s += s2 * exp2f((m2 - m) * LOG2E);
+        }
+        if (y2 > y || (y2 == y && a2 < a)) { y = y2; a = a2; zb = z2; }
+    }
+    if (lane == 0) {
+        const int row = idx ? idx[c] : c;
+        pred[row] = a;
+        conf[row] = exp2f((zb - m) * LOG2E) / s;
+    }
+}
+
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 }  // namespace
 
 // Scratch layout: [compacted X: M*D bf16][row indices: M int32][live-row count][partials: 3 x M x groups]
-size_t lmhead_workspace_bytes(int M, int D, int V, int sm_count, bool with_row_tokens) {
+size_t lmhead_workspace_bytes(int M, int D, int V, int sm_count, bool with_row_tokens, bool sampling) {
     const size_t n_tiles = (static_cast<size_t>(V) + BN - 1) / BN;
     size_t groups = static_cast<size_t>(sm_count);
     if (groups > n_tiles) groups = n_tiles;
-    size_t bytes = 3 * sizeof(float) * groups * static_cast<size_t>(M);
+    size_t bytes = (sampling ? 5 : 3) * sizeof(float) * groups * static_cast<size_t>(M);
     if (with_row_tokens)
         bytes += round_up(static_cast<size_t>(M) * D * 2, 1024) + round_up(static_cast<size_t>(M) * 4 + 4, 1024);
     return bytes;
@@ -339,7 +433,7 @@ size_t lmhead_workspace_bytes(int M, int D, int V, int sm_count, bool with_row_t
 
 int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M, int D, const void* w, int V,
                   const int32_t* row_tokens, int tok_L, int64_t tok_row_stride, int32_t mask_id,
-                  int exclude_mask_column, int32_t* pred, float* conf, cudaStream_t stream) {
+                  int exclude_mask_column, int32_t* pred, float* conf, cudaStream_t stream, const LmSampleArgs* sample) {
     const int n_tiles = (V + BN - 1) / BN;
     const int m_tiles_max = (M + BM - 1) / BM;
     int grid = ctx->sm_count;
@@ -374,17 +468,35 @@ int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M,
     rc = make_tmap_bf16_2d(ctx, &tmap_w, w, static_cast<uint64_t>(V), static_cast<uint64_t>(D), BN, BK);
     if (rc != DARE_OK) return rc;
 
-    if (cudaFuncSetAttribute(lmhead_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, LM_SMEM_BYTES) !=
-        cudaSuccess)
-        return DARE_ERR_CUDA;
     const int mask_col = (exclude_mask_column && mask_id >= 0 && mask_id < V) ? mask_id : -1;
-    lmhead_partial_kernel<<<grid, LM_THREADS, LM_SMEM_BYTES, stream>>>(tmap_x, tmap_w, M, live_rows, D, V, mask_col,
-                                                                       n_tiles, part_max, part_sum, part_arg,
-                                                                       ctx->dev_status);
-    if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
     const int rows_per_block = 8;
-    lmhead_merge_kernel<<<(M + rows_per_block - 1) / rows_per_block, rows_per_block * 32, 0, stream>>>(
-        part_max, part_sum, part_arg, grid, n_tiles, M, live_rows, idx, pred, conf);
+    LmSampling smp = {};
+    if (sample == nullptr) {
+        if (cudaFuncSetAttribute(lmhead_partial_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 LM_SMEM_BYTES) != cudaSuccess)
+            return DARE_ERR_CUDA;
+        lmhead_partial_kernel<false><<<grid, LM_THREADS, LM_SMEM_BYTES, stream>>>(
+            tmap_x, tmap_w, M, live_rows, D, V, mask_col, n_tiles, part_max, part_sum, part_arg, ctx->dev_status, smp);
+        if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
+        lmhead_merge_kernel<<<(M + rows_per_block - 1) / rows_per_block, rows_per_block * 32, 0, stream>>>(
+            part_max, part_sum, part_arg, grid, n_tiles, M, live_rows, idx, pred, conf);
+    } else {
+        smp.inv_temperature = 1.0f / sample->temperature;
+        smp.seed_lo = static_cast<uint32_t>(sample->seed & 0xffffffffu);
+        smp.seed_hi = static_cast<uint32_t>(sample->seed >> 32);
+        smp.step = sample->step;
+        smp.row_index = idx;
+        smp.part_y = reinterpret_cast<float*>(part_arg + n_part);
+        smp.part_zb = smp.part_y + n_part;
+        if (cudaFuncSetAttribute(lmhead_partial_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 LM_SMEM_BYTES) != cudaSuccess)
+            return DARE_ERR_CUDA;
+        lmhead_partial_kernel<true><<<grid, LM_THREADS, LM_SMEM_BYTES, stream>>>(
+            tmap_x, tmap_w, M, live_rows, D, V, mask_col, n_tiles, part_max, part_sum, part_arg, ctx->dev_status, smp);
+        if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
+        lmhead_merge_sample_kernel<<<(M + rows_per_block - 1) / rows_per_block, rows_per_block * 32, 0, stream>>>(
+            part_max, part_sum, part_arg, smp.part_y, smp.part_zb, grid, n_tiles, M, live_rows, idx, pred, conf);
+    }
     if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
     return DARE_OK;
 }
@@ -461,7 +573,7 @@ extern "C" int dare_lmhead_confidence_static(const void* hidden, int M, int D, c
     dare::StaticDeviceState* st = nullptr;
     int rc = dare::static_state_for_current_device(&st);
     if (rc != DARE_OK) return rc;
-    if (dare::lmhead_workspace_bytes(M, D, V, st->sm_count, row_tokens != nullptr) >
+    if (dare::lmhead_workspace_bytes(M, D, V, st->sm_count, row_tokens != nullptr, false) >
         static_cast<size_t>(DARE_LMHEAD_STATIC_SCRATCH_BYTES))
         return DARE_ERR_WORKSPACE;   // beyond the fixed scratch: use dare_lmhead_confidence with a context
     // a context-shaped view of the static state for the shared launcher; nothing here is allocated
@@ -473,6 +585,6 @@ extern "C" int dare_lmhead_confidence_static(const void* hidden, int M, int D, c
     view.dev_status = st->status;
     view.encode_tiled = st->encode;
     return dare::launch_lmhead(&view, st->scratch, hidden, M, D, w, V, row_tokens, M, 0, mask_id, exclude_mask_column,
-                               pred, conf, static_cast<cudaStream_t>(stream));
+                               pred, conf, static_cast<cudaStream_t>(stream), nullptr);
 }
 

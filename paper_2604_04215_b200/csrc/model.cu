@@ -91,7 +91,7 @@ int step_rows(dare_model* m, int32_t* tokens, int B, int64_t row_stride, int sta
     if (rc != DARE_OK) return rc;
     const int M = B * L;
     rc = dare::launch_lmhead(m->ctx, m->ctx->workspace, m->h, M, m->desc.hidden, m->lm_head, m->desc.vocab,
-                             tokens + start, L, row_stride, m->desc.mask_id, 1, pred, conf, s);
+                             tokens + start, L, row_stride, m->desc.mask_id, 1, pred, conf, s, nullptr);
     if (rc != DARE_OK) return rc;
     return dare::launch_unmask_select(tokens, B, row_stride, start, L, pred, conf, m->desc.mask_id, mode, threshold, k,
                                       n_committed, n_remaining, s);
@@ -103,7 +103,7 @@ int check_step(const dare_model* m, int B, int L, int mode, float threshold, int
     if (mode != DARE_SELECT_THRESHOLD && mode != DARE_SELECT_TOPK) return DARE_ERR_RANGE;
     if (mode == DARE_SELECT_THRESHOLD && threshold != threshold) return DARE_ERR_RANGE;
     if (mode == DARE_SELECT_TOPK && k < 1) return DARE_ERR_RANGE;
-    if (dare::lmhead_workspace_bytes(B * L, m->desc.hidden, m->desc.vocab, m->ctx->sm_count, true) > m->ctx->workspace_bytes)
+    if (dare::lmhead_workspace_bytes(B * L, m->desc.hidden, m->desc.vocab, m->ctx->sm_count, true, false) > m->ctx->workspace_bytes)
         return DARE_ERR_WORKSPACE;
     return DARE_OK;
 }
