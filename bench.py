@@ -245,8 +245,21 @@ def run_ours(args):
         float(np.mean([wl.prompt_len + ((t % steps_per_gen) // steps_per_block) * L + L for t in range(n_inst)])) + wl.suffix_cap)
     qo_bytes = 2.0 * 2 * B * L * wl.n_q_heads * wl.head_dim
     attn_gbs = (kv_bytes + qo_bytes) / (attn_ms * 1e-3) / 1e9
+    # greedy against sampled head with every row masked (the sampling epilogue draws M * V Gumbel variates)
+    full_ms = {}
+    for name, fn in (("lmhead_all_rows_ms", lambda: dare.dare_lmhead_confidence(ctx, pool[0][1], w, None, wl.mask_id, True, pred, conf, stream=stream)),
+                     ("lmhead_sample_all_rows_ms", lambda: dare.dare_lmhead_sample(ctx, pool[0][1], w, None, wl.mask_id, True, 1.0, 1, 1, pred, conf, stream=stream))):
+        for _ in range(2):
+            fn()
+        es = [torch.cuda.Event(enable_timing=True) for _ in range(9)]
+        es[0].record(stream)
+        for i in range(8):
+            fn()
+            es[i + 1].record(stream)
+        torch.cuda.synchronize()
+        full_ms[name] = float(np.median([es[i].elapsed_time(es[i + 1]) for i in range(8)]))
     breakdown = {"attn_ms": attn_ms, "lmhead_ms": lm_ms, "select_ms": sel_ms, "attn_GBps": attn_gbs,
-                 "attn_frac_hbm": attn_gbs / peaks["hbm_gbs"]}
+                 "attn_frac_hbm": attn_gbs / peaks["hbm_gbs"], **full_ms}
 
     # ---- end to end: the step's activations come from pinned host memory, results go back to the host
     n_e2e = min(args.steps, 4 * steps_per_gen)
