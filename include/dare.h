@@ -136,6 +136,22 @@ int dare_lmhead_sample(dare_ctx* ctx,
                        int32_t* pred, float* conf, void* stream);
 
 /*
+ * Logits-free log-probability of given tokens (the idea the paper cites for its fused loss kernels, Section 3.4;
+ * the rollout's old / reference log-probabilities and the likelihood estimators of Section 4.2 need exactly
+ * this): for each row m
+ *     logprob[m] = z[targets[m]] - logsumexp z,      z = hidden[m] . w^T,  z[mask_id] = -inf if exclude_mask_column
+ * with the logits kept on chip as in dare_lmhead_confidence.  -logprob is the row's cross-entropy.
+ *
+ *   targets   int32 [M]: a target outside [0, V) (or the excluded column) gives logprob = -inf
+ *   logprob   fp32 [M] out          lse  fp32 [M] out or NULL: logsumexp z
+ * Every row is evaluated.  Workspace and limits as dare_lmhead_confidence without row_tokens.
+ */
+int dare_lmhead_logprob(dare_ctx* ctx,
+                        const void* hidden, int M, int D, const void* w, int V,
+                        const int32_t* targets, int32_t mask_id, int exclude_mask_column,
+                        float* logprob, float* lse, void* stream);
+
+/*
  * Parallel unmask selection, in place on the token state (Section 3.4, "partially fixed states";
  * Section 4.2: block length 32, two tokens per step).  Per row, U = block positions whose token is
  * mask_id.  THRESHOLD: commit every i in U with conf > threshold, or the single most confident one

@@ -131,6 +131,27 @@ def lmhead_confidence(x, w, row_tokens=None, mask_id=-1, exclude_mask_column=Tru
     return {"pred": pred, "conf": conf, "logconf": logconf, "second": second, "gap_logit": gap_logit}
 
 
+def lmhead_logprob(x, w, targets, mask_id=-1, exclude_mask_column=False):
+    """Log-probability of given tokens under the LM head's softmax, per row (Section 3.4: logits-free loss).
+
+    x [M, D], w [V, D] float64; targets int [M].  z = x w^T; the mask id's logit is -inf if
+    ``exclude_mask_column``; logprob[m] = z[m, targets[m]] - logsumexp z[m].  A target outside [0, V) (or the
+    excluded column) gives -inf.  Returns (logprob float64 [M], lse float64 [M]).
+    """
+    x = np.asarray(x, dtype=np.float64)
+    w = np.asarray(w, dtype=np.float64)
+    M, V = x.shape[0], w.shape[0]
+    z = x @ w.T
+    if exclude_mask_column and 0 <= mask_id < V:
+        z[:, mask_id] = -np.inf
+    zmax = z.max(axis=1)
+    lse = zmax + np.log(np.exp(z - zmax[:, None]).sum(axis=1))
+    t = np.asarray(targets)
+    ok = (t >= 0) & (t < V)
+    zt = np.where(ok, z[np.arange(M), np.where(ok, t, 0)], -np.inf)
+    return zt - lse, lse
+
+
 def token_probability(x_row, w, token, mask_id=-1, exclude_mask_column=True):
     """Softmax probability of one given token for one row (used to judge near-ties)."""
     z = np.asarray(w, dtype=np.float64) @ np.asarray(x_row, dtype=np.float64)

@@ -22,7 +22,7 @@ DEV_WAIT_EXPIRED = 2
 
 EXPORTS = ["dare_create", "dare_destroy", "dare_status_string", "dare_device_status", "dare_sm_count",
            "dare_attn_block", "dare_lmhead_confidence", "dare_unmask_select", "dare_denoise_block",
-           "dare_lmhead_confidence_static", "dare_lmhead_sample", "dare_model_create", "dare_model_destroy", "dare_model_forward",
+           "dare_lmhead_confidence_static", "dare_lmhead_sample", "dare_lmhead_logprob", "dare_model_create", "dare_model_destroy", "dare_model_forward",
            "dare_model_step", "dare_generate", "dare_linear", "dare_linear_plan", "dare_rmsnorm", "dare_rope_kv_write"]
 
 _lib = None
@@ -64,6 +64,8 @@ def load():
     lib.dare_lmhead_confidence_static.restype = i32
     lib.dare_lmhead_sample.argtypes = [vp, vp, i32, i32, vp, i32, vp, i32, i32, f32, C.c_uint64, C.c_uint32, vp, vp, vp]
     lib.dare_lmhead_sample.restype = i32
+    lib.dare_lmhead_logprob.argtypes = [vp, vp, i32, i32, vp, i32, vp, i32, i32, vp, vp, vp]
+    lib.dare_lmhead_logprob.restype = i32
     lib.dare_unmask_select.argtypes = [vp, vp, i32, i64, i32, i32, vp, vp, i32, i32, f32, i32, vp, vp, vp]
     lib.dare_unmask_select.restype = i32
     lib.dare_denoise_block.argtypes = ([vp] + [i32] * 7 + [f32] + [vp] * 11 +   # attention operands .. lse
@@ -207,6 +209,20 @@ def dare_lmhead_sample(ctx: Context, hidden, w, row_tokens=None, mask_id: int = 
     if rc != 0 and check:
         raise DareError(rc, "dare_lmhead_sample")
     return (pred, conf) if check else rc
+
+
+def dare_lmhead_logprob(ctx: Context, hidden, w, targets, mask_id: int = -1, exclude_mask_column: bool = False,
+                        logprob=None, lse=None, stream=None, check: bool = True):
+    M, D = hidden.shape
+    V = w.shape[0]
+    if logprob is None:
+        logprob = torch.empty(M, dtype=torch.float32, device=hidden.device)
+    rc = load().dare_lmhead_logprob(ctx.handle, _ptr(hidden, torch.bfloat16), M, D, _ptr(w, torch.bfloat16), V,
+                                    _ptr(targets, torch.int32), int(mask_id), int(bool(exclude_mask_column)),
+                                    _ptr(logprob, torch.float32), _ptr(lse, torch.float32), _stream(stream))
+    if rc != 0 and check:
+        raise DareError(rc, "dare_lmhead_logprob")
+    return logprob if check else rc
 
 
 LMHEAD_STATIC_SCRATCH_BYTES = 8 << 20

@@ -168,6 +168,15 @@ int dare_lmhead_confidence(dare_ctx* ctx, const void* hidden, int M, int D, cons
                                pred, conf, static_cast<cudaStream_t>(stream), nullptr);
 }
 
+int dare_lmhead_logprob(dare_ctx* ctx, const void* hidden, int M, int D, const void* w, int V, const int32_t* targets,
+                        int32_t mask_id, int exclude_mask_column, float* logprob, float* lse, void* stream) {
+    if (!targets) return DARE_ERR_NULL;
+    int rc = check_lmhead(ctx, hidden, M, D, w, V, false, targets, logprob);
+    if (rc != DARE_OK) return rc;
+    return dare::launch_lmhead_logprob(ctx, ctx->workspace, hidden, M, D, w, V, targets, mask_id, exclude_mask_column,
+                                       logprob, lse, static_cast<cudaStream_t>(stream));
+}
+
 int dare_lmhead_sample(dare_ctx* ctx, const void* hidden, int M, int D, const void* w, int V, const int32_t* row_tokens,
                        int32_t mask_id, int exclude_mask_column, float temperature, uint64_t seed, uint32_t step,
                        int32_t* pred, float* conf, void* stream) {

@@ -32,6 +32,10 @@ int launch_unmask_select(int32_t* tokens, int B, int64_t row_stride, int block_s
                          const float* conf, int32_t mask_id, int mode, float threshold, int k, int32_t* n_committed,
                          int32_t* n_remaining, cudaStream_t stream);
 
+// log p(target) per row = z_target - logsumexp z (and optionally logsumexp z); logits never stored.
+int launch_lmhead_logprob(const dare_ctx* ctx, void* scratch, const void* hidden, int M, int D, const void* w, int V,
+                          const int32_t* targets, int32_t mask_id, int exclude_mask_column, float* logprob, float* lse_out,
+                          cudaStream_t stream);
 // Sampling epilogue of the LM head (NULL = greedy): temperature, 64-bit seed and step counter of the generator.
 struct LmSampleArgs { float temperature; uint64_t seed; uint32_t step; };
 size_t lmhead_workspace_bytes(int M, int D, int V, int sm_count, bool with_row_tokens, bool sampling);

@@ -109,6 +109,7 @@ struct LmSampling {
     float inv_temperature;
     uint32_t seed_lo, seed_hi, step;
     const int32_t* row_index;      // original row of compacted row c (NULL: identity): keys the generator
+    const int32_t* targets;        // LM_LOGPROB: target token per row
     float* part_y;                 // per partial: best perturbed score and the raw logit there
     float* part_zb;
 };
@@ -129,12 +130,18 @@ __device__ __forceinline__ float gumbel_from_word(uint32_t w) {
     return -logf(-logf(u));
 }
 
-template <bool SAMPLE>
+// MODE 0: greedy (argmax token, its probability); 1: sampling epilogue; 2: log-probability of a given target
+// token per row (the partial's third slot then carries the target's logit instead of an argmax).
+constexpr int LM_GREEDY = 0, LM_SAMPLE = 1, LM_LOGPROB = 2;
+
+template <int MODE>
 __global__ void __launch_bounds__(LM_THREADS, 1)
 lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                       int M, const int32_t* __restrict__ live_rows, int D, int V, int mask_col, int n_tiles,
                       float* __restrict__ part_max, float* __restrict__ part_sum, int32_t* __restrict__ part_arg,
                       uint32_t* __restrict__ dev_status, const LmSampling smp) {
+    constexpr bool SAMPLE = MODE == LM_SAMPLE;
+    constexpr bool LOGPROB = MODE == LM_LOGPROB;
     const int Mc = live_rows ? *live_rows : M;          // rows that need logits (uniform over the grid)
     const int m_tiles = (Mc + BM - 1) / BM;
     if (m_tiles == 0) return;
@@ -246,6 +253,12 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
                 const int row_c = m_tile * BM + row_in_tile;
                 rng_row = static_cast<uint32_t>(row_c < Mc && smp.row_index ? smp.row_index[row_c] : row_c);
             }
+            int target = -1;                                     // LOGPROB: this row's target column, its logit
+            float target_z = -INFINITY;
+            if (LOGPROB) {
+                const int row_c = m_tile * BM + row_in_tile;
+                if (row_c < Mc) target = smp.targets[row_c];
+            }
             for (int n_tile = group; n_tile < n_tiles && ok; n_tile += groups, ++it) {
                 const int acc = it & 1;
                 const uint32_t acc_phase = (it >> 1) & 1;
@@ -274,6 +287,11 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
                         const float z = __uint_as_float(v[j]);
                         if (z > cmax) { cmax = z; carg = cbase + j; }   // strict '>' keeps the lowest index
                     }
+                    if (LOGPROB && target >= cbase && target < cbase + 32) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (cbase + j == target) target_z = __uint_as_float(v[j]);   // (-inf if it is the excluded column)
+                    }
                     if (SAMPLE) {
 #pragma unroll
                         for (int q = 0; q < 8; ++q) {
@@ -292,7 +310,7 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
                         if (cmax > run_max) {   // tiles of a group come in ascending order: '>' keeps the lowest id
                             run_sum *= fast_exp2((run_max - cmax) * LOG2E);   // exp2(-inf) = 0 the first time
                             run_max = cmax;
-                            if (!SAMPLE) run_arg = carg;
+                            if (MODE == LM_GREEDY) run_arg = carg;
                         }
                         const float mb = run_max * LOG2E;
                         float s = 0.f;
@@ -309,7 +327,7 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
                 const size_t o = static_cast<size_t>(row) * groups + group;
                 part_max[o] = run_max;
                 part_sum[o] = run_sum;
-                part_arg[o] = run_arg;
+                part_arg[o] = LOGPROB ? __float_as_int(target_z) : run_arg;
                 if (SAMPLE) { smp.part_y[o] = best_y; smp.part_zb[o] = best_z; }
             }
         }
@@ -416,6 +434,41 @@ __global__ void lmhead_merge_sample_kernel(const float* __restrict__ part_max, c
     }
 }
 
+// Log-probability of the target: (z_target - max) - ln(sum of exp(z - max)); the target's logit sits in exactly one
+// partial (the others carry -inf).  Optionally also writes logsumexp z.
+__global__ void lmhead_merge_logprob_kernel(const float* __restrict__ part_max, const float* __restrict__ part_sum,
+                                            const int32_t* __restrict__ part_zt, int grid_gemm, int n_tiles, int M,
+                                            float* __restrict__ logprob, float* __restrict__ lse_out) {
+    const int c = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (c >= M) return;
+    const int groups = lm_groups(grid_gemm, (M + BM - 1) / BM, n_tiles);
+    float m = -INFINITY, s = 0.f, zt = -INFINITY;
+    const size_t base = static_cast<size_t>(c) * groups;
+    for (int t = lane; t < groups; t += 32) {
+        const float m2 = part_max[base + t], s2 = part_sum[base + t];
+        if (m2 > -INFINITY) {
+            if (m2 > m) { s = s * exp2f((m - m2) * LOG2E) + s2; m = m2; }
+            else s += s2 * exp2f((m2 - m) * LOG2E);
+        }
+        zt = fmaxf(zt, __int_as_float(part_zt[base + t]));
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const float m2 = __shfl_xor_sync(0xffffffffu, m, off);
+        const float s2 = __shfl_xor_sync(0xffffffffu, s, off);
+        zt = fmaxf(zt, __shfl_xor_sync(0xffffffffu, zt, off));
+        if (m2 > -INFINITY) {
+            if (m2 > m) { s = s * exp2f((m - m2) * LOG2E) + s2; m = m2; }
+            else s += s2 * exp2f((m2 - m) * LOG2E);
+        }
+    }
+    if (lane == 0) {
+        logprob[c] = (zt - m) - logf(s);
+        if (lse_out) lse_out[c] = m + logf(s);
+    }
+}
+
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 }  // namespace
@@ -472,10 +525,10 @@ int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M,
     const int rows_per_block = 8;
     LmSampling smp = {};
     if (sample == nullptr) {
-        if (cudaFuncSetAttribute(lmhead_partial_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(lmhead_partial_kernel<LM_GREEDY>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  LM_SMEM_BYTES) != cudaSuccess)
             return DARE_ERR_CUDA;
-        lmhead_partial_kernel<false><<<grid, LM_THREADS, LM_SMEM_BYTES, stream>>>(
+        lmhead_partial_kernel<LM_GREEDY><<<grid, LM_THREADS, LM_SMEM_BYTES, stream>>>(
             tmap_x, tmap_w, M, live_rows, D, V, mask_col, n_tiles, part_max, part_sum, part_arg, ctx->dev_status, smp);
         if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
         lmhead_merge_kernel<<<(M + rows_per_block - 1) / rows_per_block, rows_per_block * 32, 0, stream>>>(
@@ -488,10 +541,10 @@ int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M,
         smp.row_index = idx;
         smp.part_y = reinterpret_cast<float*>(part_arg + n_part);
         smp.part_zb = smp.part_y + n_part;
-        if (cudaFuncSetAttribute(lmhead_partial_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(lmhead_partial_kernel<LM_SAMPLE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  LM_SMEM_BYTES) != cudaSuccess)
             return DARE_ERR_CUDA;
-        lmhead_partial_kernel<true><<<grid, LM_THREADS, LM_SMEM_BYTES, stream>>>(
+        lmhead_partial_kernel<LM_SAMPLE><<<grid, LM_THREADS, LM_SMEM_BYTES, stream>>>(
             tmap_x, tmap_w, M, live_rows, D, V, mask_col, n_tiles, part_max, part_sum, part_arg, ctx->dev_status, smp);
         if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
         lmhead_merge_sample_kernel<<<(M + rows_per_block - 1) / rows_per_block, rows_per_block * 32, 0, stream>>>(
@@ -499,6 +552,39 @@ int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M,
     }
     if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
     return DARE_OK;
+}
+
+int launch_lmhead_logprob(const dare_ctx* ctx, void* scratch, const void* hidden, int M, int D, const void* w, int V,
+                          const int32_t* targets, int32_t mask_id, int exclude_mask_column, float* logprob, float* lse_out,
+                          cudaStream_t stream) {
+    const int n_tiles = (V + BN - 1) / BN;
+    const int m_tiles_max = (M + BM - 1) / BM;
+    int grid = ctx->sm_count;
+    if (grid > m_tiles_max * n_tiles) grid = m_tiles_max * n_tiles;
+    size_t groups_max = static_cast<size_t>(ctx->sm_count);
+    if (groups_max > static_cast<size_t>(n_tiles)) groups_max = n_tiles;
+    const size_t n_part = static_cast<size_t>(M) * groups_max;
+    float* part_max = static_cast<float*>(scratch);
+    float* part_sum = part_max + n_part;
+    int32_t* part_zt = reinterpret_cast<int32_t*>(part_sum + n_part);
+    CUtensorMap tmap_x, tmap_w;
+    int rc = make_tmap_bf16_2d(ctx, &tmap_x, hidden, static_cast<uint64_t>(M), static_cast<uint64_t>(D), BM, BK);
+    if (rc != DARE_OK) return rc;
+    rc = make_tmap_bf16_2d(ctx, &tmap_w, w, static_cast<uint64_t>(V), static_cast<uint64_t>(D), BN, BK);
+    if (rc != DARE_OK) return rc;
+    if (cudaFuncSetAttribute(lmhead_partial_kernel<LM_LOGPROB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             LM_SMEM_BYTES) != cudaSuccess)
+        return DARE_ERR_CUDA;
+    const int mask_col = (exclude_mask_column && mask_id >= 0 && mask_id < V) ? mask_id : -1;
+    LmSampling smp = {};
+    smp.targets = targets;
+    lmhead_partial_kernel<LM_LOGPROB><<<grid, LM_THREADS, LM_SMEM_BYTES, stream>>>(
+        tmap_x, tmap_w, M, nullptr, D, V, mask_col, n_tiles, part_max, part_sum, part_zt, ctx->dev_status, smp);
+    if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
+    const int rows_per_block = 8;
+    lmhead_merge_logprob_kernel<<<(M + rows_per_block - 1) / rows_per_block, rows_per_block * 32, 0, stream>>>(
+        part_max, part_sum, part_zt, grid, n_tiles, M, logprob, lse_out);
+    return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
 }
 
 }  // namespace dare

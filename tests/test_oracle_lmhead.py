@@ -99,3 +99,31 @@ def test_confidence_bounds_and_token_probability():
         assert abs(O.token_probability(x[m], w, int(r["pred"][m]), mu, True) - r["conf"][m]) < 1e-14
         tot = sum(O.token_probability(x[m], w, v, mu, True) for v in range(V))
         assert abs(tot - 1.0) < 1e-12
+
+
+def test_logprob_is_library_log_softmax_gather_and_cross_entropy():
+    """lmhead_logprob against torch: log_softmax + gather, and -cross_entropy; closed forms; exclusion; bad targets."""
+    rng = np.random.default_rng(11)
+    M, D, V = 13, 24, 97
+    x, w = rng.standard_normal((M, D)), rng.standard_normal((V, D))
+    t = rng.integers(0, V, M)
+    lp, lse = O.lmhead_logprob(x, w, t)
+    z = torch.from_numpy(x) @ torch.from_numpy(w).T
+    want = torch.log_softmax(z, dim=1).gather(1, torch.from_numpy(t)[:, None])[:, 0].numpy()
+    np.testing.assert_allclose(lp, want, atol=1e-12)
+    np.testing.assert_allclose(-lp, torch.nn.functional.cross_entropy(z, torch.from_numpy(t), reduction="none").numpy(), atol=1e-12)
+    np.testing.assert_allclose(lse, torch.logsumexp(z, dim=1).numpy(), atol=1e-12)
+    # identical weight rows: every token has probability 1 / V (1 / (V - 1) with one column excluded)
+    w1 = np.tile(rng.standard_normal((1, D)), (V, 1))
+    np.testing.assert_allclose(O.lmhead_logprob(x, w1, t)[0], -np.log(V), atol=1e-12)
+    t2 = np.where(t == 5, 6, t)
+    np.testing.assert_allclose(O.lmhead_logprob(x, w1, t2, 5, True)[0], -np.log(V - 1), atol=1e-12)
+    # the excluded column and out-of-range targets have probability zero
+    bad = np.array([5, -1, V, 3])
+    lpb, _ = O.lmhead_logprob(x[:4], w, bad, 5, True)
+    assert np.isneginf(lpb[:3]).all() and np.isfinite(lpb[3])
+    # exp(logprob) summed over all targets is 1; consistent with the greedy head's confidence
+    allp = np.stack([np.exp(O.lmhead_logprob(x[:2], w, np.full(2, v))[0]) for v in range(V)], axis=1)
+    np.testing.assert_allclose(allp.sum(axis=1), 1.0, atol=1e-12)
+    g = O.lmhead_confidence(x, w, None, -1, False)
+    np.testing.assert_allclose(np.exp(O.lmhead_logprob(x, w, g["pred"])[0]), g["conf"], rtol=1e-12)
