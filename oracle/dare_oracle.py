@@ -92,6 +92,37 @@ def attn_block(q, k_pre, v_pre, prefix_len, k_blk=None, v_blk=None,
     return out, lse
 
 
+def attn_varlen(q, k, v, cu_seqlens, scale=None):
+    """Bidirectional attention over packed variable-length sequences (Section 3.4, training-side and log-prob
+    passes: sequences are concatenated without padding and each attends to itself only).
+
+    q [T, Hq, d]; k, v [T, Hkv, d] float64 with T = total tokens; cu_seqlens int [n + 1], sequence s owns tokens
+    [cu_seqlens[s], cu_seqlens[s + 1]).  Query head h reads KV head h // (Hq / Hkv); every token of a sequence
+    sees every token of the same sequence.  Returns (o [T, Hq, d], lse [Hq, T]).
+    """
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    T, Hq, d = q.shape
+    g = Hq // k.shape[1]
+    if scale is None:
+        scale = 1.0 / np.sqrt(d)
+    out = np.zeros_like(q)
+    lse = np.full((Hq, T), -np.inf)
+    for s in range(len(cu_seqlens) - 1):
+        a, b = int(cu_seqlens[s]), int(cu_seqlens[s + 1])
+        if b <= a:
+            continue
+        for h in range(Hq):
+            sc = scale * (q[a:b, h] @ k[a:b, h // g].T)
+            m = sc.max(axis=1, keepdims=True)
+            e = np.exp(sc - m)
+            den = e.sum(axis=1, keepdims=True)
+            out[a:b, h] = (e / den) @ v[a:b, h // g]
+            lse[h, a:b] = (m + np.log(den))[:, 0]
+    return out, lse
+
+
 def lmhead_confidence(x, w, row_tokens=None, mask_id=-1, exclude_mask_column=True):
     """LM head + vocabulary softmax -> greedy token and its probability, per masked row.
 

@@ -165,3 +165,37 @@ def test_split_merge_of_partial_softmax_matches_unsplit():
     merged = (o1 * w1 + o2 * w2) / (w1 + w2)
     np.testing.assert_allclose(merged, o, atol=1e-13)
     np.testing.assert_allclose((m + np.log(w1 + w2))[..., 0], np.transpose(lse, (0, 2, 1)), atol=1e-13)
+
+
+def test_varlen_is_block_diagonal_library_attention_and_per_sequence_block_attention():
+    """attn_varlen against torch attention over the packed tokens with a block-diagonal mask, and against
+    attn_block run sequence by sequence (no prefix, the sequence as the in-place block)."""
+    rng = np.random.default_rng(21)
+    lens = [5, 1, 17, 0, 9]
+    cu = np.concatenate([[0], np.cumsum(lens)])
+    T, Hq, Hkv, d = int(cu[-1]), 6, 2, 8
+    q, k, v = rng.standard_normal((T, Hq, d)), rng.standard_normal((T, Hkv, d)), rng.standard_normal((T, Hkv, d))
+    o, lse = O.attn_varlen(q, k, v, cu)
+    seg = np.repeat(np.arange(len(lens)), lens)
+    mask = torch.from_numpy(seg[:, None] == seg[None, :])
+    tq = torch.from_numpy(q).permute(1, 0, 2)[None]
+    tk = torch.from_numpy(k).permute(1, 0, 2).repeat_interleave(Hq // Hkv, dim=0)[None]
+    tv = torch.from_numpy(v).permute(1, 0, 2).repeat_interleave(Hq // Hkv, dim=0)[None]
+    want = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, attn_mask=mask[None, None])[0].permute(1, 0, 2)
+    np.testing.assert_allclose(o, want.numpy(), atol=1e-12)
+    for s, n in enumerate(lens):
+        if n == 0:
+            continue
+        a, b = cu[s], cu[s + 1]
+        kc = np.transpose(k[a:b], (1, 0, 2))[None]
+        vc = np.transpose(v[a:b], (1, 0, 2))[None]
+        ob, lb = O.attn_block(q[a:b][None], kc, vc, np.array([0]))
+        np.testing.assert_allclose(o[a:b], ob[0], atol=1e-12)
+        np.testing.assert_allclose(lse[:, a:b], lb[0], atol=1e-12)
+    # a token of one sequence does not influence another sequence
+    k2 = k.copy()
+    k2[cu[2]] += 3.0
+    o2, _ = O.attn_varlen(q, k2, v, cu)
+    np.testing.assert_array_equal(o2[:cu[2]], o[:cu[2]])
+    np.testing.assert_array_equal(o2[cu[3]:], o[cu[3]:])
+    assert np.abs(o2[cu[2]:cu[3]] - o[cu[2]:cu[3]]).max() > 1e-3
