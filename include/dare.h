@@ -99,6 +99,22 @@ int dare_attn_block(dare_ctx* ctx,
                     void* out, float* lse, void* stream);
 
 /*
+ * Bidirectional attention over packed variable-length sequences (Section 3.4: the training-side and log-prob
+ * passes concatenate sequences without padding; each sequence attends to itself only).  Sequence s owns tokens
+ * [cu_seqlens[s], cu_seqlens[s + 1]); every token of a sequence sees every token of that sequence.
+ *
+ *   q    bf16 [total_tokens, Hq, d]      k, v  bf16 [total_tokens, Hkv, d]      out  bf16 [total_tokens, Hq, d]
+ *   cu_seqlens   int32 [n_seqs + 1], device, non-decreasing, cu_seqlens[0] = 0, cu_seqlens[n_seqs] = total_tokens
+ *   max_seqlen   host value >= the longest sequence (sizes the launch; longer sequences would be cut off)
+ *   lse          fp32 [Hq, total_tokens] or NULL
+ * Runs on the tcgen05 attention kernel.  Supported: d in {64, 128}; Hq % Hkv == 0, Hq / Hkv <= 128;
+ * n_seqs * Hkv <= 65535.  Empty sequences are allowed.
+ */
+int dare_attn_varlen(dare_ctx* ctx, int total_tokens, int n_seqs, int max_seqlen, int Hq, int Hkv, int d, float scale,
+                     const void* q, const void* k, const void* v, const int32_t* cu_seqlens,
+                     void* out, float* lse, void* stream);
+
+/*
  * Fused LM head + vocabulary softmax (Section 3.4, the logits-free idea the paper cites for its fused
  * loss kernels, applied to decoding): for each row m,
  *     z = hidden[m] . w^T  (V logits, kept on chip);  z[mask_id] = -inf if exclude_mask_column;

@@ -21,7 +21,7 @@ DEV_LEN_CLAMPED = 1
 DEV_WAIT_EXPIRED = 2
 
 EXPORTS = ["dare_create", "dare_destroy", "dare_status_string", "dare_device_status", "dare_sm_count",
-           "dare_attn_block", "dare_lmhead_confidence", "dare_unmask_select", "dare_denoise_block",
+           "dare_attn_block", "dare_attn_varlen", "dare_lmhead_confidence", "dare_unmask_select", "dare_denoise_block",
            "dare_lmhead_confidence_static", "dare_lmhead_sample", "dare_lmhead_logprob", "dare_model_create", "dare_model_destroy", "dare_model_forward",
            "dare_model_step", "dare_generate", "dare_linear", "dare_linear_plan", "dare_rmsnorm", "dare_rope_kv_write"]
 
@@ -58,6 +58,8 @@ def load():
     attn_args = [i32] * 7 + [f32] + [vp] * 12
     lib.dare_attn_block.argtypes = [vp] + attn_args
     lib.dare_attn_block.restype = i32
+    lib.dare_attn_varlen.argtypes = [vp] + [i32] * 6 + [f32] + [vp] * 7
+    lib.dare_attn_varlen.restype = i32
     lib.dare_lmhead_confidence.argtypes = [vp, vp, i32, i32, vp, i32, vp, i32, i32, vp, vp, vp]
     lib.dare_lmhead_confidence.restype = i32
     lib.dare_lmhead_confidence_static.argtypes = [vp, i32, i32, vp, i32, vp, i32, i32, vp, vp, vp]
@@ -174,6 +176,21 @@ def dare_attn_block(ctx: Context, q, k_pre, v_pre, prefix_len=None, k_blk=None, 
                                 _stream(stream))
     if rc != 0 and check:
         raise DareError(rc, "dare_attn_block")
+    return out if check else rc
+
+
+def dare_attn_varlen(ctx: Context, q, k, v, cu_seqlens, max_seqlen: int, out=None, lse=None, scale: float = 0.0,
+                     stream=None, check: bool = True):
+    total, Hq, d = q.shape
+    Hkv = k.shape[1]
+    if out is None:
+        out = torch.empty_like(q)
+    bf = torch.bfloat16
+    rc = load().dare_attn_varlen(ctx.handle, total, cu_seqlens.numel() - 1, int(max_seqlen), Hq, Hkv, d, float(scale),
+                                 _ptr(q, bf), _ptr(k, bf), _ptr(v, bf), _ptr(cu_seqlens, torch.int32), _ptr(out, bf),
+                                 _ptr(lse, torch.float32), _stream(stream))
+    if rc != 0 and check:
+        raise DareError(rc, "dare_attn_varlen")
     return out if check else rc
 
 

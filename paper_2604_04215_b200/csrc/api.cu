@@ -159,6 +159,20 @@ int dare_attn_block(dare_ctx* ctx, int B, int L, int Hq, int Hkv, int d, int pre
     return dare::launch_attn(ctx, a, static_cast<cudaStream_t>(stream));
 }
 
+int dare_attn_varlen(dare_ctx* ctx, int total_tokens, int n_seqs, int max_seqlen, int Hq, int Hkv, int d, float scale,
+                     const void* q, const void* k, const void* v, const int32_t* cu_seqlens, void* out, float* lse,
+                     void* stream) {
+    if (!ctx || !q || !k || !v || !cu_seqlens || !out) return DARE_ERR_NULL;
+    if (total_tokens < 1 || n_seqs < 1 || max_seqlen < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || Hq / Hkv > 128)
+        return DARE_ERR_SHAPE;
+    if (d != 64 && d != 128) return DARE_ERR_SHAPE;
+    if (static_cast<long long>(n_seqs) * Hkv > 65535) return DARE_ERR_SHAPE;
+    if (!(scale >= 0.f) || isinf(scale)) return DARE_ERR_RANGE;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return DARE_ERR_ALIGN;
+    return dare::launch_attn_varlen(ctx, total_tokens, n_seqs, max_seqlen, Hq, Hkv, d, scale, q, k, v, cu_seqlens, out, lse,
+                                    static_cast<cudaStream_t>(stream));
+}
+
 int dare_lmhead_confidence(dare_ctx* ctx, const void* hidden, int M, int D, const void* w, int V,
                            const int32_t* row_tokens, int32_t mask_id, int exclude_mask_column, int32_t* pred,
                            float* conf, void* stream) {

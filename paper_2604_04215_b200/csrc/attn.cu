@@ -30,6 +30,8 @@ struct AttnParams {
     int prefix_cap, suffix_cap;
     int inplace, has_suffix, splits;
     int uniform_P;                // >= 0: every row's prefix length (used when prefix_len is NULL)
+    const int32_t* cu_seqlens;    // packed variable-length mode (tcgen05 kernel): sequence b owns tokens [cu[b], cu[b+1])
+    int total_tokens;             // packed mode: rows of q / k / v
     float scale_log2;
     const __nv_bfloat16* q;
     const int32_t* prefix_len;
@@ -440,6 +442,13 @@ attn_block_tc_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_c
     const int b = unit / p.Hkv;
     const int kvh = unit % p.Hkv;
     const int pos_per_tile = 128 / p.g;            // block positions per query tile
+    // Packed variable-length mode: "rollout" b is sequence b of the packed token list; its tokens are both the
+    // queries (a block of L_eff positions, no prefix) and, in place, the keys.  K and V are [tokens, Hkv * D].
+    const bool packed = p.cu_seqlens != nullptr;
+    const int seq_base = packed ? p.cu_seqlens[b] : 0;
+    const int L_eff = packed ? p.cu_seqlens[b + 1] - seq_base : p.L;
+    if (static_cast<int>(blockIdx.x) * QT * pos_per_tile >= L_eff) return;   // (whole CTA, before anything is set up)
+    const int kv_col0 = packed ? kvh * D : 0;      // first column of this KV head in the 2-D view of K / V
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -471,18 +480,18 @@ attn_block_tc_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_c
                          : (p.uniform_P >= 0 ? p.uniform_P : (p.inplace ? p.prefix_cap - p.L : p.prefix_cap));
     const int p_max = p.inplace ? p.prefix_cap - p.L : p.prefix_cap;
     int Sx = p.has_suffix ? (p.suffix_len ? p.suffix_len[b] : p.suffix_cap) : 0;
-    if (P < 0 || P > p_max || Sx < 0 || Sx > p.suffix_cap) {
+    if (!packed && (P < 0 || P > p_max || Sx < 0 || Sx > p.suffix_cap)) {
         P = max(0, min(P, p_max));
         Sx = max(0, min(Sx, p.suffix_cap));
         if (threadIdx.x == 0) atomicOr(p.dev_status, DEV_LEN_CLAMPED);
     }
-    const int len_pre = p.inplace ? P + p.L : P;
-    const int len_blk = p.inplace ? 0 : p.L;
+    const int len_pre = packed ? L_eff : (p.inplace ? P + p.L : P);
+    const int len_blk = (packed || p.inplace) ? 0 : p.L;
     const int n_pre = (len_pre + TC_KT - 1) / TC_KT;
     const int n_blk = (len_blk + TC_KT - 1) / TC_KT;
     const int n_suf = (Sx + TC_KT - 1) / TC_KT;
     const int n_tiles = n_pre + n_blk + n_suf;
-    const int base_pre = unit * p.prefix_cap;
+    const int base_pre = packed ? seq_base : unit * p.prefix_cap;
     const int base_blk = unit * p.L;
     const int base_suf = unit * p.suffix_cap;
 
@@ -502,8 +511,8 @@ attn_block_tc_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_c
                 mbar_arrive_expect_tx(&bars->full[stage], 2 * KV_BYTES);
 #pragma unroll
                 for (int h = 0; h < NHALF; ++h) {
-                    tma_load_2d(kdst + h * HALF_K, mk, &bars->full[stage], h * 64, ti.row0);
-                    tma_load_2d(vdst + h * HALF_K, mv, &bars->full[stage], h * 64, ti.row0);
+                    tma_load_2d(kdst + h * HALF_K, mk, &bars->full[stage], kv_col0 + h * 64, ti.row0);
+                    tma_load_2d(vdst + h * HALF_K, mv, &bars->full[stage], kv_col0 + h * 64, ti.row0);
                 }
                 if (++stage == STAGES) { stage = 0; phase ^= 1; }
             }
@@ -566,8 +575,9 @@ attn_block_tc_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_c
         const int rows_in_tile = pos_per_tile * p.g;
         const int i = (blockIdx.x * QT + j) * pos_per_tile + r / p.g;   // block position
         const int h = kvh * p.g + r % p.g;                              // query head
-        const bool live = r < rows_in_tile && i < p.L;
-        const size_t qrow = ((static_cast<size_t>(b) * p.L + (live ? i : 0)) * p.Hq + (live ? h : 0)) * D;
+        const bool live = r < rows_in_tile && i < L_eff;
+        const size_t q_token = packed ? static_cast<size_t>(seq_base) : static_cast<size_t>(b) * p.L;   // first token of b
+        const size_t qrow = ((q_token + (live ? i : 0)) * p.Hq + (live ? h : 0)) * D;
         // Q row -> shared memory, K-major with the 128-byte swizzle (16-byte chunk c of row r sits at c ^ (r & 7))
         {
             const uint4* src = reinterpret_cast<const uint4*>(p.q + qrow);
@@ -689,7 +699,8 @@ attn_block_tc_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_c
             }
         }
         if (ok && live && p.lse != nullptr)
-            p.lse[(static_cast<size_t>(b) * p.Hq + h) * p.L + i] = l > 0.f ? (m_ref + log2f(l)) * LN2_F : -INFINITY;
+            p.lse[packed ? static_cast<size_t>(h) * p.total_tokens + seq_base + i
+                         : (static_cast<size_t>(b) * p.Hq + h) * p.L + i] = l > 0.f ? (m_ref + log2f(l)) * LN2_F : -INFINITY;
     }
 
     // teardown
@@ -806,6 +817,7 @@ int launch_attn(const dare_ctx* ctx, const AttnArgs& a, cudaStream_t stream) {
     p.inplace = a.k_blk == nullptr; p.has_suffix = a.k_suf != nullptr && a.suffix_cap > 0;
     p.splits = attn_plan_splits(ctx, a);
     p.uniform_P = a.prefix_len_uniform;
+    p.cu_seqlens = nullptr; p.total_tokens = 0;
     const float scale = a.scale != 0.f ? a.scale : 1.0f / sqrtf(static_cast<float>(a.d));
     p.scale_log2 = scale * LOG2E_F;
     p.q = static_cast<const __nv_bfloat16*>(a.q);
@@ -866,6 +878,32 @@ int launch_attn(const dare_ctx* ctx, const AttnArgs& a, cudaStream_t stream) {
         if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
     }
     return DARE_OK;
+}
+
+// Packed variable-length bidirectional attention on the tcgen05 kernel: sequence s = "rollout" s, its tokens are the
+// queries and, in place, the keys; K and V are 2-D [tokens, Hkv * d] views, a KV head is a column range.
+int launch_attn_varlen(const dare_ctx* ctx, int total, int n_seqs, int max_seqlen, int Hq, int Hkv, int d, float scale,
+                       const void* q, const void* k, const void* v, const int32_t* cu_seqlens, void* out, float* lse,
+                       cudaStream_t stream) {
+    AttnParams p = {};
+    p.B = n_seqs; p.L = max_seqlen; p.Hq = Hq; p.Hkv = Hkv; p.g = Hq / Hkv; p.R = max_seqlen * p.g;
+    p.prefix_cap = 0; p.suffix_cap = 0; p.inplace = 1; p.has_suffix = 0; p.splits = 1; p.uniform_P = 0;
+    p.scale_log2 = (scale != 0.f ? scale : 1.0f / sqrtf(static_cast<float>(d))) * LOG2E_F;
+    p.q = static_cast<const __nv_bfloat16*>(q);
+    p.prefix_len = nullptr; p.suffix_len = nullptr;
+    p.out = static_cast<__nv_bfloat16*>(out); p.lse = lse;
+    p.part_o = nullptr; p.part_lse = nullptr;
+    p.dev_status = ctx->dev_status;
+    p.cu_seqlens = cu_seqlens; p.total_tokens = total;
+    CUtensorMap tm[6];
+    int rc = make_tmap_bf16_2d(ctx, &tm[0], k, static_cast<uint64_t>(total), static_cast<uint64_t>(Hkv) * d, TC_KT, 64);
+    if (rc == DARE_OK) rc = make_tmap_bf16_2d(ctx, &tm[1], v, static_cast<uint64_t>(total), static_cast<uint64_t>(Hkv) * d, TC_KT, 64);
+    if (rc != DARE_OK) return rc;
+    tm[2] = tm[0]; tm[3] = tm[1]; tm[4] = tm[0]; tm[5] = tm[1];
+    const int pos_per_tile = 128 / p.g;
+    const int q_tiles = (max_seqlen + pos_per_tile - 1) / pos_per_tile;
+    if (q_tiles >= 2) return d == 128 ? launch_tc<128, 2>(tm, p, q_tiles, stream) : launch_tc<64, 2>(tm, p, q_tiles, stream);
+    return d == 128 ? launch_tc<128, 1>(tm, p, q_tiles, stream) : launch_tc<64, 1>(tm, p, q_tiles, stream);
 }
 
 }  // namespace dare

@@ -60,6 +60,9 @@ struct AttnArgs {
 int attn_plan_splits(const dare_ctx* ctx, const AttnArgs& a);
 size_t attn_workspace_bytes(const AttnArgs& a, int splits);
 int launch_attn(const dare_ctx* ctx, const AttnArgs& a, cudaStream_t stream);
+int launch_attn_varlen(const dare_ctx* ctx, int total, int n_seqs, int max_seqlen, int Hq, int Hkv, int d, float scale,
+                       const void* q, const void* k, const void* v, const int32_t* cu_seqlens, void* out, float* lse,
+                       cudaStream_t stream);
 
 // ---- layer stack (gemm.cu, layers.cu)
 enum { GEMM_EPI_STORE = 0, GEMM_EPI_RESIDUAL = 1, GEMM_EPI_SWIGLU = 2 };
