@@ -263,26 +263,45 @@ def run_ours(args):
 
     # ---- end to end: the step's activations come from pinned host memory, results go back to the host
     n_e2e = min(args.steps, 4 * steps_per_gen)
-    q_d, x_d = torch.empty_like(pool[0][0]), torch.empty_like(pool[0][1])
+    # Double-buffered: a copy stream uploads step t + 1's activations while step t computes; every step still
+    # uploads its own inputs from pinned memory and the host reads the step's counts and tokens before going on.
+    bufs = [(torch.empty_like(pool[0][0]), torch.empty_like(pool[0][1])) for _ in range(2)]
     nc_h = torch.zeros(B, dtype=torch.int32).pin_memory()
     nr_h = torch.zeros(B, dtype=torch.int32).pin_memory()
     tok_blk_h = torch.zeros(B, L, dtype=torch.int32).pin_memory()
     nc_d = torch.zeros(B, dtype=torch.int32, device="cuda")
+    copy_stream = torch.cuda.Stream()
+    uploaded = [torch.cuda.Event(), torch.cuda.Event()]
+    consumed = [torch.cuda.Event(), torch.cuda.Event()]
+
+    def upload(t):
+        qh, xh = pool_h[t % NPOOL]
+        with torch.cuda.stream(copy_stream):
+            copy_stream.wait_event(consumed[t & 1])          # the step that last read this buffer has finished
+            bufs[t & 1][0].copy_(qh, non_blocking=True)
+            bufs[t & 1][1].copy_(xh, non_blocking=True)
+            uploaded[t & 1].record(copy_stream)
+
     barrier()
+    for ev_ in consumed:
+        ev_.record(stream)
     e2e_tokens = 0
     ta = time.perf_counter()
+    upload(0)
     for t in range(n_e2e):
-        qh, xh = pool_h[t % NPOOL]
-        q_d.copy_(qh, non_blocking=True)
-        x_d.copy_(xh, non_blocking=True)
-        step(t, q_d, x_d, nc_d)
+        if t + 1 < n_e2e:
+            upload(t + 1)
+        stream.wait_event(uploaded[t & 1])
+        step(t, bufs[t & 1][0], bufs[t & 1][1], nc_d)
+        consumed[t & 1].record(stream)
         g = t % steps_per_gen
         bs = wl.prompt_len + (g // steps_per_block) * L
         nc_h.copy_(nc_d, non_blocking=True)
         nr_h.copy_(nr, non_blocking=True)
         tok_blk_h.copy_(tokens[:, bs:bs + L], non_blocking=True)
-        torch.cuda.synchronize()
+        stream.synchronize()
         e2e_tokens += int(nc_h.sum())
+    torch.cuda.synchronize()
     tb = time.perf_counter()
     e2e_s, e2e_n = reduce_step_stats(tb - ta, e2e_tokens, device="cuda")
     h2d = pool_h[0][0].numel() * 2 + pool_h[0][1].numel() * 2
