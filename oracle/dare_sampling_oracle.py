@@ -127,3 +127,46 @@ def denoise_step_sampled(q, k_pre, v_pre, prefix_len, k_blk, v_blk, k_suf, v_suf
     tok, nc, nr = O.unmask_select(tokens, block_start, L, lm["pred"], lm["conf"].astype(np.float32), mask_id, mode,
                                   threshold, k)
     return {"attn_out": o, "lse": lse, "lm": lm, "tokens": tok, "n_committed": nc, "n_remaining": nr}
+
+
+# ---------------------------------------------------------------------------------------------------------
+# Forward (corruption) process and the Monte-Carlo likelihood bound that uses it.
+
+MASK_TAG = 0x4D41534B
+
+
+def forward_mask(x0, start, length, p_mask, mask_id, seed, sample):
+    """Eq. 1 (forward process with the absorbing <MASK> state): each token of the window [start, start + length)
+    of row b independently stays x_0 with probability alpha_t = 1 - p_mask[b] and becomes <MASK> otherwise;
+    tokens outside the window (the prompt) are kept.
+
+    The uniform of position i of row b is word i % 4 of Philox4x32-10(counter = (i // 4, b, sample, MASK_TAG),
+    key = seed), mapped to u = (2 k + 1) / 2^24 as in `uniforms`; the token is masked iff u < p_mask[b]
+    (compared in float32: u is exact there).  Returns a new int32 array.
+    """
+    x = np.array(x0, dtype=np.int32, copy=True)
+    B = x.shape[0]
+    key = np.array([seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF], dtype=np.uint32)
+    n4 = (length + 3) // 4
+    for b in range(B):
+        counter = np.zeros((n4, 4), dtype=np.uint32)
+        counter[:, 0] = np.arange(n4, dtype=np.uint32)
+        counter[:, 1] = np.uint32(b)
+        counter[:, 2] = np.uint32(sample)
+        counter[:, 3] = np.uint32(MASK_TAG)
+        words = philox4x32_10(counter, key).reshape(-1)[:length]
+        u = ((2.0 * (words >> np.uint32(9)).astype(np.float64) + 1.0) / 16777216.0).astype(np.float32)
+        hit = u < np.float32(p_mask[b])
+        x[b, start:start + length][hit] = mask_id
+    return x
+
+
+def masked_nelbo(logprob, xt, start, length, mask_id, t):
+    """Eq. 2, the per-sequence term of the negative evidence lower bound for one (x_t, t) draw:
+        nelbo[b] = -(1 / t[b]) * sum over window positions l with x_t[b, l] = <MASK> of log p(x_0[b, l] | x_t).
+    logprob float [B, length] holds log p(x_0^l | x_t) for every window position (entries at unmasked positions are
+    ignored).  Returns (nelbo float64 [B], n_masked int32 [B])."""
+    lp = np.asarray(logprob, dtype=np.float64).reshape(len(t), length)
+    m = np.asarray(xt)[:, start:start + length] == mask_id
+    s = np.where(m, lp, 0.0).sum(axis=1)
+    return -s / np.asarray(t, dtype=np.float64), m.sum(axis=1).astype(np.int32)

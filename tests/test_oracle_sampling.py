@@ -104,3 +104,45 @@ def test_low_temperature_recovers_the_greedy_head_and_rows_are_skipped():
     b = SO.lmhead_sample(x, w, None, 150, True, 1.0, seed=5, step=1)["pred"]
     assert (a != greedy["pred"]).any() and (a != b).any()
     assert (a != 150).all() and (b != 150).all()
+
+
+def test_forward_process_marginals_window_and_limits():
+    """Eq. 1: P(x_t = x_0) = alpha_t per token, independently; only the window is touched; limits p = 0 and p = 1."""
+    rng = np.random.default_rng(2)
+    B, T, start, length, mask_id = 6, 5000, 100, 4800, 99
+    x0 = rng.integers(0, 90, (B, T)).astype(np.int32)
+    p = np.array([0.0, 0.1, 0.5, 0.9, 1.0, 0.3], dtype=np.float32)
+    xt = SO.forward_mask(x0, start, length, p, mask_id, seed=5, sample=0)
+    np.testing.assert_array_equal(xt[:, :start], x0[:, :start])
+    np.testing.assert_array_equal(xt[:, start + length:], x0[:, start + length:])
+    win, win0 = xt[:, start:start + length], x0[:, start:start + length]
+    assert ((win == mask_id) | (win == win0)).all()                   # a token is either kept or absorbed
+    frac = (win == mask_id).mean(axis=1)
+    assert frac[0] == 0.0 and frac[4] == 1.0
+    assert np.abs(frac - p).max() < 4 * np.sqrt(0.25 / length)
+    # neighbouring positions are masked independently: P(both) = p^2
+    both = ((win[2, :-1] == mask_id) & (win[2, 1:] == mask_id)).mean()
+    assert abs(both - 0.25) < 0.03
+    # another Monte-Carlo sample or seed gives another pattern; the same arguments the same one
+    np.testing.assert_array_equal(xt, SO.forward_mask(x0, start, length, p, mask_id, 5, 0))
+    assert (SO.forward_mask(x0, start, length, p, mask_id, 5, 1) != xt).any()
+    assert (SO.forward_mask(x0, start, length, p, mask_id, 6, 0) != xt).any()
+    # a larger p masks a superset (same uniforms, higher threshold)
+    hi = SO.forward_mask(x0, start, length, np.minimum(p + 0.2, 1.0).astype(np.float32), mask_id, 5, 0)
+    assert ((xt == mask_id) <= (hi == mask_id)).all()
+
+
+def test_masked_nelbo_hand_worked():
+    """Eq. 2 on a hand-worked case: only masked window positions count, scaled by 1 / t."""
+    mask_id = 9
+    xt = np.array([[1, 9, 3, 9, 9, 2], [4, 4, 9, 4, 4, 4]], dtype=np.int32)
+    lp = np.log(np.array([[0.5, 0.25, 0.125, 0.5], [0.1, 0.2, 0.3, 0.4]]))         # window = positions 1..4
+    nelbo, n = SO.masked_nelbo(lp, xt, 1, 4, mask_id, np.array([0.5, 0.25]))
+    # row 0: window tokens 9 3 9 9 -> masked at window offsets 0, 2, 3: -(ln .5 + ln .125 + ln .5) / 0.5
+    # row 1: window tokens 4 9 4 4 -> masked at offset 1: -ln .2 / 0.25
+    np.testing.assert_allclose(nelbo, [2 * (np.log(2) + np.log(8) + np.log(2)), 4 * np.log(5)], rtol=1e-14)
+    np.testing.assert_array_equal(n, [3, 1])
+    # with every window token masked at t = 1 it is the summed cross-entropy
+    xt2 = np.full((2, 6), mask_id, dtype=np.int32)
+    nelbo2, _ = SO.masked_nelbo(lp, xt2, 1, 4, mask_id, np.array([1.0, 1.0]))
+    np.testing.assert_allclose(nelbo2, -lp.sum(axis=1), rtol=1e-14)
