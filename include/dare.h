@@ -168,6 +168,29 @@ int dare_lmhead_logprob(dare_ctx* ctx,
                         float* logprob, float* lse, void* stream);
 
 /*
+ * Forward (corruption) process, Eq. 1: q(x_t | x_0) = Cat(alpha_t x_0 + (1 - alpha_t) m) with m the <MASK> state.
+ * Every token of the window [start, start + length) of row b independently becomes mask_id with probability
+ * p_mask[b] = 1 - alpha_t and keeps its value otherwise; tokens outside the window (the prompt) are copied.
+ * The uniform of window position i of row b is output word i % 4 of Philox4x32-10 with key = seed and counter =
+ * (i / 4, b, sample, 0x4D41534B), mapped to u = (2 k + 1) / 2^24 from its top 23 bits; masked iff u < p_mask[b].
+ * `sample` numbers the Monte-Carlo draws (Section 4.2 uses 16 per sequence).
+ *   x0  int32 [B, row_stride] in      xt  int32 [B, row_stride] out (may be x0: in place; otherwise only the
+ *   window of xt is written)          p_mask  fp32 [B], device
+ */
+int dare_forward_mask(dare_ctx* ctx, const int32_t* x0, int32_t* xt, int B, int64_t row_stride, int start, int length,
+                      const float* p_mask, int32_t mask_id, uint64_t seed, uint32_t sample, void* stream);
+
+/*
+ * Per-sequence term of the negative evidence lower bound, Eq. 2, for one draw (x_t, t):
+ *     nelbo[b] = -(1 / t[b]) * sum over window positions l with x_t[b, l] = mask_id of logprob[b, l]
+ * with logprob[b, l] = log p(x_0[b, l] | x_t) as dare_lmhead_logprob returns it for the window's rows.
+ *   logprob  fp32 [B, length]     xt  int32 [B, row_stride]     t  fp32 [B] (device, > 0)
+ *   nelbo    fp32 [B] out         n_masked  int32 [B] out or NULL
+ */
+int dare_masked_nelbo(dare_ctx* ctx, const float* logprob, const int32_t* xt, int B, int64_t row_stride, int start,
+                      int length, int32_t mask_id, const float* t, float* nelbo, int32_t* n_masked, void* stream);
+
+/*
  * Parallel unmask selection, in place on the token state (Section 3.4, "partially fixed states";
  * Section 4.2: block length 32, two tokens per step).  Per row, U = block positions whose token is
  * mask_id.  THRESHOLD: commit every i in U with conf > threshold, or the single most confident one

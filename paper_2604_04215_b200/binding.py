@@ -22,7 +22,7 @@ DEV_WAIT_EXPIRED = 2
 
 EXPORTS = ["dare_create", "dare_destroy", "dare_status_string", "dare_device_status", "dare_sm_count",
            "dare_attn_block", "dare_attn_varlen", "dare_lmhead_confidence", "dare_unmask_select", "dare_denoise_block",
-           "dare_lmhead_confidence_static", "dare_lmhead_sample", "dare_lmhead_logprob", "dare_model_create", "dare_model_destroy", "dare_model_forward",
+           "dare_lmhead_confidence_static", "dare_lmhead_sample", "dare_lmhead_logprob", "dare_forward_mask", "dare_masked_nelbo", "dare_model_create", "dare_model_destroy", "dare_model_forward",
            "dare_model_step", "dare_generate", "dare_linear", "dare_linear_plan", "dare_rmsnorm", "dare_rope_kv_write"]
 
 _lib = None
@@ -68,6 +68,10 @@ def load():
     lib.dare_lmhead_sample.restype = i32
     lib.dare_lmhead_logprob.argtypes = [vp, vp, i32, i32, vp, i32, vp, i32, i32, vp, vp, vp]
     lib.dare_lmhead_logprob.restype = i32
+    lib.dare_forward_mask.argtypes = [vp, vp, vp, i32, i64, i32, i32, vp, i32, C.c_uint64, C.c_uint32, vp]
+    lib.dare_forward_mask.restype = i32
+    lib.dare_masked_nelbo.argtypes = [vp, vp, vp, i32, i64, i32, i32, i32, vp, vp, vp, vp]
+    lib.dare_masked_nelbo.restype = i32
     lib.dare_unmask_select.argtypes = [vp, vp, i32, i64, i32, i32, vp, vp, i32, i32, f32, i32, vp, vp, vp]
     lib.dare_unmask_select.restype = i32
     lib.dare_denoise_block.argtypes = ([vp] + [i32] * 7 + [f32] + [vp] * 11 +   # attention operands .. lse
@@ -240,6 +244,34 @@ def dare_lmhead_logprob(ctx: Context, hidden, w, targets, mask_id: int = -1, exc
     if rc != 0 and check:
         raise DareError(rc, "dare_lmhead_logprob")
     return logprob if check else rc
+
+
+def dare_forward_mask(ctx: Context, x0, start: int, length: int, p_mask, mask_id: int, seed: int, sample: int, xt=None,
+                      stream=None, check: bool = True):
+    """Eq. 1.  Returns xt (a fresh copy of x0 with the window corrupted unless xt is given; xt may be x0)."""
+    B, row_stride = x0.shape
+    if xt is None:
+        xt = x0.clone()
+    rc = load().dare_forward_mask(ctx.handle, _ptr(x0, torch.int32), _ptr(xt, torch.int32), B, row_stride, int(start),
+                                  int(length), _ptr(p_mask, torch.float32), int(mask_id), int(seed) & 0xFFFFFFFFFFFFFFFF,
+                                  int(sample) & 0xFFFFFFFF, _stream(stream))
+    if rc != 0 and check:
+        raise DareError(rc, "dare_forward_mask")
+    return xt if check else rc
+
+
+def dare_masked_nelbo(ctx: Context, logprob, xt, start: int, length: int, mask_id: int, t, nelbo=None, n_masked=None,
+                      stream=None, check: bool = True):
+    """Eq. 2, one draw: nelbo [B]."""
+    B, row_stride = xt.shape
+    if nelbo is None:
+        nelbo = torch.empty(B, dtype=torch.float32, device=xt.device)
+    rc = load().dare_masked_nelbo(ctx.handle, _ptr(logprob, torch.float32), _ptr(xt, torch.int32), B, row_stride,
+                                  int(start), int(length), int(mask_id), _ptr(t, torch.float32),
+                                  _ptr(nelbo, torch.float32), _ptr(n_masked, torch.int32), _stream(stream))
+    if rc != 0 and check:
+        raise DareError(rc, "dare_masked_nelbo")
+    return nelbo if check else rc
 
 
 LMHEAD_STATIC_SCRATCH_BYTES = 8 << 20
