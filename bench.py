@@ -37,7 +37,7 @@ UNIT = "tokens/s"
 NPOOL = 4   # distinct activation sets cycled through the steps
 # dram__bytes_read.sum + dram__bytes_write.sum of one lmhead_partial_kernel launch, from the ncu capture
 # summarised in profiles/lmhead_partial_kernel_llada8b.md (W, 1.036 GB, dominates: it leaves HBM once)
-LMHEAD_TRAFFIC_BYTES = {"llada8b": 1.0497e9}
+LMHEAD_TRAFFIC_BYTES = {"llada8b": 1.0517e9}
 
 
 def _peaks():
@@ -245,10 +245,11 @@ def run_ours(args):
         float(np.mean([wl.prompt_len + ((t % steps_per_gen) // steps_per_block) * L + L for t in range(n_inst)])) + wl.suffix_cap)
     qo_bytes = 2.0 * 2 * B * L * wl.n_q_heads * wl.head_dim
     attn_gbs = (kv_bytes + qo_bytes) / (attn_ms * 1e-3) / 1e9
-    # greedy against sampled head with every row masked (the sampling epilogue draws M * V Gumbel variates)
+    # greedy against sampled head with every row masked (the sampling epilogue draws M * V Gumbel variates);
+    # skipped in the few-step runs used under the profiler
     full_ms = {}
-    for name, fn in (("lmhead_all_rows_ms", lambda: dare.dare_lmhead_confidence(ctx, pool[0][1], w, None, wl.mask_id, True, pred, conf, stream=stream)),
-                     ("lmhead_sample_all_rows_ms", lambda: dare.dare_lmhead_sample(ctx, pool[0][1], w, None, wl.mask_id, True, 1.0, 1, 1, pred, conf, stream=stream))):
+    for name, fn in (() if args.steps < 64 else (("lmhead_all_rows_ms", lambda: dare.dare_lmhead_confidence(ctx, pool[0][1], w, None, wl.mask_id, True, pred, conf, stream=stream)),
+                     ("lmhead_sample_all_rows_ms", lambda: dare.dare_lmhead_sample(ctx, pool[0][1], w, None, wl.mask_id, True, 1.0, 1, 1, pred, conf, stream=stream)))):
         for _ in range(2):
             fn()
         es = [torch.cuda.Event(enable_timing=True) for _ in range(9)]
