@@ -378,7 +378,8 @@ attn_block_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_cons
 // groups, long blocks such as the prefill).  One CTA per (one or two tiles of packed query rows, rollout x
 // KV head); the two query tiles share every K/V tile:
 //   warp 0        TMA producer: 64-key K and V tiles through a shared-memory ring (as above)
-//   warp 1        UMMA issuer:  S = Q K^T (128 x 64, K-major operands) into one of two TMEM buffers per query
+//   warp 1 (and the last warp for the second query tile)
+//                 UMMA issuer:  S = Q K^T (128 x 64, K-major operands) into one of two TMEM buffers per query
 //                 tile, then O += P V (128 x D; V is the MN-major operand, straight from the TMA tile),
 //                 accumulated in TMEM over the whole key range
 //   warps 2..5    softmax of query tile 0 (warps 6..9: tile 1): one TMEM lane = one query row per thread;
@@ -400,7 +401,7 @@ struct TcShape {
     static constexpr int FIXED = QT * Q_BYTES + QT * 2 * P_BYTES;
     static constexpr int STAGES = (226 * 1024 - 2048 - FIXED) / KV_STAGE > 6 ? 6 : (226 * 1024 - 2048 - FIXED) / KV_STAGE;
     static constexpr int SMEM = FIXED + STAGES * KV_STAGE + 1024 + 512;
-    static constexpr int THREADS = (2 + 4 * QT) * 32;
+    static constexpr int THREADS = (2 + 4 * QT + 1) * 32;             // TMA warp, MMA warp, softmax warps, second MMA warp
     static constexpr uint32_t TMEM_COLS = QT * 256;                    // per query tile: S 2 x 64 columns, O D columns
     static_assert(STAGES >= 2, "K/V ring too small");
 };
@@ -453,7 +454,7 @@ attn_block_tc_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_c
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(&bars->full[s], 1);
-            mbar_init(&bars->empty[s], 1);
+            mbar_init(&bars->empty[s], QT);                // one release per query tile's MMA thread
         }
         mbar_init(&bars->q_ready, 128 * QT);
         for (int j = 0; j < QT; ++j)
@@ -517,32 +518,32 @@ attn_block_tc_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_c
                 if (++stage == STAGES) { stage = 0; phase ^= 1; }
             }
         }
-    } else if (warp == 1) {
-        if (lane == 0) {
+    } else if (warp == 1 || warp == S::THREADS / 32 - 1) {
+        // One issuing thread per query tile (warp 1: tile 0; with two tiles the last warp: tile 1): the fixed
+        // cost of issuing a tcgen05.mma is paid per thread, so two threads keep the tensor pipe twice as busy.
+        const int j = warp == 1 ? 0 : 1;
+        if (lane == 0 && j < QT) {
             constexpr uint32_t idesc_s = umma_idesc_bf16(128, TC_KT);
             constexpr uint32_t idesc_o = umma_idesc_bf16(128, D) | UMMA_B_MN_MAJOR;
             // descriptor lower words (address >> 4 [| leading byte offset]); the upper word is a constant
-            const uint32_t q_lo = smem_u32(q_s) >> 4, kv_lo = smem_u32(kv_s) >> 4, p_lo = smem_u32(p_s) >> 4;
+            const uint32_t q_lo = (smem_u32(q_s) >> 4) + j * (S::Q_BYTES >> 4);
+            const uint32_t kv_lo = smem_u32(kv_s) >> 4, p_lo = (smem_u32(p_s) >> 4) + j * 2 * (S::P_BYTES >> 4);
             const uint32_t v_lbo = static_cast<uint32_t>(HALF_K >> 4) << 16;   // second 64 head-dim columns: one half tile on
+            const uint32_t tm_j = tmem_base + j * 256;
             bool ok = mbar_wait(&bars->q_ready, 0, abort_flag);
-            // S_j(t) = Q_j K_t^T into S buffer t & 1 of query tile j once its softmax warps have read what it held
+            // S(t) = Q K_t^T into S buffer t & 1 once the softmax warps have read what it held
             auto issue_s = [&](int t) -> bool {
                 const int stage = t % STAGES, buf = t & 1;
                 if (!mbar_wait(&bars->full[stage], (t / STAGES) & 1, abort_flag)) return false;
-                const uint32_t k_lo = kv_lo + stage * (S::KV_STAGE >> 4);
+                if (!mbar_wait(&bars->s_free[j][buf], ((t >> 1) & 1) ^ 1, abort_flag)) return false;
+                tc_fence_after_sync();
+                const uint32_t k_lo = kv_lo + stage * (S::KV_STAGE >> 4), sd = tm_j + buf * TC_KT;
+                umma_bf16_lo<false>(sd, q_lo, k_lo, idesc_s);
 #pragma unroll
-                for (int j = 0; j < QT; ++j) {
-                    if (!mbar_wait(&bars->s_free[j][buf], ((t >> 1) & 1) ^ 1, abort_flag)) return false;
-                    tc_fence_after_sync();
-#pragma unroll
-                    const uint32_t qa = q_lo + j * (S::Q_BYTES >> 4), sd = tmem_base + j * 256 + buf * TC_KT;
-                    umma_bf16_lo<false>(sd, qa, k_lo, idesc_s);
-#pragma unroll
-                    for (int kk = 1; kk < D / 16; ++kk)     // 16 channels = 32 bytes along the swizzled row: +2
-                        umma_bf16_lo<true>(sd, qa + (kk >> 2) * (HALF_Q >> 4) + 2 * (kk & 3),
-                                           k_lo + (kk >> 2) * (HALF_K >> 4) + 2 * (kk & 3), idesc_s);
-                    umma_commit(&bars->s_full[j][buf]);
-                }
+                for (int kk = 1; kk < D / 16; ++kk)     // 16 channels = 32 bytes along the swizzled row: +2
+                    umma_bf16_lo<true>(sd, q_lo + (kk >> 2) * (HALF_Q >> 4) + 2 * (kk & 3),
+                                       k_lo + (kk >> 2) * (HALF_K >> 4) + 2 * (kk & 3), idesc_s);
+                umma_commit(&bars->s_full[j][buf]);
                 return true;
             };
             if (ok && n_tiles > 0) ok = issue_s(0);
@@ -550,22 +551,17 @@ attn_block_tc_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_c
                 if (t + 1 < n_tiles && !issue_s(t + 1)) { ok = false; break; }
                 const int stage = t % STAGES, buf = t & 1;
                 const uint32_t v_lo = (kv_lo + stage * (S::KV_STAGE >> 4) + (KV_BYTES >> 4)) | v_lbo;
+                if (!mbar_wait(&bars->p_full[j][buf], (t >> 1) & 1, abort_flag)) { ok = false; break; }
+                tc_fence_after_sync();
+                // A: 16 keys further along the 128-byte row of P (+2); B: 16 key rows (2 KB) further down V
+                const uint32_t pa = p_lo + buf * (S::P_BYTES >> 4), od = tm_j + 128;
+                if (t == 0) umma_bf16_lo<false>(od, pa, v_lo, idesc_o);
+                else umma_bf16_lo<true>(od, pa, v_lo, idesc_o);
 #pragma unroll
-                for (int j = 0; j < QT; ++j) {
-                    if (!mbar_wait(&bars->p_full[j][buf], (t >> 1) & 1, abort_flag)) { ok = false; break; }
-                    tc_fence_after_sync();
-#pragma unroll
-                    // A: 16 keys further along the 128-byte row of P (+2); B: 16 key rows (2 KB) further down V
-                    const uint32_t pa = p_lo + (j * 2 + buf) * (S::P_BYTES >> 4), od = tmem_base + j * 256 + 128;
-                    if (t == 0) umma_bf16_lo<false>(od, pa, v_lo, idesc_o);
-                    else umma_bf16_lo<true>(od, pa, v_lo, idesc_o);
-#pragma unroll
-                    for (int kk = 1; kk < TC_KT / 16; ++kk)
-                        umma_bf16_lo<true>(od, pa + 2 * kk, v_lo + kk * (2048 >> 4), idesc_o);
-                    umma_commit(&bars->o_done[j][buf]);    // P buffer free again; O holds tiles 0..t
-                }
-                if (!ok) break;
-                umma_commit(&bars->empty[stage]);          // K and V of this tile have been read
+                for (int kk = 1; kk < TC_KT / 16; ++kk)
+                    umma_bf16_lo<true>(od, pa + 2 * kk, v_lo + kk * (2048 >> 4), idesc_o);
+                umma_commit(&bars->o_done[j][buf]);    // P buffer free again; O holds tiles 0..t
+                umma_commit(&bars->empty[stage]);      // this query tile is done with K and V of the tile
             }
         }
     } else {
