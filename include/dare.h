@@ -12,14 +12,19 @@
  *     dare_unmask_select      confidence-threshold / per-block top-k commit on the int32 token state
  *     dare_denoise_block      the three above, enqueued back to back
  *     dare_model_* / dare_generate   the same step with a stack of transformer layers in between, and the
- *                             whole block-by-block loop
+ *                             whole block-by-block loop (dare_linear, dare_rmsnorm, dare_rope_kv_write: its parts)
+ *     dare_lmhead_sample      the LM head with temperature + Gumbel-max sampling instead of the argmax
+ *     dare_lmhead_logprob     log-probability of given tokens (cross-entropy), logits never written either
+ *     dare_attn_varlen        bidirectional attention over packed variable-length sequences
+ *     dare_forward_mask, dare_masked_nelbo   the forward (masking) process of Eq. 1 and the bound of Eq. 2
  *
  * Conventions
  *   - Every data pointer is a DEVICE pointer unless the comment says "host".  The caller owns every
  *     buffer; the library neither frees nor keeps them after the call's stream work has run.
  *   - All entry points enqueue work on `stream` (a cudaStream_t passed as void*, NULL = default
- *     stream) and return without synchronising.  They allocate nothing; the only allocation is the
- *     workspace made once by dare_create.
+ *     stream) and return without synchronising, except where their comment says that they block
+ *     (dare_device_status, dare_model_create, dare_generate).  They allocate nothing; the only
+ *     allocations are the workspace made once by dare_create and the buffers of dare_model_create.
  *   - bf16 tensors are dense, row-major, 16-byte aligned.
  *   - Return value: DARE_OK (0) or a negative dare_status.  On any error nothing has been launched.
  *   - Data-dependent anomalies (a per-row length beyond its capacity, a wait inside a kernel that
