@@ -276,6 +276,9 @@ MODEL_WORKLOADS = {
     # small cases for element-by-element parity
     "loop_small": ModelWorkload("loop_small", 2, 256, 4, 4, 64, 768, 4096, 4095, 2, 48, 64, 32,
                                 SELECT_THRESHOLD, threshold=0.9),
+    # block diffusion with short blocks (SDAR / LLaDA2-style: block of 4, causal across blocks)
+    "loop_small_bd4": ModelWorkload("loop_small_bd4", 2, 256, 4, 2, 64, 512, 1024, 1000, 3, 24, 16, 4,
+                                    SELECT_THRESHOLD, threshold=0.95),
     "loop_small_gqa": ModelWorkload("loop_small_gqa", 3, 512, 4, 2, 128, 1280, 2048, 2000, 3, 40, 32, 16,
                                     SELECT_TOPK, k=3),
 }

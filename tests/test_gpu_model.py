@@ -171,7 +171,7 @@ def _check_lm(pred_t, conf_t, lm, n_layers):
     assert same.sum() >= 0.8 * live.sum() - 1      # near-ties (logit gap below the bar) may resolve differently
 
 
-@pytest.mark.parametrize("name", ["loop_small", "loop_small_gqa"])
+@pytest.mark.parametrize("name", ["loop_small", "loop_small_gqa", "loop_small_bd4"])
 def test_loop_small_step_by_step_and_generate(ctx, name):
     mw = I.MODEL_WORKLOADS[name]
     wts_t = I.make_model_weights(mw)
