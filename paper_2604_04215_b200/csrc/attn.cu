@@ -20,8 +20,8 @@
 namespace dare {
 namespace {
 
-constexpr int KT = 64;           // keys per tile
-constexpr int ATT_STAGES = 3;
+constexpr int KT_MAX = 64;       // keys per tile of the widest variant (sizes the launch plan)
+constexpr int ATT_MAX_STAGES = 4;
 constexpr float LOG2E_F = 1.4426950408889634f;
 constexpr float LN2_F = 0.6931471805599453f;
 
@@ -44,15 +44,15 @@ struct AttnParams {
 };
 
 struct AttBarriers {
-    uint64_t full[ATT_STAGES];
-    uint64_t empty[ATT_STAGES];
+    uint64_t full[ATT_MAX_STAGES];
+    uint64_t empty[ATT_MAX_STAGES];
     uint32_t abort_flag;
 };
 
-template <int D>
+template <int D, int KT>
 __host__ __device__ constexpr int att_stage_bytes() { return 2 * KT * D * 2; }
-template <int D>
-__host__ __device__ constexpr int att_smem_bytes() { return ATT_STAGES * att_stage_bytes<D>() + static_cast<int>(sizeof(AttBarriers)) + 1024; }
+template <int D, int KT, int STAGES>
+__host__ __device__ constexpr int att_smem_bytes() { return STAGES * att_stage_bytes<D, KT>() + static_cast<int>(sizeof(AttBarriers)) + 1024; }
 
 // Segment bookkeeping of one (row, kv head) unit: tiles of the prefix, then the block, then the suffix.
 struct TileInfo {
@@ -61,6 +61,7 @@ struct TileInfo {
     int valid;    // keys of the tile that exist (1..KT)
 };
 
+template <int KT>
 __device__ __forceinline__ TileInfo tile_info(int t, int n_pre, int n_blk, int len_pre, int len_blk, int len_suf,
                                               int base_pre, int base_blk, int base_suf) {
     TileInfo ti;
@@ -79,14 +80,15 @@ __device__ __forceinline__ TileInfo tile_info(int t, int n_pre, int n_blk, int l
 // NW row groups of 16 packed query rows; KS warps share a row group and split every 64-key tile between
 // them (KT / KS keys each), keeping separate running (max, sum, O) that are merged through shared memory at
 // the end.  More warps per SM hide the latency of the ldmatrix -> MMA -> softmax chain.
-template <int D, int NW, int KS>
-__global__ void __launch_bounds__((NW * KS + 1) * 32, (NW * KS + 1) * 32 <= 160 ? 2 : 1)
+// KT keys per tile and ATT_STAGES ring slots set the shared memory of a CTA and so how many CTAs an SM holds (CPS).
+template <int D, int NW, int KS, int KT, int ATT_STAGES, int CPS>
+__global__ void __launch_bounds__((NW * KS + 1) * 32, CPS)
 attn_block_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_constant__ CUtensorMap tm_vpre,
                   const __grid_constant__ CUtensorMap tm_kblk, const __grid_constant__ CUtensorMap tm_vblk,
                   const __grid_constant__ CUtensorMap tm_ksuf, const __grid_constant__ CUtensorMap tm_vsuf,
                   const AttnParams p) {
-    constexpr int STAGE = att_stage_bytes<D>();
-    constexpr int HALF = KT * 128;           // one 64-column half of a tile: 64 rows x 128 bytes
+    constexpr int STAGE = att_stage_bytes<D, KT>();
+    constexpr int HALF = KT * 128;           // one 64-column half of a tile: KT rows x 128 bytes
     constexpr int NHALF = D / 64;
     constexpr int KV_BYTES = KT * D * 2;
     constexpr int NCW = NW * KS;             // consumer warps
@@ -162,7 +164,7 @@ attn_block_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_cons
             int stage = 0;
             uint32_t phase = 0;
             for (int t = t_begin; t < t_end; ++t) {
-                const TileInfo ti = tile_info(t, n_pre, n_blk, len_pre, len_blk, S, base_pre, base_blk, base_suf);
+                const TileInfo ti = tile_info<KT>(t, n_pre, n_blk, len_pre, len_blk, S, base_pre, base_blk, base_suf);
                 const CUtensorMap* mk = ti.seg == 0 ? &tm_kpre : (ti.seg == 1 ? &tm_kblk : &tm_ksuf);
                 const CUtensorMap* mv = ti.seg == 0 ? &tm_vpre : (ti.seg == 1 ? &tm_vblk : &tm_vsuf);
                 if (!mbar_wait(&bars->empty[stage], phase ^ 1, abort_flag)) break;
@@ -198,7 +200,7 @@ attn_block_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_cons
         const int mi = lane >> 3, rin = lane & 7;
         const int koff = ks * KPW;           // this warp's keys inside a tile: [koff, koff + KPW)
         for (int t = t_begin; t < t_end; ++t) {
-            const TileInfo ti = tile_info(t, n_pre, n_blk, len_pre, len_blk, S, base_pre, base_blk, base_suf);
+            const TileInfo ti = tile_info<KT>(t, n_pre, n_blk, len_pre, len_blk, S, base_pre, base_blk, base_suf);
             if (!mbar_wait(&bars->full[stage], phase, abort_flag)) { ok = false; break; }
             uint8_t* kt = tiles + stage * STAGE;
             uint8_t* vt = kt + KV_BYTES;
@@ -503,7 +505,7 @@ attn_block_tc_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_c
             int stage = 0;
             uint32_t phase = 0;
             for (int t = 0; t < n_tiles; ++t) {
-                const TileInfo ti = tile_info(t, n_pre, n_blk, len_pre, len_blk, Sx, base_pre, base_blk, base_suf);
+                const TileInfo ti = tile_info<TC_KT>(t, n_pre, n_blk, len_pre, len_blk, Sx, base_pre, base_blk, base_suf);
                 const CUtensorMap* mk = ti.seg == 0 ? &tm_kpre : (ti.seg == 1 ? &tm_kblk : &tm_ksuf);
                 const CUtensorMap* mv = ti.seg == 0 ? &tm_vpre : (ti.seg == 1 ? &tm_vblk : &tm_vsuf);
                 if (!mbar_wait(&bars->empty[stage], phase ^ 1, abort_flag)) break;
@@ -592,7 +594,7 @@ attn_block_tc_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_c
         const uint32_t tm_o = tmem_base + j * 256 + 128 + lane_off;
         bool ok = true;
         for (int t = 0; t < n_tiles; ++t) {
-            const TileInfo ti = tile_info(t, n_pre, n_blk, len_pre, len_blk, Sx, base_pre, base_blk, base_suf);
+            const TileInfo ti = tile_info<TC_KT>(t, n_pre, n_blk, len_pre, len_blk, Sx, base_pre, base_blk, base_suf);
             const int buf = t & 1, stage = t % STAGES;
             if (!mbar_wait(&bars->s_full[j][buf], (t >> 1) & 1, abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
@@ -765,18 +767,29 @@ __global__ void attn_combine_kernel(const float* __restrict__ part_o, const floa
     }
 }
 
-template <int D, int NW, int KS>
+template <int D, int NW, int KS, int KT, int STAGES, int CPS>
 int launch_one(const CUtensorMap* tm, const AttnParams& p, int chunks, cudaStream_t stream) {
-    constexpr int SMEM = att_smem_bytes<D>();
-    static_assert((KS - 1) * NW * ((D / 8) * 4 + 4) * 32 * 4 <= ATT_STAGES * att_stage_bytes<D>(), "merge buffer");
-    if (cudaFuncSetAttribute(attn_block_kernel<D, NW, KS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
+    constexpr int SMEM = att_smem_bytes<D, KT, STAGES>();
+    static_assert((KS - 1) * NW * ((D / 8) * 4 + 4) * 32 * 4 <= STAGES * att_stage_bytes<D, KT>(), "merge buffer");
+    static_assert(STAGES <= ATT_MAX_STAGES && KT <= KT_MAX && KT % (16 * KS) == 0, "variant");
+    if (cudaFuncSetAttribute(attn_block_kernel<D, NW, KS, KT, STAGES, CPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
         return DARE_ERR_CUDA;
     dim3 grid(chunks, p.B * p.Hkv, p.splits);
-    attn_block_kernel<D, NW, KS><<<grid, (NW * KS + 1) * 32, SMEM, stream>>>(tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], p);
+    attn_block_kernel<D, NW, KS, KT, STAGES, CPS><<<grid, (NW * KS + 1) * 32, SMEM, stream>>>(tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], p);
     return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
 }
 
-int pick_warps(int R) { return R <= 16 ? 1 : (R <= 32 ? 2 : 4); }
+// The warp-level kernel's variants by the number of packed query rows R per (rollout, KV head):
+//   R <= 16   one row group, four key slices of a 64-key tile, 2 CTAs per SM
+//   R <= 32   two row groups, two key slices of a 64-key tile, 2 CTAs per SM (32-key tiles with two warps and
+//             4 CTAs per SM were measured slower: 58 against 45 us on 16 rollouts x 32 heads x 768 keys)
+//   larger    four row groups per 64-row chunk, 64-key tiles, 2 CTAs per SM
+struct WarpVariant { int nw, kt, per_sm; };
+WarpVariant pick_variant(int R) {
+    if (R <= 16) return {1, 64, 2};
+    if (R <= 32) return {2, 64, 2};
+    return {4, 64, 2};
+}
 
 }  // namespace
 
@@ -784,15 +797,13 @@ int attn_plan_splits(const dare_ctx* ctx, const AttnArgs& a) {
     if (use_tc_path(a)) return 1;
     const int g = a.Hq / a.Hkv;
     const int R = a.L * g;
-    const int nw = pick_warps(R);
+    const WarpVariant var = pick_variant(R);
+    const int nw = var.nw;
     const int chunks = (R + nw * 16 - 1) / (nw * 16);
     const long long units = static_cast<long long>(chunks) * a.B * a.Hkv;
-    const int smem = a.d == 128 ? att_smem_bytes<128>() : att_smem_bytes<64>();
-    int per_sm = (227 * 1024) / smem;
-    if (per_sm > 8) per_sm = 8;
-    const long long slots = static_cast<long long>(ctx->sm_count) * per_sm;
+    const long long slots = static_cast<long long>(ctx->sm_count) * var.per_sm;
     if (units >= slots) return 1;
-    const int tiles = (a.prefix_cap + (a.k_blk ? a.L : 0) + a.suffix_cap + KT - 1) / KT;
+    const int tiles = (a.prefix_cap + (a.k_blk ? a.L : 0) + a.suffix_cap + var.kt - 1) / var.kt;
     long long s = (slots + units - 1) / units;
     if (s > tiles / 2) s = tiles / 2;
     if (s > 32) s = 32;
@@ -826,6 +837,7 @@ int launch_attn(const dare_ctx* ctx, const AttnArgs& a, cudaStream_t stream) {
 
     CUtensorMap tm[6];
     const uint64_t units = static_cast<uint64_t>(a.B) * a.Hkv;
+    const uint32_t KT = static_cast<uint32_t>(use_tc_path(a) ? TC_KT : pick_variant(p.R).kt);   // rows of a K/V tile
     int rc = make_tmap_bf16_2d(ctx, &tm[0], a.k_pre, units * a.prefix_cap, a.d, KT, 64);
     if (rc == DARE_OK) rc = make_tmap_bf16_2d(ctx, &tm[1], a.v_pre, units * a.prefix_cap, a.d, KT, 64);
     if (rc != DARE_OK) return rc;
@@ -853,14 +865,16 @@ int launch_attn(const dare_ctx* ctx, const AttnArgs& a, cudaStream_t stream) {
             return a.d == 128 ? launch_tc<128, 2>(tm, p, q_tiles, stream) : launch_tc<64, 2>(tm, p, q_tiles, stream);
         return a.d == 128 ? launch_tc<128, 1>(tm, p, q_tiles, stream) : launch_tc<64, 1>(tm, p, q_tiles, stream);
     }
-    const int nw = pick_warps(p.R);
+    const int nw = pick_variant(p.R).nw;
     const int chunks = (p.R + nw * 16 - 1) / (nw * 16);
     if (a.d == 128) {
-        rc = nw == 1 ? launch_one<128, 1, 4>(tm, p, chunks, stream)
-           : nw == 2 ? launch_one<128, 2, 2>(tm, p, chunks, stream) : launch_one<128, 4, 1>(tm, p, chunks, stream);
+        rc = nw == 1 ? launch_one<128, 1, 4, 64, 3, 2>(tm, p, chunks, stream)
+           : nw == 2 ? launch_one<128, 2, 2, 64, 3, 2>(tm, p, chunks, stream)
+                     : launch_one<128, 4, 1, 64, 3, 2>(tm, p, chunks, stream);
     } else {
-        rc = nw == 1 ? launch_one<64, 1, 4>(tm, p, chunks, stream)
-           : nw == 2 ? launch_one<64, 2, 2>(tm, p, chunks, stream) : launch_one<64, 4, 1>(tm, p, chunks, stream);
+        rc = nw == 1 ? launch_one<64, 1, 4, 64, 3, 2>(tm, p, chunks, stream)
+           : nw == 2 ? launch_one<64, 2, 2, 64, 3, 2>(tm, p, chunks, stream)
+                     : launch_one<64, 4, 1, 64, 3, 2>(tm, p, chunks, stream);
     }
     if (rc != DARE_OK) return rc;
     if (p.splits > 1) {
