@@ -12,6 +12,14 @@ at exactly the places where the product path stores bf16 in memory, and states t
     has no mask left, one more forward (no LM head) rewrites its K/V from the committed tokens and the
     prefix grows by L.
 
+  * ``generate_dual``  the loop of a fully bidirectional masked model with a prefix AND a suffix cache
+    (Section 3.4, rollout with KV-cache reuse): before each block one forward of the whole sequence
+    rewrites every position's K/V from the current tokens (the still-masked future blocks included); the
+    block's steps then recompute only the block's rows against cached prefix + fresh block + cached suffix.
+    The cached K/V outside the block go stale while the block's tokens change: that approximation is the
+    algorithm, so the oracle follows its steps; what can be pinned exactly is pinned (a block forward right
+    after a refresh reproduces the refresh; one block spanning the whole sequence is the uncached model).
+
 That the two agree step by step is the pin of the cache recurrence (tests/test_oracle_model.py); the stack
 itself is pinned against an independently written torch formulation (library attention with a boolean mask,
 library rms_norm/silu, RoPE as a complex multiplication).  Nothing here is imported by the product path.
@@ -160,15 +168,20 @@ def new_cache(cfg: ModelConfig, batch, cap):
     return [(np.zeros(shp), np.zeros(shp)) for _ in range(cfg.n_layers)]
 
 
-def forward_block_cached(cfg: ModelConfig, wts: ModelWeights, tokens, start, length, cache, rounded=True):
+def forward_block_cached(cfg: ModelConfig, wts: ModelWeights, tokens, start, length, cache, rounded=True, kv_len=None):
     """The rows [start, start + length) of every rollout through the stack, against the cache.
 
     tokens int [B, row]; cache from new_cache, updated IN PLACE: each layer writes the rows' post-RoPE K/V at
     [start, start + length) and the rows attend to cache[0 : start + length) (everything before `start` is the
     prefix; the rows see each other).  With start = 0 and length = prompt length this is the prefill.
+    With kv_len > start + length the rows also see cache[start + length : kv_len) as a suffix whose K/V are
+    whatever an earlier forward left there (the dual cache of a fully bidirectional model).
     Returns the final-norm hidden states [B * length, D].
     """
     B = tokens.shape[0]
+    end = start + length
+    kv_len = end if kv_len is None else kv_len
+    assert end <= kv_len <= cache[0][0].shape[2]
     pos = np.arange(start, start + length)
     x = wts.embedding[np.asarray(tokens)[:, start:start + length].reshape(-1)]     # [B*length, D]
     plen = np.full(B, start, dtype=np.int64)
@@ -182,7 +195,11 @@ def forward_block_cached(cfg: ModelConfig, wts: ModelWeights, tokens, start, len
             qs[r] = _r(rope(q, pos, cfg.rope_base), rounded)
             kc[r, :, start:start + length] = np.transpose(_r(rope(k, pos, cfg.rope_base), rounded), (1, 0, 2))
             vc[r, :, start:start + length] = np.transpose(v, (1, 0, 2))
-        o, _ = O.attn_block(qs, kc, vc, plen)              # block stored in place behind the prefix
+        if kv_len == end:
+            o, _ = O.attn_block(qs, kc, vc, plen)          # block stored in place behind the prefix
+        else:                                              # ... and the cached suffix behind the block
+            o, _ = O.attn_block(qs, kc[:, :, :end], vc[:, :, :end], plen, None, None,
+                                kc[:, :, end:kv_len], vc[:, :, end:kv_len], None)
         o = _r(o, rounded).reshape(B * length, -1)
         x = _r(x + o @ lw.wo.T, rounded)
         x = _ffn(x, lw, cfg, rounded)
@@ -222,5 +239,46 @@ def generate(cfg, wts, tokens, prompt_len, gen_len, L, mode, threshold, k, round
             tok = res["tokens"]
             n += 1
         forward_block_cached(cfg, wts, tok, start, L, cache, rounded)   # K/V of the committed block
+        steps.append(n)
+    return tok, steps, cache
+
+
+def denoise_step_dual(cfg, wts, tokens, block_start, L, kv_len, cache, mode, threshold, k, rounded=True):
+    """One step with both caches: as denoise_step_cached, the block's rows seeing cache[0 : kv_len)."""
+    hidden = forward_block_cached(cfg, wts, tokens, block_start, L, cache, rounded, kv_len=kv_len)
+    B = tokens.shape[0]
+    row_tokens = np.asarray(tokens)[:, block_start:block_start + L].reshape(B * L)
+    lm = O.lmhead_confidence(hidden, wts.lm_head, row_tokens, cfg.mask_id, True)
+    conf32 = lm["conf"].astype(np.float32)
+    tok, nc, nr = O.unmask_select(tokens, block_start, L, lm["pred"], conf32, cfg.mask_id, mode, threshold, k)
+    return {"hidden": hidden, "lm": lm, "tokens": tok, "n_committed": nc, "n_remaining": nr}
+
+
+def generate_dual(cfg, wts, tokens, prompt_len, gen_len, L, mode, threshold, k, rounded=True, on_step=None,
+                  on_refresh=None):
+    """Dual-cache loop of a fully bidirectional model: per block, refresh every position's K/V with one forward
+    of the whole sequence [0, T), T = prompt_len + gen_len, then denoise the block against cache[0 : T) until it
+    holds no mask.  Blocks are taken left to right and the batch moves block-synchronously.
+
+    Returns (tokens int32 [B, row], steps per block, cache).  on_refresh(block, tokens, hidden [B * T, D]) and
+    on_step(block, step, tokens_before, result) are called if given.
+    """
+    tok = np.array(tokens, dtype=np.int32, copy=True)
+    B = tok.shape[0]
+    T = prompt_len + gen_len
+    cache = new_cache(cfg, B, T)
+    steps = []
+    for b in range(gen_len // L):
+        start = prompt_len + b * L
+        hidden = forward_block_cached(cfg, wts, tok, 0, T, cache, rounded)          # the refresh
+        if on_refresh is not None:
+            on_refresh(b, tok, hidden)
+        n = 0
+        while (tok[:, start:start + L] == cfg.mask_id).any():
+            res = denoise_step_dual(cfg, wts, tok, start, L, T, cache, mode, threshold, k, rounded)
+            if on_step is not None:
+                on_step(b, n, tok, res)
+            tok = res["tokens"]
+            n += 1
         steps.append(n)
     return tok, steps, cache

@@ -7,6 +7,9 @@ The paper prints no values for this loop, so the oracle is tied down by what the
     library rms_norm / silu, RoPE as a complex multiplication on re-paired channels);
   * RoPE: position 0 is the identity, norms are kept, scores depend only on position differences;
   * RMSNorm: unit root-mean-square; bf16 rounding: torch's own conversion, including ties;
+  * the dual cache: the refresh is the fully bidirectional forward; a window forward right after a refresh
+    reproduces the refresh's rows and leaves the cache unchanged; it writes only its own rows, reads the suffix
+    and nothing beyond kv_len; one block over the whole sequence makes the loop the uncached model;
   * loop counts: every rollout commits exactly G tokens; steps per block = ceil(L / k) under top-k and
     at most L under the threshold rule; prompt tokens never change; same seed, same tokens.
 """
@@ -200,3 +203,132 @@ def test_generate_is_deterministic():
     b = MO.generate(cfg, wts, tok0, mw.prompt_len, mw.gen_len, mw.block_len, O.SELECT_THRESHOLD, 0.9, 1)
     np.testing.assert_array_equal(a[0], b[0])
     assert a[1] == b[1]
+
+
+# ---------------------------------------------------------------------------------------------------------
+# Dual cache (prefix + suffix) of a fully bidirectional model
+
+def test_refresh_is_the_fully_bidirectional_forward():
+    """The refresh forward (all rows, all keys) equals the uncached forward with every position in one segment."""
+    mw = _small(batch=2)
+    cfg, wts = _cfg(mw), _weights(mw)
+    tok = I.fresh_model_tokens(mw).numpy()
+    T = mw.prompt_len + mw.gen_len
+    cache = MO.new_cache(cfg, mw.batch, T)
+    hid = MO.forward_block_cached(cfg, wts, tok, 0, T, cache, rounded=False)
+    for r in range(mw.batch):
+        full, kv = MO.forward_uncached(cfg, wts, tok[r, :T], np.zeros(T, dtype=np.int64), rounded=False)
+        np.testing.assert_allclose(hid[r * T:(r + 1) * T], full, atol=1e-9)
+        for li, (k_full, v_full) in enumerate(kv):
+            np.testing.assert_allclose(cache[li][0][r], np.transpose(k_full, (1, 0, 2)), atol=1e-9)
+            np.testing.assert_allclose(cache[li][1][r], np.transpose(v_full, (1, 0, 2)), atol=1e-9)
+
+
+@pytest.mark.parametrize("start,length", [(5, 4), (0, 5), (13, 4), (7, 3)])
+def test_window_forward_right_after_a_refresh_reproduces_it(start, length):
+    """With unchanged tokens the cached K/V are exact, so a window forward over prefix + block + suffix gives the
+    refresh's own rows and leaves the cache as it was: pins the visibility (all of [0, kv_len)), the in-place
+    positions and RoPE offsets of the window, for a window at the start, in the middle and at the end."""
+    mw = _small(batch=2)
+    cfg, wts = _cfg(mw), _weights(mw)
+    tok = I.fresh_model_tokens(mw).numpy()
+    T = mw.prompt_len + mw.gen_len
+    cache = MO.new_cache(cfg, mw.batch, T)
+    hid = MO.forward_block_cached(cfg, wts, tok, 0, T, cache, rounded=False).reshape(mw.batch, T, -1)
+    before = [(k.copy(), v.copy()) for k, v in cache]
+    win = MO.forward_block_cached(cfg, wts, tok, start, length, cache, rounded=False, kv_len=T)
+    np.testing.assert_allclose(win.reshape(mw.batch, length, -1), hid[:, start:start + length], atol=1e-9)
+    for (k0, v0), (k1, v1) in zip(before, cache):
+        np.testing.assert_allclose(k1, k0, atol=1e-9)
+        np.testing.assert_allclose(v1, v0, atol=1e-9)
+    # a window that cannot see the suffix differs (unless it is the last one)
+    if start + length < T:
+        cut = MO.forward_block_cached(cfg, wts, tok, start, length, [(k.copy(), v.copy()) for k, v in before],
+                                      rounded=False)
+        assert np.abs(cut - win).max() > 1e-6
+
+
+def test_window_forward_writes_only_its_own_rows_and_reads_the_suffix():
+    mw = _small(batch=1)
+    cfg, wts = _cfg(mw), _weights(mw)
+    tok = I.fresh_model_tokens(mw).numpy()
+    T = mw.prompt_len + mw.gen_len
+    start, L = mw.prompt_len, mw.block_len
+    cache = MO.new_cache(cfg, 1, T)
+    MO.forward_block_cached(cfg, wts, tok, 0, T, cache, rounded=False)
+    before = [(k.copy(), v.copy()) for k, v in cache]
+    tok2 = tok.copy()
+    tok2[0, start + 1] = 9                                              # a committed token inside the block
+    out = MO.forward_block_cached(cfg, wts, tok2, start, L, cache, rounded=False, kv_len=T)
+    for (k0, v0), (k1, v1) in zip(before, cache):
+        np.testing.assert_array_equal(k1[:, :, :start], k0[:, :, :start])
+        np.testing.assert_array_equal(k1[:, :, start + L:], k0[:, :, start + L:])
+        np.testing.assert_array_equal(v1[:, :, start + L:], v0[:, :, start + L:])
+    assert np.abs(cache[0][0][:, :, start + 1] - before[0][0][:, :, start + 1]).max() > 0
+    # the suffix is read: perturbing a cached suffix value changes the block's output
+    cache2 = [(k.copy(), v.copy()) for k, v in cache]
+    cache2[0][1][0, :, T - 1] += 1.0
+    out2 = MO.forward_block_cached(cfg, wts, tok2, start, L, cache2, rounded=False, kv_len=T)
+    assert np.abs(out2 - out).max() > 1e-6
+    # keys at and beyond kv_len are not read
+    cache3 = [(k.copy(), v.copy()) for k, v in cache]
+    cache3[0][1][0, :, T - 1] += 1.0
+    out3 = MO.forward_block_cached(cfg, wts, tok2, start, L, cache3, rounded=False, kv_len=T - 1)
+    out4 = MO.forward_block_cached(cfg, wts, tok2, start, L, [(k.copy(), v.copy()) for k, v in cache], rounded=False,
+                                   kv_len=T - 1)
+    np.testing.assert_array_equal(out3, out4)
+
+
+@pytest.mark.parametrize("mode,k", [(O.SELECT_THRESHOLD, 1), (O.SELECT_TOPK, 3)])
+def test_dual_loop_with_one_block_over_everything_is_the_uncached_model(mode, k):
+    """No prompt and a single block spanning the whole sequence: nothing is ever stale, so every step of the
+    dual-cache loop equals a from-scratch fully bidirectional forward of the current tokens."""
+    mw = _small(batch=2, prompt_len=0, gen_len=8, block_len=8)
+    cfg, wts = _cfg(mw), _weights(mw)
+    tok0 = I.fresh_model_tokens(mw).numpy()
+    seen = []
+
+    def on_step(b, n, tok_before, res):
+        for r in range(mw.batch):
+            full, _ = MO.forward_uncached(cfg, wts, tok_before[r, :8], np.zeros(8, dtype=np.int64), rounded=False)
+            np.testing.assert_allclose(res["hidden"][r * 8:(r + 1) * 8], full, atol=1e-9)
+        seen.append(n)
+
+    tok, steps, _ = MO.generate_dual(cfg, wts, tok0, 0, 8, 8, mode, 0.9, k, rounded=False, on_step=on_step)
+    assert len(seen) == steps[0] and (tok[:, :8] != cfg.mask_id).all()
+    if mode == O.SELECT_TOPK:
+        assert steps == [3]
+
+
+def test_dual_loop_counts_and_first_step_of_each_block():
+    """Several blocks: the first step of a block (tokens unchanged since the refresh) equals the refresh's rows for
+    that block; later steps see stale K/V outside the block and differ from a from-scratch forward; counts hold."""
+    mw = _small(batch=2)
+    cfg, wts = _cfg(mw), _weights(mw)
+    tok0 = I.fresh_model_tokens(mw).numpy()
+    T, L, P = mw.prompt_len + mw.gen_len, mw.block_len, mw.prompt_len
+    refreshed = {}
+    stale_seen = []
+
+    def on_refresh(b, tok, hidden):
+        refreshed[b] = hidden.reshape(mw.batch, T, -1).copy()
+
+    def on_step(b, n, tok_before, res):
+        start = P + b * L
+        got = res["hidden"].reshape(mw.batch, L, -1)
+        if n == 0:
+            np.testing.assert_allclose(got, refreshed[b][:, start:start + L], atol=1e-9)
+        else:
+            full = np.stack([MO.forward_uncached(cfg, wts, tok_before[r, :T], np.zeros(T, dtype=np.int64), False)[0]
+                             for r in range(mw.batch)])
+            stale_seen.append(np.abs(got - full[:, start:start + L]).max())
+
+    tok, steps, _ = MO.generate_dual(cfg, wts, tok0, P, mw.gen_len, L, O.SELECT_TOPK, 0.9, 2, rounded=False,
+                                     on_step=on_step, on_refresh=on_refresh)
+    assert steps == [2] * (mw.gen_len // L) and sorted(refreshed) == list(range(mw.gen_len // L))
+    assert (tok[:, P:] != cfg.mask_id).all()
+    np.testing.assert_array_equal(tok[:, :P], tok0[:, :P])
+    assert min(stale_seen) > 1e-6                   # staleness is real: the cached loop is an approximation
+    a = MO.generate_dual(cfg, wts, tok0, P, mw.gen_len, L, O.SELECT_TOPK, 0.9, 2)
+    b = MO.generate_dual(cfg, wts, tok0, P, mw.gen_len, L, O.SELECT_TOPK, 0.9, 2)
+    np.testing.assert_array_equal(a[0], b[0])
