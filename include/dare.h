@@ -13,6 +13,7 @@
  *     dare_denoise_block      the three above, enqueued back to back
  *     dare_model_* / dare_generate   the same step with a stack of transformer layers in between, and the
  *                             whole block-by-block loop (dare_linear, dare_rmsnorm, dare_rope_kv_write: its parts)
+ *     dare_model_*_window / dare_generate_dual   the same with a cached suffix behind the block (dual cache)
  *     dare_lmhead_sample      the LM head with temperature + Gumbel-max sampling instead of the argmax
  *     dare_lmhead_logprob     log-probability of given tokens (cross-entropy), logits never written either
  *     dare_attn_varlen        bidirectional attention over packed variable-length sequences
@@ -23,7 +24,7 @@
  *     buffer; the library neither frees nor keeps them after the call's stream work has run.
  *   - All entry points enqueue work on `stream` (a cudaStream_t passed as void*, NULL = default
  *     stream) and return without synchronising, except where their comment says that they block
- *     (dare_device_status, dare_model_create, dare_generate).  They allocate nothing; the only
+ *     (dare_device_status, dare_model_create, dare_generate, dare_generate_dual).  They allocate nothing; the only
  *     allocations are the workspace made once by dare_create and the buffers of dare_model_create.
  *   - bf16 tensors are dense, row-major, 16-byte aligned.
  *   - Return value: DARE_OK (0) or a negative dare_status.  On any error nothing has been launched.
@@ -328,6 +329,32 @@ int dare_model_step(dare_model* model, int32_t* tokens, int B, int64_t row_strid
 int dare_generate(dare_model* model, int32_t* tokens, int B, int64_t row_stride, int prompt_len, int gen_len, int L,
                   void* k_cache, void* v_cache, int cache_cap, int mode, float threshold, int k,
                   int32_t* pred, float* conf, int32_t* n_remaining, int32_t* steps_per_block, void* stream);
+
+/*
+ * Dual cache (prefix and suffix) for a fully bidirectional masked model (Section 3.4, rollout with KV-cache
+ * reuse): the rows [start, start + length) see cache[0 : kv_len) with kv_len >= start + length, i.e. also the
+ * positions behind them, whose K/V are whatever an earlier forward left in the cache.
+ *   dare_model_forward_window / dare_model_step_window: as dare_model_forward / dare_model_step with that extra
+ *     argument (kv_len = start + length gives exactly those calls).  start + length <= kv_len <= cache_cap, else
+ *     DARE_ERR_RANGE.  Enqueue on `stream`, no synchronisation.
+ *   dare_generate_dual: for each block of L positions, first one forward of ALL rows [0, T), T = prompt_len +
+ *     gen_len, seeing all of cache[0 : T) (this rewrites every position's K/V from the current tokens, the still
+ *     masked later blocks included), then the block's steps against cache[0 : T) until no rollout has a mask
+ *     left in it.  K/V outside the block are therefore as old as the last refresh while the block's tokens
+ *     change: that staleness is the method's approximation.  The model needs max_rows >= B * T
+ *     (DARE_ERR_SHAPE otherwise); prompt_len may be 0.  On return the cache holds, for each position, the K/V of
+ *     the last forward that covered it.  Other arguments as dare_generate.  This call BLOCKS until the loop has
+ *     finished.
+ */
+int dare_model_forward_window(dare_model* model, const int32_t* tokens, int B, int64_t row_stride, int start,
+                              int length, int kv_len, void* k_cache, void* v_cache, int cache_cap, void* hidden_out,
+                              void* stream);
+int dare_model_step_window(dare_model* model, int32_t* tokens, int B, int64_t row_stride, int block_start, int L,
+                           int kv_len, void* k_cache, void* v_cache, int cache_cap, int mode, float threshold, int k,
+                           int32_t* pred, float* conf, int32_t* n_committed, int32_t* n_remaining, void* stream);
+int dare_generate_dual(dare_model* model, int32_t* tokens, int B, int64_t row_stride, int prompt_len, int gen_len,
+                       int L, void* k_cache, void* v_cache, int cache_cap, int mode, float threshold, int k,
+                       int32_t* pred, float* conf, int32_t* n_remaining, int32_t* steps_per_block, void* stream);
 
 /*
  * Allocation-free variant of dare_lmhead_confidence.  (The paper has no counterpart for this entry

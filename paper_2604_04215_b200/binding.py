@@ -23,7 +23,8 @@ DEV_WAIT_EXPIRED = 2
 EXPORTS = ["dare_create", "dare_destroy", "dare_status_string", "dare_device_status", "dare_sm_count",
            "dare_attn_block", "dare_attn_varlen", "dare_lmhead_confidence", "dare_unmask_select", "dare_denoise_block",
            "dare_lmhead_confidence_static", "dare_lmhead_sample", "dare_lmhead_logprob", "dare_forward_mask", "dare_masked_nelbo", "dare_model_create", "dare_model_destroy", "dare_model_forward",
-           "dare_model_step", "dare_generate", "dare_linear", "dare_linear_plan", "dare_rmsnorm", "dare_rope_kv_write"]
+           "dare_model_step", "dare_generate", "dare_model_forward_window", "dare_model_step_window", "dare_generate_dual",
+           "dare_linear", "dare_linear_plan", "dare_rmsnorm", "dare_rope_kv_write"]
 
 _lib = None
 
@@ -90,6 +91,12 @@ def load():
     lib.dare_generate.argtypes = [vp, vp, i32, i64, i32, i32, i32, vp, vp, i32, i32, f32, i32, vp, vp, vp,
                                   C.POINTER(C.c_int32), vp]
     lib.dare_generate.restype = i32
+    lib.dare_model_forward_window.argtypes = [vp, vp, i32, i64, i32, i32, i32, vp, vp, i32, vp, vp]
+    lib.dare_model_forward_window.restype = i32
+    lib.dare_model_step_window.argtypes = [vp, vp, i32, i64, i32, i32, i32, vp, vp, i32, i32, f32, i32, vp, vp, vp, vp, vp]
+    lib.dare_model_step_window.restype = i32
+    lib.dare_generate_dual.argtypes = lib.dare_generate.argtypes
+    lib.dare_generate_dual.restype = i32
     lib.dare_linear.argtypes = [vp, i32, vp, i32, i32, vp, vp, i32, vp, vp, vp]
     lib.dare_linear.restype = i32
     lib.dare_linear_plan.argtypes = [vp, i32, i32, i32, i32, C.POINTER(C.c_int)]
@@ -455,4 +462,46 @@ def dare_generate(model: Model, tokens, prompt_len: int, gen_len: int, L: int, k
                               _ptr(n_remaining, torch.int32), steps, _stream(stream))
     if rc != 0 and check:
         raise DareError(rc, "dare_generate")
+    return list(steps) if check else rc
+
+
+def dare_model_forward_window(model: Model, tokens, start: int, length: int, kv_len: int, k_cache, v_cache,
+                              hidden_out=None, stream=None, check: bool = True):
+    """dare_model_forward with the rows seeing cache[0 : kv_len) (a cached suffix behind them)."""
+    B, row_stride = tokens.shape
+    bf = torch.bfloat16
+    rc = load().dare_model_forward_window(model.handle, _ptr(tokens, torch.int32), B, row_stride, int(start),
+                                          int(length), int(kv_len), _ptr(k_cache, bf), _ptr(v_cache, bf),
+                                          k_cache.shape[3], _ptr(hidden_out, bf), _stream(stream))
+    if rc != 0 and check:
+        raise DareError(rc, "dare_model_forward_window")
+    return rc
+
+
+def dare_model_step_window(model: Model, tokens, block_start: int, L: int, kv_len: int, k_cache, v_cache, mode: int,
+                           threshold: float, k: int, pred, conf, n_committed=None, n_remaining=None, stream=None,
+                           check: bool = True):
+    B, row_stride = tokens.shape
+    bf = torch.bfloat16
+    rc = load().dare_model_step_window(model.handle, _ptr(tokens, torch.int32), B, row_stride, int(block_start), int(L),
+                                       int(kv_len), _ptr(k_cache, bf), _ptr(v_cache, bf), k_cache.shape[3], int(mode),
+                                       float(threshold), int(k), _ptr(pred, torch.int32), _ptr(conf, torch.float32),
+                                       _ptr(n_committed, torch.int32), _ptr(n_remaining, torch.int32), _stream(stream))
+    if rc != 0 and check:
+        raise DareError(rc, "dare_model_step_window")
+    return rc
+
+
+def dare_generate_dual(model: Model, tokens, prompt_len: int, gen_len: int, L: int, k_cache, v_cache, mode: int,
+                       threshold: float, k: int, pred, conf, n_remaining, stream=None, check: bool = True):
+    """The dual-cache loop (blocks until done); returns the list of denoising steps taken per block."""
+    B, row_stride = tokens.shape
+    bf = torch.bfloat16
+    steps = (C.c_int32 * (gen_len // L))()
+    rc = load().dare_generate_dual(model.handle, _ptr(tokens, torch.int32), B, row_stride, int(prompt_len),
+                                   int(gen_len), int(L), _ptr(k_cache, bf), _ptr(v_cache, bf), k_cache.shape[3],
+                                   int(mode), float(threshold), int(k), _ptr(pred, torch.int32),
+                                   _ptr(conf, torch.float32), _ptr(n_remaining, torch.int32), steps, _stream(stream))
+    if rc != 0 and check:
+        raise DareError(rc, "dare_generate_dual")
     return list(steps) if check else rc

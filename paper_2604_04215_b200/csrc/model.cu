@@ -7,6 +7,11 @@
 // prefill (the prompt is one bidirectional segment); with start = a block's first position it is one
 // denoising step's stack, or, once the block holds no mask, the refresh that leaves the block's final K/V in
 // the cache before the prefix grows.
+//
+// A forward may also let its rows see cache[0, kv_len) with kv_len beyond the rows' own end: the positions
+// behind the rows are then a cached suffix (whatever an earlier forward wrote there).  That is the dual cache
+// of a fully bidirectional model: dare_generate_dual refreshes every position's K/V with one forward of the
+// whole sequence before each block and runs the block's steps against prefix + block + suffix.
 #include <math.h>
 #include <cuda_bf16.h>
 #include <new>
@@ -30,8 +35,9 @@ struct dare_model {
 
 namespace {
 
-int forward_rows(dare_model* m, const int32_t* tokens, int B, int64_t row_stride, int start, int length, void* k_cache,
-                 void* v_cache, int cap, void* hidden_out, cudaStream_t s) {
+// Keys visible to the rows: cache[0, kv_len), start + length <= kv_len <= cap.
+int forward_rows(dare_model* m, const int32_t* tokens, int B, int64_t row_stride, int start, int length, int kv_len,
+                 void* k_cache, void* v_cache, int cap, void* hidden_out, cudaStream_t s) {
     using namespace dare;
     const dare_model_desc& c = m->desc;
     const int rows = B * length;
@@ -54,7 +60,8 @@ int forward_rows(dare_model* m, const int32_t* tokens, int B, int64_t row_stride
         AttnArgs a;
         a.B = B; a.L = length; a.Hq = c.n_q_heads; a.Hkv = c.n_kv_heads; a.d = c.head_dim;
         a.prefix_cap = cap; a.suffix_cap = 0; a.scale = 0.f;
-        a.q = m->q; a.k_pre = kc; a.v_pre = vc; a.prefix_len = nullptr; a.prefix_len_uniform = start;
+        a.q = m->q; a.k_pre = kc; a.v_pre = vc; a.prefix_len = nullptr;
+        a.prefix_len_uniform = kv_len - length;   // in place: the kernel reads keys [0, this + length) of the cache
         a.k_blk = a.v_blk = a.k_suf = a.v_suf = nullptr; a.suffix_len = nullptr;
         a.out = m->attn; a.lse = nullptr;
         if (attn_workspace_bytes(a, attn_plan_splits(m->ctx, a)) > m->ctx->workspace_bytes) return DARE_ERR_WORKSPACE;
@@ -72,7 +79,7 @@ int forward_rows(dare_model* m, const int32_t* tokens, int B, int64_t row_stride
     return launch_rmsnorm(m->x, c.hidden, rows, c.rms_eps, hidden_out ? hidden_out : m->h, s);
 }
 
-int check_rows(const dare_model* m, const void* tokens, int B, int64_t row_stride, int start, int length,
+int check_rows(const dare_model* m, const void* tokens, int B, int64_t row_stride, int start, int length, int kv_len,
                const void* k_cache, const void* v_cache, int cap) {
     if (!m || !tokens || !k_cache || !v_cache) return DARE_ERR_NULL;
     if (B < 1 || length < 1 || B > m->max_batch) return DARE_ERR_SHAPE;
@@ -80,14 +87,15 @@ int check_rows(const dare_model* m, const void* tokens, int B, int64_t row_strid
     if (start < 0 || static_cast<long long>(start) + length > cap || cap > m->desc.max_positions ||
         static_cast<long long>(start) + length > row_stride)
         return DARE_ERR_RANGE;
+    if (kv_len < start + length || kv_len > cap) return DARE_ERR_RANGE;
     if ((reinterpret_cast<uintptr_t>(k_cache) & 15u) || (reinterpret_cast<uintptr_t>(v_cache) & 15u)) return DARE_ERR_ALIGN;
     return DARE_OK;
 }
 
-int step_rows(dare_model* m, int32_t* tokens, int B, int64_t row_stride, int start, int L, void* k_cache, void* v_cache,
-              int cap, int mode, float threshold, int k, int32_t* pred, float* conf, int32_t* n_committed,
+int step_rows(dare_model* m, int32_t* tokens, int B, int64_t row_stride, int start, int L, int kv_len, void* k_cache,
+              void* v_cache, int cap, int mode, float threshold, int k, int32_t* pred, float* conf, int32_t* n_committed,
               int32_t* n_remaining, cudaStream_t s) {
-    int rc = forward_rows(m, tokens, B, row_stride, start, L, k_cache, v_cache, cap, nullptr, s);
+    int rc = forward_rows(m, tokens, B, row_stride, start, L, kv_len, k_cache, v_cache, cap, nullptr, s);
     if (rc != DARE_OK) return rc;
     const int M = B * L;
     rc = dare::launch_lmhead(m->ctx, m->ctx->workspace, m->h, M, m->desc.hidden, m->lm_head, m->desc.vocab,
@@ -217,99 +225,174 @@ int dare_rope_kv_write(dare_model* m, const void* qkv, int B, int length, int st
                                       static_cast<cudaStream_t>(stream));
 }
 
+int dare_model_forward_window(dare_model* m, const int32_t* tokens, int B, int64_t row_stride, int start, int length,
+                              int kv_len, void* k_cache, void* v_cache, int cache_cap, void* hidden_out, void* stream) {
+    int rc = check_rows(m, tokens, B, row_stride, start, length, kv_len, k_cache, v_cache, cache_cap);
+    if (rc != DARE_OK) return rc;
+    return forward_rows(m, tokens, B, row_stride, start, length, kv_len, k_cache, v_cache, cache_cap, hidden_out,
+                        static_cast<cudaStream_t>(stream));
+}
+
 int dare_model_forward(dare_model* m, const int32_t* tokens, int B, int64_t row_stride, int start, int length,
                        void* k_cache, void* v_cache, int cache_cap, void* hidden_out, void* stream) {
-    int rc = check_rows(m, tokens, B, row_stride, start, length, k_cache, v_cache, cache_cap);
+    return dare_model_forward_window(m, tokens, B, row_stride, start, length, start + length, k_cache, v_cache,
+                                     cache_cap, hidden_out, stream);
+}
+
+int dare_model_step_window(dare_model* m, int32_t* tokens, int B, int64_t row_stride, int block_start, int L, int kv_len,
+                           void* k_cache, void* v_cache, int cache_cap, int mode, float threshold, int k, int32_t* pred,
+                           float* conf, int32_t* n_committed, int32_t* n_remaining, void* stream) {
+    int rc = check_rows(m, tokens, B, row_stride, block_start, L, kv_len, k_cache, v_cache, cache_cap);
+    if (rc == DARE_OK) rc = check_step(m, B, L, mode, threshold, k, pred, conf);
     if (rc != DARE_OK) return rc;
-    return forward_rows(m, tokens, B, row_stride, start, length, k_cache, v_cache, cache_cap, hidden_out,
-                        static_cast<cudaStream_t>(stream));
+    return step_rows(m, tokens, B, row_stride, block_start, L, kv_len, k_cache, v_cache, cache_cap, mode, threshold, k,
+                     pred, conf, n_committed, n_remaining, static_cast<cudaStream_t>(stream));
 }
 
 int dare_model_step(dare_model* m, int32_t* tokens, int B, int64_t row_stride, int block_start, int L, void* k_cache,
                     void* v_cache, int cache_cap, int mode, float threshold, int k, int32_t* pred, float* conf,
                     int32_t* n_committed, int32_t* n_remaining, void* stream) {
-    int rc = check_rows(m, tokens, B, row_stride, block_start, L, k_cache, v_cache, cache_cap);
-    if (rc == DARE_OK) rc = check_step(m, B, L, mode, threshold, k, pred, conf);
-    if (rc != DARE_OK) return rc;
-    return step_rows(m, tokens, B, row_stride, block_start, L, k_cache, v_cache, cache_cap, mode, threshold, k, pred,
-                     conf, n_committed, n_remaining, static_cast<cudaStream_t>(stream));
+    return dare_model_step_window(m, tokens, B, row_stride, block_start, L, block_start + L, k_cache, v_cache, cache_cap,
+                                  mode, threshold, k, pred, conf, n_committed, n_remaining, stream);
 }
+
+}  // extern "C"
+
+namespace {
+
+// The previous block's graph: destroyed once its launches are known to have finished.
+struct BlockGraph {
+    cudaGraph_t graph = nullptr;
+    cudaGraphExec_t exec = nullptr;
+    void destroy() {
+        if (exec) cudaGraphExecDestroy(exec);
+        if (graph) cudaGraphDestroy(graph);
+        exec = nullptr; graph = nullptr;
+    }
+};
+
+// All denoising steps of one block on the model's work stream.  The step (about forty launches with fixed
+// arguments) is captured once into a CUDA graph and replayed.
+//
+// A step whose block holds no mask any more does exactly what the refresh forward of the prefix-cache loop
+// must do (the LM head finds no live row, the selection changes nothing, the stack rewrites the block's K/V
+// from the committed tokens).  So step t + 1 is enqueued before step t's counts are read: when step t turns
+// out to have finished the block, step t + 1 was the refresh, and the GPU never waits for the host.  (In the
+// dual-cache loop that extra step is redundant and harmless: the next whole-sequence refresh rewrites the
+// same K/V.)
+int run_block(dare_model* m, int32_t* tokens, int B, int64_t row_stride, int start, int L, int kv_len, void* k_cache,
+              void* v_cache, int cap, int mode, float threshold, int k, int32_t* pred, float* conf, int32_t* n_remaining,
+              BlockGraph* old, int* steps_taken) {
+    cudaStream_t s = m->work;
+    BlockGraph cur;
+    if (cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal) != cudaSuccess) return DARE_ERR_CUDA;
+    int rc = step_rows(m, tokens, B, row_stride, start, L, kv_len, k_cache, v_cache, cap, mode, threshold, k, pred, conf,
+                       nullptr, n_remaining, s);
+    const cudaError_t end = cudaStreamEndCapture(s, &cur.graph);      // always ends the capture, also after an error
+    if (rc == DARE_OK && (end != cudaSuccess || cur.graph == nullptr)) rc = DARE_ERR_CUDA;
+    if (rc == DARE_OK && cudaGraphInstantiate(&cur.exec, cur.graph, 0) != cudaSuccess) rc = DARE_ERR_CUDA;
+    int issued = 0, taken = -1;
+    while (rc == DARE_OK && taken < 0) {
+        if (issued > L + 1) { rc = DARE_ERR_CUDA; break; }   // cannot happen: every step commits a token per row
+        const int slot = issued & 1;
+        if (cudaGraphLaunch(cur.exec, s) != cudaSuccess ||
+            cudaMemcpyAsync(m->host_counts + slot * m->max_batch, n_remaining, sizeof(int32_t) * B,
+                            cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+            cudaEventRecord(m->ev[slot], s) != cudaSuccess) {
+            rc = DARE_ERR_CUDA;
+            break;
+        }
+        ++issued;
+        if (issued >= 2) {
+            const int prev = (issued - 2) & 1;
+            if (cudaEventSynchronize(m->ev[prev]) != cudaSuccess) { rc = DARE_ERR_CUDA; break; }
+            old->destroy();      // a step of this block has finished, so every launch of the previous block has
+            bool done = true;
+            for (int r = 0; r < B; ++r) done = done && m->host_counts[prev * m->max_batch + r] == 0;
+            if (done) taken = issued - 1;   // steps 0 .. issued-2 denoised; the last one issued found no mask
+        }
+    }
+    if (old->exec) {      // (only if this block issued fewer than two steps or failed)
+        cudaStreamSynchronize(s);
+        old->destroy();
+    }
+    *old = cur;
+    *steps_taken = taken;
+    return rc;
+}
+
+// Order the model's work stream after the caller's stream (entry) / the caller's stream after it (exit).
+int enter_work_stream(dare_model* m, cudaStream_t user) {
+    if (cudaEventRecord(m->ev_in, user) != cudaSuccess || cudaStreamWaitEvent(m->work, m->ev_in, 0) != cudaSuccess)
+        return DARE_ERR_CUDA;
+    return DARE_OK;
+}
+int leave_work_stream(dare_model* m, cudaStream_t user, BlockGraph* old, int rc) {
+    const bool synced = cudaStreamSynchronize(m->work) == cudaSuccess;
+    old->destroy();
+    if (rc != DARE_OK) return rc;
+    if (!synced || cudaEventRecord(m->ev_out, m->work) != cudaSuccess ||
+        cudaStreamWaitEvent(user, m->ev_out, 0) != cudaSuccess)
+        return DARE_ERR_CUDA;
+    return DARE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+// The loops run on the model's own stream, ordered after the caller's stream at entry and before it at exit:
+// the caller's stream (possibly the legacy default stream) may not allow a capture.
 
 int dare_generate(dare_model* m, int32_t* tokens, int B, int64_t row_stride, int prompt_len, int gen_len, int L,
                   void* k_cache, void* v_cache, int cache_cap, int mode, float threshold, int k, int32_t* pred,
                   float* conf, int32_t* n_remaining, int32_t* steps_per_block, void* stream) {
     if (!n_remaining) return DARE_ERR_NULL;
     if (gen_len < 1 || L < 1 || gen_len % L != 0) return DARE_ERR_SHAPE;
-    int rc = check_rows(m, tokens, B, row_stride, 0, prompt_len, k_cache, v_cache, cache_cap);
-    if (rc == DARE_OK) rc = check_rows(m, tokens, B, row_stride, prompt_len + gen_len - L, L, k_cache, v_cache, cache_cap);
+    int rc = check_rows(m, tokens, B, row_stride, 0, prompt_len, prompt_len, k_cache, v_cache, cache_cap);
+    if (rc == DARE_OK)
+        rc = check_rows(m, tokens, B, row_stride, prompt_len + gen_len - L, L, prompt_len + gen_len, k_cache, v_cache,
+                        cache_cap);
     if (rc == DARE_OK) rc = check_step(m, B, L, mode, threshold, k, pred, conf);
     if (rc != DARE_OK) return rc;
-    // The loop runs on the model's own stream, ordered after the caller's stream at entry and before it at
-    // exit: a block's denoising step (about forty launches with fixed arguments) is captured once into a CUDA
-    // graph and replayed, which the caller's stream (possibly the legacy default stream) may not allow.
     cudaStream_t user = static_cast<cudaStream_t>(stream);
-    cudaStream_t s = m->work;
-    if (cudaEventRecord(m->ev_in, user) != cudaSuccess || cudaStreamWaitEvent(s, m->ev_in, 0) != cudaSuccess)
-        return DARE_ERR_CUDA;
-    rc = forward_rows(m, tokens, B, row_stride, 0, prompt_len, k_cache, v_cache, cache_cap, nullptr, s);
+    rc = enter_work_stream(m, user);
     if (rc != DARE_OK) return rc;
-    // A step whose block holds no mask any more does exactly what the refresh forward must do (the LM head
-    // finds no live row, the selection changes nothing, the stack rewrites the block's K/V from the committed
-    // tokens).  So step t + 1 is enqueued before step t's counts are read: when step t turns out to have
-    // finished the block, step t + 1 was the refresh, and the GPU never waits for the host.
-    cudaGraph_t old_graph = nullptr;         // the previous block's graph: destroyed once its launches are known done
-    cudaGraphExec_t old_exec = nullptr;
+    rc = forward_rows(m, tokens, B, row_stride, 0, prompt_len, prompt_len, k_cache, v_cache, cache_cap, nullptr, m->work);
+    BlockGraph old;
     for (int b = 0; b < gen_len / L && rc == DARE_OK; ++b) {
         const int start = prompt_len + b * L;
-        cudaGraph_t graph = nullptr;
-        cudaGraphExec_t exec = nullptr;
-        if (cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal) != cudaSuccess) return DARE_ERR_CUDA;
-        rc = step_rows(m, tokens, B, row_stride, start, L, k_cache, v_cache, cache_cap, mode, threshold, k, pred, conf,
-                       nullptr, n_remaining, s);
-        const cudaError_t end = cudaStreamEndCapture(s, &graph);      // always ends the capture, also after an error
-        if (rc == DARE_OK && (end != cudaSuccess || graph == nullptr)) rc = DARE_ERR_CUDA;
-        if (rc == DARE_OK && cudaGraphInstantiate(&exec, graph, 0) != cudaSuccess) rc = DARE_ERR_CUDA;
-        int issued = 0, taken = -1;
-        while (rc == DARE_OK && taken < 0) {
-            if (issued > L + 1) { rc = DARE_ERR_CUDA; break; }   // cannot happen: every step commits a token per row
-            const int slot = issued & 1;
-            if (cudaGraphLaunch(exec, s) != cudaSuccess ||
-                cudaMemcpyAsync(m->host_counts + slot * m->max_batch, n_remaining, sizeof(int32_t) * B,
-                                cudaMemcpyDeviceToHost, s) != cudaSuccess ||
-                cudaEventRecord(m->ev[slot], s) != cudaSuccess) {
-                rc = DARE_ERR_CUDA;
-                break;
-            }
-            ++issued;
-            if (issued >= 2) {
-                const int prev = (issued - 2) & 1;
-                if (cudaEventSynchronize(m->ev[prev]) != cudaSuccess) { rc = DARE_ERR_CUDA; break; }
-                if (old_exec) {      // a step of this block has finished, so every launch of the previous block has
-                    cudaGraphExecDestroy(old_exec);
-                    cudaGraphDestroy(old_graph);
-                    old_exec = nullptr; old_graph = nullptr;
-                }
-                bool done = true;
-                for (int r = 0; r < B; ++r) done = done && m->host_counts[prev * m->max_batch + r] == 0;
-                if (done) taken = issued - 1;   // steps 0 .. issued-2 denoised; the last one issued was the refresh
-            }
-        }
+        int taken = -1;
+        rc = run_block(m, tokens, B, row_stride, start, L, start + L, k_cache, v_cache, cache_cap, mode, threshold, k,
+                       pred, conf, n_remaining, &old, &taken);
         if (rc == DARE_OK && steps_per_block) steps_per_block[b] = taken;
-        if (old_exec) {      // (only if this block issued fewer than two steps or failed)
-            cudaStreamSynchronize(s);
-            cudaGraphExecDestroy(old_exec);
-            cudaGraphDestroy(old_graph);
-        }
-        old_exec = exec;
-        old_graph = graph;
     }
-    const bool synced = cudaStreamSynchronize(s) == cudaSuccess;
-    if (old_exec) cudaGraphExecDestroy(old_exec);
-    if (old_graph) cudaGraphDestroy(old_graph);
+    return leave_work_stream(m, user, &old, rc);
+}
+
+int dare_generate_dual(dare_model* m, int32_t* tokens, int B, int64_t row_stride, int prompt_len, int gen_len, int L,
+                       void* k_cache, void* v_cache, int cache_cap, int mode, float threshold, int k, int32_t* pred,
+                       float* conf, int32_t* n_remaining, int32_t* steps_per_block, void* stream) {
+    if (!n_remaining) return DARE_ERR_NULL;
+    if (prompt_len < 0 || gen_len < 1 || L < 1 || gen_len % L != 0) return DARE_ERR_SHAPE;
+    const int T = prompt_len + gen_len;
+    int rc = check_rows(m, tokens, B, row_stride, 0, T, T, k_cache, v_cache, cache_cap);   // the refresh: all rows
+    if (rc == DARE_OK) rc = check_step(m, B, L, mode, threshold, k, pred, conf);
     if (rc != DARE_OK) return rc;
-    if (!synced || cudaEventRecord(m->ev_out, s) != cudaSuccess || cudaStreamWaitEvent(user, m->ev_out, 0) != cudaSuccess)
-        return DARE_ERR_CUDA;
-    return DARE_OK;
+    cudaStream_t user = static_cast<cudaStream_t>(stream);
+    rc = enter_work_stream(m, user);
+    if (rc != DARE_OK) return rc;
+    BlockGraph old;
+    for (int b = 0; b < gen_len / L && rc == DARE_OK; ++b) {
+        const int start = prompt_len + b * L;
+        rc = forward_rows(m, tokens, B, row_stride, 0, T, T, k_cache, v_cache, cache_cap, nullptr, m->work);
+        if (rc != DARE_OK) break;
+        int taken = -1;
+        rc = run_block(m, tokens, B, row_stride, start, L, T, k_cache, v_cache, cache_cap, mode, threshold, k, pred, conf,
+                       n_remaining, &old, &taken);
+        if (rc == DARE_OK && steps_per_block) steps_per_block[b] = taken;
+    }
+    return leave_work_stream(m, user, &old, rc);
 }
 
 }  // extern "C"

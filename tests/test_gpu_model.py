@@ -241,6 +241,89 @@ def test_loop_small_step_by_step_and_generate(ctx, name):
     model.close()
 
 
+@pytest.mark.parametrize("name", ["loop_small_gqa", "loop_small_bd4"])
+def test_dual_cache_loop_step_by_step_and_generate(ctx, name):
+    """Prefix + suffix cache of a fully bidirectional model: whole-sequence refresh before each block, block steps
+    against cache[0 : T).  Teacher-forced like the prefix-cache loop; then the one-call loop."""
+    mw = I.MODEL_WORKLOADS[name]
+    wts_t = I.make_model_weights(mw)
+    cfg, wts = _cfg(mw), _oracle_weights(wts_t)
+    B, L, P, G = mw.batch, mw.block_len, mw.prompt_len, mw.gen_len
+    T = P + G
+    model = _model(ctx, mw, wts_t, max_rows=B * T)
+    tok0 = I.fresh_model_tokens(mw)
+    kc, vc = model.new_cache(B, T)
+    pred = torch.empty(B * L, dtype=torch.int32, device="cuda")
+    conf = torch.empty(B * L, dtype=torch.float32, device="cuda")
+    nc = torch.zeros(B, dtype=torch.int32, device="cuda")
+    nr = torch.zeros(B, dtype=torch.int32, device="cuda")
+    hid = torch.empty(B * T, mw.hidden, dtype=torch.bfloat16, device="cuda")
+    hid_blk = torch.empty(B * L, mw.hidden, dtype=torch.bfloat16, device="cuda")
+    ocache = MO.new_cache(cfg, B, T)
+    tok = tok0.cuda()
+    steps_manual = []
+    for b in range(G // L):
+        start = P + b * L
+        # ---- refresh: every row, every key
+        dare.dare_model_forward_window(model, tok, 0, T, T, kc, vc, hidden_out=hid)
+        torch.cuda.synchronize()
+        ref_h = MO.forward_block_cached(cfg, wts, tok.cpu().numpy(), 0, T, ocache)
+        _check_hidden(hid, ref_h, mw.n_layers)
+        for li in range(mw.n_layers):
+            _check_hidden(kc[li], ocache[li][0], li + 1)
+            _check_hidden(vc[li], ocache[li][1], li + 1)
+        # ---- a window forward right after the refresh gives the refresh's own rows (same kernels, other shapes)
+        dare.dare_model_forward_window(model, tok, start, L, T, kc, vc, hidden_out=hid_blk)
+        torch.cuda.synchronize()
+        want = hid.view(B, T, -1)[:, start:start + L].reshape(B * L, -1).float()
+        assert (hid_blk.float() - want).abs().max().item() <= HIDDEN_MAX_ABS_PER_LAYER * mw.n_layers
+        MO.forward_block_cached(cfg, wts, tok.cpu().numpy(), start, L, ocache, kv_len=T)
+        n = 0
+        while True:
+            pre = tok.cpu().numpy()
+            if not (pre[:, start:start + L] == mw.mask_id).any():
+                break
+            dare.dare_model_step_window(model, tok, start, L, T, kc, vc, mw.mode, mw.threshold, mw.k, pred, conf, nc, nr)
+            torch.cuda.synchronize()
+            res = MO.denoise_step_dual(cfg, wts, pre, start, L, T, ocache, mw.mode, mw.threshold, mw.k)
+            _check_lm(pred, conf, res["lm"], mw.n_layers)
+            want_tok, wnc, wnr = O.unmask_select(pre, start, L, pred.cpu().numpy(), conf.cpu().numpy(), mw.mask_id,
+                                                 mw.mode, mw.threshold, mw.k)
+            np.testing.assert_array_equal(tok.cpu().numpy(), want_tok)
+            np.testing.assert_array_equal(nc.cpu().numpy(), wnc)
+            np.testing.assert_array_equal(nr.cpu().numpy(), wnr)
+            for li in range(mw.n_layers):       # the block's rows were rewritten, the rest of the cache is as it was
+                _check_hidden(kc[li], ocache[li][0], li + 1)
+            n += 1
+            assert n <= L
+        steps_manual.append(n)
+    final_manual = tok.cpu().numpy()
+    assert (final_manual[:, P:] != mw.mask_id).all()
+    np.testing.assert_array_equal(final_manual[:, :P], tok0.numpy()[:, :P])
+    if mw.mode == I.SELECT_TOPK:
+        assert steps_manual == [-(-L // mw.k)] * (G // L)
+    assert ctx.device_status() == 0
+
+    # ---- the one-call loop: same tokens and steps; same cache except the last block's rows, which the loop's
+    # trailing step rewrote from the final tokens
+    tok2 = tok0.cuda()
+    kc2, vc2 = model.new_cache(B, T)
+    steps = dare.dare_generate_dual(model, tok2, P, G, L, kc2, vc2, mw.mode, mw.threshold, mw.k, pred, conf, nr)
+    np.testing.assert_array_equal(tok2.cpu().numpy(), final_manual)
+    assert steps == steps_manual
+    assert torch.equal(kc2[:, :, :, :T - L], kc[:, :, :, :T - L]) and torch.equal(vc2[:, :, :, :T - L], vc[:, :, :, :T - L])
+    assert ctx.device_status() == 0
+
+    # ---- argument checks: the window must contain the rows and fit the cache; the refresh needs max_rows >= B * T
+    assert dare.dare_model_forward_window(model, tok2, P, L, P + L - 1, kc2, vc2, check=False) == -4
+    assert dare.dare_model_forward_window(model, tok2, P, L, T + 1, kc2, vc2, check=False) == -4
+    small = _model(ctx, mw, wts_t, max_rows=B * L)
+    assert dare.dare_generate_dual(small, tok2, P, G, L, kc2, vc2, mw.mode, mw.threshold, mw.k, pred, conf, nr,
+                                   check=False) == -2
+    small.close()
+    model.close()
+
+
 class _LazyLayer:
     """fp64 views of one layer's bf16 weights, converted when touched (the full-size stack would need 7 GB)."""
 
