@@ -334,12 +334,13 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def _model_objects(dare, ctx, mw, wts_h):
+def _model_objects(dare, ctx, mw, wts_h, max_rows=None):
     layers = [{k: v.cuda() for k, v in l.items()} for l in wts_h["layers"]]
     return dare.Model(ctx, n_layers=mw.n_layers, hidden=mw.hidden, n_q_heads=mw.n_q_heads, n_kv_heads=mw.n_kv_heads,
                       head_dim=mw.head_dim, ffn=mw.ffn, vocab=mw.vocab, mask_id=mw.mask_id,
                       embedding=wts_h["embedding"].cuda(), layers=layers, lm_head=wts_h["lm_head"].cuda(),
-                      max_positions=mw.row_len, max_rows=mw.batch * max(mw.prompt_len, mw.block_len),
+                      max_positions=mw.row_len,
+                      max_rows=max_rows or mw.batch * max(mw.prompt_len, mw.block_len),
                       max_batch=mw.batch, rms_eps=mw.rms_eps, rope_base=mw.rope_base)
 
 
@@ -362,8 +363,10 @@ def run_model(args):
     wts_h = I.make_model_weights(mw)                                   # same weights on every rank
     mw_rank = I.ModelWorkload(**{**mw.__dict__, "seed": rank})         # its own prompts
     ctx = dare.Context(local)
-    model = _model_objects(dare, ctx, mw, wts_h)
+    dual = args.cache == "dual"           # whole-sequence refresh before each block, steps see prefix + block + suffix
+    model = _model_objects(dare, ctx, mw, wts_h, max_rows=mw.batch * (mw.prompt_len + mw.gen_len) if dual else None)
     B, L, P, G = mw.batch, mw.block_len, mw.prompt_len, mw.gen_len
+    loop = dare.dare_generate_dual if dual else dare.dare_generate
     tok0_h = I.fresh_model_tokens(mw_rank).pin_memory()
     tok0 = tok0_h.cuda()
     tok = tok0.clone()
@@ -378,8 +381,7 @@ def run_model(args):
 
     def generation(src):
         tok.copy_(src, non_blocking=True)
-        return dare.dare_generate(model, tok, P, G, L, kc, vc, mw.mode, mw.threshold, mw.k, pred, conf, nr,
-                                  stream=stream)
+        return loop(model, tok, P, G, L, kc, vc, mw.mode, mw.threshold, mw.k, pred, conf, nr, stream=stream)
 
     def barrier():
         torch.cuda.synchronize()
@@ -473,12 +475,15 @@ def run_model(args):
         cpu_baseline = time_model_oracle(mw, wts_h, budget_s=20.0)
     if rank == 0:
         per_fwd = 2 + 8 * mw.n_layers                   # embedding, final norm, 8 launches per layer
-        launches = n_gen * (per_fwd + (steps_taken // n_gen + G // L) * (per_fwd + 4))
+        # per generation: the prefill (prefix cache) or one refresh per block (dual cache), then per block its steps
+        # plus the trailing one, each a forward + LM head (3 kernels) + selection
+        launches = n_gen * ((G // L if dual else 1) * per_fwd + (steps_taken // n_gen + G // L) * (per_fwd + 4))
         out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps_taken, "warmup": args.warmup,
                "ms_per_step": ms_max / max(steps_taken, 1), "higher_is_better": True, "scaling": "weak",
                "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
                "config": {"workload": f"{mw.name}: {mw.n_layers} layers D{D} Hq{mw.n_q_heads}/Hkv{mw.n_kv_heads} "
-                                      f"d{mw.head_dim} F{F} V{mw.vocab} B{B} prompt{P}+gen{G} L{L} tau {mw.threshold}",
+                                      f"d{mw.head_dim} F{F} V{mw.vocab} B{B} prompt{P}+gen{G} L{L} tau {mw.threshold}, "
+                                      + ("dual cache (whole-sequence refresh per block)" if dual else "prefix cache"),
                           "generations": n_gen, "ms_per_generation": ms_max / n_gen,
                           "l2": "inputs larger than L2 (2.8 GB of weights are re-read every step)",
                           "parallelism": f"dp{world} (independent rollouts per GPU, no collective)"},
@@ -592,6 +597,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llada8b", choices=sorted(I.WORKLOADS) + sorted(I.MODEL_WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cache", default="prefix", choices=["prefix", "dual"],
+                    help="loop workloads: prefix cache (block-causal) or dual cache (bidirectional, refresh per block)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (0 = as defined)")
     args = ap.parse_args()
     if args.impl == "reference":
