@@ -98,7 +98,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     GemmBarriers* bars = reinterpret_cast<GemmBarriers*>(tiles + p.stages * stage_bytes);
     volatile uint32_t* abort_flag = &bars->abort_flag;
 
-    const int warp = threadIdx.x >> 5;
+    const int warp = warp_index_uniform();
     const int lane = threadIdx.x & 31;
     // CTA -> (K split, row item, column tile): the splits of one output tile form a cluster, row items next
     const int split = p.splits > 1 ? static_cast<int>(cluster_cta_rank()) : 0;
@@ -160,28 +160,34 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            const uint32_t idesc = umma_idesc_bf16(GM, p.bn);
-            int stage = 0;
-            uint32_t phase = 0;
-            bool ok = true;
-            for (int kb = kb_begin; kb < kb_end; ++kb) {
-                if (!mbar_wait(&bars->full[stage], phase, abort_flag)) { ok = false; break; }
-                tc_fence_after_sync();
-                const uint32_t a_addr = smem_u32(tiles + stage * stage_bytes);
-                const uint64_t b_desc = umma_desc_sw128_kmajor(a_addr + p.nsub * A_TILE_BYTES);
+        // all lanes run the loop, one elected lane issues the MMAs and their commits
+        const bool leader = elect_one_sync();
+        const uint32_t idesc = umma_idesc_bf16(GM, p.bn);
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        for (int kb = kb_begin; kb < kb_end; ++kb) {
+            ok = __all_sync(0xffffffffu, mbar_wait(&bars->full[stage], phase, abort_flag));
+            if (!ok) break;
+            tc_fence_after_sync();
+            const uint32_t a_addr = smem_u32(tiles + stage * stage_bytes);
+            const uint64_t b_desc = umma_desc_sw128_kmajor(a_addr + p.nsub * A_TILE_BYTES);
+            const uint32_t accumulate = kb > kb_begin;
+            if (leader) {
                 for (int s = 0; s < p.nsub; ++s) {
                     const uint64_t a_desc = umma_desc_sw128_kmajor(a_addr + s * A_TILE_BYTES);
 #pragma unroll
                     for (int kk = 0; kk < GK / 16; ++kk)   // +32 bytes along K per step = +2 descriptor units
                         umma_bf16(tmem_base + s * acc_stride, a_desc + 2 * kk, b_desc + 2 * kk, idesc,
-                                  (kb > kb_begin) || kk != 0);
+                                  accumulate | (kk != 0));
                 }
                 umma_commit(&bars->empty[stage]);
-                if (++stage == p.stages) { stage = 0; phase ^= 1; }
             }
-            if (ok) umma_commit(&bars->tmem_full);
+            __syncwarp();
+            if (++stage == p.stages) { stage = 0; phase ^= 1; }
         }
+        if (ok && leader) umma_commit(&bars->tmem_full);
+        __syncwarp();
     }
 
     // ---- epilogue (warps 2..9).  Warp w may touch TMEM lanes [32 * (w % 4), +32); warps 2..5 are set 0, warps

@@ -154,7 +154,7 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     LmBarriers* bars = reinterpret_cast<LmBarriers*>(tiles + STAGES * STAGE_BYTES);
     volatile uint32_t* abort_flag = &bars->abort_flag;
 
-    const int warp = threadIdx.x >> 5;
+    const int warp = warp_index_uniform();
     const int lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
@@ -203,25 +203,29 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            constexpr uint32_t idesc = umma_idesc_bf16(BM, BN);
-            int stage = 0;
-            uint32_t phase = 0;
-            int it = 0;
-            bool ok = true;
-            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-                for (int n_tile = item / m_tiles; n_tile < n_tiles && ok; n_tile += groups, ++it) {
-                    const int acc = it & 1;
-                    const uint32_t acc_phase = (it >> 1) & 1;
-                    if (!mbar_wait(&bars->tmem_empty[acc], acc_phase ^ 1, abort_flag)) { ok = false; break; }
+        // all lanes run the loops, one elected lane issues the MMAs and their commits
+        const bool leader = elect_one_sync();
+        constexpr uint32_t idesc = umma_idesc_bf16(BM, BN);
+        int stage = 0;
+        uint32_t phase = 0;
+        int it = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+            for (int n_tile = item / m_tiles; n_tile < n_tiles && ok; n_tile += groups, ++it) {
+                const int acc = it & 1;
+                const uint32_t acc_phase = (it >> 1) & 1;
+                ok = __all_sync(0xffffffffu, mbar_wait(&bars->tmem_empty[acc], acc_phase ^ 1, abort_flag));
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + acc * BN;
+                for (int kb = 0; kb < num_k; ++kb) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(&bars->full[stage], phase, abort_flag));
+                    if (!ok) break;
                     tc_fence_after_sync();
-                    const uint32_t d_tmem = tmem_base + acc * BN;
-                    for (int kb = 0; kb < num_k; ++kb) {
-                        if (!mbar_wait(&bars->full[stage], phase, abort_flag)) { ok = false; break; }
-                        tc_fence_after_sync();
-                        const uint32_t a_addr = smem_u32(tiles + stage * STAGE_BYTES);
-                        const uint64_t a_desc = umma_desc_sw128_kmajor(a_addr);
-                        const uint64_t b_desc = umma_desc_sw128_kmajor(a_addr + A_BYTES);
+                    const uint32_t a_addr = smem_u32(tiles + stage * STAGE_BYTES);
+                    const uint64_t a_desc = umma_desc_sw128_kmajor(a_addr);
+                    const uint64_t b_desc = umma_desc_sw128_kmajor(a_addr + A_BYTES);
+                    if (leader) {
 #pragma unroll
                         for (int kk = 0; kk < BK / 16; ++kk) {
                             // 16 bf16 = 32 bytes further along K inside the 128-byte swizzled row: +2 in the
@@ -229,10 +233,12 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
                             umma_bf16(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0);
                         }
                         umma_commit(&bars->empty[stage]);   // frees the stage when these MMAs have read it
-                        if (++stage == STAGES) { stage = 0; phase ^= 1; }
                     }
-                    if (ok) umma_commit(&bars->tmem_full[acc]);
+                    __syncwarp();
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
+                if (ok && leader) umma_commit(&bars->tmem_full[acc]);
+                __syncwarp();
             }
         }
     } else {

@@ -149,6 +149,25 @@ __device__ __forceinline__ void tc_fence_before_sync() {
 __device__ __forceinline__ void tc_fence_after_sync() {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 }
+// True in exactly one lane of a fully converged warp, the same lane on every call.  The MMA-issuing warps run
+// their loops with all 32 lanes (waits, counters and descriptor arithmetic stay warp-uniform, which lets the
+// compiler keep them in the uniform datapath the MMA instruction takes its operands from) and only the
+// instructions that must come from a single thread sit under this predicate.
+__device__ __forceinline__ bool elect_one_sync() {
+    uint32_t pred;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "elect.sync _|p, 0xffffffff;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(pred));
+    return pred != 0;
+}
+// The warp's index, in a form the compiler knows to be the same in all lanes.
+__device__ __forceinline__ int warp_index_uniform() {
+    return __shfl_sync(0xffffffffu, static_cast<int>(threadIdx.x >> 5), 0);
+}
 // D[tmem] (+)= A[smem] * B[smem], one thread issues.  accumulate == 0 overwrites D.
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                           uint32_t accumulate) {
