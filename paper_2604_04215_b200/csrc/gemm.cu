@@ -294,6 +294,271 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     }
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// CTA-pair variant (cta_group::2), used when the problem has at least two row tiles.  The two CTAs of a cluster
+// compute one 256-row x bn-column tile with MMAs of M = 256: each CTA loads its own 128 rows of A and only HALF
+// of the W rows of every MMA (the tensor cores exchange the halves), and holds 128 rows x bn columns of the
+// accumulator.  Per flop a CTA writes and reads a third less shared memory than a single CTA computing a
+// 128-row tile, which is what limits the single-CTA kernel.  bn may exceed 256: the tile is then made of two
+// MMAs of bn / 2 columns per K step.  SwiGLU: the even CTA loads the gate rows, the odd CTA the matching up rows,
+// so that every accumulator row holds [gate | up] column pairs.
+struct PairPlan {
+    int bn;          // accumulator columns per tile = W rows per tile and K block (both CTAs together)
+    int wcols;       // output columns per tile (bn, or bn / 2 for SwiGLU)
+    int nmma;        // MMAs per K step (1 or 2), each nchunk columns wide
+    int nchunk;
+    int stages;
+    int m_pairs, n_tiles;
+    uint32_t tmem_cols;
+};
+
+struct PairArgs {
+    int M, N, K, ldo;
+    PairPlan p;
+    __nv_bfloat16* out;
+    const __nv_bfloat16* res;
+    uint32_t* dev_status;
+};
+
+template <int EPI>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                 const __grid_constant__ CUtensorMap tmap_b2, const PairArgs g) {
+    const PairPlan& p = g.p;
+    const int half_rows = p.nchunk / 2;                      // W rows this CTA holds per MMA
+    const int chunk_bytes = half_rows * (GK * 2);
+    const int stage_bytes = A_TILE_BYTES + p.nmma * chunk_bytes;
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    GemmBarriers* bars = reinterpret_cast<GemmBarriers*>(tiles + p.stages * stage_bytes);
+    volatile uint32_t* abort_flag = &bars->abort_flag;
+
+    const int warp = warp_index_uniform();
+    const int lane = threadIdx.x & 31;
+    const int rank = static_cast<int>(cluster_cta_rank());   // 0: issues the MMAs and owns the "full" barriers
+    const int pair = blockIdx.x >> 1;
+    const int m_pair = pair % p.m_pairs;                      // row index fastest: pairs sharing W run together
+    const int n_tile = pair / p.m_pairs;
+    const int nk = (g.K + GK - 1) / GK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) {
+            mbar_init(&bars->full[s], 1);
+            mbar_init(&bars->empty[s], 1);
+        }
+        mbar_init(&bars->tmem_full, 1);
+        bars->abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(&bars->tmem_base, p.tmem_cols);
+        tmem_relinquish_pair();
+    }
+    tc_fence_before_sync();
+    cluster_sync_all();              // both CTAs' barriers exist before either CTA signals the other's
+    tc_fence_after_sync();
+    const uint32_t tmem_base = bars->tmem_base;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            prefetch_tensormap(&tmap_a);
+            prefetch_tensormap(&tmap_b);
+            if (EPI == GEMM_EPI_SWIGLU) prefetch_tensormap(&tmap_b2);
+            const CUtensorMap* tmap_w = (EPI == GEMM_EPI_SWIGLU && rank == 1) ? &tmap_b2 : &tmap_b;
+            // W row of chunk 0 for this CTA; chunk c starts w_step rows further on
+            const int w_row0 = EPI == GEMM_EPI_SWIGLU ? n_tile * p.wcols : n_tile * p.bn + rank * half_rows;
+            const int w_step = EPI == GEMM_EPI_SWIGLU ? half_rows : p.nchunk;
+            const uint32_t full0 = cluster_map_shared(smem_u32(&bars->full[0]), 0);   // the even CTA's barriers
+            int stage = 0;
+            uint32_t phase = 0;
+            for (int kb = 0; kb < nk; ++kb) {
+                if (!mbar_wait(&bars->empty[stage], phase ^ 1, abort_flag)) break;
+                uint8_t* a_dst = tiles + stage * stage_bytes;
+                uint8_t* b_dst = a_dst + A_TILE_BYTES;
+                const uint32_t full = full0 + stage * static_cast<uint32_t>(sizeof(uint64_t));
+                if (rank == 0) mbar_arrive_expect_tx(&bars->full[stage], 2 * stage_bytes);   // both CTAs' bytes
+                tma_load_2d_pair(a_dst, &tmap_a, full, kb * GK, m_pair * 2 * GM + rank * GM);
+                for (int c = 0; c < p.nmma; ++c)
+                    tma_load_2d_pair(b_dst + c * chunk_bytes, tmap_w, full, kb * GK, w_row0 + c * w_step);
+                if (++stage == p.stages) { stage = 0; phase ^= 1; }
+            }
+        }
+    } else if (warp == 1 && rank == 0) {
+        // all lanes run the loop, one elected lane issues the MMAs and their commits (which arrive in both CTAs)
+        const bool leader = elect_one_sync();
+        const uint32_t idesc = umma_idesc_bf16(2 * GM, p.nchunk);
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        for (int kb = 0; kb < nk; ++kb) {
+            ok = __all_sync(0xffffffffu, mbar_wait(&bars->full[stage], phase, abort_flag));
+            if (!ok) break;
+            tc_fence_after_sync();
+            const uint32_t a_addr = smem_u32(tiles + stage * stage_bytes);
+            const uint64_t a_desc = umma_desc_sw128_kmajor(a_addr);
+            const uint32_t accumulate = kb > 0;
+            if (leader) {
+                for (int c = 0; c < p.nmma; ++c) {
+                    const uint64_t b_desc = umma_desc_sw128_kmajor(a_addr + A_TILE_BYTES + c * chunk_bytes);
+#pragma unroll
+                    for (int kk = 0; kk < GK / 16; ++kk)   // +32 bytes along K per step = +2 descriptor units
+                        umma_bf16_pair(tmem_base + c * p.nchunk, a_desc + 2 * kk, b_desc + 2 * kk, idesc,
+                                       accumulate | (kk != 0));
+                }
+                umma_commit_pair(&bars->empty[stage], 3);
+            }
+            __syncwarp();
+            if (++stage == p.stages) { stage = 0; phase ^= 1; }
+        }
+        if (ok && leader) umma_commit_pair(&bars->tmem_full, 3);
+        __syncwarp();
+    }
+
+    // ---- epilogue (warps 2..9 of both CTAs): warp w may touch TMEM lanes [32 * (w % 4), +32); the two sets of
+    // four warps alternate over the 8-column groups of the CTA's 128 rows
+    if (warp >= 2) {
+        const int lq = warp & 3;
+        const int set = (warp - 2) >> 2;
+        const int n_groups = p.wcols / 8;
+        const int row = m_pair * 2 * GM + rank * GM + lq * 32 + lane;
+        const bool row_ok = row < g.M;
+        const size_t row_off = static_cast<size_t>(row) * g.ldo;
+        const int col_base = n_tile * p.wcols;
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(lq * 32) << 16);
+        mbar_wait(&bars->tmem_full, 0, abort_flag);     // (a wait that gave up leaves the abort flag set)
+        tc_fence_after_sync();
+        __syncwarp();
+        if (!*abort_flag) {
+            for (int gi = set; gi < n_groups; gi += 2) {
+                uint32_t v[8];
+                float f[8], u[8];
+                if (EPI == GEMM_EPI_SWIGLU) {
+                    const int j = gi * 8, c = j / half_rows;
+                    const int gcol = c * p.nchunk + (j - c * half_rows);
+                    uint32_t w[8];
+                    tmem_ld_8cols(taddr + gcol, v);
+                    tmem_ld_8cols(taddr + gcol + half_rows, w);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) u[k] = __uint_as_float(w[k]);
+                } else {
+                    tmem_ld_8cols(taddr + gi * 8, v);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) u[k] = 0.f;
+                }
+#pragma unroll
+                for (int k = 0; k < 8; ++k) f[k] = __uint_as_float(v[k]);
+                const int col = col_base + gi * 8;
+                if (row_ok && col < g.N) store_group<EPI>(f, u, g.out, g.res, row_off + col);
+            }
+        }
+    }
+
+    // teardown: neither CTA may leave while its partner can still signal its barriers or read its tiles
+    tc_fence_before_sync();
+    cluster_sync_all();
+    if (*abort_flag) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) {}   // let copies in flight land before the shared memory goes away
+        if (threadIdx.x == 0) atomicOr(g.dev_status, DEV_WAIT_EXPIRED);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc_pair(tmem_base, p.tmem_cols);
+    }
+}
+
+template <int EPI>
+int launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tb2, const PairArgs& g,
+                cudaStream_t stream, int* max_clusters_query) {
+    if (cudaFuncSetAttribute(gemm_pair_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_BYTES) !=
+        cudaSuccess)
+        return DARE_ERR_CUDA;
+    const long long ctas = 2LL * g.p.m_pairs * g.p.n_tiles;
+    if (ctas > 0x7fffffffLL) return DARE_ERR_SHAPE;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(ctas), 1, 1);
+    cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = GEMM_SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    if (max_clusters_query) {
+        cfg.gridDim = dim3(2048u, 1, 1);
+        return cudaOccupancyMaxActiveClusters(max_clusters_query, gemm_pair_kernel<EPI>, &cfg) == cudaSuccess
+                   ? DARE_OK : DARE_ERR_CUDA;
+    }
+    return cudaLaunchKernelEx(&cfg, gemm_pair_kernel<EPI>, ta, tb, tb2, g) == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
+}
+
+// CTA pairs of the pair kernel that can be resident at once (cached; 0 = it cannot run).
+int max_active_pairs() {
+    static int cache = -1;
+    if (cache < 0) {
+        PairArgs g{};
+        g.p.m_pairs = g.p.n_tiles = 1;
+        CUtensorMap dummy{};
+        int n = 0;
+        if (launch_pair<GEMM_EPI_STORE>(dummy, dummy, dummy, g, nullptr, &n) != DARE_OK) n = 0;
+        cache = n;
+    }
+    return cache;
+}
+
+// Tile shape for the pair kernel.  Per K block a CTA's time is the largest of: its MMA time (nchunk / 2 cycles
+// per MMA plus ~20 to issue it), its shared-memory traffic (the stage written by the copies plus, per MMA, 4 KB of
+// A and its half of W read by the tensor core) at 128 bytes per cycle, and the operand delivery at ~55 bytes
+// per cycle; a launch takes as many rounds as the pairs need on the device.  cost_out: the model's cycles.
+PairPlan pair_plan(int epi, int M, int N, int K, double* cost_out) {
+    PairPlan best{};
+    double best_cost = 1e300;
+    const int resident = max_active_pairs();
+    const int nk = (K + GK - 1) / GK;
+    const int m_pairs = (M + 2 * GM - 1) / (2 * GM);
+    const int ring = GEMM_SMEM_BYTES - 1024 - 256;
+    if (resident >= 1) {
+        for (int nmma = 1; nmma <= 2; ++nmma) {
+            for (int nchunk = 256; nchunk >= 32; nchunk -= 16) {
+                const int bn = nmma * nchunk;
+                const int wcols = epi == GEMM_EPI_SWIGLU ? bn / 2 : bn;
+                if (wcols > ((N + 7) / 8) * 8 + 15 && bn > 32) continue;      // wider than the whole output
+                const int half_rows = nchunk / 2;
+                const int stage_bytes = A_TILE_BYTES + nmma * half_rows * GK * 2;
+                int stages = ring / stage_bytes;
+                if (stages > MAX_STAGES) stages = MAX_STAGES;
+                if (stages < 3) continue;
+                const int n_tiles = (N + wcols - 1) / wcols;
+                const long long tiles = static_cast<long long>(m_pairs) * n_tiles;
+                const long long rounds = (tiles + resident - 1) / resident;
+                const double mma = nmma * 4 * (nchunk / 2.0 + 20.0);
+                const double smem = (stage_bytes + nmma * 4 * (4096.0 + half_rows * 32.0)) / 128.0;
+                const double ld = stage_bytes / 55.0;
+                double per_kb = mma > smem ? mma : smem;
+                if (ld > per_kb) per_kb = ld;
+                const double cost = rounds * (nk * per_kb + 2500.0 + wcols * 14.0);
+                if (cost < best_cost) {
+                    best_cost = cost;
+                    best.bn = bn; best.wcols = wcols; best.nmma = nmma; best.nchunk = nchunk; best.stages = stages;
+                    best.m_pairs = m_pairs; best.n_tiles = n_tiles;
+                    uint32_t cols = 32;
+                    while (cols < static_cast<uint32_t>(bn)) cols <<= 1;
+                    best.tmem_cols = cols;
+                }
+            }
+        }
+    }
+    if (cost_out) *cost_out = best_cost;
+    return best;
+}
+
 template <int EPI>
 int launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tb2, const GemmArgs& g,
                cudaStream_t stream, int* max_clusters_query) {
@@ -391,7 +656,16 @@ GemmPlan gemm_plan(int epi, int M, int N, int K, int sm_count) {
 
 }  // namespace
 
+// The pair kernel serves every problem with more than one row tile.
+bool use_pair_kernel(int M, const PairPlan& pp) { return M > GM && pp.bn != 0; }
+
 int gemm_plan_describe(const dare_ctx* ctx, int epi, int M, int N, int K, int* out) {
+    const PairPlan pp = pair_plan(epi, M, N, K, nullptr);
+    if (use_pair_kernel(M, pp)) {
+        out[0] = 2; out[1] = pp.bn; out[2] = pp.wcols; out[3] = 1; out[4] = pp.stages;
+        out[5] = pp.m_pairs; out[6] = pp.n_tiles; out[7] = max_active_pairs();
+        return DARE_OK;
+    }
     const GemmPlan p = gemm_plan(epi, M, N, K, ctx->sm_count);
     out[0] = p.nsub; out[1] = p.bn; out[2] = p.wcols; out[3] = p.splits; out[4] = p.stages;
     out[5] = p.m_items; out[6] = p.n_tiles; out[7] = p.splits > 1 ? max_active_clusters(p.splits) : 0;
@@ -402,6 +676,28 @@ int launch_gemm(const dare_ctx* ctx, int epi, const void* a, int M, int K, const
                 void* out, const void* res, int ldo, cudaStream_t stream) {
     if (M < 1 || N < 8 || K < 8 || (N % 8) || (K % 8) || (ldo % 8)) return DARE_ERR_SHAPE;
     if (epi < GEMM_EPI_STORE || epi > GEMM_EPI_SWIGLU) return DARE_ERR_RANGE;
+    const PairPlan pp = pair_plan(epi, M, N, K, nullptr);
+    if (use_pair_kernel(M, pp)) {
+        PairArgs pg;
+        pg.M = M; pg.N = N; pg.K = K; pg.ldo = ldo;
+        pg.p = pp;
+        pg.out = static_cast<__nv_bfloat16*>(out);
+        pg.res = static_cast<const __nv_bfloat16*>(res);
+        pg.dev_status = ctx->dev_status;
+        CUtensorMap pa, pb, pb2;
+        int prc = make_tmap_bf16_2d(ctx, &pa, a, static_cast<uint64_t>(M), static_cast<uint64_t>(K), GM, GK);
+        if (prc != DARE_OK) return prc;
+        const uint32_t half_rows = static_cast<uint32_t>(pp.nchunk / 2);
+        prc = make_tmap_bf16_2d(ctx, &pb, w, static_cast<uint64_t>(N), static_cast<uint64_t>(K), half_rows, GK);
+        if (prc != DARE_OK) return prc;
+        if (epi == GEMM_EPI_SWIGLU) {
+            prc = make_tmap_bf16_2d(ctx, &pb2, w2, static_cast<uint64_t>(N), static_cast<uint64_t>(K), half_rows, GK);
+            if (prc != DARE_OK) return prc;
+            return launch_pair<GEMM_EPI_SWIGLU>(pa, pb, pb2, pg, stream, nullptr);
+        }
+        return epi == GEMM_EPI_STORE ? launch_pair<GEMM_EPI_STORE>(pa, pb, pb, pg, stream, nullptr)
+                                     : launch_pair<GEMM_EPI_RESIDUAL>(pa, pb, pb, pg, stream, nullptr);
+    }
     GemmArgs g;
     g.M = M; g.N = N; g.K = K; g.ldo = ldo;
     g.p = gemm_plan(epi, M, N, K, ctx->sm_count);
