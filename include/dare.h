@@ -291,9 +291,12 @@ int dare_model_destroy(dare_model* model);
 enum { DARE_LINEAR_STORE = 0, DARE_LINEAR_RESIDUAL = 1, DARE_LINEAR_SWIGLU = 2 };
 int dare_linear(dare_ctx* ctx, int epilogue, const void* a, int M, int K, const void* w, const void* w2, int N,
                 void* out, const void* residual, void* stream);
-/* The launch shape dare_linear picks for a problem (no launch): plan_out (HOST int[8]) = {row tiles per CTA,
- * W rows per tile, output columns per tile, CTAs along K per output tile (they form a cluster), pipeline
- * stages, row items, column tiles, clusters of that size resident at once (0 without a K split)}. */
+/* The launch shape dare_linear picks for a problem (no launch): plan_out (HOST int[8]) = {row tiles per work
+ * item, W rows per tile, output columns per tile, CTAs along K per output tile, pipeline stages, row items,
+ * column tiles, clusters resident at once}.  M > 128: a work item is a PAIR of CTAs (a cluster of two) that
+ * computes two row tiles with 256-row MMAs; entry 3 is 1 and entry 7 the number of resident pairs.
+ * M <= 128: one CTA per (row tile, column tile, K slice); the K slices of a tile form a cluster and entry 7
+ * is 0 without a K split. */
 int dare_linear_plan(dare_ctx* ctx, int epilogue, int M, int K, int N, int* plan_out);
 int dare_rmsnorm(dare_ctx* ctx, const void* x, int n_rows, int D, float eps, void* y, void* stream);
 int dare_rope_kv_write(dare_model* model, const void* qkv, int B, int length, int start, void* q_out,

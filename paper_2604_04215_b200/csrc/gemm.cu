@@ -1,6 +1,8 @@
 // Dense bf16 projections of the layer stack on the tcgen05 tensor cores: out = epilogue(A W^T).
 //
-// A [M, K] activations and W [N, K] weights are both K-major bf16.  One CTA computes one output tile of up to
+// A [M, K] activations and W [N, K] weights are both K-major bf16.  Problems with two or more row tiles run on
+// CTA pairs (gemm_pair_kernel, further down); the single-CTA kernel described here serves the rest and is the
+// shape the pair kernel is derived from.  One CTA computes one output tile of up to
 // two 128-row tiles by `bn` columns over a range of K:
 //   warp 0      TMA producer: one or two A tiles [128 x 64] and a W tile [bn x 64] per stage (128-byte swizzle)
 //   warp 1      UMMA issuer: 128 x bn x 16 MMAs, one fp32 accumulator in TMEM per row tile
