@@ -117,7 +117,6 @@ attn_block_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_cons
         fence_barrier_init();
     }
     __syncthreads();
-    grid_dependency_sync();      // everything below reads what earlier kernels of the stream wrote
 
     // lengths (clamped to capacity; a clamp is reported, never trapped on)
     int P = p.prefix_len ? p.prefix_len[b]
@@ -449,7 +448,6 @@ attn_block_tc_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_c
     // Packed variable-length mode: "rollout" b is sequence b of the packed token list; its tokens are both the
     // queries (a block of L_eff positions, no prefix) and, in place, the keys.  K and V are [tokens, Hkv * D].
     const bool packed = p.cu_seqlens != nullptr;
-    grid_dependency_sync();      // the lengths below may come from the previous kernel of the stream
     const int seq_base = packed ? p.cu_seqlens[b] : 0;
     const int L_eff = packed ? p.cu_seqlens[b + 1] - seq_base : p.L;
     if (static_cast<int>(blockIdx.x) * QT * pos_per_tile >= L_eff) return;   // (whole CTA, before anything is set up)
@@ -724,8 +722,8 @@ int launch_tc(const CUtensorMap* tm, const AttnParams& p, int q_tiles, cudaStrea
     if (cudaFuncSetAttribute(attn_block_tc_kernel<D, QT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
         return DARE_ERR_CUDA;
     dim3 grid((q_tiles + QT - 1) / QT, p.B * p.Hkv, 1);
-    return launch_overlapped(attn_block_tc_kernel<D, QT>, grid, dim3(TcShape<D, QT>::THREADS), SMEM, stream, 1, tm[0], tm[1],
-                             tm[2], tm[3], tm[4], tm[5], p);
+    attn_block_tc_kernel<D, QT><<<grid, TcShape<D, QT>::THREADS, SMEM, stream>>>(tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], p);
+    return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
 }
 
 // The tensor-core tile is worth it when a tile's 128 rows are mostly real query rows.
@@ -742,7 +740,6 @@ template <int D>
 __global__ void attn_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_lse, int splits,
                                     size_t n_rows, int L, int Hq, __nv_bfloat16* __restrict__ out,
                                     float* __restrict__ lse) {
-    grid_dependency_sync();
     const size_t row = static_cast<size_t>(blockIdx.x) * (blockDim.x / (D / 4)) + threadIdx.x / (D / 4);
     const int c4 = threadIdx.x % (D / 4);
     if (row >= n_rows) return;
@@ -778,8 +775,8 @@ int launch_one(const CUtensorMap* tm, const AttnParams& p, int chunks, cudaStrea
     if (cudaFuncSetAttribute(attn_block_kernel<D, NW, KS, KT, STAGES, CPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
         return DARE_ERR_CUDA;
     dim3 grid(chunks, p.B * p.Hkv, p.splits);
-    return launch_overlapped(attn_block_kernel<D, NW, KS, KT, STAGES, CPS>, grid, dim3((NW * KS + 1) * 32), SMEM, stream, 1,
-                             tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], p);
+    attn_block_kernel<D, NW, KS, KT, STAGES, CPS><<<grid, (NW * KS + 1) * 32, SMEM, stream>>>(tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], p);
+    return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
 }
 
 // The warp-level kernel's variants by the number of packed query rows R per (rollout, KV head):
@@ -884,11 +881,11 @@ int launch_attn(const dare_ctx* ctx, const AttnArgs& a, cudaStream_t stream) {
         const int tpr = a.d / 4;                    // threads per row
         const int rows_per_block = 256 / tpr;
         const unsigned blocks = static_cast<unsigned>((n_rows + rows_per_block - 1) / rows_per_block);
-        rc = a.d == 128 ? launch_overlapped(attn_combine_kernel<128>, dim3(blocks), dim3(256), 0, stream, 1, p.part_o,
-                                            p.part_lse, p.splits, n_rows, a.L, a.Hq, p.out, p.lse)
-                        : launch_overlapped(attn_combine_kernel<64>, dim3(blocks), dim3(256), 0, stream, 1, p.part_o,
-                                            p.part_lse, p.splits, n_rows, a.L, a.Hq, p.out, p.lse);
-        if (rc != DARE_OK) return rc;
+        if (a.d == 128)
+            attn_combine_kernel<128><<<blocks, 256, 0, stream>>>(p.part_o, p.part_lse, p.splits, n_rows, a.L, a.Hq, p.out, p.lse);
+        else
+            attn_combine_kernel<64><<<blocks, 256, 0, stream>>>(p.part_o, p.part_lse, p.splits, n_rows, a.L, a.Hq, p.out, p.lse);
+        if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
     }
     return DARE_OK;
 }

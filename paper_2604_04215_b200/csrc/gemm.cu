@@ -128,7 +128,6 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     tc_fence_after_sync();
     const uint32_t tmem_base = bars->tmem_base;
     const int acc_stride = p.nsub == 2 ? 256 : 0;   // accumulator of row tile s starts at column s * 256
-    grid_dependency_sync();      // set-up done; the operands may come from the previous kernel of the stream
 
     if (warp == 0) {
         if (lane == 0) {
@@ -362,7 +361,6 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     cluster_sync_all();              // both CTAs' barriers exist before either CTA signals the other's
     tc_fence_after_sync();
     const uint32_t tmem_base = bars->tmem_base;
-    grid_dependency_sync();          // set-up done; the operands may come from the previous kernel of the stream
 
     if (warp == 0) {
         if (lane == 0) {
@@ -488,17 +486,14 @@ int launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap&
     cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
     cfg.dynamicSmemBytes = GEMM_SMEM_BYTES;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // see launch_overlapped (internal.h)
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 2;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
     if (max_clusters_query) {
-        cfg.numAttrs = 1;
         cfg.gridDim = dim3(2048u, 1, 1);
         return cudaOccupancyMaxActiveClusters(max_clusters_query, gemm_pair_kernel<EPI>, &cfg) == cudaSuccess
                    ? DARE_OK : DARE_ERR_CUDA;
@@ -579,17 +574,14 @@ int launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& 
     cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
     cfg.dynamicSmemBytes = GEMM_SMEM_BYTES;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = static_cast<unsigned>(g.p.splits);
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // see launch_overlapped (internal.h)
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 2;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = static_cast<unsigned>(g.p.splits);
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
     if (max_clusters_query) {     // how many clusters of this size the device runs at once (plan input)
-        cfg.numAttrs = 1;
         cfg.gridDim = dim3(static_cast<unsigned>(g.p.splits) * 1024u, 1, 1);
         return cudaOccupancyMaxActiveClusters(max_clusters_query, gemm_bf16_kernel<EPI>, &cfg) == cudaSuccess
                    ? DARE_OK : DARE_ERR_CUDA;

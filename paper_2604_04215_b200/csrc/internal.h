@@ -24,34 +24,6 @@ struct dare_ctx {
 
 namespace dare {
 
-// Launches `kernel` with programmatic stream serialization: its CTAs may be scheduled while the previous kernel
-// of the stream is still running, and block in grid_dependency_sync() (ptx.cuh) until that kernel has
-// completed.  EVERY kernel launched this way calls grid_dependency_sync() in all its threads before it touches
-// global memory; the ordering of a chain of such kernels rests on that.  cluster_x > 1 launches clusters.
-template <typename... P, typename... A>
-inline int launch_overlapped(void (*kernel)(P...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
-                             unsigned cluster_x, A&&... args) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = grid;
-    cfg.blockDim = block;
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    unsigned n = 1;
-    if (cluster_x > 1) {
-        attr[1].id = cudaLaunchAttributeClusterDimension;
-        attr[1].val.clusterDim.x = cluster_x;
-        attr[1].val.clusterDim.y = 1;
-        attr[1].val.clusterDim.z = 1;
-        n = 2;
-    }
-    cfg.attrs = attr;
-    cfg.numAttrs = n;
-    return cudaLaunchKernelEx(&cfg, kernel, static_cast<P>(args)...) == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
-}
-
 // bf16 2-D row-major tensor [rows, cols] -> tensor map with a [box_rows, 64] box and 128-byte swizzle.
 int make_tmap_bf16_2d(const dare_ctx* ctx, CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols,
                       uint32_t box_rows, uint32_t box_cols);

@@ -17,7 +17,6 @@ __device__ __forceinline__ float hi_f(uint32_t w) { return __uint_as_float(w & 0
 __global__ void __launch_bounds__(ROWS_PER_BLOCK * 32)
 embed_gather_kernel(const uint4* __restrict__ emb, int D8, int V, const int32_t* __restrict__ tokens, int64_t row_stride,
                     int start, int length, int n_rows, uint4* __restrict__ x) {
-    grid_dependency_sync();
     const int m = blockIdx.x * ROWS_PER_BLOCK + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (m >= n_rows) return;
@@ -31,7 +30,6 @@ embed_gather_kernel(const uint4* __restrict__ emb, int D8, int V, const int32_t*
 // y = x / sqrt(mean(x^2) + eps), weight 1.  Two passes over the row (the second one hits L1/L2).
 __global__ void __launch_bounds__(ROWS_PER_BLOCK * 32)
 rmsnorm_kernel(const uint4* __restrict__ x, int D8, int n_rows, float eps, uint4* __restrict__ y) {
-    grid_dependency_sync();
     const int m = blockIdx.x * ROWS_PER_BLOCK + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (m >= n_rows) return;
@@ -77,7 +75,6 @@ __global__ void __launch_bounds__(128)
 rope_kv_write_kernel(const __nv_bfloat16* __restrict__ qkv, int Hq, int Hkv, int d, int start, int length,
                      const float2* __restrict__ cs, __nv_bfloat16* __restrict__ q_out,
                      __nv_bfloat16* __restrict__ k_cache, __nv_bfloat16* __restrict__ v_cache, int cap) {
-    grid_dependency_sync();
     const int m = blockIdx.x;
     const int b = m / length, i = m % length, p = start + i;
     const int half = d / 2, cpb = half / 8;                 // 8-channel chunks per half head
@@ -116,15 +113,15 @@ rope_kv_write_kernel(const __nv_bfloat16* __restrict__ qkv, int Hq, int Hkv, int
 
 int launch_embed(const void* emb, int D, int V, const int32_t* tokens, int64_t row_stride, int start, int length,
                  int n_rows, void* x, cudaStream_t stream) {
-    return launch_overlapped(embed_gather_kernel, dim3((n_rows + ROWS_PER_BLOCK - 1) / ROWS_PER_BLOCK),
-                             dim3(ROWS_PER_BLOCK * 32), 0, stream, 1, static_cast<const uint4*>(emb), D / 8, V, tokens,
-                             row_stride, start, length, n_rows, static_cast<uint4*>(x));
+    embed_gather_kernel<<<(n_rows + ROWS_PER_BLOCK - 1) / ROWS_PER_BLOCK, ROWS_PER_BLOCK * 32, 0, stream>>>(
+        static_cast<const uint4*>(emb), D / 8, V, tokens, row_stride, start, length, n_rows, static_cast<uint4*>(x));
+    return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
 }
 
 int launch_rmsnorm(const void* x, int D, int n_rows, float eps, void* y, cudaStream_t stream) {
-    return launch_overlapped(rmsnorm_kernel, dim3((n_rows + ROWS_PER_BLOCK - 1) / ROWS_PER_BLOCK),
-                             dim3(ROWS_PER_BLOCK * 32), 0, stream, 1, static_cast<const uint4*>(x), D / 8, n_rows, eps,
-                             static_cast<uint4*>(y));
+    rmsnorm_kernel<<<(n_rows + ROWS_PER_BLOCK - 1) / ROWS_PER_BLOCK, ROWS_PER_BLOCK * 32, 0, stream>>>(
+        static_cast<const uint4*>(x), D / 8, n_rows, eps, static_cast<uint4*>(y));
+    return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
 }
 
 int launch_rope_table(float* cs, int n_pos, int half, double base, cudaStream_t stream) {
@@ -135,10 +132,12 @@ int launch_rope_table(float* cs, int n_pos, int half, double base, cudaStream_t 
 
 int launch_rope_kv_write(const void* qkv, int n_rows, int Hq, int Hkv, int d, int start, int length, const float* cs,
                          void* q_out, void* k_cache, void* v_cache, int cap, cudaStream_t stream) {
-    return launch_overlapped(rope_kv_write_kernel, dim3(n_rows), dim3(128), 0, stream, 1,
-                             static_cast<const __nv_bfloat16*>(qkv), Hq, Hkv, d, start, length,
-                             reinterpret_cast<const float2*>(cs), static_cast<__nv_bfloat16*>(q_out),
-                             static_cast<__nv_bfloat16*>(k_cache), static_cast<__nv_bfloat16*>(v_cache), cap);
+    rope_kv_write_kernel<<<n_rows, 128, 0, stream>>>(static_cast<const __nv_bfloat16*>(qkv), Hq, Hkv, d, start, length,
+                                                     reinterpret_cast<const float2*>(cs),
+                                                     static_cast<__nv_bfloat16*>(q_out),
+                                                     static_cast<__nv_bfloat16*>(k_cache),
+                                                     static_cast<__nv_bfloat16*>(v_cache), cap);
+    return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
 }
 
 }  // namespace dare

@@ -67,7 +67,6 @@ lmhead_compact_kernel(const uint4* __restrict__ x, int M, int D8, const int32_t*
                       int32_t* __restrict__ count, int32_t* __restrict__ pred, float* __restrict__ conf) {
     __shared__ int s_base;
     __shared__ int s_flag[CP_ROWS];
-    grid_dependency_sync();
     const int row0 = blockIdx.x * CP_ROWS;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) s_base = 0;
@@ -143,7 +142,6 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
                       uint32_t* __restrict__ dev_status, const LmSampling smp) {
     constexpr bool SAMPLE = MODE == LM_SAMPLE;
     constexpr bool LOGPROB = MODE == LM_LOGPROB;
-    grid_dependency_sync();                             // the row count below comes from the previous kernel
     const int Mc = live_rows ? *live_rows : M;          // rows that need logits (uniform over the grid)
     const int m_tiles = (Mc + BM - 1) / BM;
     if (m_tiles == 0) return;
@@ -363,7 +361,6 @@ __global__ void lmhead_merge_kernel(const float* __restrict__ part_max, const fl
                                     const int32_t* __restrict__ part_arg, int grid_gemm, int n_tiles, int M,
                                     const int32_t* __restrict__ live_rows, const int32_t* __restrict__ idx,
                                     int32_t* __restrict__ pred, float* __restrict__ conf) {
-    grid_dependency_sync();
     const int c = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     const int Mc = live_rows ? *live_rows : M;
@@ -405,7 +402,6 @@ __global__ void lmhead_merge_sample_kernel(const float* __restrict__ part_max, c
                                            const float* __restrict__ part_zb, int grid_gemm, int n_tiles, int M,
                                            const int32_t* __restrict__ live_rows, const int32_t* __restrict__ idx,
                                            int32_t* __restrict__ pred, float* __restrict__ conf) {
-    grid_dependency_sync();
     const int c = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     const int Mc = live_rows ? *live_rows : M;
@@ -449,7 +445,6 @@ __global__ void lmhead_merge_sample_kernel(const float* __restrict__ part_max, c
 __global__ void lmhead_merge_logprob_kernel(const float* __restrict__ part_max, const float* __restrict__ part_sum,
                                             const int32_t* __restrict__ part_zt, int grid_gemm, int n_tiles, int M,
                                             float* __restrict__ logprob, float* __restrict__ lse_out) {
-    grid_dependency_sync();
     const int c = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (c >= M) return;
@@ -514,10 +509,10 @@ int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M,
         live_rows = idx + M;
         cur += round_up(static_cast<size_t>(M) * 4 + 4, 1024);
         x_gemm = xc;
-        if (launch_overlapped(lmhead_compact_kernel, dim3((M + CP_ROWS - 1) / CP_ROWS), dim3(CP_ROWS * 32), 0, stream, 1,
-                              static_cast<const uint4*>(hidden), M, D / 8, row_tokens, tok_L, tok_row_stride, mask_id,
-                              static_cast<uint4*>(xc), idx, live_rows, pred, conf) != DARE_OK)
-            return DARE_ERR_CUDA;
+        lmhead_compact_kernel<<<(M + CP_ROWS - 1) / CP_ROWS, CP_ROWS * 32, 0, stream>>>(
+            static_cast<const uint4*>(hidden), M, D / 8, row_tokens, tok_L, tok_row_stride, mask_id,
+            static_cast<uint4*>(xc), idx, live_rows, pred, conf);
+        if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
     }
     size_t groups_max = static_cast<size_t>(ctx->sm_count);
     if (groups_max > static_cast<size_t>(n_tiles)) groups_max = n_tiles;
@@ -539,14 +534,11 @@ int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M,
         if (cudaFuncSetAttribute(lmhead_partial_kernel<LM_GREEDY>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  LM_SMEM_BYTES) != cudaSuccess)
             return DARE_ERR_CUDA;
-        if (launch_overlapped(lmhead_partial_kernel<LM_GREEDY>, dim3(grid), dim3(LM_THREADS), LM_SMEM_BYTES, stream, 1,
-                              tmap_x, tmap_w, M, live_rows, D, V, mask_col, n_tiles, part_max, part_sum, part_arg,
-                              ctx->dev_status, smp) != DARE_OK)
-            return DARE_ERR_CUDA;
-        if (launch_overlapped(lmhead_merge_kernel, dim3((M + rows_per_block - 1) / rows_per_block),
-                              dim3(rows_per_block * 32), 0, stream, 1, part_max, part_sum, part_arg, grid, n_tiles, M,
-                              live_rows, idx, pred, conf) != DARE_OK)
-            return DARE_ERR_CUDA;
+        lmhead_partial_kernel<LM_GREEDY><<<grid, LM_THREADS, LM_SMEM_BYTES, stream>>>(
+            tmap_x, tmap_w, M, live_rows, D, V, mask_col, n_tiles, part_max, part_sum, part_arg, ctx->dev_status, smp);
+        if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
+        lmhead_merge_kernel<<<(M + rows_per_block - 1) / rows_per_block, rows_per_block * 32, 0, stream>>>(
+            part_max, part_sum, part_arg, grid, n_tiles, M, live_rows, idx, pred, conf);
     } else {
         smp.inv_temperature = 1.0f / sample->temperature;
         smp.seed_lo = static_cast<uint32_t>(sample->seed & 0xffffffffu);
@@ -558,15 +550,13 @@ int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M,
         if (cudaFuncSetAttribute(lmhead_partial_kernel<LM_SAMPLE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  LM_SMEM_BYTES) != cudaSuccess)
             return DARE_ERR_CUDA;
-        if (launch_overlapped(lmhead_partial_kernel<LM_SAMPLE>, dim3(grid), dim3(LM_THREADS), LM_SMEM_BYTES, stream, 1,
-                              tmap_x, tmap_w, M, live_rows, D, V, mask_col, n_tiles, part_max, part_sum, part_arg,
-                              ctx->dev_status, smp) != DARE_OK)
-            return DARE_ERR_CUDA;
-        if (launch_overlapped(lmhead_merge_sample_kernel, dim3((M + rows_per_block - 1) / rows_per_block),
-                              dim3(rows_per_block * 32), 0, stream, 1, part_max, part_sum, part_arg, smp.part_y,
-                              smp.part_zb, grid, n_tiles, M, live_rows, idx, pred, conf) != DARE_OK)
-            return DARE_ERR_CUDA;
+        lmhead_partial_kernel<LM_SAMPLE><<<grid, LM_THREADS, LM_SMEM_BYTES, stream>>>(
+            tmap_x, tmap_w, M, live_rows, D, V, mask_col, n_tiles, part_max, part_sum, part_arg, ctx->dev_status, smp);
+        if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
+        lmhead_merge_sample_kernel<<<(M + rows_per_block - 1) / rows_per_block, rows_per_block * 32, 0, stream>>>(
+            part_max, part_sum, part_arg, smp.part_y, smp.part_zb, grid, n_tiles, M, live_rows, idx, pred, conf);
     }
+    if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
     return DARE_OK;
 }
 
@@ -594,14 +584,13 @@ int launch_lmhead_logprob(const dare_ctx* ctx, void* scratch, const void* hidden
     const int mask_col = (exclude_mask_column && mask_id >= 0 && mask_id < V) ? mask_id : -1;
     LmSampling smp = {};
     smp.targets = targets;
-    if (launch_overlapped(lmhead_partial_kernel<LM_LOGPROB>, dim3(grid), dim3(LM_THREADS), LM_SMEM_BYTES, stream, 1,
-                          tmap_x, tmap_w, M, static_cast<const int32_t*>(nullptr), D, V, mask_col, n_tiles, part_max,
-                          part_sum, part_zt, ctx->dev_status, smp) != DARE_OK)
-        return DARE_ERR_CUDA;
+    lmhead_partial_kernel<LM_LOGPROB><<<grid, LM_THREADS, LM_SMEM_BYTES, stream>>>(
+        tmap_x, tmap_w, M, nullptr, D, V, mask_col, n_tiles, part_max, part_sum, part_zt, ctx->dev_status, smp);
+    if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
     const int rows_per_block = 8;
-    return launch_overlapped(lmhead_merge_logprob_kernel, dim3((M + rows_per_block - 1) / rows_per_block),
-                             dim3(rows_per_block * 32), 0, stream, 1, part_max, part_sum, part_zt, grid, n_tiles, M,
-                             logprob, lse_out);
+    lmhead_merge_logprob_kernel<<<(M + rows_per_block - 1) / rows_per_block, rows_per_block * 32, 0, stream>>>(
+        part_max, part_sum, part_zt, grid, n_tiles, M, logprob, lse_out);
+    return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
 }
 
 }  // namespace dare

@@ -69,17 +69,6 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     return true;
 }
 
-// ---------------------------------------------------------------- programmatic dependent launch
-// Kernels are launched so that their CTAs may become resident while the previous kernel of the stream is still
-// running (launch_overlapped in internal.h).  This call blocks until that kernel has completed and its memory
-// writes are visible, and then lets the next kernel of the stream start its own launch.  Nothing that a
-// predecessor writes may be read, and nothing it reads or writes may be written, before this call; without the
-// launch attribute it does nothing.
-__device__ __forceinline__ void grid_dependency_sync() {
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-}
-
 // ---------------------------------------------------------------- thread-block cluster
 __device__ __forceinline__ uint32_t cluster_cta_rank() {
     uint32_t r;

@@ -5,7 +5,6 @@
 #include <math.h>
 
 #include "internal.h"
-#include "ptx.cuh"
 
 namespace dare {
 namespace {
@@ -17,7 +16,6 @@ __global__ void __launch_bounds__(SEL_THREADS)
 unmask_select_kernel(int32_t* __restrict__ tokens, int64_t row_stride, int block_start, int L,
                      const int32_t* __restrict__ pred, const float* __restrict__ conf, int32_t mask_id, int mode,
                      float threshold, int k, int32_t* __restrict__ n_committed, int32_t* __restrict__ n_remaining) {
-    grid_dependency_sync();
     extern __shared__ float s_conf[];   // [L]; -inf for NaN; positions that are not masked hold NaN as "absent"
     __shared__ int s_masked, s_above, s_commit;
     const int r = blockIdx.x;
@@ -75,9 +73,10 @@ int launch_unmask_select(int32_t* tokens, int B, int64_t row_stride, int block_s
                          const float* conf, int32_t mask_id, int mode, float threshold, int k, int32_t* n_committed,
                          int32_t* n_remaining, cudaStream_t stream) {
     if (L > SEL_MAX_L) return DARE_ERR_SHAPE;
-    return launch_overlapped(unmask_select_kernel, dim3(B), dim3(SEL_THREADS), L * sizeof(float), stream, 1, tokens,
-                             row_stride, block_start, L, pred, conf, mask_id, mode, threshold, k, n_committed,
-                             n_remaining);
+    unmask_select_kernel<<<B, SEL_THREADS, L * sizeof(float), stream>>>(tokens, row_stride, block_start, L, pred, conf,
+                                                                        mask_id, mode, threshold, k, n_committed,
+                                                                        n_remaining);
+    return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
 }
 
 }  // namespace dare
