@@ -294,7 +294,8 @@ int dare_linear(dare_ctx* ctx, int epilogue, const void* a, int M, int K, const 
 /* The launch shape dare_linear picks for a problem (no launch): plan_out (HOST int[8]) = {row tiles per work
  * item, W rows per tile, output columns per tile, CTAs along K per output tile, pipeline stages, row items,
  * column tiles, clusters resident at once}.  M > 128: a work item is a PAIR of CTAs (a cluster of two) that
- * computes two row tiles with 256-row MMAs; entry 3 is 1 and entry 7 the number of resident pairs.
+ * computes two row tiles with 256-row MMAs; entry 3 is the number of pairs along K (1 or 2; two pairs form a
+ * cluster of four CTAs) and entry 7 the number of such clusters resident at once.
  * M <= 128: one CTA per (row tile, column tile, K slice); the K slices of a tile form a cluster and entry 7
  * is 0 without a K split. */
 int dare_linear_plan(dare_ctx* ctx, int epilogue, int M, int K, int N, int* plan_out);

@@ -304,11 +304,16 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 // 128-row tile, which is what limits the single-CTA kernel.  bn may exceed 256: the tile is then made of two
 // MMAs of bn / 2 columns per K step.  SwiGLU: the even CTA loads the gate rows, the odd CTA the matching up rows,
 // so that every accumulator row holds [gate | up] column pairs.
+// K split (long K, few output tiles): two pairs form a cluster of four CTAs (ranks 0, 1 = first half of K, ranks 2,
+// 3 = second half).  After the main loop each CTA hands the accumulator column groups it does not own to the CTA
+// with the same rows in the other pair, through distributed shared memory into that CTA's idle operand ring; both
+// add in the same order (first half + second half) and each applies the epilogue to the groups it owns.
 struct PairPlan {
     int bn;          // accumulator columns per tile = W rows per tile and K block (both CTAs together)
     int wcols;       // output columns per tile (bn, or bn / 2 for SwiGLU)
     int nmma;        // MMAs per K step (1 or 2), each nchunk columns wide
     int nchunk;
+    int splits;      // pairs along K per output tile (1 or 2); two pairs form a cluster of four CTAs
     int stages;
     int m_pairs, n_tiles;
     uint32_t tmem_cols;
@@ -338,11 +343,15 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 
     const int warp = warp_index_uniform();
     const int lane = threadIdx.x & 31;
-    const int rank = static_cast<int>(cluster_cta_rank());   // 0: issues the MMAs and owns the "full" barriers
-    const int pair = blockIdx.x >> 1;
-    const int m_pair = pair % p.m_pairs;                      // row index fastest: pairs sharing W run together
-    const int n_tile = pair / p.m_pairs;
+    const int rank4 = static_cast<int>(cluster_cta_rank());
+    const int rank = rank4 & 1;                               // 0: issues the MMAs and owns the "full" barriers
+    const int split = rank4 >> 1;                             // which part of K this pair computes
+    const int tile = blockIdx.x / (2 * p.splits);
+    const int m_pair = tile % p.m_pairs;                      // row index fastest: pairs sharing W run together
+    const int n_tile = tile / p.m_pairs;
     const int nk = (g.K + GK - 1) / GK;
+    const int kb_begin = static_cast<int>(static_cast<long long>(nk) * split / p.splits);
+    const int kb_end = static_cast<int>(static_cast<long long>(nk) * (split + 1) / p.splits);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
@@ -371,10 +380,10 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             // W row of chunk 0 for this CTA; chunk c starts w_step rows further on
             const int w_row0 = EPI == GEMM_EPI_SWIGLU ? n_tile * p.wcols : n_tile * p.bn + rank * half_rows;
             const int w_step = EPI == GEMM_EPI_SWIGLU ? half_rows : p.nchunk;
-            const uint32_t full0 = cluster_map_shared(smem_u32(&bars->full[0]), 0);   // the even CTA's barriers
+            const uint32_t full0 = cluster_map_shared(smem_u32(&bars->full[0]), rank4 & ~1);   // the even CTA's barriers
             int stage = 0;
             uint32_t phase = 0;
-            for (int kb = 0; kb < nk; ++kb) {
+            for (int kb = kb_begin; kb < kb_end; ++kb) {
                 if (!mbar_wait(&bars->empty[stage], phase ^ 1, abort_flag)) break;
                 uint8_t* a_dst = tiles + stage * stage_bytes;
                 uint8_t* b_dst = a_dst + A_TILE_BYTES;
@@ -390,16 +399,17 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         // all lanes run the loop, one elected lane issues the MMAs and their commits (which arrive in both CTAs)
         const bool leader = elect_one_sync();
         const uint32_t idesc = umma_idesc_bf16(2 * GM, p.nchunk);
+        const uint16_t pair_mask = static_cast<uint16_t>(3u << rank4);     // this CTA (even rank) and the next
         int stage = 0;
         uint32_t phase = 0;
         bool ok = true;
-        for (int kb = 0; kb < nk; ++kb) {
+        for (int kb = kb_begin; kb < kb_end; ++kb) {
             ok = __all_sync(0xffffffffu, mbar_wait(&bars->full[stage], phase, abort_flag));
             if (!ok) break;
             tc_fence_after_sync();
             const uint32_t a_addr = smem_u32(tiles + stage * stage_bytes);
             const uint64_t a_desc = umma_desc_sw128_kmajor(a_addr);
-            const uint32_t accumulate = kb > 0;
+            const uint32_t accumulate = kb > kb_begin;
             if (leader) {
                 for (int c = 0; c < p.nmma; ++c) {
                     const uint64_t b_desc = umma_desc_sw128_kmajor(a_addr + A_TILE_BYTES + c * chunk_bytes);
@@ -408,53 +418,83 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                         umma_bf16_pair(tmem_base + c * p.nchunk, a_desc + 2 * kk, b_desc + 2 * kk, idesc,
                                        accumulate | (kk != 0));
                 }
-                umma_commit_pair(&bars->empty[stage], 3);
+                umma_commit_pair(&bars->empty[stage], pair_mask);
             }
             __syncwarp();
             if (++stage == p.stages) { stage = 0; phase ^= 1; }
         }
-        if (ok && leader) umma_commit_pair(&bars->tmem_full, 3);
+        if (ok && leader) umma_commit_pair(&bars->tmem_full, pair_mask);
         __syncwarp();
     }
 
-    // ---- epilogue (warps 2..9 of both CTAs): warp w may touch TMEM lanes [32 * (w % 4), +32); the two sets of
-    // four warps alternate over the 8-column groups of the CTA's 128 rows
-    if (warp >= 2) {
-        const int lq = warp & 3;
-        const int set = (warp - 2) >> 2;
-        const int n_groups = p.wcols / 8;
-        const int row = m_pair * 2 * GM + rank * GM + lq * 32 + lane;
-        const bool row_ok = row < g.M;
-        const size_t row_off = static_cast<size_t>(row) * g.ldo;
-        const int col_base = n_tile * p.wcols;
-        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(lq * 32) << 16);
+    // ---- epilogue (warps 2..9 of every CTA): warp w may touch TMEM lanes [32 * (w % 4), +32); the two sets of
+    // four warps alternate over the 8-column groups of the CTA's 128 rows.  With a K split, group gi belongs to
+    // the pair (gi / 2) % 2; the other pair's CTA with the same rows sends its partial into slot gi of this
+    // CTA's idle ring ([group][row][8 floats]).
+    const bool epi_warp = warp >= 2;
+    const int lq = warp & 3;
+    const int set = epi_warp ? (warp - 2) >> 2 : 0;
+    const int n_groups = p.wcols / 8;
+    const int row_local = lq * 32 + lane;
+    const int row = m_pair * 2 * GM + rank * GM + row_local;
+    const bool row_ok = row < g.M;
+    const size_t row_off = static_cast<size_t>(row) * g.ldo;
+    const int col_base = n_tile * p.wcols;
+    const uint32_t taddr = tmem_base + (static_cast<uint32_t>(lq * 32) << 16);
+    if (epi_warp) {
         mbar_wait(&bars->tmem_full, 0, abort_flag);     // (a wait that gave up leaves the abort flag set)
         tc_fence_after_sync();
-        __syncwarp();
-        if (!*abort_flag) {
+    }
+    __syncwarp();
+    if (p.splits > 1) {
+        cluster_sync_all();                              // every CTA of the cluster is done with its ring
+        if (epi_warp) {
+            const uint32_t ring = smem_u32(tiles);
             for (int gi = set; gi < n_groups; gi += 2) {
+                if (((gi >> 1) & 1) == split) continue;  // mine: stays here
                 uint32_t v[8];
-                float f[8], u[8];
-                if (EPI == GEMM_EPI_SWIGLU) {
-                    const int j = gi * 8, c = j / half_rows;
-                    const int gcol = c * p.nchunk + (j - c * half_rows);
-                    uint32_t w[8];
-                    tmem_ld_8cols(taddr + gcol, v);
-                    tmem_ld_8cols(taddr + gcol + half_rows, w);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) u[k] = __uint_as_float(w[k]);
-                } else {
-                    tmem_ld_8cols(taddr + gi * 8, v);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) u[k] = 0.f;
-                }
-#pragma unroll
-                for (int k = 0; k < 8; ++k) f[k] = __uint_as_float(v[k]);
-                const int col = col_base + gi * 8;
-                if (row_ok && col < g.N) store_group<EPI>(f, u, g.out, g.res, row_off + col);
+                tmem_ld_8cols(taddr + gi * 8, v);
+                tmem_ld_wait();
+                const uint32_t local = ring + ((static_cast<uint32_t>(gi) * GM + row_local) << 5);
+                const uint32_t remote = cluster_map_shared(local, static_cast<uint32_t>(rank4 ^ 2));
+                st_shared_cluster_v4(remote, v[0], v[1], v[2], v[3]);
+                st_shared_cluster_v4(remote + 16, v[4], v[5], v[6], v[7]);
             }
+        }
+        cluster_sync_all();                              // the partials of the groups this CTA owns have arrived
+    }
+    if (epi_warp && !*abort_flag) {
+        for (int gi = set; gi < n_groups; gi += 2) {
+            if (p.splits > 1 && ((gi >> 1) & 1) != split) continue;
+            uint32_t v[8];
+            float f[8], u[8];
+            if (EPI == GEMM_EPI_SWIGLU) {
+                const int j = gi * 8, c = j / half_rows;
+                const int gcol = c * p.nchunk + (j - c * half_rows);
+                uint32_t w[8];
+                tmem_ld_8cols(taddr + gcol, v);
+                tmem_ld_8cols(taddr + gcol + half_rows, w);
+                tmem_ld_wait();
+#pragma unroll
+                for (int k = 0; k < 8; ++k) u[k] = __uint_as_float(w[k]);
+            } else {
+                tmem_ld_8cols(taddr + gi * 8, v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int k = 0; k < 8; ++k) u[k] = 0.f;
+            }
+#pragma unroll
+            for (int k = 0; k < 8; ++k) f[k] = __uint_as_float(v[k]);
+            if (p.splits > 1) {
+                // first half of K + second half of K, in that order in both pairs
+                const float4* q = reinterpret_cast<const float4*>(tiles + ((static_cast<size_t>(gi) * GM + row_local) << 5));
+                const float4 a = q[0], c = q[1];
+                const float o[8] = {a.x, a.y, a.z, a.w, c.x, c.y, c.z, c.w};
+#pragma unroll
+                for (int k = 0; k < 8; ++k) f[k] = split == 0 ? f[k] + o[k] : o[k] + f[k];
+            }
+            const int col = col_base + gi * 8;
+            if (row_ok && col < g.N) store_group<EPI>(f, u, g.out, g.res, row_off + col);
         }
     }
 
@@ -479,7 +519,7 @@ int launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap&
     if (cudaFuncSetAttribute(gemm_pair_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_BYTES) !=
         cudaSuccess)
         return DARE_ERR_CUDA;
-    const long long ctas = 2LL * g.p.m_pairs * g.p.n_tiles;
+    const long long ctas = 2LL * g.p.splits * g.p.m_pairs * g.p.n_tiles;
     if (ctas > 0x7fffffffLL) return DARE_ERR_SHAPE;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(ctas), 1, 1);
@@ -488,45 +528,48 @@ int launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap&
     cfg.stream = stream;
     cudaLaunchAttribute attr;
     attr.id = cudaLaunchAttributeClusterDimension;
-    attr.val.clusterDim.x = 2;
+    attr.val.clusterDim.x = static_cast<unsigned>(2 * g.p.splits);
     attr.val.clusterDim.y = 1;
     attr.val.clusterDim.z = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
     if (max_clusters_query) {
-        cfg.gridDim = dim3(2048u, 1, 1);
+        cfg.gridDim = dim3(4096u, 1, 1);
         return cudaOccupancyMaxActiveClusters(max_clusters_query, gemm_pair_kernel<EPI>, &cfg) == cudaSuccess
                    ? DARE_OK : DARE_ERR_CUDA;
     }
     return cudaLaunchKernelEx(&cfg, gemm_pair_kernel<EPI>, ta, tb, tb2, g) == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
 }
 
-// CTA pairs of the pair kernel that can be resident at once (cached; 0 = it cannot run).
-int max_active_pairs() {
-    static int cache = -1;
-    if (cache < 0) {
+// Clusters of `splits` CTA pairs of the pair kernel that can be resident at once (cached; 0 = they cannot run).
+int max_active_pairs(int splits = 1) {
+    static int cache[3] = {-1, -1, -1};
+    if (cache[splits] < 0) {
         PairArgs g{};
         g.p.m_pairs = g.p.n_tiles = 1;
+        g.p.splits = splits;
         CUtensorMap dummy{};
         int n = 0;
         if (launch_pair<GEMM_EPI_STORE>(dummy, dummy, dummy, g, nullptr, &n) != DARE_OK) n = 0;
-        cache = n;
+        cache[splits] = n;
     }
-    return cache;
+    return cache[splits];
 }
 
 // Tile shape for the pair kernel.  Per K block a CTA's time is the largest of: its MMA time (nchunk / 2 cycles
-// per MMA plus ~20 to issue it), its shared-memory traffic (the stage written by the copies plus, per MMA, 4 KB of
+// per MMA plus the ~45 measured on top of that), its shared-memory traffic (the stage written by the copies plus, per MMA, 4 KB of
 // A and its half of W read by the tensor core) at 128 bytes per cycle, and the operand delivery at ~55 bytes
 // per cycle; a launch takes as many rounds as the pairs need on the device.  cost_out: the model's cycles.
 PairPlan pair_plan(int epi, int M, int N, int K, double* cost_out) {
     PairPlan best{};
     double best_cost = 1e300;
-    const int resident = max_active_pairs();
     const int nk = (K + GK - 1) / GK;
     const int m_pairs = (M + 2 * GM - 1) / (2 * GM);
     const int ring = GEMM_SMEM_BYTES - 1024 - 256;
-    if (resident >= 1) {
+    for (int splits = 1; splits <= 2; ++splits) {
+        if (splits > 1 && (epi == GEMM_EPI_SWIGLU || nk < 32)) break;
+        const int resident = max_active_pairs(splits);
+        if (resident < 1) continue;
         for (int nmma = 1; nmma <= 2; ++nmma) {
             for (int nchunk = 256; nchunk >= 32; nchunk -= 16) {
                 const int bn = nmma * nchunk;
@@ -537,19 +580,22 @@ PairPlan pair_plan(int epi, int M, int N, int K, double* cost_out) {
                 int stages = ring / stage_bytes;
                 if (stages > MAX_STAGES) stages = MAX_STAGES;
                 if (stages < 3) continue;
+                if (splits > 1 && (wcols / 8) * GM * 32 > stages * stage_bytes) continue;   // partials must fit the ring
                 const int n_tiles = (N + wcols - 1) / wcols;
                 const long long tiles = static_cast<long long>(m_pairs) * n_tiles;
                 const long long rounds = (tiles + resident - 1) / resident;
-                const double mma = nmma * 4 * (nchunk / 2.0 + 20.0);
+                const double kb = static_cast<double>((nk + splits - 1) / splits);
+                const double mma = nmma * 4 * (nchunk / 2.0 + 45.0);
                 const double smem = (stage_bytes + nmma * 4 * (4096.0 + half_rows * 32.0)) / 128.0;
                 const double ld = stage_bytes / 55.0;
                 double per_kb = mma > smem ? mma : smem;
                 if (ld > per_kb) per_kb = ld;
-                const double cost = rounds * (nk * per_kb + 2500.0 + wcols * 14.0);
+                const double epilogue = wcols * 14.0 / splits + (splits > 1 ? 6000.0 : 0.0);   // two cluster barriers, exchange
+                const double cost = rounds * (kb * per_kb + 2500.0 + epilogue);
                 if (cost < best_cost) {
                     best_cost = cost;
                     best.bn = bn; best.wcols = wcols; best.nmma = nmma; best.nchunk = nchunk; best.stages = stages;
-                    best.m_pairs = m_pairs; best.n_tiles = n_tiles;
+                    best.splits = splits; best.m_pairs = m_pairs; best.n_tiles = n_tiles;
                     uint32_t cols = 32;
                     while (cols < static_cast<uint32_t>(bn)) cols <<= 1;
                     best.tmem_cols = cols;
@@ -664,8 +710,8 @@ bool use_pair_kernel(int M, const PairPlan& pp) { return M > GM && pp.bn != 0; }
 int gemm_plan_describe(const dare_ctx* ctx, int epi, int M, int N, int K, int* out) {
     const PairPlan pp = pair_plan(epi, M, N, K, nullptr);
     if (use_pair_kernel(M, pp)) {
-        out[0] = 2; out[1] = pp.bn; out[2] = pp.wcols; out[3] = 1; out[4] = pp.stages;
-        out[5] = pp.m_pairs; out[6] = pp.n_tiles; out[7] = max_active_pairs();
+        out[0] = 2; out[1] = pp.bn; out[2] = pp.wcols; out[3] = pp.splits; out[4] = pp.stages;
+        out[5] = pp.m_pairs; out[6] = pp.n_tiles; out[7] = max_active_pairs(pp.splits);
         return DARE_OK;
     }
     const GemmPlan p = gemm_plan(epi, M, N, K, ctx->sm_count);
