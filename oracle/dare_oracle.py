@@ -183,6 +183,37 @@ def lmhead_logprob(x, w, targets, mask_id=-1, exclude_mask_column=False):
     return zt - lse, lse
 
 
+def lmhead_logprob_backward(x, w, targets, grad_logprob, mask_id=-1, exclude_mask_column=False):
+    """Gradient of sum_m grad_logprob[m] * logprob[m] (lmhead_logprob) with respect to x and w: the backward of
+    the logits-free loss of Section 3.4 (the actor update differentiates the per-token log-probabilities).
+
+    With p = softmax(z) over the non-excluded columns:  d logprob[m] / d z[m, v] = 1[v = targets[m]] - p[m, v]
+    (0 in the excluded column), so
+        dz = grad_logprob[:, None] * (onehot(targets) - p),   dx = dz @ w,   dw = dz^T @ x.
+    Rows whose target is outside [0, V) or is the excluded column have logprob = -inf and take no part
+    (their dz is 0).  Returns (dx float64 [M, D], dw float64 [V, D], dz float64 [M, V]).
+    """
+    x = np.asarray(x, dtype=np.float64)
+    w = np.asarray(w, dtype=np.float64)
+    g = np.asarray(grad_logprob, dtype=np.float64)
+    M, V = x.shape[0], w.shape[0]
+    z = x @ w.T
+    excluded = exclude_mask_column and 0 <= mask_id < V
+    if excluded:
+        z[:, mask_id] = -np.inf
+    e = np.exp(z - z.max(axis=1, keepdims=True))
+    p = e / e.sum(axis=1, keepdims=True)
+    t = np.asarray(targets)
+    ok = (t >= 0) & (t < V)
+    if excluded:
+        ok &= t != mask_id
+    onehot = np.zeros((M, V))
+    onehot[np.nonzero(ok)[0], t[ok]] = 1.0
+    dz = g[:, None] * (onehot - p)
+    dz[~ok] = 0.0
+    return dz @ w, dz.T @ x, dz
+
+
 def token_probability(x_row, w, token, mask_id=-1, exclude_mask_column=True):
     """Softmax probability of one given token for one row (used to judge near-ties)."""
     z = np.asarray(w, dtype=np.float64) @ np.asarray(x_row, dtype=np.float64)

@@ -127,3 +127,55 @@ def test_logprob_is_library_log_softmax_gather_and_cross_entropy():
     np.testing.assert_allclose(allp.sum(axis=1), 1.0, atol=1e-12)
     g = O.lmhead_confidence(x, w, None, -1, False)
     np.testing.assert_allclose(np.exp(O.lmhead_logprob(x, w, g["pred"])[0]), g["conf"], rtol=1e-12)
+
+
+def test_logprob_backward_is_autograd_and_finite_differences():
+    """lmhead_logprob_backward against torch autograd of log_softmax + gather (a library routine written
+    independently of the oracle), against central differences of the oracle's own forward, and by invariants."""
+    import torch
+    rng = np.random.default_rng(11)
+    M, D, V, mu = 7, 12, 23, 5
+    x, w = rng.standard_normal((M, D)), rng.standard_normal((V, D)) * 0.5
+    t = rng.integers(0, V, M)
+    t[t == mu] = 6
+    g = rng.standard_normal(M)
+    for excl in (False, True):
+        dx, dw, dz = O.lmhead_logprob_backward(x, w, t, g, mu, excl)
+        xt = torch.tensor(x, requires_grad=True)
+        wt = torch.tensor(w, requires_grad=True)
+        z = xt @ wt.T
+        if excl:
+            z = z.masked_fill(torch.arange(V)[None, :] == mu, float("-inf"))
+        lp = torch.log_softmax(z, dim=1).gather(1, torch.tensor(t)[:, None])[:, 0]
+        (lp * torch.tensor(g)).sum().backward()
+        np.testing.assert_allclose(dx, xt.grad.numpy(), atol=1e-12)
+        np.testing.assert_allclose(dw, wt.grad.numpy(), atol=1e-12)
+        # invariants: each row of dz sums to 0 (softmax is shift invariant); the excluded column gets nothing
+        np.testing.assert_allclose(dz.sum(axis=1), 0.0, atol=1e-12)
+        if excl:
+            assert (dz[:, mu] == 0).all() and (dw[mu] == 0).all()
+    # central differences of the forward oracle on a few coordinates
+    f = lambda xx, ww: float((g * O.lmhead_logprob(xx, ww, t, mu, True)[0]).sum())
+    dx, dw, _ = O.lmhead_logprob_backward(x, w, t, g, mu, True)
+    h = 1e-6
+    for (i, j) in [(0, 0), (3, 7), (6, 11)]:
+        xp, xm = x.copy(), x.copy()
+        xp[i, j] += h
+        xm[i, j] -= h
+        assert abs((f(xp, w) - f(xm, w)) / (2 * h) - dx[i, j]) < 1e-6
+    for (v, j) in [(0, 0), (int(t[2]), 3), (22, 11)]:
+        wp, wm = w.copy(), w.copy()
+        wp[v, j] += h
+        wm[v, j] -= h
+        assert abs((f(x, wp) - f(x, wm)) / (2 * h) - dw[v, j]) < 1e-6
+    # a row with zero upstream gradient, an out-of-range target or the excluded column as target contributes nothing
+    g2 = g.copy()
+    g2[1] = 0.0
+    t2 = t.copy()
+    t2[2], t2[4] = -1, mu
+    dx2, dw2, dz2 = O.lmhead_logprob_backward(x, w, t2, g2, mu, True)
+    assert (dz2[[1, 2, 4]] == 0).all() and (dx2[[1, 2, 4]] == 0).all()
+    keep = np.array([0, 3, 5, 6])
+    dxk, dwk, _ = O.lmhead_logprob_backward(x[keep], w, t2[keep], g2[keep], mu, True)
+    np.testing.assert_allclose(dw2, dwk, atol=1e-12)
+    np.testing.assert_allclose(dx2[keep], dxk, atol=1e-12)
