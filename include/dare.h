@@ -16,6 +16,7 @@
  *     dare_model_*_window / dare_generate_dual   the same with a cached suffix behind the block (dual cache)
  *     dare_lmhead_sample      the LM head with temperature + Gumbel-max sampling instead of the argmax
  *     dare_lmhead_logprob     log-probability of given tokens (cross-entropy), logits never written either
+ *     dare_lmhead_logprob_backward   its gradient with respect to the hidden states and the weights
  *     dare_attn_varlen        bidirectional attention over packed variable-length sequences
  *     dare_forward_mask, dare_masked_nelbo   the forward (masking) process of Eq. 1 and the bound of Eq. 2
  *
@@ -333,6 +334,30 @@ int dare_model_step(dare_model* model, int32_t* tokens, int B, int64_t row_strid
 int dare_generate(dare_model* model, int32_t* tokens, int B, int64_t row_stride, int prompt_len, int gen_len, int L,
                   void* k_cache, void* v_cache, int cache_cap, int mode, float threshold, int k,
                   int32_t* pred, float* conf, int32_t* n_remaining, int32_t* steps_per_block, void* stream);
+
+/*
+ * Backward of dare_lmhead_logprob (Section 3.4: the actor update differentiates the per-token log-probabilities;
+ * the logits are recomputed, never stored).  For L = sum_m grad_logprob[m] * logprob[m]:
+ *     dz[m, v]  = grad_logprob[m] * (1[v = targets[m]] - exp(z[m, v] - lse[m]))   (0 in the excluded column;
+ *                 a row whose target is outside [0, V) or is the excluded column gets dz = 0)
+ *     d_hidden  = dz . w           bf16 [M, D]
+ *     d_w       = dz^T . hidden    bf16 [V, D]
+ * hidden bf16 [M, D]; w bf16 [V, D]; w_t bf16 [D, V] = the transpose of w, kept by the caller (dare_transpose_bf16
+ * makes it; it changes only when the weights do); targets int32 [M]; lse fp32 [M] = the logsumexp that
+ * dare_lmhead_logprob returned for the same inputs; grad_logprob fp32 [M].
+ * dz bf16 [M, V] and dzt bf16 [V, M]: caller-provided scratch for the gradient of the logits in both orientations
+ * (2 * M * V * 2 bytes together: the caller bounds them by the rows it passes per call; d_w of several calls add up
+ * on the caller's side).  Products accumulate in fp32 and are rounded to bf16 once.
+ * Supported: M, D, V multiples of 8; the ctx workspace must hold M * D * 2 bytes (DARE_ERR_WORKSPACE otherwise).
+ * Enqueues on `stream`, no synchronisation.
+ *
+ * dare_transpose_bf16: out [cols, rows] = transpose of in [rows, cols] (bf16, dense, out != in, rows <= 2 097 120).
+ */
+int dare_lmhead_logprob_backward(dare_ctx* ctx, const void* hidden, int M, int D, const void* w, const void* w_t,
+                                 int V, const int32_t* targets, int32_t mask_id, int exclude_mask_column,
+                                 const float* lse, const float* grad_logprob, void* dz, void* dzt, void* d_hidden,
+                                 void* d_w, void* stream);
+int dare_transpose_bf16(dare_ctx* ctx, const void* in, int rows, int cols, void* out, void* stream);
 
 /*
  * Dual cache (prefix and suffix) for a fully bidirectional masked model (Section 3.4, rollout with KV-cache

@@ -22,7 +22,7 @@ DEV_WAIT_EXPIRED = 2
 
 EXPORTS = ["dare_create", "dare_destroy", "dare_status_string", "dare_device_status", "dare_sm_count",
            "dare_attn_block", "dare_attn_varlen", "dare_lmhead_confidence", "dare_unmask_select", "dare_denoise_block",
-           "dare_lmhead_confidence_static", "dare_lmhead_sample", "dare_lmhead_logprob", "dare_forward_mask", "dare_masked_nelbo", "dare_model_create", "dare_model_destroy", "dare_model_forward",
+           "dare_lmhead_confidence_static", "dare_lmhead_sample", "dare_lmhead_logprob", "dare_lmhead_logprob_backward", "dare_transpose_bf16", "dare_forward_mask", "dare_masked_nelbo", "dare_model_create", "dare_model_destroy", "dare_model_forward",
            "dare_model_step", "dare_generate", "dare_model_forward_window", "dare_model_step_window", "dare_generate_dual",
            "dare_linear", "dare_linear_plan", "dare_rmsnorm", "dare_rope_kv_write"]
 
@@ -69,6 +69,10 @@ def load():
     lib.dare_lmhead_sample.restype = i32
     lib.dare_lmhead_logprob.argtypes = [vp, vp, i32, i32, vp, i32, vp, i32, i32, vp, vp, vp]
     lib.dare_lmhead_logprob.restype = i32
+    lib.dare_lmhead_logprob_backward.argtypes = [vp, vp, i32, i32, vp, vp, i32, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp]
+    lib.dare_lmhead_logprob_backward.restype = i32
+    lib.dare_transpose_bf16.argtypes = [vp, vp, i32, i32, vp, vp]
+    lib.dare_transpose_bf16.restype = i32
     lib.dare_forward_mask.argtypes = [vp, vp, vp, i32, i64, i32, i32, vp, i32, C.c_uint64, C.c_uint32, vp]
     lib.dare_forward_mask.restype = i32
     lib.dare_masked_nelbo.argtypes = [vp, vp, vp, i32, i64, i32, i32, i32, vp, vp, vp, vp]
@@ -251,6 +255,37 @@ def dare_lmhead_logprob(ctx: Context, hidden, w, targets, mask_id: int = -1, exc
     if rc != 0 and check:
         raise DareError(rc, "dare_lmhead_logprob")
     return logprob if check else rc
+
+
+def dare_transpose_bf16(ctx: Context, a, out=None, stream=None, check: bool = True):
+    rows, cols = a.shape
+    if out is None:
+        out = torch.empty(cols, rows, dtype=torch.bfloat16, device=a.device)
+    rc = load().dare_transpose_bf16(ctx.handle, _ptr(a, torch.bfloat16), rows, cols, _ptr(out, torch.bfloat16),
+                                    _stream(stream))
+    if rc != 0 and check:
+        raise DareError(rc, "dare_transpose_bf16")
+    return out if check else rc
+
+
+def dare_lmhead_logprob_backward(ctx: Context, hidden, w, w_t, targets, lse, grad_logprob, mask_id: int = -1,
+                                 exclude_mask_column: bool = False, dz=None, dzt=None, d_hidden=None, d_w=None,
+                                 stream=None, check: bool = True):
+    """Gradient of sum(grad_logprob * logprob) with respect to hidden and w.  Returns (d_hidden, d_w, dz, dzt)."""
+    M, D = hidden.shape
+    V = w.shape[0]
+    bf, dev = torch.bfloat16, hidden.device
+    dz = torch.empty(M, V, dtype=bf, device=dev) if dz is None else dz
+    dzt = torch.empty(V, M, dtype=bf, device=dev) if dzt is None else dzt
+    d_hidden = torch.empty(M, D, dtype=bf, device=dev) if d_hidden is None else d_hidden
+    d_w = torch.empty(V, D, dtype=bf, device=dev) if d_w is None else d_w
+    rc = load().dare_lmhead_logprob_backward(ctx.handle, _ptr(hidden, bf), M, D, _ptr(w, bf), _ptr(w_t, bf), V,
+                                             _ptr(targets, torch.int32), int(mask_id), int(bool(exclude_mask_column)),
+                                             _ptr(lse, torch.float32), _ptr(grad_logprob, torch.float32), _ptr(dz, bf),
+                                             _ptr(dzt, bf), _ptr(d_hidden, bf), _ptr(d_w, bf), _stream(stream))
+    if rc != 0 and check:
+        raise DareError(rc, "dare_lmhead_logprob_backward")
+    return (d_hidden, d_w, dz, dzt) if check else rc
 
 
 def dare_forward_mask(ctx: Context, x0, start: int, length: int, p_mask, mask_id: int, seed: int, sample: int, xt=None,

@@ -15,7 +15,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdare.so")
-SOURCES = ["api.cu", "lmhead.cu", "attn.cu", "select.cu", "gemm.cu", "layers.cu", "model.cu", "diffusion.cu"]
+SOURCES = ["api.cu", "lmhead.cu", "attn.cu", "select.cu", "gemm.cu", "layers.cu", "model.cu", "diffusion.cu", "backward.cu"]
 HEADERS = ["ptx.cuh", "internal.h", os.path.join("..", "..", "include", "dare.h")]
 
 

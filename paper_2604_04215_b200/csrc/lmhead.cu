@@ -112,6 +112,13 @@ struct LmSampling {
     const int32_t* targets;        // LM_LOGPROB: target token per row
     float* part_y;                 // per partial: best perturbed score and the raw logit there
     float* part_zb;
+    // LM_GRAD: per-row logsumexp of the forward pass and upstream gradient; outputs dz [M, V] and its transpose
+    // [V, ldm] (bf16)
+    const float* lse;
+    const float* grad;
+    __nv_bfloat16* dz;
+    __nv_bfloat16* dzt;
+    int ldm;
 };
 
 __device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1) {
@@ -132,7 +139,9 @@ __device__ __forceinline__ float gumbel_from_word(uint32_t w) {
 
 // MODE 0: greedy (argmax token, its probability); 1: sampling epilogue; 2: log-probability of a given target
 // token per row (the partial's third slot then carries the target's logit instead of an argmax).
-constexpr int LM_GREEDY = 0, LM_SAMPLE = 1, LM_LOGPROB = 2;
+// MODE 3: gradient of the log-probability with respect to the logits, g * (onehot(target) - softmax), written as
+// bf16 in both orientations (the two products of the backward pass take it from there); no partials.
+constexpr int LM_GREEDY = 0, LM_SAMPLE = 1, LM_LOGPROB = 2, LM_GRAD = 3;
 
 template <int MODE>
 __global__ void __launch_bounds__(LM_THREADS, 1)
@@ -142,6 +151,7 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
                       uint32_t* __restrict__ dev_status, const LmSampling smp) {
     constexpr bool SAMPLE = MODE == LM_SAMPLE;
     constexpr bool LOGPROB = MODE == LM_LOGPROB;
+    constexpr bool GRAD = MODE == LM_GRAD;
     const int Mc = live_rows ? *live_rows : M;          // rows that need logits (uniform over the grid)
     const int m_tiles = (Mc + BM - 1) / BM;
     if (m_tiles == 0) return;
@@ -265,6 +275,14 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
                 const int row_c = m_tile * BM + row_in_tile;
                 if (row_c < Mc) target = smp.targets[row_c];
             }
+            float g_row = 0.f, lse2 = 0.f;                       // GRAD: upstream gradient, logsumexp * log2(e)
+            const int row_g = m_tile * BM + row_in_tile;
+            if (GRAD && row_g < Mc) {
+                target = smp.targets[row_g];
+                // a target outside the vocabulary or in the excluded column has log-probability -inf: no gradient
+                if (target >= 0 && target < V && target != mask_col) g_row = smp.grad[row_g];
+                lse2 = smp.lse[row_g] * LOG2E;
+            }
             for (int n_tile = group; n_tile < n_tiles && ok; n_tile += groups, ++it) {
                 const int acc = it & 1;
                 const uint32_t acc_phase = (it >> 1) & 1;
@@ -279,6 +297,40 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
                     tmem_ld_32cols(taddr + c * 32, v);
                     tmem_ld_wait();
                     const int cbase = col0 + c * 32;
+                    if (GRAD) {
+                        // dz = g * (1[col = target] - exp(z - lse)); 0 beyond the vocabulary and in the excluded column
+                        if (row_g < Mc) {
+                            uint32_t packed[16];
+#pragma unroll
+                            for (int j = 0; j < 32; j += 2) {
+                                float d2[2];
+#pragma unroll
+                                for (int e = 0; e < 2; ++e) {
+                                    const int col = cbase + j + e;
+                                    const float pr = fast_exp2(fmaf(__uint_as_float(v[j + e]), LOG2E, -lse2));
+                                    float d = g_row * ((col == target ? 1.0f : 0.0f) - pr);
+                                    if (col >= V || col == mask_col) d = 0.f;
+                                    d2[e] = d;
+                                }
+                                packed[j >> 1] = pack_bf16(d2[0], d2[1]);
+                            }
+                            __nv_bfloat16* dz_row = smp.dz + static_cast<size_t>(row_g) * V + cbase;
+#pragma unroll
+                            for (int q = 0; q < 4; ++q)       // V is a multiple of 8: a group of 8 columns is inside or outside
+                                if (cbase + q * 8 < V)
+                                    *reinterpret_cast<uint4*>(dz_row + q * 8) =
+                                        make_uint4(packed[q * 4], packed[q * 4 + 1], packed[q * 4 + 2], packed[q * 4 + 3]);
+                            // transposed copy: the lanes of a warp are consecutive rows, so each column is one 64-byte run
+                            unsigned short* dzt_col = reinterpret_cast<unsigned short*>(smp.dzt) +
+                                                      static_cast<size_t>(cbase) * smp.ldm + row_g;
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (cbase + j < V)
+                                    dzt_col[static_cast<size_t>(j) * smp.ldm] =
+                                        static_cast<unsigned short>(j & 1 ? packed[j >> 1] >> 16 : packed[j >> 1] & 0xffffu);
+                        }
+                        continue;
+                    }
                     float cmax = -INFINITY;
                     int carg = ARG_NONE;
                     if (edge) {
@@ -329,7 +381,7 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
                 mbar_arrive(&bars->tmem_empty[acc]);
             }
             const int row = m_tile * BM + row_in_tile;
-            if (ok && row < Mc) {
+            if (!GRAD && ok && row < Mc) {
                 const size_t o = static_cast<size_t>(row) * groups + group;
                 part_max[o] = run_max;
                 part_sum[o] = run_sum;
@@ -590,6 +642,36 @@ int launch_lmhead_logprob(const dare_ctx* ctx, void* scratch, const void* hidden
     const int rows_per_block = 8;
     lmhead_merge_logprob_kernel<<<(M + rows_per_block - 1) / rows_per_block, rows_per_block * 32, 0, stream>>>(
         part_max, part_sum, part_zt, grid, n_tiles, M, logprob, lse_out);
+    return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
+}
+
+// dz[m, v] = grad[m] * (1[v = targets[m]] - exp(z[m, v] - lse[m])) as bf16 [M, V] and transposed [V, ldm]
+// (ldm >= M; columns [M, ldm) of the transpose are not written).
+int launch_lmhead_grad(const dare_ctx* ctx, const void* hidden, int M, int D, const void* w, int V,
+                       const int32_t* targets, int32_t mask_id, int exclude_mask_column, const float* lse,
+                       const float* grad, void* dz, void* dzt, int ldm, cudaStream_t stream) {
+    const int n_tiles = (V + BN - 1) / BN;
+    const int m_tiles_max = (M + BM - 1) / BM;
+    int grid = ctx->sm_count;
+    if (grid > m_tiles_max * n_tiles) grid = m_tiles_max * n_tiles;
+    CUtensorMap tmap_x, tmap_w;
+    int rc = make_tmap_bf16_2d(ctx, &tmap_x, hidden, static_cast<uint64_t>(M), static_cast<uint64_t>(D), BM, BK);
+    if (rc != DARE_OK) return rc;
+    rc = make_tmap_bf16_2d(ctx, &tmap_w, w, static_cast<uint64_t>(V), static_cast<uint64_t>(D), BN, BK);
+    if (rc != DARE_OK) return rc;
+    if (cudaFuncSetAttribute(lmhead_partial_kernel<LM_GRAD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             LM_SMEM_BYTES) != cudaSuccess)
+        return DARE_ERR_CUDA;
+    const int mask_col = (exclude_mask_column && mask_id >= 0 && mask_id < V) ? mask_id : -1;
+    LmSampling smp = {};
+    smp.targets = targets;
+    smp.lse = lse;
+    smp.grad = grad;
+    smp.dz = static_cast<__nv_bfloat16*>(dz);
+    smp.dzt = static_cast<__nv_bfloat16*>(dzt);
+    smp.ldm = ldm;
+    lmhead_partial_kernel<LM_GRAD><<<grid, LM_THREADS, LM_SMEM_BYTES, stream>>>(
+        tmap_x, tmap_w, M, nullptr, D, V, mask_col, n_tiles, nullptr, nullptr, nullptr, ctx->dev_status, smp);
     return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
 }
 
