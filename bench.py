@@ -248,8 +248,24 @@ def run_ours(args):
     # greedy against sampled head with every row masked (the sampling epilogue draws M * V Gumbel variates);
     # skipped in the few-step runs used under the profiler
     full_ms = {}
+    bwd = {}
+    if args.steps >= 64 and wl.M % 8 == 0 and wl.vocab % 8 == 0:
+        # log-probability head and its backward on all rows (the likelihood / actor-update side of the same head)
+        M_, V_ = wl.M, wl.vocab
+        tg = I.uniform_int(1, I.TID_TOK, (M_,), 0, V_ - 1).cuda()
+        gl = torch.ones(M_, dtype=torch.float32, device="cuda")
+        lse_b = torch.empty(M_, dtype=torch.float32, device="cuda")
+        lp_b = torch.empty(M_, dtype=torch.float32, device="cuda")
+        w_t = dare.dare_transpose_bf16(ctx, w)
+        bf = torch.bfloat16
+        bwd = {"dz": torch.empty(M_, V_, dtype=bf, device="cuda"), "dzt": torch.empty(V_, M_, dtype=bf, device="cuda"),
+               "d_hidden": torch.empty(M_, wl.hidden, dtype=bf, device="cuda"),
+               "d_w": torch.empty(V_, wl.hidden, dtype=bf, device="cuda")}
+        logprob_fn = lambda: dare.dare_lmhead_logprob(ctx, pool[0][1], w, tg, wl.mask_id, True, logprob=lp_b, lse=lse_b, stream=stream)
+        backward_fn = lambda: dare.dare_lmhead_logprob_backward(ctx, pool[0][1], w, w_t, tg, lse_b, gl, wl.mask_id, True, stream=stream, **bwd)
     for name, fn in (() if args.steps < 64 else (("lmhead_all_rows_ms", lambda: dare.dare_lmhead_confidence(ctx, pool[0][1], w, None, wl.mask_id, True, pred, conf, stream=stream)),
-                     ("lmhead_sample_all_rows_ms", lambda: dare.dare_lmhead_sample(ctx, pool[0][1], w, None, wl.mask_id, True, 1.0, 1, 1, pred, conf, stream=stream)))):
+                     ("lmhead_sample_all_rows_ms", lambda: dare.dare_lmhead_sample(ctx, pool[0][1], w, None, wl.mask_id, True, 1.0, 1, 1, pred, conf, stream=stream)))
+                     + ((("lmhead_logprob_all_rows_ms", logprob_fn), ("lmhead_logprob_backward_all_rows_ms", backward_fn)) if bwd else ())):
         for _ in range(2):
             fn()
         es = [torch.cuda.Event(enable_timing=True) for _ in range(9)]

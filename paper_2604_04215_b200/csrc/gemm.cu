@@ -463,8 +463,28 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         }
         cluster_sync_all();                              // the partials of the groups this CTA owns have arrived
     }
+    // Without a K split and without the SwiGLU pairing a thread takes 32 accumulator columns per load (one wait per
+    // 64 output bytes); the last n_groups % 4 groups, and the other cases, go 8 columns at a time.
+    int g_begin = set;
+    if (EPI != GEMM_EPI_SWIGLU && p.splits == 1 && epi_warp && !*abort_flag) {
+        const int n_chunks = n_groups / 4;
+        for (int ci = set; ci < n_chunks; ci += 2) {
+            uint32_t v[32];
+            tmem_ld_32cols(taddr + ci * 32, v);
+            tmem_ld_wait();
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                float f[8], u[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) { f[k] = __uint_as_float(v[q * 8 + k]); u[k] = 0.f; }
+                const int col = col_base + ci * 32 + q * 8;
+                if (row_ok && col < g.N) store_group<EPI>(f, u, g.out, g.res, row_off + col);
+            }
+        }
+        g_begin = n_chunks * 4 + set;
+    }
     if (epi_warp && !*abort_flag) {
-        for (int gi = set; gi < n_groups; gi += 2) {
+        for (int gi = g_begin; gi < n_groups; gi += 2) {
             if (p.splits > 1 && ((gi >> 1) & 1) != split) continue;
             uint32_t v[8];
             float f[8], u[8];
