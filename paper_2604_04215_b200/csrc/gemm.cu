@@ -314,6 +314,7 @@ struct PairPlan {
     int nmma;        // MMAs per K step (1 or 2), each nchunk columns wide
     int nchunk;
     int splits;      // pairs along K per output tile (1 or 2); two pairs form a cluster of four CTAs
+    int resident;    // clusters of this shape the device holds at once
     int stages;
     int m_pairs, n_tiles;
     uint32_t tmem_cols;
@@ -327,6 +328,31 @@ struct PairArgs {
     uint32_t* dev_status;
 };
 
+struct PairBarriers {
+    uint64_t full[MAX_STAGES];
+    uint64_t empty[MAX_STAGES];
+    uint64_t tmem_full[2];       // accumulator buffer ready (arrives in both CTAs)
+    uint64_t tmem_empty[2];      // accumulator buffer drained by the epilogue warps of both CTAs (even CTA's is used)
+    uint32_t tmem_base;
+    uint32_t abort_flag;
+};
+constexpr int PAIR_EPI_WARPS = 8;
+
+// Arrive on the mbarrier at this CTA's shared-memory address `bar` in CTA `rank` of the cluster.
+__device__ __forceinline__ void mbar_arrive_cluster(uint64_t* bar, uint32_t rank) {
+    asm volatile(
+        "{\n"
+        ".reg .b32 remote;\n"
+        "mapa.shared::cluster.u32 remote, %0, %1;\n"
+        "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [remote];\n"
+        "}\n" ::"r"(smem_u32(bar)),
+        "r"(rank)
+        : "memory");
+}
+
+// Persistent: cluster c computes tiles c, c + #clusters, ... (row index fastest).  The copies run ahead into the
+// next tile, and with bn <= 256 two accumulator buffers alternate, so a tile's epilogue overlaps the next tile's
+// main loop.  With a K split every cluster has exactly one tile (the exchange needs the idle ring).
 template <int EPI>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
@@ -338,7 +364,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    GemmBarriers* bars = reinterpret_cast<GemmBarriers*>(tiles + p.stages * stage_bytes);
+    PairBarriers* bars = reinterpret_cast<PairBarriers*>(tiles + p.stages * stage_bytes);
     volatile uint32_t* abort_flag = &bars->abort_flag;
 
     const int warp = warp_index_uniform();
@@ -346,19 +372,24 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     const int rank4 = static_cast<int>(cluster_cta_rank());
     const int rank = rank4 & 1;                               // 0: issues the MMAs and owns the "full" barriers
     const int split = rank4 >> 1;                             // which part of K this pair computes
-    const int tile = blockIdx.x / (2 * p.splits);
-    const int m_pair = tile % p.m_pairs;                      // row index fastest: pairs sharing W run together
-    const int n_tile = tile / p.m_pairs;
+    const int cluster_size = 2 * p.splits;
+    const int cluster_id = blockIdx.x / cluster_size;
+    const int n_clusters = gridDim.x / cluster_size;
+    const int total_tiles = p.m_pairs * p.n_tiles;
     const int nk = (g.K + GK - 1) / GK;
     const int kb_begin = static_cast<int>(static_cast<long long>(nk) * split / p.splits);
     const int kb_end = static_cast<int>(static_cast<long long>(nk) * (split + 1) / p.splits);
+    const int n_acc = p.bn <= 256 ? 2 : 1;                   // accumulator buffers (256 columns apart)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
             mbar_init(&bars->full[s], 1);
             mbar_init(&bars->empty[s], 1);
         }
-        mbar_init(&bars->tmem_full, 1);
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(&bars->tmem_full[a], 1);
+            mbar_init(&bars->tmem_empty[a], 2 * PAIR_EPI_WARPS);
+        }
         bars->abort_flag = 0;
         fence_barrier_init();
     }
@@ -367,7 +398,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         tmem_relinquish_pair();
     }
     tc_fence_before_sync();
-    cluster_sync_all();              // both CTAs' barriers exist before either CTA signals the other's
+    cluster_sync_all();              // every CTA's barriers exist before another CTA signals them
     tc_fence_after_sync();
     const uint32_t tmem_base = bars->tmem_base;
 
@@ -377,148 +408,174 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             prefetch_tensormap(&tmap_b);
             if (EPI == GEMM_EPI_SWIGLU) prefetch_tensormap(&tmap_b2);
             const CUtensorMap* tmap_w = (EPI == GEMM_EPI_SWIGLU && rank == 1) ? &tmap_b2 : &tmap_b;
-            // W row of chunk 0 for this CTA; chunk c starts w_step rows further on
-            const int w_row0 = EPI == GEMM_EPI_SWIGLU ? n_tile * p.wcols : n_tile * p.bn + rank * half_rows;
-            const int w_step = EPI == GEMM_EPI_SWIGLU ? half_rows : p.nchunk;
+            const int w_step = EPI == GEMM_EPI_SWIGLU ? half_rows : p.nchunk;   // rows from one chunk to the next
             const uint32_t full0 = cluster_map_shared(smem_u32(&bars->full[0]), rank4 & ~1);   // the even CTA's barriers
             int stage = 0;
             uint32_t phase = 0;
-            for (int kb = kb_begin; kb < kb_end; ++kb) {
-                if (!mbar_wait(&bars->empty[stage], phase ^ 1, abort_flag)) break;
-                uint8_t* a_dst = tiles + stage * stage_bytes;
-                uint8_t* b_dst = a_dst + A_TILE_BYTES;
-                const uint32_t full = full0 + stage * static_cast<uint32_t>(sizeof(uint64_t));
-                if (rank == 0) mbar_arrive_expect_tx(&bars->full[stage], 2 * stage_bytes);   // both CTAs' bytes
-                tma_load_2d_pair(a_dst, &tmap_a, full, kb * GK, m_pair * 2 * GM + rank * GM);
-                for (int c = 0; c < p.nmma; ++c)
-                    tma_load_2d_pair(b_dst + c * chunk_bytes, tmap_w, full, kb * GK, w_row0 + c * w_step);
-                if (++stage == p.stages) { stage = 0; phase ^= 1; }
+            bool ok = true;
+            for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters) {
+                const int m_pair = tile % p.m_pairs, n_tile = tile / p.m_pairs;
+                const int w_row0 = EPI == GEMM_EPI_SWIGLU ? n_tile * p.wcols : n_tile * p.bn + rank * half_rows;
+                for (int kb = kb_begin; kb < kb_end; ++kb) {
+                    if (!mbar_wait(&bars->empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
+                    uint8_t* a_dst = tiles + stage * stage_bytes;
+                    uint8_t* b_dst = a_dst + A_TILE_BYTES;
+                    const uint32_t full = full0 + stage * static_cast<uint32_t>(sizeof(uint64_t));
+                    if (rank == 0) mbar_arrive_expect_tx(&bars->full[stage], 2 * stage_bytes);   // both CTAs' bytes
+                    tma_load_2d_pair(a_dst, &tmap_a, full, kb * GK, m_pair * 2 * GM + rank * GM);
+                    for (int c = 0; c < p.nmma; ++c)
+                        tma_load_2d_pair(b_dst + c * chunk_bytes, tmap_w, full, kb * GK, w_row0 + c * w_step);
+                    if (++stage == p.stages) { stage = 0; phase ^= 1; }
+                }
             }
         }
     } else if (warp == 1 && rank == 0) {
-        // all lanes run the loop, one elected lane issues the MMAs and their commits (which arrive in both CTAs)
+        // all lanes run the loops, one elected lane issues the MMAs and their commits (which arrive in both CTAs)
         const bool leader = elect_one_sync();
         const uint32_t idesc = umma_idesc_bf16(2 * GM, p.nchunk);
         const uint16_t pair_mask = static_cast<uint16_t>(3u << rank4);     // this CTA (even rank) and the next
         int stage = 0;
         uint32_t phase = 0;
+        int it = 0;
         bool ok = true;
-        for (int kb = kb_begin; kb < kb_end; ++kb) {
-            ok = __all_sync(0xffffffffu, mbar_wait(&bars->full[stage], phase, abort_flag));
+        for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters, ++it) {
+            const int acc = it % n_acc;
+            const uint32_t acc_phase = (it / n_acc) & 1;
+            ok = __all_sync(0xffffffffu, mbar_wait(&bars->tmem_empty[acc], acc_phase ^ 1, abort_flag));
             if (!ok) break;
             tc_fence_after_sync();
-            const uint32_t a_addr = smem_u32(tiles + stage * stage_bytes);
-            const uint64_t a_desc = umma_desc_sw128_kmajor(a_addr);
-            const uint32_t accumulate = kb > kb_begin;
-            if (leader) {
-                for (int c = 0; c < p.nmma; ++c) {
-                    const uint64_t b_desc = umma_desc_sw128_kmajor(a_addr + A_TILE_BYTES + c * chunk_bytes);
+            const uint32_t d_tmem = tmem_base + acc * 256;
+            for (int kb = kb_begin; kb < kb_end; ++kb) {
+                ok = __all_sync(0xffffffffu, mbar_wait(&bars->full[stage], phase, abort_flag));
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t a_addr = smem_u32(tiles + stage * stage_bytes);
+                const uint64_t a_desc = umma_desc_sw128_kmajor(a_addr);
+                const uint32_t accumulate = kb > kb_begin;
+                if (leader) {
+                    for (int c = 0; c < p.nmma; ++c) {
+                        const uint64_t b_desc = umma_desc_sw128_kmajor(a_addr + A_TILE_BYTES + c * chunk_bytes);
 #pragma unroll
-                    for (int kk = 0; kk < GK / 16; ++kk)   // +32 bytes along K per step = +2 descriptor units
-                        umma_bf16_pair(tmem_base + c * p.nchunk, a_desc + 2 * kk, b_desc + 2 * kk, idesc,
-                                       accumulate | (kk != 0));
+                        for (int kk = 0; kk < GK / 16; ++kk)   // +32 bytes along K per step = +2 descriptor units
+                            umma_bf16_pair(d_tmem + c * p.nchunk, a_desc + 2 * kk, b_desc + 2 * kk, idesc,
+                                           accumulate | (kk != 0));
+                    }
+                    umma_commit_pair(&bars->empty[stage], pair_mask);
                 }
-                umma_commit_pair(&bars->empty[stage], pair_mask);
+                __syncwarp();
+                if (++stage == p.stages) { stage = 0; phase ^= 1; }
             }
+            if (ok && leader) umma_commit_pair(&bars->tmem_full[acc], pair_mask);
             __syncwarp();
-            if (++stage == p.stages) { stage = 0; phase ^= 1; }
         }
-        if (ok && leader) umma_commit_pair(&bars->tmem_full, pair_mask);
-        __syncwarp();
     }
+    __syncwarp();      // (the lanes of the producer and MMA warps walk the tile loop below together)
 
     // ---- epilogue (warps 2..9 of every CTA): warp w may touch TMEM lanes [32 * (w % 4), +32); the two sets of
-    // four warps alternate over the 8-column groups of the CTA's 128 rows.  With a K split, group gi belongs to
-    // the pair (gi / 2) % 2; the other pair's CTA with the same rows sends its partial into slot gi of this
+    // four warps alternate over the column groups of the CTA's 128 rows.  With a K split, 8-column group gi belongs
+    // to the pair (gi / 2) % 2; the other pair's CTA with the same rows sends its partial into slot gi of this
     // CTA's idle ring ([group][row][8 floats]).
     const bool epi_warp = warp >= 2;
     const int lq = warp & 3;
     const int set = epi_warp ? (warp - 2) >> 2 : 0;
     const int n_groups = p.wcols / 8;
     const int row_local = lq * 32 + lane;
-    const int row = m_pair * 2 * GM + rank * GM + row_local;
-    const bool row_ok = row < g.M;
-    const size_t row_off = static_cast<size_t>(row) * g.ldo;
-    const int col_base = n_tile * p.wcols;
-    const uint32_t taddr = tmem_base + (static_cast<uint32_t>(lq * 32) << 16);
-    if (epi_warp) {
-        mbar_wait(&bars->tmem_full, 0, abort_flag);     // (a wait that gave up leaves the abort flag set)
-        tc_fence_after_sync();
-    }
-    __syncwarp();
-    if (p.splits > 1) {
-        cluster_sync_all();                              // every CTA of the cluster is done with its ring
-        if (epi_warp) {
-            const uint32_t ring = smem_u32(tiles);
-            for (int gi = set; gi < n_groups; gi += 2) {
-                if (((gi >> 1) & 1) == split) continue;  // mine: stays here
-                uint32_t v[8];
-                tmem_ld_8cols(taddr + gi * 8, v);
-                tmem_ld_wait();
-                const uint32_t local = ring + ((static_cast<uint32_t>(gi) * GM + row_local) << 5);
-                const uint32_t remote = cluster_map_shared(local, static_cast<uint32_t>(rank4 ^ 2));
-                st_shared_cluster_v4(remote, v[0], v[1], v[2], v[3]);
-                st_shared_cluster_v4(remote + 16, v[4], v[5], v[6], v[7]);
-            }
+    int it = 0;
+    bool epi_ok = true;
+    for (int tile = cluster_id; tile < total_tiles; tile += n_clusters, ++it) {
+        const int m_pair = tile % p.m_pairs, n_tile = tile / p.m_pairs;
+        const int acc = it % n_acc;
+        const uint32_t acc_phase = (it / n_acc) & 1;
+        const int row = m_pair * 2 * GM + rank * GM + row_local;
+        const bool row_ok = row < g.M;
+        const size_t row_off = static_cast<size_t>(row) * g.ldo;
+        const int col_base = n_tile * p.wcols;
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(lq * 32) << 16) + acc * 256;
+        if (epi_warp && epi_ok) {
+            epi_ok = mbar_wait(&bars->tmem_full[acc], acc_phase, abort_flag);   // (a wait that gave up leaves the abort flag set)
+            tc_fence_after_sync();
         }
-        cluster_sync_all();                              // the partials of the groups this CTA owns have arrived
-    }
-    // Without a K split and without the SwiGLU pairing a thread takes 32 accumulator columns per load (one wait per
-    // 64 output bytes); the last n_groups % 4 groups, and the other cases, go 8 columns at a time.
-    int g_begin = set;
-    if (EPI != GEMM_EPI_SWIGLU && p.splits == 1 && epi_warp && !*abort_flag) {
-        const int n_chunks = n_groups / 4;
-        for (int ci = set; ci < n_chunks; ci += 2) {
-            uint32_t v[32];
-            tmem_ld_32cols(taddr + ci * 32, v);
-            tmem_ld_wait();
+        __syncwarp();
+        if (p.splits > 1) {              // (one tile per cluster in this case)
+            cluster_sync_all();                              // every CTA of the cluster is done with its ring
+            if (epi_warp) {
+                const uint32_t ring = smem_u32(tiles);
+                for (int gi = set; gi < n_groups; gi += 2) {
+                    if (((gi >> 1) & 1) == split) continue;  // mine: stays here
+                    uint32_t v[8];
+                    tmem_ld_8cols(taddr + gi * 8, v);
+                    tmem_ld_wait();
+                    const uint32_t local = ring + ((static_cast<uint32_t>(gi) * GM + row_local) << 5);
+                    const uint32_t remote = cluster_map_shared(local, static_cast<uint32_t>(rank4 ^ 2));
+                    st_shared_cluster_v4(remote, v[0], v[1], v[2], v[3]);
+                    st_shared_cluster_v4(remote + 16, v[4], v[5], v[6], v[7]);
+                }
+            }
+            cluster_sync_all();                              // the partials of the groups this CTA owns have arrived
+        }
+        if (!epi_warp) continue;
+        const bool live = epi_ok && !*abort_flag;
+        // Without a K split and without the SwiGLU pairing a thread takes 32 accumulator columns per load (one wait
+        // per 64 output bytes); the last n_groups % 4 groups, and the other cases, go 8 columns at a time.
+        int g_begin = set;
+        if (EPI != GEMM_EPI_SWIGLU && p.splits == 1 && live) {
+            const int n_chunks = n_groups / 4;
+            for (int ci = set; ci < n_chunks; ci += 2) {
+                uint32_t v[32];
+                tmem_ld_32cols(taddr + ci * 32, v);
+                tmem_ld_wait();
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
+                for (int q = 0; q < 4; ++q) {
+                    float f[8], u[8];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) { f[k] = __uint_as_float(v[q * 8 + k]); u[k] = 0.f; }
+                    const int col = col_base + ci * 32 + q * 8;
+                    if (row_ok && col < g.N) store_group<EPI>(f, u, g.out, g.res, row_off + col);
+                }
+            }
+            g_begin = n_chunks * 4 + set;
+        }
+        if (live) {
+            for (int gi = g_begin; gi < n_groups; gi += 2) {
+                if (p.splits > 1 && ((gi >> 1) & 1) != split) continue;
+                uint32_t v[8];
                 float f[8], u[8];
+                if (EPI == GEMM_EPI_SWIGLU) {
+                    const int j = gi * 8, c = j / half_rows;
+                    const int gcol = c * p.nchunk + (j - c * half_rows);
+                    uint32_t w[8];
+                    tmem_ld_8cols(taddr + gcol, v);
+                    tmem_ld_8cols(taddr + gcol + half_rows, w);
+                    tmem_ld_wait();
 #pragma unroll
-                for (int k = 0; k < 8; ++k) { f[k] = __uint_as_float(v[q * 8 + k]); u[k] = 0.f; }
-                const int col = col_base + ci * 32 + q * 8;
+                    for (int k = 0; k < 8; ++k) u[k] = __uint_as_float(w[k]);
+                } else {
+                    tmem_ld_8cols(taddr + gi * 8, v);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) u[k] = 0.f;
+                }
+#pragma unroll
+                for (int k = 0; k < 8; ++k) f[k] = __uint_as_float(v[k]);
+                if (p.splits > 1) {
+                    // first half of K + second half of K, in that order in both pairs
+                    const float4* q = reinterpret_cast<const float4*>(tiles + ((static_cast<size_t>(gi) * GM + row_local) << 5));
+                    const float4 a = q[0], c = q[1];
+                    const float o[8] = {a.x, a.y, a.z, a.w, c.x, c.y, c.z, c.w};
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) f[k] = split == 0 ? f[k] + o[k] : o[k] + f[k];
+                }
+                const int col = col_base + gi * 8;
                 if (row_ok && col < g.N) store_group<EPI>(f, u, g.out, g.res, row_off + col);
             }
         }
-        g_begin = n_chunks * 4 + set;
-    }
-    if (epi_warp && !*abort_flag) {
-        for (int gi = g_begin; gi < n_groups; gi += 2) {
-            if (p.splits > 1 && ((gi >> 1) & 1) != split) continue;
-            uint32_t v[8];
-            float f[8], u[8];
-            if (EPI == GEMM_EPI_SWIGLU) {
-                const int j = gi * 8, c = j / half_rows;
-                const int gcol = c * p.nchunk + (j - c * half_rows);
-                uint32_t w[8];
-                tmem_ld_8cols(taddr + gcol, v);
-                tmem_ld_8cols(taddr + gcol + half_rows, w);
-                tmem_ld_wait();
-#pragma unroll
-                for (int k = 0; k < 8; ++k) u[k] = __uint_as_float(w[k]);
-            } else {
-                tmem_ld_8cols(taddr + gi * 8, v);
-                tmem_ld_wait();
-#pragma unroll
-                for (int k = 0; k < 8; ++k) u[k] = 0.f;
-            }
-#pragma unroll
-            for (int k = 0; k < 8; ++k) f[k] = __uint_as_float(v[k]);
-            if (p.splits > 1) {
-                // first half of K + second half of K, in that order in both pairs
-                const float4* q = reinterpret_cast<const float4*>(tiles + ((static_cast<size_t>(gi) * GM + row_local) << 5));
-                const float4 a = q[0], c = q[1];
-                const float o[8] = {a.x, a.y, a.z, a.w, c.x, c.y, c.z, c.w};
-#pragma unroll
-                for (int k = 0; k < 8; ++k) f[k] = split == 0 ? f[k] + o[k] : o[k] + f[k];
-            }
-            const int col = col_base + gi * 8;
-            if (row_ok && col < g.N) store_group<EPI>(f, u, g.out, g.res, row_off + col);
-        }
+        // this warp has read its part of the buffer: tell the even CTA's MMA warp
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(&bars->tmem_empty[acc], static_cast<uint32_t>(rank4 & ~1));
     }
 
-    // teardown: neither CTA may leave while its partner can still signal its barriers or read its tiles
+    // teardown: no CTA may leave while a partner can still signal its barriers or read its tiles
     tc_fence_before_sync();
     cluster_sync_all();
     if (*abort_flag) {
@@ -539,7 +596,10 @@ int launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap&
     if (cudaFuncSetAttribute(gemm_pair_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_BYTES) !=
         cudaSuccess)
         return DARE_ERR_CUDA;
-    const long long ctas = 2LL * g.p.splits * g.p.m_pairs * g.p.n_tiles;
+    // one cluster per tile with a K split; otherwise as many clusters as the device holds, each walking the tiles
+    long long clusters = static_cast<long long>(g.p.m_pairs) * g.p.n_tiles;
+    if (g.p.splits == 1 && !max_clusters_query && clusters > g.p.resident) clusters = g.p.resident;
+    const long long ctas = 2LL * g.p.splits * clusters;
     if (ctas > 0x7fffffffLL) return DARE_ERR_SHAPE;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(ctas), 1, 1);
@@ -568,6 +628,7 @@ int max_active_pairs(int splits = 1) {
         PairArgs g{};
         g.p.m_pairs = g.p.n_tiles = 1;
         g.p.splits = splits;
+        g.p.resident = 1;
         CUtensorMap dummy{};
         int n = 0;
         if (launch_pair<GEMM_EPI_STORE>(dummy, dummy, dummy, g, nullptr, &n) != DARE_OK) n = 0;
@@ -616,9 +677,8 @@ PairPlan pair_plan(int epi, int M, int N, int K, double* cost_out) {
                     best_cost = cost;
                     best.bn = bn; best.wcols = wcols; best.nmma = nmma; best.nchunk = nchunk; best.stages = stages;
                     best.splits = splits; best.m_pairs = m_pairs; best.n_tiles = n_tiles;
-                    uint32_t cols = 32;
-                    while (cols < static_cast<uint32_t>(bn)) cols <<= 1;
-                    best.tmem_cols = cols;
+                    best.resident = resident;
+                    best.tmem_cols = 512;       // two buffers of up to 256 columns, or one of up to 512
                 }
             }
         }
