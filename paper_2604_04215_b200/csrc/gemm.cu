@@ -328,6 +328,71 @@ struct PairArgs {
     uint32_t* dev_status;
 };
 
+// 4 x 4 transpose of 16-byte pieces inside every group of four lanes.  In: v[q] = piece q of this lane's row.
+// Out: v[i] = piece (lane % 4) of the row of lane (lane & ~3) + i.  Its own inverse.  All lanes take part.
+__device__ __forceinline__ void quad_transpose(uint4 (&v)[4], int lane) {
+#pragma unroll
+    for (int m = 1; m <= 2; m <<= 1) {
+        const bool hi = (lane & m) != 0;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            if (q & m) continue;
+            const uint4 send = hi ? v[q] : v[q ^ m];
+            uint4 recv;
+            recv.x = __shfl_xor_sync(0xffffffffu, send.x, m);
+            recv.y = __shfl_xor_sync(0xffffffffu, send.y, m);
+            recv.z = __shfl_xor_sync(0xffffffffu, send.z, m);
+            recv.w = __shfl_xor_sync(0xffffffffu, send.w, m);
+            if (hi) v[q] = recv; else v[q ^ m] = recv;
+        }
+    }
+}
+
+// Stores 32 consecutive output columns of the 32 rows a warp owns (lane = row, f = this row's values; SwiGLU
+// already applied).  The values are rounded to bf16, transposed among each four lanes and written so that one
+// store instruction covers 8 rows x 64 contiguous bytes instead of 32 rows x 16 bytes; the residual, if any, is
+// read the same way and transposed back before the add.  row0 = the warp's first row; all lanes must call.
+template <int EPI>
+__device__ __forceinline__ void store_chunk32(float (&f)[32], int lane, int row0, int n_rows_total, int col0, int n_cols_total,
+                                              int ldo, __nv_bfloat16* out, const __nv_bfloat16* res) {
+    const int my_col = col0 + (lane & 3) * 8;             // after the transpose: this lane's 8 columns ...
+    const int my_row0 = row0 + (lane & ~3);               // ... of rows my_row0 + i, i = 0..3
+    const bool col_ok = my_col < n_cols_total;            // (columns come in whole groups of 8)
+    if (EPI == GEMM_EPI_RESIDUAL) {
+        uint4 r[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int row = my_row0 + i;
+            r[i] = (col_ok && row < n_rows_total)
+                       ? *reinterpret_cast<const uint4*>(res + static_cast<size_t>(row) * ldo + my_col)
+                       : make_uint4(0u, 0u, 0u, 0u);
+        }
+        quad_transpose(r, lane);                           // back to lane = row: r[q] = columns 8q .. 8q+7 of my row
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            f[q * 8 + 0] += bf16_lo(r[q].x); f[q * 8 + 1] += bf16_hi(r[q].x);
+            f[q * 8 + 2] += bf16_lo(r[q].y); f[q * 8 + 3] += bf16_hi(r[q].y);
+            f[q * 8 + 4] += bf16_lo(r[q].z); f[q * 8 + 5] += bf16_hi(r[q].z);
+            f[q * 8 + 6] += bf16_lo(r[q].w); f[q * 8 + 7] += bf16_hi(r[q].w);
+        }
+    }
+    uint4 o[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        o[q].x = pack_bf16(f[q * 8 + 0], f[q * 8 + 1]);
+        o[q].y = pack_bf16(f[q * 8 + 2], f[q * 8 + 3]);
+        o[q].z = pack_bf16(f[q * 8 + 4], f[q * 8 + 5]);
+        o[q].w = pack_bf16(f[q * 8 + 6], f[q * 8 + 7]);
+    }
+    quad_transpose(o, lane);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int row = my_row0 + i;
+        if (col_ok && row < n_rows_total)
+            *reinterpret_cast<uint4*>(out + static_cast<size_t>(row) * ldo + my_col) = o[i];
+    }
+}
+
 struct PairBarriers {
     uint64_t full[MAX_STAGES];
     uint64_t empty[MAX_STAGES];
@@ -515,23 +580,40 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         }
         if (!epi_warp) continue;
         const bool live = epi_ok && !*abort_flag;
-        // Without a K split and without the SwiGLU pairing a thread takes 32 accumulator columns per load (one wait
-        // per 64 output bytes); the last n_groups % 4 groups, and the other cases, go 8 columns at a time.
+        // Without a K split the output goes 32 columns at a time through store_chunk32 (coalesced stores); the
+        // last n_groups % 4 groups, and the K-split case, go 8 columns at a time with one 16-byte store per lane.
         int g_begin = set;
-        if (EPI != GEMM_EPI_SWIGLU && p.splits == 1 && live) {
+        if (p.splits == 1) {             // (warp-uniform: store_chunk32 shuffles)
             const int n_chunks = n_groups / 4;
+            const int warp_row0 = m_pair * 2 * GM + rank * GM + lq * 32;
             for (int ci = set; ci < n_chunks; ci += 2) {
-                uint32_t v[32];
-                tmem_ld_32cols(taddr + ci * 32, v);
-                tmem_ld_wait();
+                float f[32];
+                if (EPI == GEMM_EPI_SWIGLU) {
+                    uint32_t vg[32], vu[32];
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    float f[8], u[8];
+                    for (int q = 0; q < 4; ++q) {          // each group of 8 output columns has its gate and up columns
+                        const int j = (ci * 4 + q) * 8, c = j / half_rows;
+                        const int gcol = c * p.nchunk + (j - c * half_rows);
+                        uint32_t a8[8], b8[8];
+                        tmem_ld_8cols(taddr + gcol, a8);
+                        tmem_ld_8cols(taddr + gcol + half_rows, b8);
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) { f[k] = __uint_as_float(v[q * 8 + k]); u[k] = 0.f; }
-                    const int col = col_base + ci * 32 + q * 8;
-                    if (row_ok && col < g.N) store_group<EPI>(f, u, g.out, g.res, row_off + col);
+                        for (int k = 0; k < 8; ++k) { vg[q * 8 + k] = a8[k]; vu[q * 8 + k] = b8[k]; }
+                    }
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int k = 0; k < 32; ++k) {
+                        const float gte = __uint_as_float(vg[k]);
+                        f[k] = __fdividef(gte, 1.0f + __expf(-gte)) * __uint_as_float(vu[k]);   // silu(g) * u
+                    }
+                } else {
+                    uint32_t v[32];
+                    tmem_ld_32cols(taddr + ci * 32, v);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int k = 0; k < 32; ++k) f[k] = __uint_as_float(v[k]);
                 }
+                if (live) store_chunk32<EPI>(f, lane, warp_row0, g.M, col_base + ci * 32, g.N, g.ldo, g.out, g.res);
             }
             g_begin = n_chunks * 4 + set;
         }
