@@ -52,7 +52,9 @@ def close_bf16(got, ref, steps=1.0, floor=1e-3):
                                    (512, 4096, 12288),     # two row tiles per CTA, 176-column tiles
                                    (500, 12288, 4096),     # K split three ways, ragged last row tile
                                    (512, 4096, 4096),      # K split two ways
-                                   (1100, 512, 1000)])     # many row items, odd number of row tiles
+                                   (1100, 512, 1000),      # many row items, odd number of row tiles
+                                   (5000, 320, 1536),      # more tiles than resident CTA pairs: each pair walks several
+                                   (9000, 128, 512)])      # ... with two accumulator buffers in turn, short K
 def test_linear_store_and_residual(ctx, M, K, N):
     a = I.normal_bf16(1, I.TID_X, (M, K))
     w = I.normal_bf16(1, I.TID_W, (N, K), 0.05)
@@ -72,7 +74,8 @@ def test_linear_store_and_residual(ctx, M, K, N):
     assert ctx.device_status() == 0
 
 
-@pytest.mark.parametrize("M,K,F", [(200, 256, 392), (512, 512, 1024), (32, 128, 128), (512, 4096, 12288)])
+@pytest.mark.parametrize("M,K,F", [(200, 256, 392), (512, 512, 1024), (32, 128, 128), (512, 4096, 12288),
+                                   (6000, 256, 1024)])     # several tiles per CTA pair
 def test_linear_swiglu(ctx, M, K, F):
     a = I.normal_bf16(2, I.TID_X, (M, K))
     wg = I.normal_bf16(2, I.TID_W, (F, K), 0.1)
