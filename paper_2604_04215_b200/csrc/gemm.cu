@@ -403,18 +403,6 @@ struct PairBarriers {
 };
 constexpr int PAIR_EPI_WARPS = 8;
 
-// Arrive on the mbarrier at this CTA's shared-memory address `bar` in CTA `rank` of the cluster.
-__device__ __forceinline__ void mbar_arrive_cluster(uint64_t* bar, uint32_t rank) {
-    asm volatile(
-        "{\n"
-        ".reg .b32 remote;\n"
-        "mapa.shared::cluster.u32 remote, %0, %1;\n"
-        "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [remote];\n"
-        "}\n" ::"r"(smem_u32(bar)),
-        "r"(rank)
-        : "memory");
-}
-
 // Persistent: cluster c computes tiles c, c + #clusters, ... (row index fastest).  The copies run ahead into the
 // next tile, and with bn <= 256 two accumulator buffers alternate, so a tile's epilogue overlaps the next tile's
 // main loop.  With a K split every cluster has exactly one tile (the exchange needs the idle ring).

@@ -16,6 +16,7 @@
 // partials of a row into (token, confidence) and scatters them to the row's original position.
 #include <math.h>
 #include <mutex>
+#include <type_traits>
 
 #include "internal.h"
 #include "ptx.cuh"
@@ -44,6 +45,21 @@ struct LmBarriers {
     uint32_t abort_flag;
 };
 constexpr int LM_SMEM_BYTES = STAGES * STAGE_BYTES + static_cast<int>(sizeof(LmBarriers)) + 1024;
+// CTA-pair mode (cta_group::2): two CTAs of a cluster take two row tiles against the same W tiles with MMAs of
+// M = 256; each CTA loads its own X tile and only half of the W tile, which takes a third off the shared-memory
+// traffic per flop that limits the single-CTA mode (tensor pipe 83 % -> 93 % busy in the projections).
+constexpr int PSTAGES = 6;
+constexpr int PB_BYTES = (BN / 2) * BK * 2;
+constexpr int PSTAGE_BYTES = A_BYTES + PB_BYTES;
+struct LmPairBarriers {
+    uint64_t full[PSTAGES];
+    uint64_t empty[PSTAGES];
+    uint64_t tmem_full[2];
+    uint64_t tmem_empty[2];
+    uint32_t tmem_base;
+    uint32_t abort_flag;
+};
+constexpr int LM_PAIR_SMEM_BYTES = PSTAGES * PSTAGE_BYTES + static_cast<int>(sizeof(LmPairBarriers)) + 1024;
 
 // Number of vocabulary groups for a grid of `grid` CTAs and `m_tiles` row tiles (same formula on the host,
 // in the GEMM and in the merge kernel).
@@ -52,6 +68,16 @@ __host__ __device__ inline int lm_groups(int grid, int m_tiles, int n_tiles) {
     if (g < 1) g = 1;
     if (g > n_tiles) g = n_tiles;
     return g;
+}
+
+// Pairs pay when the row tiles come in twos (an odd tile would drag an empty partner along).  The row count is
+// only known on the device, so both kernels are launched and the one whose mode does not apply returns at once.
+__host__ __device__ inline bool lm_pair_mode(int m_tiles, int allow_pair) {
+    return allow_pair && m_tiles >= 2 && (m_tiles & 1) == 0;
+}
+// Vocabulary groups in the mode that applies: pairs count as one CTA and two row tiles as one.
+__host__ __device__ inline int lm_groups_mode(int grid, int m_tiles, int n_tiles, int allow_pair) {
+    return lm_pair_mode(m_tiles, allow_pair) ? lm_groups(grid / 2, m_tiles / 2, n_tiles) : lm_groups(grid, m_tiles, n_tiles);
 }
 
 __device__ __forceinline__ int32_t row_token(const int32_t* row_tokens, int tok_L, int64_t tok_row_stride, int m) {
@@ -143,48 +169,58 @@ __device__ __forceinline__ float gumbel_from_word(uint32_t w) {
 // bf16 in both orientations (the two products of the backward pass take it from there); no partials.
 constexpr int LM_GREEDY = 0, LM_SAMPLE = 1, LM_LOGPROB = 2, LM_GRAD = 3;
 
-template <int MODE>
+template <int MODE, bool PAIR>
 __global__ void __launch_bounds__(LM_THREADS, 1)
 lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                       int M, const int32_t* __restrict__ live_rows, int D, int V, int mask_col, int n_tiles,
                       float* __restrict__ part_max, float* __restrict__ part_sum, int32_t* __restrict__ part_arg,
-                      uint32_t* __restrict__ dev_status, const LmSampling smp) {
+                      uint32_t* __restrict__ dev_status, const LmSampling smp, int allow_pair) {
+    constexpr int NSTAGES = PAIR ? PSTAGES : STAGES;
+    constexpr int STAGE_SZ = PAIR ? PSTAGE_BYTES : STAGE_BYTES;
+    using Barriers = typename std::conditional<PAIR, LmPairBarriers, LmBarriers>::type;
     constexpr bool SAMPLE = MODE == LM_SAMPLE;
     constexpr bool LOGPROB = MODE == LM_LOGPROB;
     constexpr bool GRAD = MODE == LM_GRAD;
     const int Mc = live_rows ? *live_rows : M;          // rows that need logits (uniform over the grid)
     const int m_tiles = (Mc + BM - 1) / BM;
     if (m_tiles == 0) return;
-    const int groups = lm_groups(gridDim.x, m_tiles, n_tiles);
-    const int n_items = m_tiles * groups;
-    if (static_cast<int>(blockIdx.x) >= n_items) return;
+    if (lm_pair_mode(m_tiles, allow_pair) != PAIR) return;        // the other kernel does this launch's work
+    // PAIR: a work unit is a cluster of two CTAs, an item two row tiles (one per CTA) and a vocabulary group
+    const int rank = PAIR ? static_cast<int>(cluster_cta_rank()) : 0;
+    const int unit = PAIR ? blockIdx.x >> 1 : blockIdx.x;
+    const int n_units = PAIR ? gridDim.x >> 1 : gridDim.x;
+    const int item_rows = PAIR ? m_tiles >> 1 : m_tiles;             // row tiles (pairs of them) to walk
+    const int groups = lm_groups(n_units, item_rows, n_tiles);
+    const int n_items = item_rows * groups;
+    if (unit >= n_items) return;                                    // (both CTAs of a pair alike)
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    LmBarriers* bars = reinterpret_cast<LmBarriers*>(tiles + STAGES * STAGE_BYTES);
+    Barriers* bars = reinterpret_cast<Barriers*>(tiles + NSTAGES * STAGE_SZ);
     volatile uint32_t* abort_flag = &bars->abort_flag;
 
     const int warp = warp_index_uniform();
     const int lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) {
+        for (int s = 0; s < NSTAGES; ++s) {
             mbar_init(&bars->full[s], 1);
             mbar_init(&bars->empty[s], 1);
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(&bars->tmem_full[a], 1);
-            mbar_init(&bars->tmem_empty[a], 128);
+            mbar_init(&bars->tmem_empty[a], PAIR ? 8 : 128);   // PAIR: one arrival per epilogue warp of both CTAs
         }
         bars->abort_flag = 0;
         fence_barrier_init();
     }
     if (warp == 1) {
-        tmem_alloc(&bars->tmem_base, TMEM_COLS);
-        tmem_relinquish();
+        if (PAIR) { tmem_alloc_pair(&bars->tmem_base, TMEM_COLS); tmem_relinquish_pair(); }
+        else { tmem_alloc(&bars->tmem_base, TMEM_COLS); tmem_relinquish(); }
     }
     tc_fence_before_sync();
-    __syncthreads();
+    if (PAIR) cluster_sync_all();     // both CTAs' barriers exist before either signals the other's
+    else __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = bars->tmem_base;
     const int num_k = (D + BK - 1) / BK;
@@ -197,31 +233,41 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-                const int m_tile = item % m_tiles;
-                for (int n_tile = item / m_tiles; n_tile < n_tiles && ok; n_tile += groups) {
+            // PAIR: the even CTA's "full" barriers count the bytes of both CTAs' copies
+            const uint32_t full0 = PAIR ? cluster_map_shared(smem_u32(&bars->full[0]), 0) : 0u;
+            for (int item = unit; item < n_items && ok; item += n_units) {
+                const int m_tile = PAIR ? 2 * (item % item_rows) + rank : item % item_rows;
+                for (int n_tile = item / item_rows; n_tile < n_tiles && ok; n_tile += groups) {
                     for (int kb = 0; kb < num_k; ++kb) {
                         if (!mbar_wait(&bars->empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
-                        uint8_t* a_dst = tiles + stage * STAGE_BYTES;
+                        uint8_t* a_dst = tiles + stage * STAGE_SZ;
                         uint8_t* b_dst = a_dst + A_BYTES;
-                        mbar_arrive_expect_tx(&bars->full[stage], STAGE_BYTES);
-                        tma_load_2d(a_dst, &tmap_x, &bars->full[stage], kb * BK, m_tile * BM);
-                        tma_load_2d(b_dst, &tmap_w, &bars->full[stage], kb * BK, n_tile * BN);
-                        if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                        if (PAIR) {
+                            const uint32_t full = full0 + stage * static_cast<uint32_t>(sizeof(uint64_t));
+                            if (rank == 0) mbar_arrive_expect_tx(&bars->full[stage], 2 * STAGE_SZ);
+                            tma_load_2d_pair(a_dst, &tmap_x, full, kb * BK, m_tile * BM);
+                            tma_load_2d_pair(b_dst, &tmap_w, full, kb * BK, n_tile * BN + rank * (BN / 2));
+                        } else {
+                            mbar_arrive_expect_tx(&bars->full[stage], STAGE_SZ);
+                            tma_load_2d(a_dst, &tmap_x, &bars->full[stage], kb * BK, m_tile * BM);
+                            tma_load_2d(b_dst, &tmap_w, &bars->full[stage], kb * BK, n_tile * BN);
+                        }
+                        if (++stage == NSTAGES) { stage = 0; phase ^= 1; }
                     }
                 }
             }
         }
-    } else if (warp == 1) {
-        // all lanes run the loops, one elected lane issues the MMAs and their commits
+    } else if (warp == 1 && rank == 0) {
+        // all lanes run the loops, one elected lane issues the MMAs and their commits (PAIR: the even CTA issues
+        // for both, and the commits arrive on both CTAs' barriers)
         const bool leader = elect_one_sync();
-        constexpr uint32_t idesc = umma_idesc_bf16(BM, BN);
+        constexpr uint32_t idesc = umma_idesc_bf16(PAIR ? 2 * BM : BM, BN);
         int stage = 0;
         uint32_t phase = 0;
         int it = 0;
         bool ok = true;
-        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-            for (int n_tile = item / m_tiles; n_tile < n_tiles && ok; n_tile += groups, ++it) {
+        for (int item = unit; item < n_items && ok; item += n_units) {
+            for (int n_tile = item / item_rows; n_tile < n_tiles && ok; n_tile += groups, ++it) {
                 const int acc = it & 1;
                 const uint32_t acc_phase = (it >> 1) & 1;
                 ok = __all_sync(0xffffffffu, mbar_wait(&bars->tmem_empty[acc], acc_phase ^ 1, abort_flag));
@@ -232,7 +278,7 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
                     ok = __all_sync(0xffffffffu, mbar_wait(&bars->full[stage], phase, abort_flag));
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const uint32_t a_addr = smem_u32(tiles + stage * STAGE_BYTES);
+                    const uint32_t a_addr = smem_u32(tiles + stage * STAGE_SZ);
                     const uint64_t a_desc = umma_desc_sw128_kmajor(a_addr);
                     const uint64_t b_desc = umma_desc_sw128_kmajor(a_addr + A_BYTES);
                     if (leader) {
@@ -240,26 +286,32 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
                         for (int kk = 0; kk < BK / 16; ++kk) {
                             // 16 bf16 = 32 bytes further along K inside the 128-byte swizzled row: +2 in the
                             // descriptor's 16-byte address units
-                            umma_bf16(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0);
+                            if (PAIR) umma_bf16_pair(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0);
+                            else umma_bf16(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0);
                         }
-                        umma_commit(&bars->empty[stage]);   // frees the stage when these MMAs have read it
+                        // frees the stage when these MMAs have read it
+                        if (PAIR) umma_commit_pair(&bars->empty[stage], 3);
+                        else umma_commit(&bars->empty[stage]);
                     }
                     __syncwarp();
-                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                    if (++stage == NSTAGES) { stage = 0; phase ^= 1; }
                 }
-                if (ok && leader) umma_commit(&bars->tmem_full[acc]);
+                if (ok && leader) {
+                    if (PAIR) umma_commit_pair(&bars->tmem_full[acc], 3);
+                    else umma_commit(&bars->tmem_full[acc]);
+                }
                 __syncwarp();
             }
         }
-    } else {
+    } else if (warp >= 2) {
         // epilogue: warp w may touch TMEM lanes [32 * (w % 4), +32)
         const int lq = warp & 3;
         const int row_in_tile = lq * 32 + lane;
         int it = 0;
         bool ok = true;
-        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-            const int m_tile = item % m_tiles;
-            const int group = item / m_tiles;
+        for (int item = unit; item < n_items && ok; item += n_units) {
+            const int m_tile = PAIR ? 2 * (item % item_rows) + rank : item % item_rows;
+            const int group = item / item_rows;
             float run_max = -INFINITY;
             float run_sum = 0.f;
             int run_arg = ARG_NONE;
@@ -286,7 +338,9 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
             for (int n_tile = group; n_tile < n_tiles && ok; n_tile += groups, ++it) {
                 const int acc = it & 1;
                 const uint32_t acc_phase = (it >> 1) & 1;
-                if (!mbar_wait(&bars->tmem_full[acc], acc_phase, abort_flag)) { ok = false; break; }
+                ok = mbar_wait(&bars->tmem_full[acc], acc_phase, abort_flag);
+                if (PAIR) ok = __all_sync(0xffffffffu, ok);      // the warp arrives as one further down
+                if (!ok) break;
                 tc_fence_after_sync();
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(lq * 32) << 16) + acc * BN;
                 const int col0 = n_tile * BN;
@@ -378,7 +432,12 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
                     }
                 }
                 tc_fence_before_sync();
-                mbar_arrive(&bars->tmem_empty[acc]);
+                if (PAIR) {           // one arrival per warp, on the even CTA's barrier
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(&bars->tmem_empty[acc], 0);
+                } else {
+                    mbar_arrive(&bars->tmem_empty[acc]);
+                }
             }
             const int row = m_tile * BM + row_in_tile;
             if (!GRAD && ok && row < Mc) {
@@ -391,9 +450,10 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
         }
     }
 
-    // teardown
+    // teardown (PAIR: neither CTA leaves while its partner can still signal its barriers or read its tiles)
     tc_fence_before_sync();
-    __syncthreads();
+    if (PAIR) cluster_sync_all();
+    else __syncthreads();
     if (*abort_flag) {
         // give copies still in flight time to land before the shared memory is released
         const long long t0 = clock64();
@@ -403,7 +463,8 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     }
     if (warp == 1) {
         tc_fence_after_sync();
-        tmem_dealloc(tmem_base, TMEM_COLS);
+        if (PAIR) tmem_dealloc_pair(tmem_base, TMEM_COLS);
+        else tmem_dealloc(tmem_base, TMEM_COLS);
     }
 }
 
@@ -412,12 +473,12 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
 __global__ void lmhead_merge_kernel(const float* __restrict__ part_max, const float* __restrict__ part_sum,
                                     const int32_t* __restrict__ part_arg, int grid_gemm, int n_tiles, int M,
                                     const int32_t* __restrict__ live_rows, const int32_t* __restrict__ idx,
-                                    int32_t* __restrict__ pred, float* __restrict__ conf) {
+                                    int32_t* __restrict__ pred, float* __restrict__ conf, int allow_pair) {
     const int c = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     const int Mc = live_rows ? *live_rows : M;
     if (c >= Mc) return;
-    const int groups = lm_groups(grid_gemm, (Mc + BM - 1) / BM, n_tiles);
+    const int groups = lm_groups_mode(grid_gemm, (Mc + BM - 1) / BM, n_tiles, allow_pair);
     float m = -INFINITY, s = 0.f;
     int a = ARG_NONE;
     const size_t base = static_cast<size_t>(c) * groups;
@@ -453,12 +514,12 @@ __global__ void lmhead_merge_sample_kernel(const float* __restrict__ part_max, c
                                            const int32_t* __restrict__ part_arg, const float* __restrict__ part_y,
                                            const float* __restrict__ part_zb, int grid_gemm, int n_tiles, int M,
                                            const int32_t* __restrict__ live_rows, const int32_t* __restrict__ idx,
-                                           int32_t* __restrict__ pred, float* __restrict__ conf) {
+                                           int32_t* __restrict__ pred, float* __restrict__ conf, int allow_pair) {
     const int c = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     const int Mc = live_rows ? *live_rows : M;
     if (c >= Mc) return;
-    const int groups = lm_groups(grid_gemm, (Mc + BM - 1) / BM, n_tiles);
+    const int groups = lm_groups_mode(grid_gemm, (Mc + BM - 1) / BM, n_tiles, allow_pair);
     float m = -INFINITY, s = 0.f, y = -INFINITY, zb = -INFINITY;
     int a = ARG_NONE;
     const size_t base = static_cast<size_t>(c) * groups;
@@ -496,11 +557,11 @@ __global__ void lmhead_merge_sample_kernel(const float* __restrict__ part_max, c
 // partial (the others carry -inf).  Optionally also writes logsumexp z.
 __global__ void lmhead_merge_logprob_kernel(const float* __restrict__ part_max, const float* __restrict__ part_sum,
                                             const int32_t* __restrict__ part_zt, int grid_gemm, int n_tiles, int M,
-                                            float* __restrict__ logprob, float* __restrict__ lse_out) {
+                                            float* __restrict__ logprob, float* __restrict__ lse_out, int allow_pair) {
     const int c = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (c >= M) return;
-    const int groups = lm_groups(grid_gemm, (M + BM - 1) / BM, n_tiles);
+    const int groups = lm_groups_mode(grid_gemm, (M + BM - 1) / BM, n_tiles, allow_pair);
     float m = -INFINITY, s = 0.f, zt = -INFINITY;
     const size_t base = static_cast<size_t>(c) * groups;
     for (int t = lane; t < groups; t += 32) {
@@ -528,6 +589,78 @@ __global__ void lmhead_merge_logprob_kernel(const float* __restrict__ part_max, 
 }
 
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Whether clusters of two CTAs of the pair-mode kernel can run on this device (asked once).
+int lm_pair_available() {
+    static int cache = -1;
+    if (cache < 0) {
+        int n = 0;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2048, 1, 1);
+        cfg.blockDim = dim3(LM_THREADS, 1, 1);
+        cfg.dynamicSmemBytes = LM_PAIR_SMEM_BYTES;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        if (cudaFuncSetAttribute(lmhead_partial_kernel<LM_GREEDY, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 LM_PAIR_SMEM_BYTES) != cudaSuccess ||
+            cudaOccupancyMaxActiveClusters(&n, lmhead_partial_kernel<LM_GREEDY, true>, &cfg) != cudaSuccess)
+            n = 0;
+        cache = n > 0 ? 1 : 0;
+    }
+    return cache;
+}
+
+// The GEMM part of a head: the single-CTA kernel, the CTA-pair kernel, or (when the row count is only known on
+// the device) both, of which the one whose mode does not apply returns at once.  *allow_pair_out tells the
+// merge kernel which rule was in force.
+template <int MODE>
+int launch_partial(const dare_ctx* ctx, int grid, const CUtensorMap& tmap_x, const void* w, int M,
+                   const int32_t* live_rows, int D, int V, int mask_col, int n_tiles, float* part_max, float* part_sum,
+                   int32_t* part_arg, const LmSampling& smp, cudaStream_t stream, int* allow_pair_out) {
+    const int allow_pair = (grid >= 2 && lm_pair_available()) ? 1 : 0;
+    *allow_pair_out = allow_pair;
+    const int m_tiles_host = (M + BM - 1) / BM;
+    const bool pair_known = live_rows == nullptr && lm_pair_mode(m_tiles_host, allow_pair);
+    const bool run_single = !allow_pair || live_rows != nullptr || !pair_known;
+    const bool run_pair = allow_pair && (live_rows != nullptr || pair_known);
+    if (run_single) {
+        CUtensorMap tmap_w;
+        int rc = make_tmap_bf16_2d(ctx, &tmap_w, w, static_cast<uint64_t>(V), static_cast<uint64_t>(D), BN, BK);
+        if (rc != DARE_OK) return rc;
+        if (cudaFuncSetAttribute(lmhead_partial_kernel<MODE, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 LM_SMEM_BYTES) != cudaSuccess)
+            return DARE_ERR_CUDA;
+        lmhead_partial_kernel<MODE, false><<<grid, LM_THREADS, LM_SMEM_BYTES, stream>>>(
+            tmap_x, tmap_w, M, live_rows, D, V, mask_col, n_tiles, part_max, part_sum, part_arg, ctx->dev_status, smp,
+            allow_pair);
+        if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
+    }
+    if (run_pair) {
+        CUtensorMap tmap_wh;      // half a W tile per CTA
+        int rc = make_tmap_bf16_2d(ctx, &tmap_wh, w, static_cast<uint64_t>(V), static_cast<uint64_t>(D), BN / 2, BK);
+        if (rc != DARE_OK) return rc;
+        if (cudaFuncSetAttribute(lmhead_partial_kernel<MODE, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 LM_PAIR_SMEM_BYTES) != cudaSuccess)
+            return DARE_ERR_CUDA;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(static_cast<unsigned>(grid & ~1), 1, 1);
+        cfg.blockDim = dim3(LM_THREADS, 1, 1);
+        cfg.dynamicSmemBytes = LM_PAIR_SMEM_BYTES;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, lmhead_partial_kernel<MODE, true>, tmap_x, tmap_wh, M, live_rows, D, V, mask_col,
+                               n_tiles, part_max, part_sum, part_arg, ctx->dev_status, smp, allow_pair) != cudaSuccess)
+            return DARE_ERR_CUDA;
+    }
+    return DARE_OK;
+}
 
 }  // namespace
 
@@ -573,24 +706,20 @@ int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M,
     float* part_sum = part_max + n_part;
     int32_t* part_arg = reinterpret_cast<int32_t*>(part_sum + n_part);
 
-    CUtensorMap tmap_x, tmap_w;
+    CUtensorMap tmap_x;
     int rc = make_tmap_bf16_2d(ctx, &tmap_x, x_gemm, static_cast<uint64_t>(M), static_cast<uint64_t>(D), BM, BK);
-    if (rc != DARE_OK) return rc;
-    rc = make_tmap_bf16_2d(ctx, &tmap_w, w, static_cast<uint64_t>(V), static_cast<uint64_t>(D), BN, BK);
     if (rc != DARE_OK) return rc;
 
     const int mask_col = (exclude_mask_column && mask_id >= 0 && mask_id < V) ? mask_id : -1;
     const int rows_per_block = 8;
     LmSampling smp = {};
+    int allow_pair = 0;
     if (sample == nullptr) {
-        if (cudaFuncSetAttribute(lmhead_partial_kernel<LM_GREEDY>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 LM_SMEM_BYTES) != cudaSuccess)
-            return DARE_ERR_CUDA;
-        lmhead_partial_kernel<LM_GREEDY><<<grid, LM_THREADS, LM_SMEM_BYTES, stream>>>(
-            tmap_x, tmap_w, M, live_rows, D, V, mask_col, n_tiles, part_max, part_sum, part_arg, ctx->dev_status, smp);
-        if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
+        rc = launch_partial<LM_GREEDY>(ctx, grid, tmap_x, w, M, live_rows, D, V, mask_col, n_tiles, part_max, part_sum,
+                                       part_arg, smp, stream, &allow_pair);
+        if (rc != DARE_OK) return rc;
         lmhead_merge_kernel<<<(M + rows_per_block - 1) / rows_per_block, rows_per_block * 32, 0, stream>>>(
-            part_max, part_sum, part_arg, grid, n_tiles, M, live_rows, idx, pred, conf);
+            part_max, part_sum, part_arg, grid, n_tiles, M, live_rows, idx, pred, conf, allow_pair);
     } else {
         smp.inv_temperature = 1.0f / sample->temperature;
         smp.seed_lo = static_cast<uint32_t>(sample->seed & 0xffffffffu);
@@ -599,14 +728,12 @@ int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M,
         smp.row_index = idx;
         smp.part_y = reinterpret_cast<float*>(part_arg + n_part);
         smp.part_zb = smp.part_y + n_part;
-        if (cudaFuncSetAttribute(lmhead_partial_kernel<LM_SAMPLE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 LM_SMEM_BYTES) != cudaSuccess)
-            return DARE_ERR_CUDA;
-        lmhead_partial_kernel<LM_SAMPLE><<<grid, LM_THREADS, LM_SMEM_BYTES, stream>>>(
-            tmap_x, tmap_w, M, live_rows, D, V, mask_col, n_tiles, part_max, part_sum, part_arg, ctx->dev_status, smp);
-        if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
+        rc = launch_partial<LM_SAMPLE>(ctx, grid, tmap_x, w, M, live_rows, D, V, mask_col, n_tiles, part_max, part_sum,
+                                       part_arg, smp, stream, &allow_pair);
+        if (rc != DARE_OK) return rc;
         lmhead_merge_sample_kernel<<<(M + rows_per_block - 1) / rows_per_block, rows_per_block * 32, 0, stream>>>(
-            part_max, part_sum, part_arg, smp.part_y, smp.part_zb, grid, n_tiles, M, live_rows, idx, pred, conf);
+            part_max, part_sum, part_arg, smp.part_y, smp.part_zb, grid, n_tiles, M, live_rows, idx, pred, conf,
+            allow_pair);
     }
     if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
     return DARE_OK;
@@ -625,23 +752,19 @@ int launch_lmhead_logprob(const dare_ctx* ctx, void* scratch, const void* hidden
     float* part_max = static_cast<float*>(scratch);
     float* part_sum = part_max + n_part;
     int32_t* part_zt = reinterpret_cast<int32_t*>(part_sum + n_part);
-    CUtensorMap tmap_x, tmap_w;
+    CUtensorMap tmap_x;
     int rc = make_tmap_bf16_2d(ctx, &tmap_x, hidden, static_cast<uint64_t>(M), static_cast<uint64_t>(D), BM, BK);
     if (rc != DARE_OK) return rc;
-    rc = make_tmap_bf16_2d(ctx, &tmap_w, w, static_cast<uint64_t>(V), static_cast<uint64_t>(D), BN, BK);
-    if (rc != DARE_OK) return rc;
-    if (cudaFuncSetAttribute(lmhead_partial_kernel<LM_LOGPROB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             LM_SMEM_BYTES) != cudaSuccess)
-        return DARE_ERR_CUDA;
     const int mask_col = (exclude_mask_column && mask_id >= 0 && mask_id < V) ? mask_id : -1;
     LmSampling smp = {};
     smp.targets = targets;
-    lmhead_partial_kernel<LM_LOGPROB><<<grid, LM_THREADS, LM_SMEM_BYTES, stream>>>(
-        tmap_x, tmap_w, M, nullptr, D, V, mask_col, n_tiles, part_max, part_sum, part_zt, ctx->dev_status, smp);
-    if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
+    int allow_pair = 0;
+    rc = launch_partial<LM_LOGPROB>(ctx, grid, tmap_x, w, M, nullptr, D, V, mask_col, n_tiles, part_max, part_sum, part_zt,
+                                    smp, stream, &allow_pair);
+    if (rc != DARE_OK) return rc;
     const int rows_per_block = 8;
     lmhead_merge_logprob_kernel<<<(M + rows_per_block - 1) / rows_per_block, rows_per_block * 32, 0, stream>>>(
-        part_max, part_sum, part_zt, grid, n_tiles, M, logprob, lse_out);
+        part_max, part_sum, part_zt, grid, n_tiles, M, logprob, lse_out, allow_pair);
     return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
 }
 
@@ -654,14 +777,9 @@ int launch_lmhead_grad(const dare_ctx* ctx, const void* hidden, int M, int D, co
     const int m_tiles_max = (M + BM - 1) / BM;
     int grid = ctx->sm_count;
     if (grid > m_tiles_max * n_tiles) grid = m_tiles_max * n_tiles;
-    CUtensorMap tmap_x, tmap_w;
+    CUtensorMap tmap_x;
     int rc = make_tmap_bf16_2d(ctx, &tmap_x, hidden, static_cast<uint64_t>(M), static_cast<uint64_t>(D), BM, BK);
     if (rc != DARE_OK) return rc;
-    rc = make_tmap_bf16_2d(ctx, &tmap_w, w, static_cast<uint64_t>(V), static_cast<uint64_t>(D), BN, BK);
-    if (rc != DARE_OK) return rc;
-    if (cudaFuncSetAttribute(lmhead_partial_kernel<LM_GRAD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             LM_SMEM_BYTES) != cudaSuccess)
-        return DARE_ERR_CUDA;
     const int mask_col = (exclude_mask_column && mask_id >= 0 && mask_id < V) ? mask_id : -1;
     LmSampling smp = {};
     smp.targets = targets;
@@ -670,9 +788,9 @@ int launch_lmhead_grad(const dare_ctx* ctx, const void* hidden, int M, int D, co
     smp.dz = static_cast<__nv_bfloat16*>(dz);
     smp.dzt = static_cast<__nv_bfloat16*>(dzt);
     smp.ldm = ldm;
-    lmhead_partial_kernel<LM_GRAD><<<grid, LM_THREADS, LM_SMEM_BYTES, stream>>>(
-        tmap_x, tmap_w, M, nullptr, D, V, mask_col, n_tiles, nullptr, nullptr, nullptr, ctx->dev_status, smp);
-    return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
+    int allow_pair = 0;
+    return launch_partial<LM_GRAD>(ctx, grid, tmap_x, w, M, nullptr, D, V, mask_col, n_tiles, nullptr, nullptr, nullptr, smp,
+                                   stream, &allow_pair);
 }
 
 }  // namespace dare
