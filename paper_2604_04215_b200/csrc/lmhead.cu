@@ -6,6 +6,8 @@
 //   warps 2..5  epilogue: each thread owns one row (one TMEM lane), streams the 256 logits of the tile
 //               through registers and keeps (running max, sum of exp, argmax); no cross-thread traffic
 // The two accumulators let the epilogue of tile i overlap the MMAs of tile i+1.
+// A second instantiation runs the same roles on CTA pairs (cta_group::2, MMAs of 256 rows, half a W tile per CTA);
+// see lm_pair_mode below for when it is the one that works.
 //
 // Only rows that are still masked need logits.  A first small kernel compacts those rows of X into a dense
 // buffer (and answers the committed rows directly); the GEMM reads the number of live rows from device
