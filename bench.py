@@ -342,8 +342,9 @@ def run_ours(args):
                           "l2": "inputs larger than L2 (W 1.04 GB and KV cache 0.2 GB are re-read every step)",
                           "parallelism": f"dp{world} (independent rollouts per GPU, no collective)"},
                "clocks": clocks, "e2e": e2e, # per step: attention, row compaction, the LM-head GEMM in its two instantiations (single CTAs and CTA
-               # pairs: the one whose mode does not apply to the step's row count returns at once), merge, selection
-               "gpu_launches": (attn_launches + 5) * args.steps,
+               # pairs: the one whose mode does not apply to the step's row count returns at once), and the merge
+               # kernel, which also does the selection for blocks of at most 32 positions
+               "gpu_launches": (attn_launches + (4 if L <= 32 else 5)) * args.steps,
                "roofline": roofline, "breakdown": breakdown, "cpu_baseline": cpu_baseline}
         print(json.dumps(out))
     ctx.close()
@@ -495,8 +496,8 @@ def run_model(args):
         per_fwd = 2 + 8 * mw.n_layers                   # embedding, final norm, 8 launches per layer
         # per generation: the prefill (prefix cache) or one refresh per block (dual cache), then per block its steps
         # plus the trailing one, each a forward + LM head (4 kernels: compaction, the GEMM in its two
-        # instantiations, merge) + selection
-        launches = n_gen * ((G // L if dual else 1) * per_fwd + (steps_taken // n_gen + G // L) * (per_fwd + 5))
+        # instantiations, merge with the selection folded in for L <= 32, else a fifth kernel)
+        launches = n_gen * ((G // L if dual else 1) * per_fwd + (steps_taken // n_gen + G // L) * (per_fwd + (4 if L <= 32 else 5)))
         out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps_taken, "warmup": args.warmup,
                "ms_per_step": ms_max / max(steps_taken, 1), "higher_is_better": True, "scaling": "weak",
                "vs_baseline": None, "dtype": "bf16", "data": "synthetic",

@@ -236,6 +236,11 @@ int dare_denoise_block(dare_ctx* ctx, int B, int L, int Hq, int Hkv, int d, int 
     if (rc != DARE_OK) return rc;
     // The LM head reads each row's current token straight from the token state: row m = (r, i) lives at
     // tokens[r * row_stride + block_start + i].
+    if (L <= dare::LMHEAD_SELECT_MAX_L) {      // short blocks: the selection rides on the head's merge kernel
+        const dare::LmSelectArgs sel = {tokens + block_start, B, mode, threshold, k, n_committed, n_remaining};
+        return dare::launch_lmhead(ctx, ctx->workspace, hidden, M, D, w, V, tokens + block_start, L, row_stride, mask_id,
+                                   exclude_mask_column, pred, conf, s, nullptr, &sel);
+    }
     rc = dare::launch_lmhead(ctx, ctx->workspace, hidden, M, D, w, V, tokens + block_start, L, row_stride, mask_id,
                              exclude_mask_column, pred, conf, s, nullptr);
     if (rc != DARE_OK) return rc;

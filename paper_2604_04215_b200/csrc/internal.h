@@ -40,9 +40,14 @@ int launch_lmhead_logprob(const dare_ctx* ctx, void* scratch, const void* hidden
 struct LmSampleArgs { float temperature; uint64_t seed; uint32_t step; };
 size_t lmhead_workspace_bytes(int M, int D, int V, int sm_count, bool with_row_tokens, bool sampling);
 // Token of LM-head row m (to skip committed rows) = row_tokens[(m / tok_L) * tok_row_stride + m % tok_L].
+// Unmask selection folded into the head's last kernel (greedy head on a block of at most LMHEAD_SELECT_MAX_L
+// positions whose tokens are given by row_tokens = tokens + block_start, tok_L = L): the caller then skips
+// launch_unmask_select.  tokens_block is the same address as row_tokens, writable.
+constexpr int LMHEAD_SELECT_MAX_L = 32;
+struct LmSelectArgs { int32_t* tokens_block; int B; int mode; float threshold; int k; int32_t* n_committed; int32_t* n_remaining; };
 int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M, int D, const void* w, int V,
                   const int32_t* row_tokens, int tok_L, int64_t tok_row_stride, int32_t mask_id, int exclude_mask_column, int32_t* pred, float* conf,
-                  cudaStream_t stream, const LmSampleArgs* sample);
+                  cudaStream_t stream, const LmSampleArgs* sample, const LmSelectArgs* select = nullptr);
 
 struct AttnArgs {
     int B, L, Hq, Hkv, d, prefix_cap, suffix_cap;

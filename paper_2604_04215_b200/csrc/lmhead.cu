@@ -470,20 +470,13 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     }
 }
 
-// One warp per live row: fold the row's partial triples (one per vocabulary group) into (token, confidence)
-// and write them at the row's original position.
-__global__ void lmhead_merge_kernel(const float* __restrict__ part_max, const float* __restrict__ part_sum,
-                                    const int32_t* __restrict__ part_arg, int grid_gemm, int n_tiles, int M,
-                                    const int32_t* __restrict__ live_rows, const int32_t* __restrict__ idx,
-                                    int32_t* __restrict__ pred, float* __restrict__ conf, int allow_pair) {
-    const int c = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    const int Mc = live_rows ? *live_rows : M;
-    if (c >= Mc) return;
-    const int groups = lm_groups_mode(grid_gemm, (Mc + BM - 1) / BM, n_tiles, allow_pair);
+// Fold of one row's partial triples by a warp: returns (argmax token, sum of exp relative to the maximum) in all
+// lanes.  Ties of the maximum go to the lowest token id.
+__device__ __forceinline__ void merge_row_partials(const float* __restrict__ part_max, const float* __restrict__ part_sum,
+                                                   const int32_t* __restrict__ part_arg, size_t base, int groups, int lane,
+                                                   int& a_out, float& s_out) {
     float m = -INFINITY, s = 0.f;
     int a = ARG_NONE;
-    const size_t base = static_cast<size_t>(c) * groups;
     for (int t = lane; t < groups; t += 32) {
         const float m2 = part_max[base + t];
         const float s2 = part_sum[base + t];
@@ -503,10 +496,114 @@ __global__ void lmhead_merge_kernel(const float* __restrict__ part_max, const fl
             else { s += s2 * exp2f((m2 - m) * LOG2E); if (m2 == m && a2 < a) a = a2; }
         }
     }
+    a_out = a;
+    s_out = s;
+}
+
+// One warp per live row: fold the row's partial triples (one per vocabulary group) into (token, confidence)
+// and write them at the row's original position.
+__global__ void lmhead_merge_kernel(const float* __restrict__ part_max, const float* __restrict__ part_sum,
+                                    const int32_t* __restrict__ part_arg, int grid_gemm, int n_tiles, int M,
+                                    const int32_t* __restrict__ live_rows, const int32_t* __restrict__ idx,
+                                    int32_t* __restrict__ pred, float* __restrict__ conf, int allow_pair) {
+    const int c = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    const int Mc = live_rows ? *live_rows : M;
+    if (c >= Mc) return;
+    const int groups = lm_groups_mode(grid_gemm, (Mc + BM - 1) / BM, n_tiles, allow_pair);
+    int a;
+    float s;
+    merge_row_partials(part_max, part_sum, part_arg, static_cast<size_t>(c) * groups, groups, lane, a, s);
     if (lane == 0) {
         const int row = idx ? idx[c] : c;
         pred[row] = a;
         conf[row] = 1.0f / s;   // exp(max - logsumexp) with the sum taken relative to the max
+    }
+}
+
+// Merge and unmask selection in one kernel, for blocks of at most 32 positions: one CTA per rollout, one warp per
+// block position.  A warp whose position is still masked finds its row's place among the compacted rows (from the
+// compaction kernel's sorted row list: other CTAs change the token state meanwhile), folds the row's partials and writes
+// (pred, conf); then the CTA applies the selection rule of select.cu to the block: rank by counting, bit for bit
+// the same decisions as the separate kernel takes from the same (pred, conf).
+struct LmSelect {
+    int32_t* tokens_block;      // tokens + block_start (row b at + b * row_stride)
+    int64_t row_stride;
+    int mode;
+    float threshold;
+    int k;
+    int32_t* n_committed;
+    int32_t* n_remaining;
+};
+__global__ void __launch_bounds__(1024)
+lmhead_merge_select_kernel(const float* __restrict__ part_max, const float* __restrict__ part_sum,
+                           const int32_t* __restrict__ part_arg, int grid_gemm, int n_tiles, int L,
+                           const int32_t* __restrict__ live_rows, const int32_t* __restrict__ idx, int32_t mask_id,
+                           int32_t* __restrict__ pred, float* __restrict__ conf, int allow_pair, const LmSelect sel) {
+    __shared__ int s_before;
+    __shared__ int s_flag[32];
+    __shared__ float s_conf[32];
+    __shared__ int32_t s_pred[32];
+    const int b = blockIdx.x;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;      // warp = block position (blockDim = 32 L)
+    const int Mc = *live_rows;
+    if (threadIdx.x == 0) {
+        // compacted rows that belong to earlier rollouts = first entry of the ascending row list that is >= b * L
+        int lo = 0, hi = Mc;
+        while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if (idx[mid] < b * L) lo = mid + 1; else hi = mid;
+        }
+        s_before = lo;
+    }
+    int32_t* row = sel.tokens_block + static_cast<int64_t>(b) * sel.row_stride;
+    const bool masked = row[warp] == mask_id;
+    if (lane == 0) s_flag[warp] = masked ? 1 : 0;
+    __syncthreads();
+    if (masked) {
+        int c = s_before;
+        for (int i = 0; i < warp; ++i) c += s_flag[i];
+        const int groups = lm_groups_mode(grid_gemm, (Mc + BM - 1) / BM, n_tiles, allow_pair);
+        int a;
+        float s;
+        merge_row_partials(part_max, part_sum, part_arg, static_cast<size_t>(c) * groups, groups, lane, a, s);
+        if (lane == 0) {
+            float cf = 1.0f / s;
+            pred[b * L + warp] = a;
+            conf[b * L + warp] = cf;
+            if (cf != cf) cf = -INFINITY;
+            s_conf[warp] = cf;
+            s_pred[warp] = a;
+        }
+    } else if (lane == 0) {
+        s_conf[warp] = __int_as_float(0x7fc00000);      // absent
+    }
+    __syncthreads();
+    if (warp != 0) return;
+    // selection (warp 0, lane = block position)
+    const float cf = lane < L ? s_conf[lane] : __int_as_float(0x7fc00000);
+    const bool is_masked = cf == cf;
+    const unsigned masked_set = __ballot_sync(0xffffffffu, is_masked);
+    const unsigned above_set = __ballot_sync(0xffffffffu, is_masked && cf > sel.threshold);
+    bool commit = false;
+    if (is_masked) {
+        if (sel.mode == DARE_SELECT_THRESHOLD && above_set != 0u) {
+            commit = cf > sel.threshold;
+        } else {
+            const int want = sel.mode == DARE_SELECT_TOPK ? sel.k : 1;
+            int rank = 0;
+            for (int j = 0; j < L; ++j) {
+                const float cj = s_conf[j];
+                rank += (cj > cf || (cj == cf && j < lane)) ? 1 : 0;   // NaN (absent) compares false
+            }
+            commit = rank < want;
+        }
+    }
+    if (commit) row[lane] = s_pred[lane];
+    const unsigned commit_set = __ballot_sync(0xffffffffu, commit);
+    if (lane == 0) {
+        if (sel.n_committed) sel.n_committed[b] = __popc(commit_set);
+        if (sel.n_remaining) sel.n_remaining[b] = __popc(masked_set) - __popc(commit_set);
     }
 }
 
@@ -679,7 +776,10 @@ size_t lmhead_workspace_bytes(int M, int D, int V, int sm_count, bool with_row_t
 
 int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M, int D, const void* w, int V,
                   const int32_t* row_tokens, int tok_L, int64_t tok_row_stride, int32_t mask_id,
-                  int exclude_mask_column, int32_t* pred, float* conf, cudaStream_t stream, const LmSampleArgs* sample) {
+                  int exclude_mask_column, int32_t* pred, float* conf, cudaStream_t stream, const LmSampleArgs* sample,
+                  const LmSelectArgs* select) {
+    if (select && (sample || !row_tokens || tok_L > LMHEAD_SELECT_MAX_L || tok_L < 1 || M != select->B * tok_L))
+        return DARE_ERR_SHAPE;
     const int n_tiles = (V + BN - 1) / BN;
     const int m_tiles_max = (M + BM - 1) / BM;
     int grid = ctx->sm_count;
@@ -720,8 +820,18 @@ int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M,
         rc = launch_partial<LM_GREEDY>(ctx, grid, tmap_x, w, M, live_rows, D, V, mask_col, n_tiles, part_max, part_sum,
                                        part_arg, smp, stream, &allow_pair);
         if (rc != DARE_OK) return rc;
-        lmhead_merge_kernel<<<(M + rows_per_block - 1) / rows_per_block, rows_per_block * 32, 0, stream>>>(
-            part_max, part_sum, part_arg, grid, n_tiles, M, live_rows, idx, pred, conf, allow_pair);
+        if (select) {
+            LmSelect sel;
+            sel.tokens_block = select->tokens_block; sel.row_stride = tok_row_stride; sel.mode = select->mode;
+            sel.threshold = select->threshold; sel.k = select->k;
+            sel.n_committed = select->n_committed; sel.n_remaining = select->n_remaining;
+            lmhead_merge_select_kernel<<<select->B, 32 * tok_L, 0, stream>>>(part_max, part_sum, part_arg, grid, n_tiles,
+                                                                             tok_L, live_rows, idx, mask_id, pred, conf,
+                                                                             allow_pair, sel);
+        } else {
+            lmhead_merge_kernel<<<(M + rows_per_block - 1) / rows_per_block, rows_per_block * 32, 0, stream>>>(
+                part_max, part_sum, part_arg, grid, n_tiles, M, live_rows, idx, pred, conf, allow_pair);
+        }
     } else {
         smp.inv_temperature = 1.0f / sample->temperature;
         smp.seed_lo = static_cast<uint32_t>(sample->seed & 0xffffffffu);

@@ -98,6 +98,11 @@ int step_rows(dare_model* m, int32_t* tokens, int B, int64_t row_stride, int sta
     int rc = forward_rows(m, tokens, B, row_stride, start, L, kv_len, k_cache, v_cache, cap, nullptr, s);
     if (rc != DARE_OK) return rc;
     const int M = B * L;
+    if (L <= dare::LMHEAD_SELECT_MAX_L) {      // short blocks: the selection rides on the head's merge kernel
+        const dare::LmSelectArgs sel = {tokens + start, B, mode, threshold, k, n_committed, n_remaining};
+        return dare::launch_lmhead(m->ctx, m->ctx->workspace, m->h, M, m->desc.hidden, m->lm_head, m->desc.vocab,
+                                   tokens + start, L, row_stride, m->desc.mask_id, 1, pred, conf, s, nullptr, &sel);
+    }
     rc = dare::launch_lmhead(m->ctx, m->ctx->workspace, m->h, M, m->desc.hidden, m->lm_head, m->desc.vocab,
                              tokens + start, L, row_stride, m->desc.mask_id, 1, pred, conf, s, nullptr);
     if (rc != DARE_OK) return rc;
