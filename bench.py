@@ -280,13 +280,16 @@ def run_ours(args):
 
     # ---- end to end: the step's activations come from pinned host memory, results go back to the host
     n_e2e = min(args.steps, 4 * steps_per_gen)
-    # Double-buffered: a copy stream uploads step t + 1's activations while step t computes; every step still
-    # uploads its own inputs from pinned memory and the host reads the step's counts and tokens before going on.
+    # Double-buffered both ways: a copy stream uploads step t + 1's activations while step t computes, and the host
+    # reads step t's counts and tokens (copied to pinned memory right behind the step) while step t + 1 runs: the
+    # step does not depend on the host, so the host stays one step behind, as dare_generate does.  Every step still
+    # uploads its own inputs from pinned memory and every step's results are read on the host.
     bufs = [(torch.empty_like(pool[0][0]), torch.empty_like(pool[0][1])) for _ in range(2)]
-    nc_h = torch.zeros(B, dtype=torch.int32).pin_memory()
-    nr_h = torch.zeros(B, dtype=torch.int32).pin_memory()
-    tok_blk_h = torch.zeros(B, L, dtype=torch.int32).pin_memory()
-    nc_d = torch.zeros(B, dtype=torch.int32, device="cuda")
+    nc_h = [torch.zeros(B, dtype=torch.int32).pin_memory() for _ in range(2)]
+    nr_h = [torch.zeros(B, dtype=torch.int32).pin_memory() for _ in range(2)]
+    tok_blk_h = [torch.zeros(B, L, dtype=torch.int32).pin_memory() for _ in range(2)]
+    nc_d = [torch.zeros(B, dtype=torch.int32, device="cuda") for _ in range(2)]
+    read_back = [torch.cuda.Event(), torch.cuda.Event()]
     copy_stream = torch.cuda.Stream()
     uploaded = [torch.cuda.Event(), torch.cuda.Event()]
     consumed = [torch.cuda.Event(), torch.cuda.Event()]
@@ -309,15 +312,19 @@ def run_ours(args):
         if t + 1 < n_e2e:
             upload(t + 1)
         stream.wait_event(uploaded[t & 1])
-        step(t, bufs[t & 1][0], bufs[t & 1][1], nc_d)
+        step(t, bufs[t & 1][0], bufs[t & 1][1], nc_d[t & 1])
         consumed[t & 1].record(stream)
         g = t % steps_per_gen
         bs = wl.prompt_len + (g // steps_per_block) * L
-        nc_h.copy_(nc_d, non_blocking=True)
-        nr_h.copy_(nr, non_blocking=True)
-        tok_blk_h.copy_(tokens[:, bs:bs + L], non_blocking=True)
-        stream.synchronize()
-        e2e_tokens += int(nc_h.sum())
+        nc_h[t & 1].copy_(nc_d[t & 1], non_blocking=True)
+        nr_h[t & 1].copy_(nr, non_blocking=True)
+        tok_blk_h[t & 1].copy_(tokens[:, bs:bs + L], non_blocking=True)
+        read_back[t & 1].record(stream)
+        if t >= 1:
+            read_back[(t - 1) & 1].synchronize()
+            e2e_tokens += int(nc_h[(t - 1) & 1].sum())
+    read_back[(n_e2e - 1) & 1].synchronize()
+    e2e_tokens += int(nc_h[(n_e2e - 1) & 1].sum())
     torch.cuda.synchronize()
     tb = time.perf_counter()
     e2e_s, e2e_n = reduce_step_stats(tb - ta, e2e_tokens, device="cuda")
