@@ -106,6 +106,19 @@ def test_lmhead_without_exclusion_and_with_committed_rows(ctx):
     _lm_case(ctx, 130, 256, 1024, 1023, seed=6, with_rows=True)
 
 
+@pytest.mark.parametrize("M,D,V,mu,with_rows", [
+    (256, 320, 2600, 7, False),        # two row tiles known on the host: the CTA-pair kernel alone is launched
+    (500, 128, 1000, 999, False),      # four row tiles, ragged last one
+    (600, 256, 2048, 5, True),         # 200 masked rows = two tiles, known only on the device: pairs do the work
+    (1400, 64, 1200, 3, True),         # 467 masked rows = four tiles
+    (900, 64, 1200, 3, True),          # 300 masked rows = three tiles: the single-CTA kernel does the work
+])
+def test_lmhead_single_and_pair_modes(ctx, M, D, V, mu, with_rows):
+    """The LM-head GEMM has a single-CTA and a CTA-pair instantiation; which one works depends on the number of
+    128-row tiles of masked rows (even: pairs), decided on the device when rows are skipped."""
+    _lm_case(ctx, M, D, V, mu, seed=M + D, with_rows=with_rows)
+
+
 def test_lmhead_tie_break_lowest_index_and_mask_column(ctx):
     """Identical weight rows: all admissible columns tie exactly; lowest admissible id wins, conf = 1/(V-1)."""
     M, D, V = 64, 128, 700
