@@ -10,7 +10,8 @@
  *     dare_lmhead_confidence  LM head + vocabulary softmax -> (argmax token, max probability) per row,
  *                             logits never written to memory
  *     dare_unmask_select      confidence-threshold / per-block top-k commit on the int32 token state
- *     dare_denoise_block      the three above, enqueued back to back
+ *     dare_denoise_block      the three above, enqueued back to back (dare_denoise_block_sampled: with the
+ *                             sampled head)
  *     dare_model_* / dare_generate   the same step with a stack of transformer layers in between, and the
  *                             whole block-by-block loop (dare_linear, dare_rmsnorm, dare_rope_kv_write: its parts)
  *     dare_model_*_window / dare_generate_dual   the same with a cached suffix behind the block (dual cache)
@@ -234,6 +235,21 @@ int dare_denoise_block(dare_ctx* ctx,
                        int mode, float threshold, int k,
                        int32_t* pred, float* conf,
                        int32_t* n_committed, int32_t* n_remaining, void* stream);
+
+/*
+ * The same step with the sampled head (Section 4.2: several different rollouts per prompt): dare_attn_block, then
+ * dare_lmhead_sample on the block's rows (temperature, seed and step counter as there), then dare_unmask_select on
+ * the sampled tokens and their temperature-1 probabilities.  Same buffers and rules as dare_denoise_block;
+ * temperature must be finite and > 0 (DARE_ERR_RANGE otherwise).
+ */
+int dare_denoise_block_sampled(dare_ctx* ctx, int B, int L, int Hq, int Hkv, int d, int prefix_cap, int suffix_cap,
+                               float scale, const void* q, const void* k_pre, const void* v_pre,
+                               const int32_t* prefix_len, const void* k_blk, const void* v_blk, const void* k_suf,
+                               const void* v_suf, const int32_t* suffix_len, void* attn_out, float* lse,
+                               const void* hidden, int D, const void* w, int V, int32_t mask_id,
+                               int exclude_mask_column, float temperature, uint64_t seed, uint32_t step,
+                               int32_t* tokens, int64_t row_stride, int block_start, int mode, float threshold, int k,
+                               int32_t* pred, float* conf, int32_t* n_committed, int32_t* n_remaining, void* stream);
 
 /*
  * ---------------------------------------------------------------------------------------------------------

@@ -21,7 +21,7 @@ DEV_LEN_CLAMPED = 1
 DEV_WAIT_EXPIRED = 2
 
 EXPORTS = ["dare_create", "dare_destroy", "dare_status_string", "dare_device_status", "dare_sm_count",
-           "dare_attn_block", "dare_attn_varlen", "dare_lmhead_confidence", "dare_unmask_select", "dare_denoise_block",
+           "dare_attn_block", "dare_attn_varlen", "dare_lmhead_confidence", "dare_unmask_select", "dare_denoise_block", "dare_denoise_block_sampled",
            "dare_lmhead_confidence_static", "dare_lmhead_sample", "dare_lmhead_logprob", "dare_lmhead_logprob_backward", "dare_transpose_bf16", "dare_forward_mask", "dare_masked_nelbo", "dare_model_create", "dare_model_destroy", "dare_model_forward",
            "dare_model_step", "dare_generate", "dare_model_forward_window", "dare_model_step_window", "dare_generate_dual",
            "dare_linear", "dare_linear_plan", "dare_rmsnorm", "dare_rope_kv_write"]
@@ -84,6 +84,10 @@ def load():
                                         vp, i64, i32, i32, f32, i32,             # tokens, stride, start, mode, thr, k
                                         vp, vp, vp, vp, vp])                     # pred, conf, n_comm, n_rem, stream
     lib.dare_denoise_block.restype = i32
+    lib.dare_denoise_block_sampled.argtypes = ([vp] + [i32] * 7 + [f32] + [vp] * 11 +
+                                               [vp, i32, vp, i32, i32, i32, f32, C.c_uint64, C.c_uint32,
+                                                vp, i64, i32, i32, f32, i32, vp, vp, vp, vp, vp])
+    lib.dare_denoise_block_sampled.restype = i32
     lib.dare_model_create.argtypes = [vp, C.POINTER(ModelDesc), vp, C.POINTER(LayerWeights), vp, C.POINTER(vp)]
     lib.dare_model_create.restype = i32
     lib.dare_model_destroy.argtypes = [vp]
@@ -374,6 +378,31 @@ def dare_denoise_block(ctx: Context, q, k_pre, v_pre, prefix_len, k_blk, v_blk, 
         _ptr(n_remaining, torch.int32), _stream(stream))
     if rc != 0 and check:
         raise DareError(rc, "dare_denoise_block")
+    return rc
+
+
+def dare_denoise_block_sampled(ctx: Context, q, k_pre, v_pre, prefix_len, k_blk, v_blk, k_suf, v_suf, suffix_len,
+                               attn_out, lse, hidden, w, mask_id: int, exclude_mask_column: bool, temperature: float,
+                               seed: int, step: int, tokens, block_start: int, mode: int, threshold: float, k: int,
+                               pred, conf, n_committed=None, n_remaining=None, scale: float = 0.0, stream=None,
+                               check: bool = True):
+    B, L, Hq, d = q.shape
+    Hkv, prefix_cap = k_pre.shape[1], k_pre.shape[2]
+    suffix_cap = k_suf.shape[2] if k_suf is not None else 0
+    D = hidden.shape[1]
+    V = w.shape[0]
+    bf = torch.bfloat16
+    rc = load().dare_denoise_block_sampled(
+        ctx.handle, B, L, Hq, Hkv, d, prefix_cap, suffix_cap, float(scale),
+        _ptr(q, bf), _ptr(k_pre, bf), _ptr(v_pre, bf), _ptr(prefix_len, torch.int32), _ptr(k_blk, bf), _ptr(v_blk, bf),
+        _ptr(k_suf, bf), _ptr(v_suf, bf), _ptr(suffix_len, torch.int32), _ptr(attn_out, bf), _ptr(lse, torch.float32),
+        _ptr(hidden, bf), D, _ptr(w, bf), V, int(mask_id), int(bool(exclude_mask_column)), float(temperature),
+        int(seed) & 0xFFFFFFFFFFFFFFFF, int(step) & 0xFFFFFFFF,
+        _ptr(tokens, torch.int32), tokens.shape[1], int(block_start), int(mode), float(threshold), int(k),
+        _ptr(pred, torch.int32), _ptr(conf, torch.float32), _ptr(n_committed, torch.int32),
+        _ptr(n_remaining, torch.int32), _stream(stream))
+    if rc != 0 and check:
+        raise DareError(rc, "dare_denoise_block_sampled")
     return rc
 
 

@@ -248,4 +248,37 @@ int dare_denoise_block(dare_ctx* ctx, int B, int L, int Hq, int Hkv, int d, int 
                                       n_committed, n_remaining, s);
 }
 
+// The step with the sampled head: as dare_denoise_block, the token of every masked row drawn by temperature +
+// Gumbel-max sampling (dare_lmhead_sample), its confidence the temperature-1 probability of that token.
+int dare_denoise_block_sampled(dare_ctx* ctx, int B, int L, int Hq, int Hkv, int d, int prefix_cap, int suffix_cap,
+                               float scale, const void* q, const void* k_pre, const void* v_pre,
+                               const int32_t* prefix_len, const void* k_blk, const void* v_blk, const void* k_suf,
+                               const void* v_suf, const int32_t* suffix_len, void* attn_out, float* lse,
+                               const void* hidden, int D, const void* w, int V, int32_t mask_id, int exclude_mask_column,
+                               float temperature, uint64_t seed, uint32_t step, int32_t* tokens, int64_t row_stride,
+                               int block_start, int mode, float threshold, int k, int32_t* pred, float* conf,
+                               int32_t* n_committed, int32_t* n_remaining, void* stream) {
+    dare::AttnArgs a;
+    int rc = check_attn(ctx, B, L, Hq, Hkv, d, prefix_cap, suffix_cap, scale, q, k_pre, v_pre, k_blk, v_blk, k_suf,
+                        v_suf, attn_out, &a);
+    if (rc != DARE_OK) return rc;
+    a.prefix_len = prefix_len; a.suffix_len = suffix_len; a.lse = lse;
+    if (static_cast<long long>(B) * L > 0x7fffffffLL) return DARE_ERR_SHAPE;
+    const int M = B * L;
+    rc = check_lmhead(ctx, hidden, M, D, w, V, true, pred, conf, true);
+    if (rc != DARE_OK) return rc;
+    if (!(temperature > 0.f) || isinf(temperature)) return DARE_ERR_RANGE;
+    rc = check_select(tokens, B, row_stride, block_start, L, pred, conf, mode, threshold, k);
+    if (rc != DARE_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    rc = dare::launch_attn(ctx, a, s);
+    if (rc != DARE_OK) return rc;
+    const dare::LmSampleArgs smp = {temperature, seed, step};
+    rc = dare::launch_lmhead(ctx, ctx->workspace, hidden, M, D, w, V, tokens + block_start, L, row_stride, mask_id,
+                             exclude_mask_column, pred, conf, s, &smp);
+    if (rc != DARE_OK) return rc;
+    return dare::launch_unmask_select(tokens, B, row_stride, block_start, L, pred, conf, mask_id, mode, threshold, k,
+                                      n_committed, n_remaining, s);
+}
+
 }  // extern "C"

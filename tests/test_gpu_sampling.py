@@ -178,3 +178,46 @@ def test_llada8b_full_size_sampled_rows(ctx):
     assert ((c_all[~done] > 0) & (c_all[~done] <= 1.0)).all()
     assert (p_all[~done] != wl.mask_id).all() and (p_all[~done] >= 0).all() and (p_all[~done] < wl.vocab).all()
     assert len(np.unique(p_all[~done])) > 0.9 * (~done).sum()          # high-entropy logits: almost all tokens differ
+
+
+def test_sampled_step_on_the_tiny_workload(ctx):
+    """dare_denoise_block_sampled over 6 iterations of config 1 (planted confidences, so that the threshold rule
+    commits varying numbers of tokens): attention and sampled head against the oracle from the GPU's pre-step state,
+    selection bit-exact from the GPU's own tokens and confidences."""
+    from _util import check_attn
+    wl = I.WORKLOADS["tiny"]
+    w = I.make_weights(wl)
+    caches = I.make_caches(wl)
+    wd, kp, vp = w.cuda(), caches[0].cuda(), caches[1].cuda()
+    tok_d = I.fresh_tokens(wl).cuda()
+    T, seed = 0.9, 0xC0FFEE1234
+    w64 = f64(w)
+    for it in range(6):
+        si = I.make_step(wl, step=it, planted=True, w=w, caches=caches)
+        pre = tok_d.cpu().numpy()
+        attn_out = torch.empty_like(si.q, device="cuda")
+        pred = torch.empty(wl.M, dtype=torch.int32, device="cuda")
+        conf = torch.empty(wl.M, dtype=torch.float32, device="cuda")
+        nc = torch.zeros(wl.batch, dtype=torch.int32, device="cuda")
+        nr = torch.zeros(wl.batch, dtype=torch.int32, device="cuda")
+        dare.dare_denoise_block_sampled(ctx, si.q.cuda(), kp, vp, si.prefix_len.cuda(), si.k_blk.cuda(), si.v_blk.cuda(),
+                                        None, None, None, attn_out, None, si.x.cuda(), wd, wl.mask_id, True, T, seed, it,
+                                        tok_d, si.block_start, wl.mode, wl.threshold, wl.k, pred, conf, nc, nr)
+        torch.cuda.synchronize()
+        assert ctx.device_status() == 0
+        ref = SO.denoise_step_sampled(f64(si.q), f64(si.k_pre), f64(si.v_pre), si.prefix_len.numpy(), f64(si.k_blk),
+                                      f64(si.v_blk), None, None, None, f64(si.x), w64, pre, si.block_start, wl.block_len,
+                                      wl.mask_id, wl.mode, wl.threshold, wl.k, T, seed, it)
+        check_attn(attn_out, ref["attn_out"])
+        rows = pre[:, si.block_start:si.block_start + wl.block_len].reshape(-1)
+        _check(pred, conf, ref["lm"], f64(si.x), w64, rows, wl.mask_id, True, T, seed, it)
+        want, wnc, wnr = O.unmask_select(pre, si.block_start, wl.block_len, pred.cpu().numpy(), conf.cpu().numpy(),
+                                         wl.mask_id, wl.mode, wl.threshold, wl.k)
+        np.testing.assert_array_equal(tok_d.cpu().numpy(), want)
+        np.testing.assert_array_equal(nc.cpu().numpy(), wnc)
+        np.testing.assert_array_equal(nr.cpu().numpy(), wnr)
+        assert wnc.min() >= 1 or (rows != wl.mask_id).all()
+    assert dare.dare_denoise_block_sampled(ctx, si.q.cuda(), kp, vp, si.prefix_len.cuda(), si.k_blk.cuda(),
+                                           si.v_blk.cuda(), None, None, None, attn_out, None, si.x.cuda(), wd, wl.mask_id,
+                                           True, 0.0, seed, 0, tok_d, si.block_start, wl.mode, wl.threshold, wl.k, pred,
+                                           conf, nc, nr, check=False) == -4
