@@ -34,6 +34,10 @@ constexpr int A_BYTES = BM * BK * 2;
 constexpr int B_BYTES = BN * BK * 2;
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int LM_THREADS = 192;
+// The sampling epilogue does several times the arithmetic of the greedy one per logit (a generator block and two
+// logarithms): it gets two sets of four epilogue warps that take alternate 32-column chunks of every tile.
+constexpr int LM_SAMPLE_THREADS = 320;
+__host__ __device__ constexpr int lm_threads(int mode) { return mode == 1 ? LM_SAMPLE_THREADS : LM_THREADS; }
 constexpr uint32_t TMEM_COLS = 512;
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr int ARG_NONE = 0x7fffffff;
@@ -43,6 +47,7 @@ struct LmBarriers {
     uint64_t empty[STAGES];
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
+    uint64_t exch_full, exch_empty;      // two epilogue sets: hand-over of the second set's running values
     uint32_t tmem_base;
     uint32_t abort_flag;
 };
@@ -58,6 +63,7 @@ struct LmPairBarriers {
     uint64_t empty[PSTAGES];
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
+    uint64_t exch_full, exch_empty;
     uint32_t tmem_base;
     uint32_t abort_flag;
 };
@@ -172,7 +178,7 @@ __device__ __forceinline__ float gumbel_from_word(uint32_t w) {
 constexpr int LM_GREEDY = 0, LM_SAMPLE = 1, LM_LOGPROB = 2, LM_GRAD = 3;
 
 template <int MODE, bool PAIR>
-__global__ void __launch_bounds__(LM_THREADS, 1)
+__global__ void __launch_bounds__(lm_threads(MODE), 1)
 lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                       int M, const int32_t* __restrict__ live_rows, int D, int V, int mask_col, int n_tiles,
                       float* __restrict__ part_max, float* __restrict__ part_sum, int32_t* __restrict__ part_arg,
@@ -183,6 +189,8 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     constexpr bool SAMPLE = MODE == LM_SAMPLE;
     constexpr bool LOGPROB = MODE == LM_LOGPROB;
     constexpr bool GRAD = MODE == LM_GRAD;
+    constexpr int EPI_SETS = SAMPLE ? 2 : 1;                 // sets of four epilogue warps
+    __shared__ float s_exch[5][BM];                          // (max, sum, best y, its logit, its column) per row
     const int Mc = live_rows ? *live_rows : M;          // rows that need logits (uniform over the grid)
     const int m_tiles = (Mc + BM - 1) / BM;
     if (m_tiles == 0) return;
@@ -211,8 +219,11 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(&bars->tmem_full[a], 1);
-            mbar_init(&bars->tmem_empty[a], PAIR ? 8 : 128);   // PAIR: one arrival per epilogue warp of both CTAs
+            // every epilogue thread arrives (PAIR: one arrival per epilogue warp of both CTAs)
+            mbar_init(&bars->tmem_empty[a], (PAIR ? 8 : 128) * EPI_SETS);
         }
+        mbar_init(&bars->exch_full, 128);
+        mbar_init(&bars->exch_empty, 128);
         bars->abort_flag = 0;
         fence_barrier_init();
     }
@@ -308,10 +319,12 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     } else if (warp >= 2) {
         // epilogue: warp w may touch TMEM lanes [32 * (w % 4), +32)
         const int lq = warp & 3;
+        const int set = (warp - 2) >> 2;
         const int row_in_tile = lq * 32 + lane;
         int it = 0;
+        int items_done = 0;
         bool ok = true;
-        for (int item = unit; item < n_items && ok; item += n_units) {
+        for (int item = unit; item < n_items && ok; item += n_units, ++items_done) {
             const int m_tile = PAIR ? 2 * (item % item_rows) + rank : item % item_rows;
             const int group = item / item_rows;
             float run_max = -INFINITY;
@@ -348,7 +361,7 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
                 const int col0 = n_tile * BN;
                 const bool edge = (col0 + BN > V) || (mask_col >= col0 && mask_col < col0 + BN);
 #pragma unroll 1
-                for (int c = 0; c < BN / 32; ++c) {
+                for (int c = set; c < BN / 32; c += EPI_SETS) {
                     uint32_t v[32];
                     tmem_ld_32cols(taddr + c * 32, v);
                     tmem_ld_wait();
@@ -441,8 +454,33 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
                     mbar_arrive(&bars->tmem_empty[acc]);
                 }
             }
+            if (EPI_SETS == 2 && ok) {
+                // the second set hands its running values to the first, which folds them into its own: the larger
+                // perturbed score wins, the lower column on a tie (each set saw its columns in ascending order)
+                const uint32_t par = items_done & 1;
+                if (set == 1) {
+                    ok = mbar_wait(&bars->exch_empty, par ^ 1, abort_flag);
+                    s_exch[0][row_in_tile] = run_max; s_exch[1][row_in_tile] = run_sum;
+                    s_exch[2][row_in_tile] = best_y; s_exch[3][row_in_tile] = best_z;
+                    s_exch[4][row_in_tile] = __int_as_float(run_arg);
+                    mbar_arrive(&bars->exch_full);          // (release: the values above are visible to the waiter)
+                } else {
+                    ok = mbar_wait(&bars->exch_full, par, abort_flag);
+                    if (ok) {
+                        const float m2 = s_exch[0][row_in_tile], s2 = s_exch[1][row_in_tile];
+                        const float y2 = s_exch[2][row_in_tile], z2 = s_exch[3][row_in_tile];
+                        const int a2 = __float_as_int(s_exch[4][row_in_tile]);
+                        mbar_arrive(&bars->exch_empty);
+                        if (m2 > -INFINITY) {
+                            if (m2 > run_max) { run_sum = run_sum * fast_exp2((run_max - m2) * LOG2E) + s2; run_max = m2; }
+                            else run_sum += s2 * fast_exp2((m2 - run_max) * LOG2E);
+                        }
+                        if (y2 > best_y || (y2 == best_y && a2 < run_arg)) { best_y = y2; best_z = z2; run_arg = a2; }
+                    }
+                }
+            }
             const int row = m_tile * BM + row_in_tile;
-            if (!GRAD && ok && row < Mc) {
+            if (!GRAD && ok && row < Mc && set == 0) {
                 const size_t o = static_cast<size_t>(row) * groups + group;
                 part_max[o] = run_max;
                 part_sum[o] = run_sum;
@@ -732,7 +770,7 @@ int launch_partial(const dare_ctx* ctx, int grid, const CUtensorMap& tmap_x, con
         if (cudaFuncSetAttribute(lmhead_partial_kernel<MODE, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  LM_SMEM_BYTES) != cudaSuccess)
             return DARE_ERR_CUDA;
-        lmhead_partial_kernel<MODE, false><<<grid, LM_THREADS, LM_SMEM_BYTES, stream>>>(
+        lmhead_partial_kernel<MODE, false><<<grid, lm_threads(MODE), LM_SMEM_BYTES, stream>>>(
             tmap_x, tmap_w, M, live_rows, D, V, mask_col, n_tiles, part_max, part_sum, part_arg, ctx->dev_status, smp,
             allow_pair);
         if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
@@ -746,7 +784,7 @@ int launch_partial(const dare_ctx* ctx, int grid, const CUtensorMap& tmap_x, con
             return DARE_ERR_CUDA;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(static_cast<unsigned>(grid & ~1), 1, 1);
-        cfg.blockDim = dim3(LM_THREADS, 1, 1);
+        cfg.blockDim = dim3(lm_threads(MODE), 1, 1);
         cfg.dynamicSmemBytes = LM_PAIR_SMEM_BYTES;
         cfg.stream = stream;
         cudaLaunchAttribute attr;
