@@ -439,6 +439,13 @@ def run_model(args):
         raise RuntimeError("the loop left masks behind or the device status word is non-zero")
     ms_max, committed_all = reduce_step_stats(ms, committed, device="cuda")
     value = committed_all / (ms_max * 1e-3)
+    if world > 1:
+        # the one exchange of the sharded job: every rank gets all rollouts' final tokens (outside the timed region;
+        # B * (P + G) int32 per rank)
+        from paper_2604_04215_b200.dist import gather_tokens
+        all_tok = gather_tokens(tok)
+        if all_tok.shape[0] != world * B or not bool((all_tok[:, P:] != mw.mask_id).all()):
+            raise RuntimeError("gathered tokens are incomplete")
 
     # ---- the projections of one layer at the step's row count, timed one by one for the roofline
     M = B * L
