@@ -282,3 +282,48 @@ def generate_dual(cfg, wts, tokens, prompt_len, gen_len, L, mode, threshold, k, 
             n += 1
         steps.append(n)
     return tok, steps, cache
+
+
+# ---------------------------------------------------------------------------------------------------------
+# The cached loop with the sampled head (RL rollouts draw several different responses per prompt, Section 4.2).
+
+STEP_BLOCK_SHIFT = 16      # generator step counter of step n of block b: (b << 16) + n
+
+
+def denoise_step_cached_sampled(cfg, wts, tokens, block_start, L, cache, mode, threshold, k, temperature, seed, step,
+                                rounded=True, kv_len=None):
+    """One step of the loop with temperature + Gumbel-max sampling in place of the argmax (see
+    dare_sampling_oracle.lmhead_sample): stack on the block's rows, sampled head on the still-masked rows (the
+    generator is keyed by the row's index b * L + i in the block's row list and by `step`), selection on the
+    sampled tokens' temperature-1 probabilities."""
+    from . import dare_sampling_oracle as SO
+    hidden = forward_block_cached(cfg, wts, tokens, block_start, L, cache, rounded, kv_len=kv_len)
+    B = tokens.shape[0]
+    row_tokens = np.asarray(tokens)[:, block_start:block_start + L].reshape(B * L)
+    lm = SO.lmhead_sample(hidden, wts.lm_head, row_tokens, cfg.mask_id, True, temperature, seed, step)
+    conf32 = lm["conf"].astype(np.float32)
+    tok, nc, nr = O.unmask_select(tokens, block_start, L, lm["pred"], conf32, cfg.mask_id, mode, threshold, k)
+    return {"hidden": hidden, "lm": lm, "tokens": tok, "n_committed": nc, "n_remaining": nr}
+
+
+def generate_sampled(cfg, wts, tokens, prompt_len, gen_len, L, mode, threshold, k, temperature, seed, rounded=True,
+                     on_step=None):
+    """`generate` with the sampled head; step n of block b uses the generator step counter (b << 16) + n."""
+    tok = np.array(tokens, dtype=np.int32, copy=True)
+    B = tok.shape[0]
+    cache = new_cache(cfg, B, prompt_len + gen_len)
+    forward_block_cached(cfg, wts, tok, 0, prompt_len, cache, rounded)
+    steps = []
+    for b in range(gen_len // L):
+        start = prompt_len + b * L
+        n = 0
+        while (tok[:, start:start + L] == cfg.mask_id).any():
+            res = denoise_step_cached_sampled(cfg, wts, tok, start, L, cache, mode, threshold, k, temperature, seed,
+                                              (b << STEP_BLOCK_SHIFT) + n, rounded)
+            if on_step is not None:
+                on_step(b, n, tok, res)
+            tok = res["tokens"]
+            n += 1
+        forward_block_cached(cfg, wts, tok, start, L, cache, rounded)   # K/V of the committed block
+        steps.append(n)
+    return tok, steps, cache

@@ -332,3 +332,38 @@ def test_dual_loop_counts_and_first_step_of_each_block():
     a = MO.generate_dual(cfg, wts, tok0, P, mw.gen_len, L, O.SELECT_TOPK, 0.9, 2)
     b = MO.generate_dual(cfg, wts, tok0, P, mw.gen_len, L, O.SELECT_TOPK, 0.9, 2)
     np.testing.assert_array_equal(a[0], b[0])
+
+
+# ---------------------------------------------------------------------------------------------------------
+# The loop with the sampled head
+
+def test_sampled_loop_limits_counts_and_determinism():
+    """T -> 0 gives the greedy loop's tokens; the same seed the same tokens, another seed others; every rollout
+    commits all G tokens under top-k in ceil(L / k) steps per block; steps of different blocks and different steps
+    of a block use different generator counters (identical hidden rows would otherwise repeat their draws)."""
+    mw = _small(batch=2)
+    cfg, wts = _cfg(mw), _weights(mw)
+    tok0 = I.fresh_model_tokens(mw).numpy()
+    P, G, L = mw.prompt_len, mw.gen_len, mw.block_len
+    greedy, gsteps, _ = MO.generate(cfg, wts, tok0, P, G, L, O.SELECT_TOPK, 0.9, 2, rounded=False)
+    cold, csteps, _ = MO.generate_sampled(cfg, wts, tok0, P, G, L, O.SELECT_TOPK, 0.9, 2, 1e-7, 5, rounded=False)
+    np.testing.assert_array_equal(cold, greedy)
+    assert csteps == gsteps == [2] * (G // L)
+    seen = []
+    a, _, _ = MO.generate_sampled(cfg, wts, tok0, P, G, L, O.SELECT_TOPK, 0.9, 2, 1.0, 5, rounded=False,
+                                  on_step=lambda b, n, t, r: seen.append((b, n)))
+    b_, _, _ = MO.generate_sampled(cfg, wts, tok0, P, G, L, O.SELECT_TOPK, 0.9, 2, 1.0, 5, rounded=False)
+    c, _, _ = MO.generate_sampled(cfg, wts, tok0, P, G, L, O.SELECT_TOPK, 0.9, 2, 1.0, 6, rounded=False)
+    np.testing.assert_array_equal(a, b_)
+    assert (a != c).any() and (a != greedy).any()
+    assert (a[:, P:] != cfg.mask_id).all() and (a[:, :P] == tok0[:, :P]).all()
+    assert seen == [(b, n) for b in range(G // L) for n in range(2)]
+    # the step counter reaches the generator: the same state sampled under two counters differs
+    cache = MO.new_cache(cfg, mw.batch, P + G)
+    MO.forward_block_cached(cfg, wts, tok0, 0, P, cache, False)
+    r1 = MO.denoise_step_cached_sampled(cfg, wts, tok0, P, L, [(k.copy(), v.copy()) for k, v in cache], O.SELECT_TOPK,
+                                        0.9, 2, 1.0, 5, (0 << 16) + 0, False)
+    r2 = MO.denoise_step_cached_sampled(cfg, wts, tok0, P, L, [(k.copy(), v.copy()) for k, v in cache], O.SELECT_TOPK,
+                                        0.9, 2, 1.0, 5, (1 << 16) + 0, False)
+    assert (r1["lm"]["pred"] != r2["lm"]["pred"]).any()
+    np.testing.assert_allclose(r1["hidden"], r2["hidden"], atol=0)
