@@ -393,6 +393,8 @@ def run_model(args):
     model = _model_objects(dare, ctx, mw, wts_h, max_rows=mw.batch * (mw.prompt_len + mw.gen_len) if dual else None)
     B, L, P, G = mw.batch, mw.block_len, mw.prompt_len, mw.gen_len
     loop = dare.dare_generate_dual if dual else dare.dare_generate
+    if args.temperature > 0:              # sampled rollouts (temperature + Gumbel-max) instead of the argmax
+        dare.dare_model_set_sampling(model, args.temperature, 1234 + rank, 0)
     tok0_h = I.fresh_model_tokens(mw_rank).pin_memory()
     tok0 = tok0_h.cuda()
     tok = tok0.clone()
@@ -517,7 +519,8 @@ def run_model(args):
                "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
                "config": {"workload": f"{mw.name}: {mw.n_layers} layers D{D} Hq{mw.n_q_heads}/Hkv{mw.n_kv_heads} "
                                       f"d{mw.head_dim} F{F} V{mw.vocab} B{B} prompt{P}+gen{G} L{L} tau {mw.threshold}, "
-                                      + ("dual cache (whole-sequence refresh per block)" if dual else "prefix cache"),
+                                      + ("dual cache (whole-sequence refresh per block)" if dual else "prefix cache")
+                                      + (f", sampled head T={args.temperature}" if args.temperature > 0 else ""),
                           "generations": n_gen, "ms_per_generation": ms_max / n_gen,
                           "l2": "inputs larger than L2 (2.8 GB of weights are re-read every step)",
                           "parallelism": f"dp{world} (independent rollouts per GPU, no collective)"},
@@ -631,6 +634,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llada8b", choices=sorted(I.WORKLOADS) + sorted(I.MODEL_WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--temperature", type=float, default=0.0,
+                    help="loop workloads: > 0 samples the tokens (temperature + Gumbel-max) instead of the argmax")
     ap.add_argument("--cache", default="prefix", choices=["prefix", "dual"],
                     help="loop workloads: prefix cache (block-causal) or dual cache (bidirectional, refresh per block)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (0 = as defined)")

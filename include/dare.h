@@ -376,6 +376,20 @@ int dare_lmhead_logprob_backward(dare_ctx* ctx, const void* hidden, int M, int D
 int dare_transpose_bf16(dare_ctx* ctx, const void* in, int rows, int cols, void* out, void* stream);
 
 /*
+ * Sampled head for the model calls (Section 4.2: several different rollouts per prompt).  After
+ * dare_model_set_sampling(model, temperature > 0, seed, first_step, stream), dare_model_step, dare_model_step_window,
+ * dare_generate and dare_generate_dual draw every masked row's token by temperature + Gumbel-max sampling
+ * (dare_lmhead_sample; confidence = temperature-1 probability of the drawn token) instead of taking the argmax.
+ * The generator's step counter lives on the device: the call sets it to first_step (enqueued on `stream`) and
+ * every step adds one, so consecutive dare_model_step calls use first_step, first_step + 1, ...; the loops set it to
+ * (block index << 16) at the start of each block, so step n of block b uses (b << 16) + n.  The generator's row
+ * index is the row's index b * L + i among the block's rows.  temperature = 0 switches back to the argmax (the
+ * default); negative, NaN or infinite values give DARE_ERR_RANGE.  The ctx workspace must cover the sampled head
+ * (5 instead of 3 floats per partial), else the step calls return DARE_ERR_WORKSPACE.
+ */
+int dare_model_set_sampling(dare_model* model, float temperature, uint64_t seed, uint32_t first_step, void* stream);
+
+/*
  * Dual cache (prefix and suffix) for a fully bidirectional masked model (Section 3.4, rollout with KV-cache
  * reuse): the rows [start, start + length) see cache[0 : kv_len) with kv_len >= start + length, i.e. also the
  * positions behind them, whose K/V are whatever an earlier forward left in the cache.

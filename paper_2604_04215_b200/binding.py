@@ -23,7 +23,7 @@ DEV_WAIT_EXPIRED = 2
 EXPORTS = ["dare_create", "dare_destroy", "dare_status_string", "dare_device_status", "dare_sm_count",
            "dare_attn_block", "dare_attn_varlen", "dare_lmhead_confidence", "dare_unmask_select", "dare_denoise_block", "dare_denoise_block_sampled",
            "dare_lmhead_confidence_static", "dare_lmhead_sample", "dare_lmhead_logprob", "dare_lmhead_logprob_backward", "dare_transpose_bf16", "dare_forward_mask", "dare_masked_nelbo", "dare_model_create", "dare_model_destroy", "dare_model_forward",
-           "dare_model_step", "dare_generate", "dare_model_forward_window", "dare_model_step_window", "dare_generate_dual",
+           "dare_model_step", "dare_generate", "dare_model_set_sampling", "dare_model_forward_window", "dare_model_step_window", "dare_generate_dual",
            "dare_linear", "dare_linear_plan", "dare_rmsnorm", "dare_rope_kv_write"]
 
 _lib = None
@@ -99,6 +99,8 @@ def load():
     lib.dare_generate.argtypes = [vp, vp, i32, i64, i32, i32, i32, vp, vp, i32, i32, f32, i32, vp, vp, vp,
                                   C.POINTER(C.c_int32), vp]
     lib.dare_generate.restype = i32
+    lib.dare_model_set_sampling.argtypes = [vp, f32, C.c_uint64, C.c_uint32, vp]
+    lib.dare_model_set_sampling.restype = i32
     lib.dare_model_forward_window.argtypes = [vp, vp, i32, i64, i32, i32, i32, vp, vp, i32, vp, vp]
     lib.dare_model_forward_window.restype = i32
     lib.dare_model_step_window.argtypes = [vp, vp, i32, i64, i32, i32, i32, vp, vp, i32, i32, f32, i32, vp, vp, vp, vp, vp]
@@ -569,3 +571,13 @@ def dare_generate_dual(model: Model, tokens, prompt_len: int, gen_len: int, L: i
     if rc != 0 and check:
         raise DareError(rc, "dare_generate_dual")
     return list(steps) if check else rc
+
+
+def dare_model_set_sampling(model: Model, temperature: float, seed: int = 0, first_step: int = 0, stream=None,
+                            check: bool = True):
+    """temperature > 0: the model's step and loop calls sample; 0: back to the argmax."""
+    rc = load().dare_model_set_sampling(model.handle, float(temperature), int(seed) & 0xFFFFFFFFFFFFFFFF,
+                                        int(first_step) & 0xFFFFFFFF, _stream(stream))
+    if rc != 0 and check:
+        raise DareError(rc, "dare_model_set_sampling")
+    return rc

@@ -37,7 +37,9 @@ int launch_lmhead_logprob(const dare_ctx* ctx, void* scratch, const void* hidden
                           const int32_t* targets, int32_t mask_id, int exclude_mask_column, float* logprob, float* lse_out,
                           cudaStream_t stream);
 // Sampling epilogue of the LM head (NULL = greedy): temperature, 64-bit seed and step counter of the generator.
-struct LmSampleArgs { float temperature; uint64_t seed; uint32_t step; };
+// step_dev (optional, device): added to `step`; the head's last kernel then increments it, so that a step replayed
+// from a CUDA graph draws fresh noise every time.
+struct LmSampleArgs { float temperature; uint64_t seed; uint32_t step; uint32_t* step_dev = nullptr; };
 size_t lmhead_workspace_bytes(int M, int D, int V, int sm_count, bool with_row_tokens, bool sampling);
 // Token of LM-head row m (to skip committed rows) = row_tokens[(m / tok_L) * tok_row_stride + m % tok_L].
 // Unmask selection folded into the head's last kernel (greedy head on a block of at most LMHEAD_SELECT_MAX_L

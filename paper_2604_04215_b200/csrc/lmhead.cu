@@ -142,6 +142,7 @@ lmhead_compact_kernel(const uint4* __restrict__ x, int M, int D8, const int32_t*
 struct LmSampling {
     float inv_temperature;
     uint32_t seed_lo, seed_hi, step;
+    const uint32_t* step_dev;      // optional device word added to `step`
     const int32_t* row_index;      // original row of compacted row c (NULL: identity): keys the generator
     const int32_t* targets;        // LM_LOGPROB: target token per row
     float* part_y;                 // per partial: best perturbed score and the raw logit there
@@ -331,8 +332,9 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
             float run_sum = 0.f;
             int run_arg = ARG_NONE;
             float best_y = -INFINITY, best_z = -INFINITY;       // SAMPLE: best perturbed score, raw logit there
-            uint32_t rng_row = 0;
+            uint32_t rng_row = 0, rng_step = 0;
             if (SAMPLE) {
+                rng_step = smp.step + (smp.step_dev ? *smp.step_dev : 0u);
                 const int row_c = m_tile * BM + row_in_tile;
                 rng_row = static_cast<uint32_t>(row_c < Mc && smp.row_index ? smp.row_index[row_c] : row_c);
             }
@@ -422,7 +424,7 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
                     if (SAMPLE) {
 #pragma unroll
                         for (int q = 0; q < 8; ++q) {
-                            const uint4 w4 = philox4x32_10(make_uint4(static_cast<uint32_t>(cbase >> 2) + q, rng_row, smp.step,
+                            const uint4 w4 = philox4x32_10(make_uint4(static_cast<uint32_t>(cbase >> 2) + q, rng_row, rng_step,
                                                                       0x44415245u), smp.seed_lo, smp.seed_hi);
                             const uint32_t ww[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
@@ -651,7 +653,9 @@ __global__ void lmhead_merge_sample_kernel(const float* __restrict__ part_max, c
                                            const int32_t* __restrict__ part_arg, const float* __restrict__ part_y,
                                            const float* __restrict__ part_zb, int grid_gemm, int n_tiles, int M,
                                            const int32_t* __restrict__ live_rows, const int32_t* __restrict__ idx,
-                                           int32_t* __restrict__ pred, float* __restrict__ conf, int allow_pair) {
+                                           int32_t* __restrict__ pred, float* __restrict__ conf, int allow_pair,
+                                           uint32_t* __restrict__ step_dev) {
+    if (step_dev && blockIdx.x == 0 && threadIdx.x == 0) *step_dev += 1;   // the GEMM kernels before this one read it
     const int c = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     const int Mc = live_rows ? *live_rows : M;
@@ -875,6 +879,7 @@ int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M,
         smp.seed_lo = static_cast<uint32_t>(sample->seed & 0xffffffffu);
         smp.seed_hi = static_cast<uint32_t>(sample->seed >> 32);
         smp.step = sample->step;
+        smp.step_dev = sample->step_dev;
         smp.row_index = idx;
         smp.part_y = reinterpret_cast<float*>(part_arg + n_part);
         smp.part_zb = smp.part_y + n_part;
@@ -883,7 +888,7 @@ int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M,
         if (rc != DARE_OK) return rc;
         lmhead_merge_sample_kernel<<<(M + rows_per_block - 1) / rows_per_block, rows_per_block * 32, 0, stream>>>(
             part_max, part_sum, part_arg, smp.part_y, smp.part_zb, grid, n_tiles, M, live_rows, idx, pred, conf,
-            allow_pair);
+            allow_pair, sample->step_dev);
     }
     if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
     return DARE_OK;

@@ -31,9 +31,15 @@ struct dare_model {
     cudaEvent_t ev[2];
     cudaStream_t work;             // the loop runs here: a block's step is captured once into a CUDA graph
     cudaEvent_t ev_in, ev_out;     // order the work stream after / before the caller's stream
+    // sampled head (dare_model_set_sampling): temperature 0 = greedy; the device word counts the steps
+    float sample_temperature;
+    uint64_t sample_seed;
+    uint32_t* step_counter;
 };
 
 namespace {
+
+__global__ void set_word_kernel(uint32_t* p, uint32_t v) { *p = v; }
 
 // Keys visible to the rows: cache[0, kv_len), start + length <= kv_len <= cap.
 int forward_rows(dare_model* m, const int32_t* tokens, int B, int64_t row_stride, int start, int length, int kv_len,
@@ -98,6 +104,15 @@ int step_rows(dare_model* m, int32_t* tokens, int B, int64_t row_stride, int sta
     int rc = forward_rows(m, tokens, B, row_stride, start, L, kv_len, k_cache, v_cache, cap, nullptr, s);
     if (rc != DARE_OK) return rc;
     const int M = B * L;
+    if (m->sample_temperature > 0.f) {          // sampled head, then the separate selection kernel
+        dare::LmSampleArgs smp;
+        smp.temperature = m->sample_temperature; smp.seed = m->sample_seed; smp.step = 0; smp.step_dev = m->step_counter;
+        rc = dare::launch_lmhead(m->ctx, m->ctx->workspace, m->h, M, m->desc.hidden, m->lm_head, m->desc.vocab,
+                                 tokens + start, L, row_stride, m->desc.mask_id, 1, pred, conf, s, &smp);
+        if (rc != DARE_OK) return rc;
+        return dare::launch_unmask_select(tokens, B, row_stride, start, L, pred, conf, m->desc.mask_id, mode, threshold,
+                                          k, n_committed, n_remaining, s);
+    }
     if (L <= dare::LMHEAD_SELECT_MAX_L) {      // short blocks: the selection rides on the head's merge kernel
         const dare::LmSelectArgs sel = {tokens + start, B, mode, threshold, k, n_committed, n_remaining};
         return dare::launch_lmhead(m->ctx, m->ctx->workspace, m->h, M, m->desc.hidden, m->lm_head, m->desc.vocab,
@@ -116,7 +131,8 @@ int check_step(const dare_model* m, int B, int L, int mode, float threshold, int
     if (mode != DARE_SELECT_THRESHOLD && mode != DARE_SELECT_TOPK) return DARE_ERR_RANGE;
     if (mode == DARE_SELECT_THRESHOLD && threshold != threshold) return DARE_ERR_RANGE;
     if (mode == DARE_SELECT_TOPK && k < 1) return DARE_ERR_RANGE;
-    if (dare::lmhead_workspace_bytes(B * L, m->desc.hidden, m->desc.vocab, m->ctx->sm_count, true, false) > m->ctx->workspace_bytes)
+    if (dare::lmhead_workspace_bytes(B * L, m->desc.hidden, m->desc.vocab, m->ctx->sm_count, true,
+                                     m->sample_temperature > 0.f) > m->ctx->workspace_bytes)
         return DARE_ERR_WORKSPACE;
     return DARE_OK;
 }
@@ -145,6 +161,7 @@ int dare_model_create(dare_ctx* ctx, const dare_model_desc* desc, const void* em
     m->rope_cs = nullptr; m->x = m->h = m->qkv = m->q = m->attn = m->act = nullptr; m->host_counts = nullptr;
     m->ev[0] = m->ev[1] = nullptr;
     m->work = nullptr; m->ev_in = m->ev_out = nullptr;
+    m->sample_temperature = 0.f; m->sample_seed = 0; m->step_counter = nullptr;
     bool ok = m->layers != nullptr;
     if (ok) for (int l = 0; l < c.n_layers; ++l) m->layers[l] = layers[l];
     const size_t rows = static_cast<size_t>(c.max_rows);
@@ -156,6 +173,8 @@ int dare_model_create(dare_ctx* ctx, const dare_model_desc* desc, const void* em
     ok = ok && cudaMalloc(&m->q, rows * nq * 2) == cudaSuccess;
     ok = ok && cudaMalloc(&m->attn, rows * nq * 2) == cudaSuccess;
     ok = ok && cudaMalloc(&m->act, rows * c.ffn * 2) == cudaSuccess;
+    ok = ok && cudaMalloc(reinterpret_cast<void**>(&m->step_counter), sizeof(uint32_t)) == cudaSuccess;
+    ok = ok && cudaMemset(m->step_counter, 0, sizeof(uint32_t)) == cudaSuccess;
     ok = ok && cudaMallocHost(reinterpret_cast<void**>(&m->host_counts), sizeof(int32_t) * 2 * c.max_batch) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&m->ev[0], cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&m->ev[1], cudaEventDisableTiming) == cudaSuccess;
@@ -178,6 +197,7 @@ int dare_model_destroy(dare_model* m) {
     cudaSetDevice(m->ctx->device);
     cudaFree(m->rope_cs); cudaFree(m->x); cudaFree(m->h); cudaFree(m->qkv); cudaFree(m->q); cudaFree(m->attn);
     cudaFree(m->act);
+    cudaFree(m->step_counter);
     if (m->host_counts) cudaFreeHost(m->host_counts);
     if (m->ev[0]) cudaEventDestroy(m->ev[0]);
     if (m->ev[1]) cudaEventDestroy(m->ev[1]);
@@ -187,6 +207,15 @@ int dare_model_destroy(dare_model* m) {
     delete[] m->layers;
     delete m;
     return DARE_OK;
+}
+
+int dare_model_set_sampling(dare_model* m, float temperature, uint64_t seed, uint32_t first_step, void* stream) {
+    if (!m) return DARE_ERR_NULL;
+    if (!(temperature >= 0.f) || isinf(temperature)) return DARE_ERR_RANGE;
+    m->sample_temperature = temperature;
+    m->sample_seed = seed;
+    set_word_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(m->step_counter, first_step);
+    return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
 }
 
 int dare_linear(dare_ctx* ctx, int epilogue, const void* a, int M, int K, const void* w, const void* w2, int N, void* out,
@@ -368,6 +397,8 @@ int dare_generate(dare_model* m, int32_t* tokens, int B, int64_t row_stride, int
     for (int b = 0; b < gen_len / L && rc == DARE_OK; ++b) {
         const int start = prompt_len + b * L;
         int taken = -1;
+        if (m->sample_temperature > 0.f)       // step n of block b draws with the counter (b << 16) + n
+            set_word_kernel<<<1, 1, 0, m->work>>>(m->step_counter, static_cast<uint32_t>(b) << 16);
         rc = run_block(m, tokens, B, row_stride, start, L, start + L, k_cache, v_cache, cache_cap, mode, threshold, k,
                        pred, conf, n_remaining, &old, &taken);
         if (rc == DARE_OK && steps_per_block) steps_per_block[b] = taken;
@@ -393,6 +424,8 @@ int dare_generate_dual(dare_model* m, int32_t* tokens, int B, int64_t row_stride
         rc = forward_rows(m, tokens, B, row_stride, 0, T, T, k_cache, v_cache, cache_cap, nullptr, m->work);
         if (rc != DARE_OK) break;
         int taken = -1;
+        if (m->sample_temperature > 0.f)
+            set_word_kernel<<<1, 1, 0, m->work>>>(m->step_counter, static_cast<uint32_t>(b) << 16);
         rc = run_block(m, tokens, B, row_stride, start, L, T, k_cache, v_cache, cache_cap, mode, threshold, k, pred, conf,
                        n_remaining, &old, &taken);
         if (rc == DARE_OK && steps_per_block) steps_per_block[b] = taken;

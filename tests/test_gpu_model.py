@@ -327,6 +327,101 @@ def test_dual_cache_loop_step_by_step_and_generate(ctx, name):
     model.close()
 
 
+@pytest.mark.parametrize("name", ["loop_small_gqa", "loop_small_bd4"])
+def test_sampled_loop_step_by_step_and_generate(ctx, name):
+    """The loop with the sampled head (dare_model_set_sampling): teacher-forced steps against the oracle's sampled
+    step with the same generator counter (block << 16) + step, then the one-call loop, then back to the argmax."""
+    from oracle import dare_sampling_oracle as SO
+    mw = I.MODEL_WORKLOADS[name]
+    wts_t = I.make_model_weights(mw)
+    cfg, wts = _cfg(mw), _oracle_weights(wts_t)
+    model = _model(ctx, mw, wts_t)
+    B, L, P, G = mw.batch, mw.block_len, mw.prompt_len, mw.gen_len
+    T, seed = 1.0, 0x5EED0123456789
+    tok0 = I.fresh_model_tokens(mw)
+    pred = torch.empty(B * L, dtype=torch.int32, device="cuda")
+    conf = torch.empty(B * L, dtype=torch.float32, device="cuda")
+    nc = torch.zeros(B, dtype=torch.int32, device="cuda")
+    nr = torch.zeros(B, dtype=torch.int32, device="cuda")
+
+    # greedy reference run of the one-call loop, before sampling is switched on
+    tok_g = tok0.cuda()
+    kc_g, vc_g = model.new_cache(B, mw.row_len)
+    steps_g = dare.dare_generate(model, tok_g, P, G, L, kc_g, vc_g, mw.mode, mw.threshold, mw.k, pred, conf, nr)
+
+    kc, vc = model.new_cache(B, mw.row_len)
+    tok = tok0.cuda()
+    dare.dare_model_forward(model, tok, 0, P, kc, vc)
+    ocache = MO.new_cache(cfg, B, mw.row_len)
+    MO.forward_block_cached(cfg, wts, tok0.numpy(), 0, P, ocache)
+    y_gap = LOGIT_GAP / T
+    steps_manual, n_rows, n_same = [], 0, 0
+    for b in range(G // L):
+        start = P + b * L
+        n = 0
+        while True:
+            pre = tok.cpu().numpy()
+            if not (pre[:, start:start + L] == mw.mask_id).any():
+                break
+            step = (b << 16) + n
+            dare.dare_model_set_sampling(model, T, seed, step)
+            dare.dare_model_step(model, tok, start, L, kc, vc, mw.mode, mw.threshold, mw.k, pred, conf, nc, nr)
+            torch.cuda.synchronize()
+            res = MO.denoise_step_cached_sampled(cfg, wts, pre, start, L, ocache, mw.mode, mw.threshold, mw.k, T, seed, step)
+            lm = res["lm"]
+            p_gpu, c_gpu = pred.cpu().numpy(), conf.cpu().numpy().astype(np.float64)
+            live = np.isfinite(lm["conf"])
+            assert (p_gpu[~live] == lm["pred"][~live]).all() and np.isneginf(c_gpu[~live]).all()
+            must = live & (lm["gap_y"] > y_gap)
+            assert (p_gpu[must] == lm["pred"][must]).all(), "sampled token differs where the best score leads clearly"
+            rows = pre[:, start:start + L].reshape(-1)
+            for m in np.nonzero(live & (p_gpu != lm["pred"]))[0]:       # a near-tie under the oracle's own scores
+                y = SO.perturbed_score(res["hidden"][m], wts.lm_head, int(p_gpu[m]), int(m), mw.mask_id, True, T, seed, step)
+                assert y >= lm["y_best"][m] - y_gap
+            same = live & (p_gpu == lm["pred"])
+            assert np.abs(np.log(c_gpu[same]) - lm["logconf"][same]).max(initial=0) <= \
+                LOGCONF_ABS_BASE + LOGCONF_ABS_PER_LAYER * mw.n_layers
+            n_rows += int(live.sum())
+            n_same += int(same.sum())
+            want, wnc, wnr = O.unmask_select(pre, start, L, p_gpu, conf.cpu().numpy(), mw.mask_id, mw.mode, mw.threshold,
+                                             mw.k)
+            np.testing.assert_array_equal(tok.cpu().numpy(), want)
+            np.testing.assert_array_equal(nc.cpu().numpy(), wnc)
+            np.testing.assert_array_equal(nr.cpu().numpy(), wnr)
+            n += 1
+            assert n <= L
+        steps_manual.append(n)
+        dare.dare_model_forward(model, tok, start, L, kc, vc)
+        MO.forward_block_cached(cfg, wts, tok.cpu().numpy(), start, L, ocache)
+    assert n_same >= 0.85 * n_rows                       # near-ties are the exception
+    final_manual = tok.cpu().numpy()
+    assert (final_manual[:, P:] != mw.mask_id).all()
+    assert (final_manual != tok_g.cpu().numpy()).any()   # sampling changed the rollouts
+    assert ctx.device_status() == 0
+
+    # ---- the one-call loop draws the same tokens (it sets the counter per block and counts the steps on the device)
+    tok2 = tok0.cuda()
+    kc2, vc2 = model.new_cache(B, mw.row_len)
+    dare.dare_model_set_sampling(model, T, seed, 0)
+    steps = dare.dare_generate(model, tok2, P, G, L, kc2, vc2, mw.mode, mw.threshold, mw.k, pred, conf, nr)
+    np.testing.assert_array_equal(tok2.cpu().numpy(), final_manual)
+    assert steps == steps_manual
+    # another seed, other rollouts
+    tok3 = tok0.cuda()
+    dare.dare_model_set_sampling(model, T, seed + 1, 0)
+    dare.dare_generate(model, tok3, P, G, L, kc2, vc2, mw.mode, mw.threshold, mw.k, pred, conf, nr)
+    assert (tok3.cpu().numpy() != final_manual).any()
+
+    # ---- temperature 0 switches back to the argmax
+    assert dare.dare_model_set_sampling(model, -1.0, 0, 0, check=False) == -4
+    dare.dare_model_set_sampling(model, 0.0)
+    tok4 = tok0.cuda()
+    steps4 = dare.dare_generate(model, tok4, P, G, L, kc2, vc2, mw.mode, mw.threshold, mw.k, pred, conf, nr)
+    assert torch.equal(tok4, tok_g) and steps4 == steps_g
+    assert ctx.device_status() == 0
+    model.close()
+
+
 class _LazyLayer:
     """fp64 views of one layer's bf16 weights, converted when touched (the full-size stack would need 7 GB)."""
 
