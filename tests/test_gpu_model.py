@@ -422,6 +422,51 @@ def test_sampled_loop_step_by_step_and_generate(ctx, name):
     model.close()
 
 
+def test_likelihood_estimator_through_the_stack(ctx):
+    """The Monte-Carlo likelihood bound of Section 4.2 end to end on a small model: forward masking of the response
+    (Eq. 1), a fully bidirectional forward of the corrupted sequence, the log-probability head on the response
+    positions, the NELBO term (Eq. 2); the same chain in the oracle.  Two draws, averaged."""
+    from oracle import dare_sampling_oracle as SO
+    mw = I.MODEL_WORKLOADS["loop_small_gqa"]
+    wts_t = I.make_model_weights(mw)
+    cfg, wts = _cfg(mw), _oracle_weights(wts_t)
+    B, P, G = mw.batch, mw.prompt_len, mw.gen_len
+    T = P + G
+    model = _model(ctx, mw, wts_t, max_rows=B * T)
+    x0 = I.uniform_int(9, I.TID_TOK, (B, T), 0, mw.mask_id - 1)            # a finished sequence: no mask anywhere
+    t = torch.tensor([0.25, 0.6, 1.0][:B], dtype=torch.float32)
+    kc, vc = model.new_cache(B, T)
+    hid = torch.empty(B * T, mw.hidden, dtype=torch.bfloat16, device="cuda")
+    lm_head = wts_t["lm_head"].cuda()
+    est_gpu, est_ref = np.zeros(B), np.zeros(B)
+    for sample in range(2):
+        xt = dare.dare_forward_mask(ctx, x0.cuda(), P, G, t.cuda(), mw.mask_id, 31, sample)
+        xt_ref = SO.forward_mask(x0.numpy(), P, G, t.numpy(), mw.mask_id, 31, sample)
+        np.testing.assert_array_equal(xt.cpu().numpy(), xt_ref)
+        dare.dare_model_forward_window(model, xt, 0, T, T, kc, vc, hidden_out=hid)
+        h_resp = hid.view(B, T, -1)[:, P:].reshape(B * G, -1).contiguous()
+        targets = x0[:, P:].contiguous().view(-1)
+        lp = dare.dare_lmhead_logprob(ctx, h_resp, lm_head, targets.cuda(), mw.mask_id, True)
+        n = torch.zeros(B, dtype=torch.int32, device="cuda")
+        nelbo = dare.dare_masked_nelbo(ctx, lp, xt, P, G, mw.mask_id, t.cuda(), n_masked=n)
+        torch.cuda.synchronize()
+        # the oracle's chain: whole sequence in one bidirectional segment
+        lp_ref = np.zeros((B, G))
+        for r in range(B):
+            full, _ = MO.forward_uncached(cfg, wts, xt_ref[r], np.zeros(T, dtype=np.int64))
+            lp_ref[r], _ = O.lmhead_logprob(full[P:], wts.lm_head, x0.numpy()[r, P:], mw.mask_id, True)
+        ref, n_ref = SO.masked_nelbo(lp_ref, xt_ref, P, G, mw.mask_id, t.numpy())
+        np.testing.assert_array_equal(n.cpu().numpy(), n_ref)
+        # per masked token the log-probability may be off by the head's bar plus the stack's (as for log-confidences)
+        per_token = LOGCONF_ABS_BASE + LOGCONF_ABS_PER_LAYER * mw.n_layers
+        assert (np.abs(nelbo.cpu().numpy() - ref) <= per_token * n_ref / t.numpy()).all()
+        est_gpu += nelbo.cpu().numpy() / 2
+        est_ref += ref / 2
+    np.testing.assert_allclose(est_gpu, est_ref, rtol=5e-3)
+    assert ctx.device_status() == 0
+    model.close()
+
+
 class _LazyLayer:
     """fp64 views of one layer's bf16 weights, converted when touched (the full-size stack would need 7 GB)."""
 
