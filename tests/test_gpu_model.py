@@ -412,6 +412,19 @@ def test_sampled_loop_step_by_step_and_generate(ctx, name):
     dare.dare_generate(model, tok3, P, G, L, kc2, vc2, mw.mode, mw.threshold, mw.k, pred, conf, nr)
     assert (tok3.cpu().numpy() != final_manual).any()
 
+    # ---- the dual-cache loop samples too: reproducible for a seed, complete, different from its argmax run
+    big = _model(ctx, mw, wts_t, max_rows=B * (P + G))
+    kd, vd = big.new_cache(B, P + G)
+    runs = []
+    for temp in (T, T, 0.0):
+        dare.dare_model_set_sampling(big, temp, seed, 0)
+        td = tok0.cuda()
+        dare.dare_generate_dual(big, td, P, G, L, kd, vd, mw.mode, mw.threshold, mw.k, pred, conf, nr)
+        assert bool((td[:, P:] != mw.mask_id).all())
+        runs.append(td.clone())
+    assert torch.equal(runs[0], runs[1]) and not torch.equal(runs[0], runs[2])
+    big.close()
+
     # ---- temperature 0 switches back to the argmax
     assert dare.dare_model_set_sampling(model, -1.0, 0, 0, check=False) == -4
     dare.dare_model_set_sampling(model, 0.0)
