@@ -34,6 +34,13 @@
  *     ran out of its bounded time) never trap: they set bits in a device status word that
  *     dare_device_status reads.
  *   - One ctx serves one stream at a time (the workspace is shared by consecutive calls).
+ *   - Work is launched on the CURRENT CUDA device, which must be the one the ctx was created on: every entry
+ *     point that takes a ctx (or a model) returns DARE_ERR_DEVICE otherwise, before anything is enqueued.
+ *     dare_create, dare_destroy, dare_model_create and dare_model_destroy work on the ctx's device and put the
+ *     caller's current device back before they return.
+ *   - A ctx keeps the TMA tensor maps it has encoded (keyed by base address, shape and tile box; a map depends on
+ *     nothing else, so an entry never goes stale): a loop that passes the same buffers every step encodes each
+ *     map once.  The kernels' shared-memory limits are likewise raised once per kernel and device.
  */
 #ifndef DARE_H_
 #define DARE_H_
@@ -55,7 +62,8 @@ typedef enum {
     DARE_ERR_RANGE = -4,       /* scalar out of range (k < 1, NaN threshold, mask id, window)   */
     DARE_ERR_WORKSPACE = -5,   /* ctx workspace too small for this call                         */
     DARE_ERR_CUDA = -6,        /* a CUDA runtime/driver call failed                             */
-    DARE_ERR_UNSUPPORTED = -7  /* device is not sm_100                                          */
+    DARE_ERR_UNSUPPORTED = -7, /* device is not sm_100                                          */
+    DARE_ERR_DEVICE = -8       /* the current CUDA device is not the context's (or a buffer's) device */
 } dare_status;
 
 /* bits of the device status word */
@@ -68,6 +76,10 @@ enum { DARE_SELECT_THRESHOLD = 0, DARE_SELECT_TOPK = 1 };
  * *out (host) receives the handle.  Allocates device memory; call outside any stream capture. */
 int dare_create(dare_ctx** out, int device, size_t workspace_bytes);
 int dare_destroy(dare_ctx* ctx);
+
+/* Counters of the ctx's tensor-map cache since dare_create (HOST pointers): calls that found their map and
+ * calls that had to encode one. */
+int dare_tmap_cache_stats(const dare_ctx* ctx, uint64_t* hits, uint64_t* misses);
 
 /* Static string for a status code (host pointer, never NULL). */
 const char* dare_status_string(int status);
@@ -433,15 +445,22 @@ int dare_generate_dual(dare_model* model, int32_t* tokens, int B, int64_t row_st
  *     returned and nothing is launched (use the ctx variant for larger problems).
  *   - The first call on each device looks up the device address of the scratch array and a driver entry
  *     point; make that first call before starting any stream capture.
- *   - All calls on a device share the one scratch array.  Nothing in it needs to start at zero (every
- *     entry that is read has been written by the same call), but two calls whose GPU work overlaps
- *     (different streams, or several host threads) race on it: serialise them on one stream.
- *   - Data-dependent status bits of this variant go to an internal word that is not exposed.
+ *   - All calls on a device share the one scratch array.  Nothing in it needs to start at zero: in a call
+ *     that runs to completion every entry that is read has been written by that call.  Two calls whose GPU
+ *     work overlaps (different streams, or several host threads) race on it: serialise them on one stream.
+ *   - hidden, w, row_tokens, pred and conf must live on the current device (DARE_ERR_DEVICE otherwise).
+ *   - Data-dependent status bits of this variant go to a word inside the library that
+ *     dare_lmhead_static_status reads.  If DARE_DEV_WAIT_EXPIRED is set there, a bounded wait inside the
+ *     kernel gave up: parts of the scratch were then NOT written by that call and its pred / conf may have
+ *     been folded from an earlier call's leftovers -- discard them.
  */
 #define DARE_LMHEAD_STATIC_SCRATCH_BYTES (8u << 20)
 int dare_lmhead_confidence_static(const void* hidden, int M, int D, const void* w, int V,
                                   const int32_t* row_tokens, int32_t mask_id, int exclude_mask_column,
                                   int32_t* pred, float* conf, void* stream);
+/* Synchronises `stream`, copies the status word of the allocation-free calls on the current device to
+ * *host_out (host) and clears it.  Allocates nothing. */
+int dare_lmhead_static_status(void* stream, uint32_t* host_out);
 
 #ifdef __cplusplus
 }

@@ -21,6 +21,7 @@ DEV_LEN_CLAMPED = 1
 DEV_WAIT_EXPIRED = 2
 
 EXPORTS = ["dare_create", "dare_destroy", "dare_status_string", "dare_device_status", "dare_sm_count",
+           "dare_tmap_cache_stats", "dare_lmhead_static_status",
            "dare_attn_block", "dare_attn_varlen", "dare_lmhead_confidence", "dare_unmask_select", "dare_denoise_block", "dare_denoise_block_sampled",
            "dare_lmhead_confidence_static", "dare_lmhead_sample", "dare_lmhead_logprob", "dare_lmhead_logprob_backward", "dare_transpose_bf16", "dare_forward_mask", "dare_masked_nelbo", "dare_model_create", "dare_model_destroy", "dare_model_forward",
            "dare_model_step", "dare_generate", "dare_model_set_sampling", "dare_model_forward_window", "dare_model_step_window", "dare_generate_dual",
@@ -56,6 +57,10 @@ def load():
     lib.dare_device_status.restype = i32
     lib.dare_sm_count.argtypes = [vp]
     lib.dare_sm_count.restype = i32
+    lib.dare_tmap_cache_stats.argtypes = [vp, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
+    lib.dare_tmap_cache_stats.restype = i32
+    lib.dare_lmhead_static_status.argtypes = [vp, C.POINTER(C.c_uint32)]
+    lib.dare_lmhead_static_status.restype = i32
     attn_args = [i32] * 7 + [f32] + [vp] * 12
     lib.dare_attn_block.argtypes = [vp] + attn_args
     lib.dare_attn_block.restype = i32
@@ -136,6 +141,9 @@ def _ptr(t: Optional[torch.Tensor], dtype=None):
         return None
     if not t.is_cuda or not t.is_contiguous():
         raise ValueError("expected a contiguous CUDA tensor")
+    # the library launches on the current device (and refuses a context of another one): the buffers must live there
+    if t.device.index != torch.cuda.current_device():
+        raise ValueError(f"tensor on cuda:{t.device.index}, but the current device is cuda:{torch.cuda.current_device()}")
     if dtype is not None and t.dtype != dtype:
         raise ValueError(f"expected dtype {dtype}, got {t.dtype}")
     return C.c_void_p(t.data_ptr())
@@ -173,6 +181,14 @@ class Context:
     @property
     def sm_count(self) -> int:
         return load().dare_sm_count(self.handle)
+
+    def tmap_cache_stats(self):
+        """(hits, misses) of the context's tensor-map cache since it was created."""
+        hits, misses = C.c_uint64(0), C.c_uint64(0)
+        rc = load().dare_tmap_cache_stats(self.handle, C.byref(hits), C.byref(misses))
+        if rc != 0:
+            raise DareError(rc, "dare_tmap_cache_stats")
+        return int(hits.value), int(misses.value)
 
     def device_status(self, stream=None) -> int:
         out = C.c_uint32(0)
@@ -345,6 +361,15 @@ def dare_lmhead_confidence_static(hidden, w, row_tokens=None, mask_id: int = -1,
     if rc != 0 and check:
         raise DareError(rc, "dare_lmhead_confidence_static")
     return (pred, conf) if check else rc
+
+
+def dare_lmhead_static_status(stream=None) -> int:
+    """Reads and clears the status word of the allocation-free LM-head calls on the current device (blocks)."""
+    out = C.c_uint32(0)
+    rc = load().dare_lmhead_static_status(_stream(stream), C.byref(out))
+    if rc != 0:
+        raise DareError(rc, "dare_lmhead_static_status")
+    return int(out.value)
 
 
 def dare_unmask_select(ctx: Context, tokens, block_start: int, L: int, pred, conf, mask_id: int, mode: int,

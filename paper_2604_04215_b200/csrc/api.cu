@@ -10,6 +10,20 @@ namespace dare {
 
 int make_tmap_bf16_2d(const dare_ctx* ctx, CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols,
                       uint32_t box_rows, uint32_t box_cols) {
+    TmapCache::Slot* slot = nullptr;
+    if (ctx->tmaps) {
+        uint64_t h = (reinterpret_cast<uintptr_t>(base) >> 4) * 0x9E3779B97F4A7C15ull;
+        h ^= (rows * 0xC2B2AE3D27D4EB4Full) ^ (cols << 17) ^ (static_cast<uint64_t>(box_rows) << 7) ^ box_cols;
+        h ^= h >> 29;
+        slot = &ctx->tmaps->slot[h % TmapCache::SLOTS];
+        if (slot->valid && slot->base == base && slot->rows == rows && slot->cols == cols &&
+            slot->box_rows == box_rows && slot->box_cols == box_cols) {
+            *out = slot->map;
+            ++ctx->tmaps->hits;
+            return DARE_OK;
+        }
+        ++ctx->tmaps->misses;
+    }
     cuuint64_t dims[2] = {cols, rows};
     cuuint64_t strides[1] = {cols * 2};   // bytes, dimension 1
     cuuint32_t box[2] = {box_cols, box_rows};
@@ -17,7 +31,13 @@ int make_tmap_bf16_2d(const dare_ctx* ctx, CUtensorMap* out, const void* base, u
     CUresult r = ctx->encode_tiled(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides,
                                    box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? DARE_OK : DARE_ERR_CUDA;
+    if (r != CUDA_SUCCESS) return DARE_ERR_CUDA;
+    if (slot) {
+        slot->base = base; slot->rows = rows; slot->cols = cols; slot->box_rows = box_rows; slot->box_cols = box_cols;
+        slot->map = *out;
+        slot->valid = true;
+    }
+    return DARE_OK;
 }
 
 }  // namespace dare
@@ -30,6 +50,7 @@ int check_attn(const dare_ctx* ctx, int B, int L, int Hq, int Hkv, int d, int pr
                const void* q, const void* k_pre, const void* v_pre, const void* k_blk, const void* v_blk,
                const void* k_suf, const void* v_suf, const void* out, dare::AttnArgs* a) {
     if (!ctx || !q || !k_pre || !v_pre || !out) return DARE_ERR_NULL;
+    if (int rc = dare::check_current_device(ctx)) return rc;
     if ((k_blk == nullptr) != (v_blk == nullptr)) return DARE_ERR_NULL;
     if ((k_suf == nullptr) != (v_suf == nullptr)) return DARE_ERR_NULL;
     if (B < 1 || L < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv != 0) return DARE_ERR_SHAPE;
@@ -54,6 +75,7 @@ int check_attn(const dare_ctx* ctx, int B, int L, int Hq, int Hkv, int d, int pr
 int check_lmhead(const dare_ctx* ctx, const void* hidden, int M, int D, const void* w, int V, bool with_row_tokens,
                  const void* pred, const void* conf, bool sampling = false) {
     if (!ctx || !hidden || !w || !pred || !conf) return DARE_ERR_NULL;
+    if (int rc = dare::check_current_device(ctx)) return rc;
     if (M < 1 || D < 8 || D % 8 != 0 || V < 2) return DARE_ERR_SHAPE;
     if (!aligned16(hidden) || !aligned16(w)) return DARE_ERR_ALIGN;
     if (dare::lmhead_workspace_bytes(M, D, V, ctx->sm_count, with_row_tokens, sampling) > ctx->workspace_bytes)
@@ -84,9 +106,12 @@ int dare_create(dare_ctx** out, int device, size_t workspace_bytes) {
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return DARE_ERR_CUDA;
     if (prop.major != 10) return DARE_ERR_UNSUPPORTED;
-    if (cudaSetDevice(device) != cudaSuccess) return DARE_ERR_CUDA;
+    dare::DeviceScope scope(device);      // the caller's current device is put back on return
+    if (!scope.ok()) return DARE_ERR_CUDA;
     dare_ctx* ctx = new (std::nothrow) dare_ctx();
     if (!ctx) return DARE_ERR_CUDA;
+    ctx->tmaps = new (std::nothrow) TmapCache();      // value-initialised: every slot invalid
+    if (!ctx->tmaps) { delete ctx; return DARE_ERR_CUDA; }
     ctx->device = device;
     ctx->sm_count = prop.multiProcessorCount;
     ctx->workspace_bytes = workspace_bytes ? workspace_bytes : (size_t(256) << 20);
@@ -96,6 +121,7 @@ int dare_create(dare_ctx** out, int device, size_t workspace_bytes) {
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
         qres != cudaDriverEntryPointSuccess || fn == nullptr) {
+        delete ctx->tmaps;
         delete ctx;
         return DARE_ERR_CUDA;
     }
@@ -105,6 +131,7 @@ int dare_create(dare_ctx** out, int device, size_t workspace_bytes) {
         cudaMemset(ctx->dev_status, 0, sizeof(uint32_t)) != cudaSuccess) {
         if (ctx->workspace) cudaFree(ctx->workspace);
         if (ctx->dev_status) cudaFree(ctx->dev_status);
+        delete ctx->tmaps;
         delete ctx;
         return DARE_ERR_CUDA;
     }
@@ -114,10 +141,18 @@ int dare_create(dare_ctx** out, int device, size_t workspace_bytes) {
 
 int dare_destroy(dare_ctx* ctx) {
     if (!ctx) return DARE_ERR_NULL;
-    cudaSetDevice(ctx->device);
+    dare::DeviceScope scope(ctx->device);
     cudaFree(ctx->workspace);
     cudaFree(ctx->dev_status);
+    delete ctx->tmaps;
     delete ctx;
+    return DARE_OK;
+}
+
+int dare_tmap_cache_stats(const dare_ctx* ctx, uint64_t* hits, uint64_t* misses) {
+    if (!ctx || !hits || !misses) return DARE_ERR_NULL;
+    *hits = ctx->tmaps ? ctx->tmaps->hits : 0;
+    *misses = ctx->tmaps ? ctx->tmaps->misses : 0;
     return DARE_OK;
 }
 
@@ -131,12 +166,14 @@ const char* dare_status_string(int status) {
         case DARE_ERR_WORKSPACE: return "context workspace too small";
         case DARE_ERR_CUDA: return "CUDA call failed";
         case DARE_ERR_UNSUPPORTED: return "device is not sm_100";
+        case DARE_ERR_DEVICE: return "the current CUDA device is not the one the context or buffers belong to";
         default: return "unknown status";
     }
 }
 
 int dare_device_status(dare_ctx* ctx, void* stream, uint32_t* host_out) {
     if (!ctx || !host_out) return DARE_ERR_NULL;
+    if (int rc = dare::check_current_device(ctx)) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (cudaMemcpyAsync(host_out, ctx->dev_status, sizeof(uint32_t), cudaMemcpyDeviceToHost, s) != cudaSuccess)
         return DARE_ERR_CUDA;
@@ -163,6 +200,7 @@ int dare_attn_varlen(dare_ctx* ctx, int total_tokens, int n_seqs, int max_seqlen
                      const void* q, const void* k, const void* v, const int32_t* cu_seqlens, void* out, float* lse,
                      void* stream) {
     if (!ctx || !q || !k || !v || !cu_seqlens || !out) return DARE_ERR_NULL;
+    if (int rc = dare::check_current_device(ctx)) return rc;
     if (total_tokens < 1 || n_seqs < 1 || max_seqlen < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || Hq / Hkv > 128)
         return DARE_ERR_SHAPE;
     if (d != 64 && d != 128) return DARE_ERR_SHAPE;
@@ -206,6 +244,7 @@ int dare_unmask_select(dare_ctx* ctx, int32_t* tokens, int B, int64_t row_stride
                        const int32_t* pred, const float* conf, int32_t mask_id, int mode, float threshold, int k,
                        int32_t* n_committed, int32_t* n_remaining, void* stream) {
     if (!ctx) return DARE_ERR_NULL;
+    if (int rc = dare::check_current_device(ctx)) return rc;
     int rc = check_select(tokens, B, row_stride, block_start, L, pred, conf, mode, threshold, k);
     if (rc != DARE_OK) return rc;
     return dare::launch_unmask_select(tokens, B, row_stride, block_start, L, pred, conf, mask_id, mode, threshold, k,

@@ -719,8 +719,8 @@ attn_block_tc_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_c
 template <int D, int QT>
 int launch_tc(const CUtensorMap* tm, const AttnParams& p, int q_tiles, cudaStream_t stream) {
     constexpr int SMEM = TcShape<D, QT>::SMEM;
-    if (cudaFuncSetAttribute(attn_block_tc_kernel<D, QT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
-        return DARE_ERR_CUDA;
+    static std::atomic<uint64_t> smem_set{0};
+    if (ensure_dynamic_smem(smem_set, attn_block_tc_kernel<D, QT>, SMEM) != DARE_OK) return DARE_ERR_CUDA;
     dim3 grid((q_tiles + QT - 1) / QT, p.B * p.Hkv, 1);
     attn_block_tc_kernel<D, QT><<<grid, TcShape<D, QT>::THREADS, SMEM, stream>>>(tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], p);
     return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
@@ -772,8 +772,8 @@ int launch_one(const CUtensorMap* tm, const AttnParams& p, int chunks, cudaStrea
     constexpr int SMEM = att_smem_bytes<D, KT, STAGES>();
     static_assert((KS - 1) * NW * ((D / 8) * 4 + 4) * 32 * 4 <= STAGES * att_stage_bytes<D, KT>(), "merge buffer");
     static_assert(STAGES <= ATT_MAX_STAGES && KT <= KT_MAX && KT % (16 * KS) == 0, "variant");
-    if (cudaFuncSetAttribute(attn_block_kernel<D, NW, KS, KT, STAGES, CPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
-        return DARE_ERR_CUDA;
+    static std::atomic<uint64_t> smem_set{0};
+    if (ensure_dynamic_smem(smem_set, attn_block_kernel<D, NW, KS, KT, STAGES, CPS>, SMEM) != DARE_OK) return DARE_ERR_CUDA;
     dim3 grid(chunks, p.B * p.Hkv, p.splits);
     attn_block_kernel<D, NW, KS, KT, STAGES, CPS><<<grid, (NW * KS + 1) * 32, SMEM, stream>>>(tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], p);
     return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;

@@ -52,6 +52,7 @@ extern "C" {
 
 int dare_transpose_bf16(dare_ctx* ctx, const void* in, int rows, int cols, void* out, void* stream) {
     if (!ctx || !in || !out) return DARE_ERR_NULL;
+    if (int rc = dare::check_current_device(ctx)) return rc;
     if (rows < 1 || cols < 1) return DARE_ERR_SHAPE;
     if (in == out) return DARE_ERR_RANGE;
     // the tile grid puts the row tiles on the y axis (65 535 at most): transpose the longer side along x
@@ -64,6 +65,7 @@ int dare_lmhead_logprob_backward(dare_ctx* ctx, const void* hidden, int M, int D
                                  const float* grad_logprob, void* dz, void* dzt, void* d_hidden, void* d_w, void* stream) {
     if (!ctx || !hidden || !w || !w_t || !targets || !lse || !grad_logprob || !dz || !dzt || !d_hidden || !d_w)
         return DARE_ERR_NULL;
+    if (int rc = dare::check_current_device(ctx)) return rc;
     if (M < 8 || D < 8 || V < 8 || (M % 8) || (D % 8) || (V % 8)) return DARE_ERR_SHAPE;
     if (!dare::aligned16(hidden) || !dare::aligned16(w) || !dare::aligned16(w_t) || !dare::aligned16(dz) ||
         !dare::aligned16(dzt) || !dare::aligned16(d_hidden) || !dare::aligned16(d_w))

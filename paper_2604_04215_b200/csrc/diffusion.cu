@@ -98,6 +98,7 @@ extern "C" {
 int dare_forward_mask(dare_ctx* ctx, const int32_t* x0, int32_t* xt, int B, int64_t row_stride, int start, int length,
                       const float* p_mask, int32_t mask_id, uint64_t seed, uint32_t sample, void* stream) {
     if (!ctx || !x0 || !xt || !p_mask) return DARE_ERR_NULL;
+    if (int rc = dare::check_current_device(ctx)) return rc;
     if (B < 1 || B > 65535 || length < 1) return DARE_ERR_SHAPE;
     if (start < 0 || row_stride < 1 || static_cast<int64_t>(start) + length > row_stride) return DARE_ERR_RANGE;
     return dare::launch_forward_mask(x0, xt, B, row_stride, start, length, p_mask, mask_id, seed, sample,
@@ -107,6 +108,7 @@ int dare_forward_mask(dare_ctx* ctx, const int32_t* x0, int32_t* xt, int B, int6
 int dare_masked_nelbo(dare_ctx* ctx, const float* logprob, const int32_t* xt, int B, int64_t row_stride, int start,
                       int length, int32_t mask_id, const float* t, float* nelbo, int32_t* n_masked, void* stream) {
     if (!ctx || !logprob || !xt || !t || !nelbo) return DARE_ERR_NULL;
+    if (int rc = dare::check_current_device(ctx)) return rc;
     if (B < 1 || length < 1) return DARE_ERR_SHAPE;
     if (start < 0 || row_stride < 1 || static_cast<int64_t>(start) + length > row_stride) return DARE_ERR_RANGE;
     return dare::launch_masked_nelbo(logprob, xt, B, row_stride, start, length, mask_id, t, nelbo, n_masked,

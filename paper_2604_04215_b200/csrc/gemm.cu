@@ -663,9 +663,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 template <int EPI>
 int launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tb2, const PairArgs& g,
                 cudaStream_t stream, int* max_clusters_query) {
-    if (cudaFuncSetAttribute(gemm_pair_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_BYTES) !=
-        cudaSuccess)
-        return DARE_ERR_CUDA;
+    static std::atomic<uint64_t> smem_set{0};
+    if (ensure_dynamic_smem(smem_set, gemm_pair_kernel<EPI>, GEMM_SMEM_BYTES) != DARE_OK) return DARE_ERR_CUDA;
     // one cluster per tile with a K split; otherwise as many clusters as the device holds, each walking the tiles
     long long clusters = static_cast<long long>(g.p.m_pairs) * g.p.n_tiles;
     if (g.p.splits == 1 && !max_clusters_query && clusters > g.p.resident) clusters = g.p.resident;
@@ -760,9 +759,8 @@ PairPlan pair_plan(int epi, int M, int N, int K, double* cost_out) {
 template <int EPI>
 int launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tb2, const GemmArgs& g,
                cudaStream_t stream, int* max_clusters_query) {
-    if (cudaFuncSetAttribute(gemm_bf16_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_BYTES) !=
-        cudaSuccess)
-        return DARE_ERR_CUDA;
+    static std::atomic<uint64_t> smem_set{0};
+    if (ensure_dynamic_smem(smem_set, gemm_bf16_kernel<EPI>, GEMM_SMEM_BYTES) != DARE_OK) return DARE_ERR_CUDA;
     const long long ctas = static_cast<long long>(g.p.m_items) * g.p.n_tiles * g.p.splits;
     if (ctas > 0x7fffffffLL) return DARE_ERR_SHAPE;
     cudaLaunchConfig_t cfg = {};

@@ -13,6 +13,23 @@ typedef CUresult (*dare_encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuui
                                          CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
                                          CUtensorMapFloatOOBfill);
 
+// Encoded tensor maps, kept per context.  A map is a pure function of (base address, rows, columns, box): it holds no
+// state of the memory it describes, so an entry can never go stale -- a buffer that was freed and allocated again at
+// the same address with the same shape gets the same, still correct, map.  The rollout passes the same buffers every
+// step, so after the first step no call encodes anything.  Direct-mapped, a colliding key overwrites.
+struct TmapCache {
+    static constexpr int SLOTS = 1024;
+    struct Slot {
+        const void* base;
+        uint64_t rows, cols;
+        uint32_t box_rows, box_cols;
+        bool valid;
+        CUtensorMap map;
+    };
+    Slot slot[SLOTS];
+    uint64_t hits, misses;
+};
+
 struct dare_ctx {
     int device;
     int sm_count;
@@ -20,9 +37,50 @@ struct dare_ctx {
     size_t workspace_bytes;
     uint32_t* dev_status;   // device word, bits DARE_DEV_*
     dare_encode_tiled_fn encode_tiled;
+    TmapCache* tmaps;       // host memory; NULL = encode on every call
 };
 
+#include <atomic>
+
 namespace dare {
+
+// Raising a kernel's dynamic shared-memory limit is needed once per kernel and device, not per launch: `done` is a
+// static of the launching function (one per kernel instantiation), bit d = set on device d.
+template <typename Kernel>
+inline int ensure_dynamic_smem(std::atomic<uint64_t>& done, Kernel kernel, int bytes) {
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess) return DARE_ERR_CUDA;
+    const uint64_t bit = (device >= 0 && device < 64) ? (uint64_t(1) << device) : 0;
+    if (bit && (done.load(std::memory_order_acquire) & bit)) return DARE_OK;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess)
+        return DARE_ERR_CUDA;
+    if (bit) done.fetch_or(bit, std::memory_order_release);
+    return DARE_OK;
+}
+
+// Makes `device` current for the lifetime of the object and puts the previous device back afterwards (the create
+// and destroy calls allocate and free on the context's device whatever the caller's current device is).
+class DeviceScope {
+public:
+    explicit DeviceScope(int device) : prev_(-1), ok_(false) {
+        if (cudaGetDevice(&prev_) != cudaSuccess) { prev_ = -1; return; }
+        ok_ = prev_ == device || cudaSetDevice(device) == cudaSuccess;
+        if (prev_ == device) prev_ = -1;      // nothing to restore
+    }
+    ~DeviceScope() { if (prev_ >= 0) cudaSetDevice(prev_); }
+    bool ok() const { return ok_; }
+private:
+    int prev_;
+    bool ok_;
+};
+
+// The entry points launch on the CURRENT device with the context's workspace and status word: a context that
+// belongs to another device must be refused before anything is enqueued.
+inline int check_current_device(const dare_ctx* ctx) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return DARE_ERR_CUDA;
+    return dev == ctx->device ? DARE_OK : DARE_ERR_DEVICE;
+}
 
 // bf16 2-D row-major tensor [rows, cols] -> tensor map with a [box_rows, 64] box and 128-byte swizzle.
 int make_tmap_bf16_2d(const dare_ctx* ctx, CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols,

@@ -771,9 +771,8 @@ int launch_partial(const dare_ctx* ctx, int grid, const CUtensorMap& tmap_x, con
         CUtensorMap tmap_w;
         int rc = make_tmap_bf16_2d(ctx, &tmap_w, w, static_cast<uint64_t>(V), static_cast<uint64_t>(D), BN, BK);
         if (rc != DARE_OK) return rc;
-        if (cudaFuncSetAttribute(lmhead_partial_kernel<MODE, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 LM_SMEM_BYTES) != cudaSuccess)
-            return DARE_ERR_CUDA;
+        static std::atomic<uint64_t> smem_set{0};
+        if (ensure_dynamic_smem(smem_set, lmhead_partial_kernel<MODE, false>, LM_SMEM_BYTES) != DARE_OK) return DARE_ERR_CUDA;
         lmhead_partial_kernel<MODE, false><<<grid, lm_threads(MODE), LM_SMEM_BYTES, stream>>>(
             tmap_x, tmap_w, M, live_rows, D, V, mask_col, n_tiles, part_max, part_sum, part_arg, ctx->dev_status, smp,
             allow_pair);
@@ -783,8 +782,8 @@ int launch_partial(const dare_ctx* ctx, int grid, const CUtensorMap& tmap_x, con
         CUtensorMap tmap_wh;      // half a W tile per CTA
         int rc = make_tmap_bf16_2d(ctx, &tmap_wh, w, static_cast<uint64_t>(V), static_cast<uint64_t>(D), BN / 2, BK);
         if (rc != DARE_OK) return rc;
-        if (cudaFuncSetAttribute(lmhead_partial_kernel<MODE, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 LM_PAIR_SMEM_BYTES) != cudaSuccess)
+        static std::atomic<uint64_t> smem_set_pair{0};
+        if (ensure_dynamic_smem(smem_set_pair, lmhead_partial_kernel<MODE, true>, LM_PAIR_SMEM_BYTES) != DARE_OK)
             return DARE_ERR_CUDA;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(static_cast<unsigned>(grid & ~1), 1, 1);
@@ -969,6 +968,7 @@ static __device__ uint32_t g_lm_static_status;
 
 struct StaticDeviceState {
     bool ready = false;
+    int device = -1;
     void* scratch = nullptr;        // device address of g_lm_static_scratch on this device
     uint32_t* status = nullptr;     // device address of g_lm_static_status on this device
     int sm_count = 0;
@@ -1002,6 +1002,7 @@ int static_state_for_current_device(StaticDeviceState** out) {
             qres != cudaDriverEntryPointSuccess || fn == nullptr)
             return DARE_ERR_CUDA;
         st.encode = reinterpret_cast<dare_encode_tiled_fn>(fn);
+        st.device = dev;
         st.ready = true;
     }
     *out = &st;
@@ -1023,9 +1024,20 @@ extern "C" int dare_lmhead_confidence_static(const void* hidden, int M, int D, c
     if (dare::lmhead_workspace_bytes(M, D, V, st->sm_count, row_tokens != nullptr, false) >
         static_cast<size_t>(DARE_LMHEAD_STATIC_SCRATCH_BYTES))
         return DARE_ERR_WORKSPACE;   // beyond the fixed scratch: use dare_lmhead_confidence with a context
+    // The kernels run on the current device with that device's scratch: a buffer that lives on another GPU would be
+    // read or written through the wrong address space.  Asking where a pointer lives allocates nothing.
+    const void* bufs[5] = {hidden, w, row_tokens, pred, conf};
+    for (const void* p : bufs) {
+        if (!p) continue;
+        cudaPointerAttributes attr;
+        if (cudaPointerGetAttributes(&attr, p) != cudaSuccess) return DARE_ERR_CUDA;
+        if ((attr.type == cudaMemoryTypeDevice || attr.type == cudaMemoryTypeManaged) && attr.device != st->device)
+            return DARE_ERR_DEVICE;
+    }
     // a context-shaped view of the static state for the shared launcher; nothing here is allocated
     dare_ctx view;
-    view.device = -1;
+    view.tmaps = nullptr;
+    view.device = st->device;
     view.sm_count = st->sm_count;
     view.workspace = st->scratch;
     view.workspace_bytes = DARE_LMHEAD_STATIC_SCRATCH_BYTES;
@@ -1035,3 +1047,17 @@ extern "C" int dare_lmhead_confidence_static(const void* hidden, int M, int D, c
                                pred, conf, static_cast<cudaStream_t>(stream), nullptr);
 }
 
+
+// Reads and clears the status word of the allocation-free calls on the current device (bits DARE_DEV_*), after
+// everything enqueued on `stream` so far has run.  Allocates nothing.
+extern "C" int dare_lmhead_static_status(void* stream, uint32_t* host_out) {
+    if (!host_out) return DARE_ERR_NULL;
+    dare::StaticDeviceState* st = nullptr;
+    int rc = dare::static_state_for_current_device(&st);
+    if (rc != DARE_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(host_out, st->status, sizeof(uint32_t), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaMemsetAsync(st->status, 0, sizeof(uint32_t), s) != cudaSuccess || cudaStreamSynchronize(s) != cudaSuccess)
+        return DARE_ERR_CUDA;
+    return DARE_OK;
+}

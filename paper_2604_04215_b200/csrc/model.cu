@@ -88,6 +88,7 @@ int forward_rows(dare_model* m, const int32_t* tokens, int B, int64_t row_stride
 int check_rows(const dare_model* m, const void* tokens, int B, int64_t row_stride, int start, int length, int kv_len,
                const void* k_cache, const void* v_cache, int cap) {
     if (!m || !tokens || !k_cache || !v_cache) return DARE_ERR_NULL;
+    if (int rc = dare::check_current_device(m->ctx)) return rc;
     if (B < 1 || length < 1 || B > m->max_batch) return DARE_ERR_SHAPE;
     if (static_cast<long long>(B) * length > m->desc.max_rows) return DARE_ERR_SHAPE;
     if (start < 0 || static_cast<long long>(start) + length > cap || cap > m->desc.max_positions ||
@@ -153,7 +154,8 @@ int dare_model_create(dare_ctx* ctx, const dare_model_desc* desc, const void* em
     if (c.mask_id < 0 || c.mask_id >= c.vocab || !(c.rms_eps >= 0.f) || !(c.rope_base > 1.f)) return DARE_ERR_RANGE;
     for (int l = 0; l < c.n_layers; ++l)
         if (!layers[l].wqkv || !layers[l].wo || !layers[l].wg || !layers[l].wu || !layers[l].wd) return DARE_ERR_NULL;
-    if (cudaSetDevice(ctx->device) != cudaSuccess) return DARE_ERR_CUDA;
+    dare::DeviceScope scope(ctx->device);
+    if (!scope.ok()) return DARE_ERR_CUDA;
     dare_model* m = new (std::nothrow) dare_model();
     if (!m) return DARE_ERR_CUDA;
     m->ctx = ctx; m->desc = c; m->embedding = embedding; m->lm_head = lm_head; m->max_batch = c.max_batch;
@@ -194,7 +196,7 @@ int dare_model_create(dare_ctx* ctx, const dare_model_desc* desc, const void* em
 
 int dare_model_destroy(dare_model* m) {
     if (!m) return DARE_ERR_NULL;
-    cudaSetDevice(m->ctx->device);
+    dare::DeviceScope scope(m->ctx->device);
     cudaFree(m->rope_cs); cudaFree(m->x); cudaFree(m->h); cudaFree(m->qkv); cudaFree(m->q); cudaFree(m->attn);
     cudaFree(m->act);
     cudaFree(m->step_counter);
@@ -211,6 +213,7 @@ int dare_model_destroy(dare_model* m) {
 
 int dare_model_set_sampling(dare_model* m, float temperature, uint64_t seed, uint32_t first_step, void* stream) {
     if (!m) return DARE_ERR_NULL;
+    if (int rc = dare::check_current_device(m->ctx)) return rc;
     if (!(temperature >= 0.f) || isinf(temperature)) return DARE_ERR_RANGE;
     m->sample_temperature = temperature;
     m->sample_seed = seed;
@@ -221,6 +224,7 @@ int dare_model_set_sampling(dare_model* m, float temperature, uint64_t seed, uin
 int dare_linear(dare_ctx* ctx, int epilogue, const void* a, int M, int K, const void* w, const void* w2, int N, void* out,
                 const void* residual, void* stream) {
     if (!ctx || !a || !w || !out) return DARE_ERR_NULL;
+    if (int rc = dare::check_current_device(ctx)) return rc;
     if (epilogue == DARE_LINEAR_SWIGLU && !w2) return DARE_ERR_NULL;
     if (epilogue == DARE_LINEAR_RESIDUAL && !residual) return DARE_ERR_NULL;
     if (epilogue < DARE_LINEAR_STORE || epilogue > DARE_LINEAR_SWIGLU) return DARE_ERR_RANGE;
@@ -239,6 +243,7 @@ int dare_linear_plan(dare_ctx* ctx, int epilogue, int M, int K, int N, int* plan
 
 int dare_rmsnorm(dare_ctx* ctx, const void* x, int n_rows, int D, float eps, void* y, void* stream) {
     if (!ctx || !x || !y) return DARE_ERR_NULL;
+    if (int rc = dare::check_current_device(ctx)) return rc;
     if (n_rows < 1 || D < 8 || D % 8) return DARE_ERR_SHAPE;
     if (!(eps >= 0.f)) return DARE_ERR_RANGE;
     if ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(y)) & 15u) return DARE_ERR_ALIGN;
@@ -248,6 +253,7 @@ int dare_rmsnorm(dare_ctx* ctx, const void* x, int n_rows, int D, float eps, voi
 int dare_rope_kv_write(dare_model* m, const void* qkv, int B, int length, int start, void* q_out, void* k_cache,
                        void* v_cache, int cache_cap, void* stream) {
     if (!m || !qkv || !q_out || !k_cache || !v_cache) return DARE_ERR_NULL;
+    if (int rc = dare::check_current_device(m->ctx)) return rc;
     if (B < 1 || length < 1) return DARE_ERR_SHAPE;
     if (start < 0 || static_cast<long long>(start) + length > cache_cap || cache_cap > m->desc.max_positions)
         return DARE_ERR_RANGE;

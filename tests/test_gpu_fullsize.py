@@ -106,5 +106,16 @@ def test_dream7b_full_size():
     assert nc.sum() > len(nc)                      # planted confidences pass tau = 0.9 somewhere
 
 
+def test_dream7b_full_size_as_stated():
+    nc = _run_full("dream7b", block_index=0, step_in_block=0, planted=False)
+    assert (nc == 1).all()                         # confidences ~1e-3 << tau: the at-least-one rule commits one per rollout
+
+
+def test_dualcache_full_size_uniform_prefix_4096():
+    """Every prefix at 4096 and every suffix at 1024: the KV-bound case the benchmark times."""
+    nc = _run_full("dualcache", block_index=0, step_in_block=0, planted=False, ragged=False)
+    assert (nc == 1).all()
+
+
 def test_dualcache_full_size_ragged():
     _run_full("dualcache", block_index=0, step_in_block=0, planted=False, ragged=True)

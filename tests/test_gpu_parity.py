@@ -291,3 +291,65 @@ def test_bad_arguments_are_rejected_before_any_launch(ctx):
     assert dare.dare_lmhead_confidence(small, xb, wb, check=False) == -5                   # workspace too small
     small.close()
     torch.cuda.synchronize()
+
+
+def test_tensor_map_cache_hits_on_the_same_buffers_and_misses_on_new_ones():
+    """The context keeps encoded tensor maps keyed by (address, shape, box).  The same step on the same buffers must
+    hit; other buffers of the same shapes must miss and still give the right result (each against the oracle); a
+    buffer freed and allocated again with another shape, possibly at the same address, must give the new shape's
+    result."""
+    wl = I.scaled(I.WORKLOADS["tiny"], batch=3)
+    ctx = dare.Context(0)
+
+    def run(si, bufs=None):
+        d = bufs or {k: getattr(si, k).cuda() for k in ("q", "k_pre", "v_pre", "k_blk", "v_blk", "x", "w")}
+        tok = si.tokens.cuda()
+        out = torch.empty_like(d["q"])
+        pred = torch.empty(wl.M, dtype=torch.int32, device="cuda")
+        conf = torch.empty(wl.M, dtype=torch.float32, device="cuda")
+        dare.dare_denoise_block(ctx, d["q"], d["k_pre"], d["v_pre"], si.prefix_len.cuda(), d["k_blk"], d["v_blk"], None,
+                                None, None, out, None, d["x"], d["w"], wl.mask_id, True, tok, si.block_start, wl.mode,
+                                wl.threshold, wl.k, pred, conf, None, None)
+        torch.cuda.synchronize()
+        ref = O.denoise_step(f64(si.q), f64(si.k_pre), f64(si.v_pre), si.prefix_len.numpy(), f64(si.k_blk), f64(si.v_blk),
+                             None, None, None, f64(si.x), f64(si.w), si.tokens.numpy(), si.block_start, wl.block_len,
+                             wl.mask_id, wl.mode, wl.threshold, wl.k)
+        check_attn(out, ref["attn_out"])
+        check_lmhead(pred, conf, ref["lm"], f64(si.x), f64(si.w), wl.mask_id, True, O)
+        return d
+
+    a = I.make_step(wl, step=0, planted=True)
+    b = I.make_step(wl, step=1, planted=True)
+    bufs_a = run(a)
+    h0, m0 = ctx.tmap_cache_stats()
+    assert m0 > 0
+    run(a, bufs_a)                                   # same buffers: every map is found
+    h1, m1 = ctx.tmap_cache_stats()
+    assert m1 == m0 and h1 - h0 == h0 + m0         # as many look-ups as the first run made, all found
+    bufs_b = run(b)                                  # same shapes at other addresses: encoded anew, results of b
+    h2, m2 = ctx.tmap_cache_stats()
+    assert m2 > m1
+    run(a, bufs_a)                                   # and a's maps are still right
+    # free a's LM-head input and let the allocator hand the memory out again for another shape
+    M, D = bufs_a["x"].shape
+    del bufs_a, bufs_b
+    x2 = I.normal_bf16(5, I.TID_X, (2 * M, D // 2))
+    w2 = I.normal_bf16(5, I.TID_W, (300, D // 2), 0.05)
+    pred, conf = dare.dare_lmhead_confidence(ctx, x2.cuda(), w2.cuda(), None, 7, True)
+    torch.cuda.synchronize()
+    ref = O.lmhead_confidence(f64(x2), f64(w2), None, 7, True)
+    check_lmhead(pred, conf, ref, f64(x2), f64(w2), 7, True, O)
+    assert ctx.device_status() == 0
+    ctx.close()
+
+
+@pytest.mark.skipif(not torch.cuda.is_available() or torch.cuda.device_count() < 2, reason="needs two GPUs")
+def test_context_of_another_device_is_refused():
+    """Nothing is launched: the call returns DARE_ERR_DEVICE before it touches the other GPU's workspace."""
+    ctx = dare.Context(1)
+    assert torch.cuda.current_device() == 0          # dare_create put the current device back
+    tok = torch.zeros(2, 8, dtype=torch.int32, device="cuda:0")
+    pred = torch.zeros(2, 4, dtype=torch.int32, device="cuda:0")
+    conf = torch.zeros(2, 4, dtype=torch.float32, device="cuda:0")
+    assert dare.dare_unmask_select(ctx, tok, 0, 4, pred, conf, 5, dare.SELECT_TOPK, 0.0, 1, check=False) == -8
+    ctx.close()

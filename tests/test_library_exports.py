@@ -31,7 +31,7 @@ def test_library_exports_every_declared_symbol():
 def test_status_strings_need_no_gpu():
     lib = binding.load()
     assert lib.dare_status_string(0) == b"ok"
-    for code in range(-7, 0):
+    for code in range(-8, 0):
         assert lib.dare_status_string(code) not in (b"ok", b"unknown status")
     assert lib.dare_status_string(-99) == b"unknown status"
 
@@ -44,3 +44,40 @@ def test_product_path_never_touches_the_oracle():
             if fn.endswith((".py", ".cu", ".cuh", ".h")):
                 text = open(os.path.join(base, fn)).read()
                 assert not re.search(r"(from|import)\s+oracle|oracle[/.]\w|dare_oracle", text), fn
+
+
+def test_binding_refuses_a_tensor_that_is_not_on_the_current_device(monkeypatch):
+    """The library launches on the current device and checks that the context belongs to it (DARE_ERR_DEVICE); the
+    binding closes the other half: a buffer on another GPU is refused before its address reaches the library.
+    Checked with a stand-in for a tensor, so that no GPU is needed."""
+    import pytest
+    import torch
+
+    class FakeDevice:
+        index = 1
+
+    class FakeTensor:
+        is_cuda = True
+        dtype = torch.int32
+        device = FakeDevice()
+
+        def is_contiguous(self):
+            return True
+
+        def data_ptr(self):
+            return 0x1000
+
+    monkeypatch.setattr(torch.cuda, "current_device", lambda: 0)
+    with pytest.raises(ValueError, match="current device"):
+        binding._ptr(FakeTensor(), torch.int32)
+    monkeypatch.setattr(torch.cuda, "current_device", lambda: 1)
+    assert binding._ptr(FakeTensor(), torch.int32).value == 0x1000
+
+
+def test_null_context_is_refused_before_anything_else():
+    lib = binding.load()
+    out = ctypes.c_uint32(0)
+    assert lib.dare_device_status(None, None, ctypes.byref(out)) == -1
+    h, m = ctypes.c_uint64(0), ctypes.c_uint64(0)
+    assert lib.dare_tmap_cache_stats(None, ctypes.byref(h), ctypes.byref(m)) == -1
+    assert lib.dare_status_string(-8).startswith(b"the current CUDA device")

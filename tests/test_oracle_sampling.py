@@ -146,3 +146,84 @@ def test_masked_nelbo_hand_worked():
     xt2 = np.full((2, 6), mask_id, dtype=np.int32)
     nelbo2, _ = SO.masked_nelbo(lp, xt2, 1, 4, mask_id, np.array([1.0, 1.0]))
     np.testing.assert_allclose(nelbo2, -lp.sum(axis=1), rtol=1e-14)
+
+
+def test_perturbed_score_is_the_winning_score_of_the_sampled_head_and_is_keyed_by_row_and_step():
+    """perturbed_score judges near-ties in the GPU tests, so a wrong row, step or seed key, a dropped temperature or
+    a forgotten mask column there must show: at the sampled token it has to reproduce the head's own best score,
+    at every other token it has to stay below it, and it is rebuilt here from the uniforms without the function."""
+    rng = np.random.default_rng(3)
+    M, V, D, mask_id, T, seed, step = 7, 90, 12, 40, 0.6, 0xABCDEF0123, 9
+    x, w = rng.standard_normal((M, D)), rng.standard_normal((V, D))
+    res = SO.lmhead_sample(x, w, None, mask_id, True, T, seed, step)
+    for m in range(M):
+        ys = np.array([SO.perturbed_score(x[m], w, v, m, mask_id, True, T, seed, step) for v in range(V)])
+        assert int(np.argmax(ys)) == res["pred"][m]
+        assert ys[res["pred"][m]] == res["y_best"][m]
+        assert ys[mask_id] == -np.inf                                       # the excluded column can never win
+        second = np.sort(ys)[-2]
+        np.testing.assert_allclose(res["gap_y"][m], ys.max() - second, rtol=1e-12)
+        # rebuilt from the definition: z / T - ln(-ln u), u of (seed, row m, step)
+        u = SO.uniforms(seed, m, step, V)
+        z = w @ x[m]
+        want = z / T - np.log(-np.log(u))
+        keep = np.arange(V) != mask_id
+        np.testing.assert_allclose(ys[keep], want[keep], rtol=1e-13)
+        # another row, step or seed key gives other scores; without the exclusion flag the mask column is finite
+        assert SO.perturbed_score(x[m], w, 3, m + 1, mask_id, True, T, seed, step) != ys[3]
+        assert SO.perturbed_score(x[m], w, 3, m, mask_id, True, T, seed, step + 1) != ys[3]
+        assert SO.perturbed_score(x[m], w, 3, m, mask_id, True, T, seed + 1, step) != ys[3]
+        assert np.isfinite(SO.perturbed_score(x[m], w, mask_id, m, mask_id, False, T, seed, step))
+
+
+def _tiny_step_inputs(rng, B=2, L=4, Hq=2, Hkv=1, d=8, P=5, V=30, mask_id=29):
+    D = Hq * d
+    q = rng.standard_normal((B, L, Hq, d))
+    k_pre, v_pre = rng.standard_normal((B, Hkv, P + L, d)), rng.standard_normal((B, Hkv, P + L, d))
+    plen = np.array([P, P - 2][:B])
+    x, w = rng.standard_normal((B * L, D)), rng.standard_normal((V, D))
+    tokens = rng.integers(0, mask_id, (B, P + L + 3)).astype(np.int32)
+    tokens[:, P:P + L] = mask_id
+    tokens[0, P + 1] = 4                                                    # one position already committed
+    return q, k_pre, v_pre, plen, x, w, tokens, P, L, mask_id
+
+
+def test_sampled_step_is_attention_plus_sampled_head_plus_selection_and_reduces_to_the_greedy_step():
+    rng = np.random.default_rng(4)
+    q, k_pre, v_pre, plen, x, w, tokens, P, L, mask_id = _tiny_step_inputs(rng)
+    T, seed, step = 0.8, 77, 3
+    for mode, thr, k in ((O.SELECT_THRESHOLD, 0.2, 0), (O.SELECT_TOPK, 0.0, 2)):
+        res = SO.denoise_step_sampled(q, k_pre, v_pre, plen, None, None, None, None, None, x, w, tokens, P, L, mask_id,
+                                      mode, thr, k, T, seed, step)
+        # composition of the three separately pinned parts, on the same inputs
+        o, lse = O.attn_block(q, k_pre, v_pre, plen)
+        np.testing.assert_array_equal(res["attn_out"], o)
+        np.testing.assert_array_equal(res["lse"], lse)
+        lm = SO.lmhead_sample(x, w, tokens[:, P:P + L].reshape(-1), mask_id, True, T, seed, step)
+        np.testing.assert_array_equal(res["lm"]["pred"], lm["pred"])
+        np.testing.assert_array_equal(res["lm"]["conf"], lm["conf"])
+        tok, nc, nr = O.unmask_select(tokens, P, L, lm["pred"], lm["conf"].astype(np.float32), mask_id, mode, thr, k)
+        np.testing.assert_array_equal(res["tokens"], tok)
+        np.testing.assert_array_equal(res["n_committed"], nc)
+        np.testing.assert_array_equal(res["n_remaining"], nr)
+        # invariants of a step: committed positions and everything outside the block keep their tokens; a commit
+        # removes a mask; the committed row of the block echoes its token with confidence -inf
+        assert res["tokens"][0, P + 1] == 4 and res["lm"]["pred"][1] == 4 and np.isneginf(res["lm"]["conf"][1])
+        outside = np.ones_like(tokens, dtype=bool)
+        outside[:, P:P + L] = False
+        np.testing.assert_array_equal(res["tokens"][outside], tokens[outside])
+        assert (nc >= 1).all() and (nc + nr == (tokens[:, P:P + L] == mask_id).sum(axis=1)).all()
+        # T -> 0: the sampled step is the greedy step
+        cold = SO.denoise_step_sampled(q, k_pre, v_pre, plen, None, None, None, None, None, x, w, tokens, P, L, mask_id,
+                                       mode, thr, k, 1e-7, seed, step)
+        greedy = O.denoise_step(q, k_pre, v_pre, plen, None, None, None, None, None, x, w, tokens, P, L, mask_id, mode,
+                                thr, k)
+        np.testing.assert_array_equal(cold["tokens"], greedy["tokens"])
+        np.testing.assert_array_equal(cold["n_committed"], greedy["n_committed"])
+        np.testing.assert_allclose(cold["lm"]["conf"], greedy["lm"]["conf"], rtol=1e-12)
+    # the step index keys the noise: another step draws other tokens somewhere
+    a = SO.denoise_step_sampled(q, k_pre, v_pre, plen, None, None, None, None, None, x, w, tokens, P, L, mask_id,
+                                O.SELECT_TOPK, 0.0, 4, 1.5, seed, 0)["lm"]["pred"]
+    b = SO.denoise_step_sampled(q, k_pre, v_pre, plen, None, None, None, None, None, x, w, tokens, P, L, mask_id,
+                                O.SELECT_TOPK, 0.0, 4, 1.5, seed, 1)["lm"]["pred"]
+    assert (a != b).any()

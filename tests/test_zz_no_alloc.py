@@ -7,13 +7,17 @@ dare_lmhead_confidence_static serves callers that cannot call cudaMalloc (and th
 context): its scratch is a fixed array inside the library.  Same kernels, so the results must agree with
 dare_lmhead_confidence on the same inputs within the LM-head bars of the other tests -- here they are
 required to be identical.  Two different problems are run back to back because the scratch array keeps the
-previous call's contents.
+previous call's contents.  The results are also held against the fp64 oracle directly, with the same bars as the
+context-based entry point.
 """
 import pytest
 import torch
 
+from oracle import dare_oracle as O
 from paper_2604_04215_b200 import binding as dare
 from paper_2604_04215_b200 import inputs as I
+
+from _util import check_lmhead, f64
 
 pytestmark = pytest.mark.gpu
 
@@ -52,6 +56,12 @@ def test_static_entry_matches_context_entry_on_two_calls_in_a_row():
             assert torch.equal(torch.isfinite(c), live)
             assert (c[live] - wc[live]).abs().max().item() <= 1e-3      # the suite's confidence bar
             assert torch.equal(c[live], wc[live])                        # and in fact bit-identical
+    # against the oracle itself, not only against the other entry point
+    for (x, w, rt, mu), (p, c) in zip(problems, outs[1]):
+        x64, w64 = f64(x.cpu()), f64(w.cpu())
+        ref = O.lmhead_confidence(x64, w64, None if rt is None else rt.cpu().numpy(), mu, True)
+        check_lmhead(p, c, ref, x64, w64, mu, True, O)
+    assert dare.dare_lmhead_static_status() == 0                 # no clamp, no expired wait in any of the calls
     ctx.close()
 
 
