@@ -90,6 +90,11 @@ int dare_device_status(dare_ctx* ctx, void* stream, uint32_t* host_out);
 /* Number of SMs the ctx's device reports (launch shapes are sized from it). */
 int dare_sm_count(const dare_ctx* ctx);
 
+/* Kernels the library has launched in this process since it was loaded, counted on the host at each launch
+ * (a step replayed from a CUDA graph counts its kernels once per replay).  Differences of two readings count
+ * the launches in between. */
+uint64_t dare_kernel_launches(void);
+
 /*
  * Block-bidirectional attention against the caches (Section 2.1; Section 3.4).
  * For every row r, query head h (KV head h / (Hq/Hkv)) and block position i:

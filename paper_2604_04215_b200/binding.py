@@ -21,7 +21,7 @@ DEV_LEN_CLAMPED = 1
 DEV_WAIT_EXPIRED = 2
 
 EXPORTS = ["dare_create", "dare_destroy", "dare_status_string", "dare_device_status", "dare_sm_count",
-           "dare_tmap_cache_stats", "dare_lmhead_static_status",
+           "dare_tmap_cache_stats", "dare_lmhead_static_status", "dare_kernel_launches",
            "dare_attn_block", "dare_attn_varlen", "dare_lmhead_confidence", "dare_unmask_select", "dare_denoise_block", "dare_denoise_block_sampled",
            "dare_lmhead_confidence_static", "dare_lmhead_sample", "dare_lmhead_logprob", "dare_lmhead_logprob_backward", "dare_transpose_bf16", "dare_forward_mask", "dare_masked_nelbo", "dare_model_create", "dare_model_destroy", "dare_model_forward",
            "dare_model_step", "dare_generate", "dare_model_set_sampling", "dare_model_forward_window", "dare_model_step_window", "dare_generate_dual",
@@ -59,6 +59,8 @@ def load():
     lib.dare_sm_count.restype = i32
     lib.dare_tmap_cache_stats.argtypes = [vp, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
     lib.dare_tmap_cache_stats.restype = i32
+    lib.dare_kernel_launches.argtypes = []
+    lib.dare_kernel_launches.restype = C.c_uint64
     lib.dare_lmhead_static_status.argtypes = [vp, C.POINTER(C.c_uint32)]
     lib.dare_lmhead_static_status.restype = i32
     attn_args = [i32] * 7 + [f32] + [vp] * 12
@@ -361,6 +363,11 @@ def dare_lmhead_confidence_static(hidden, w, row_tokens=None, mask_id: int = -1,
     if rc != 0 and check:
         raise DareError(rc, "dare_lmhead_confidence_static")
     return (pred, conf) if check else rc
+
+
+def dare_kernel_launches() -> int:
+    """Kernels launched by the library in this process so far (host-side count)."""
+    return int(load().dare_kernel_launches())
 
 
 def dare_lmhead_static_status(stream=None) -> int:

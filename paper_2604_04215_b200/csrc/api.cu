@@ -8,6 +8,8 @@
 
 namespace dare {
 
+std::atomic<uint64_t> g_kernel_launches{0};
+
 int make_tmap_bf16_2d(const dare_ctx* ctx, CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols,
                       uint32_t box_rows, uint32_t box_cols) {
     TmapCache::Slot* slot = nullptr;
@@ -183,6 +185,8 @@ int dare_device_status(dare_ctx* ctx, void* stream, uint32_t* host_out) {
 }
 
 int dare_sm_count(const dare_ctx* ctx) { return ctx ? ctx->sm_count : DARE_ERR_NULL; }
+
+uint64_t dare_kernel_launches(void) { return dare::g_kernel_launches.load(std::memory_order_relaxed); }
 
 int dare_attn_block(dare_ctx* ctx, int B, int L, int Hq, int Hkv, int d, int prefix_cap, int suffix_cap, float scale,
                     const void* q, const void* k_pre, const void* v_pre, const int32_t* prefix_len, const void* k_blk,

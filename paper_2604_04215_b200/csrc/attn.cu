@@ -722,7 +722,7 @@ int launch_tc(const CUtensorMap* tm, const AttnParams& p, int q_tiles, cudaStrea
     static std::atomic<uint64_t> smem_set{0};
     if (ensure_dynamic_smem(smem_set, attn_block_tc_kernel<D, QT>, SMEM) != DARE_OK) return DARE_ERR_CUDA;
     dim3 grid((q_tiles + QT - 1) / QT, p.B * p.Hkv, 1);
-    attn_block_tc_kernel<D, QT><<<grid, TcShape<D, QT>::THREADS, SMEM, stream>>>(tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], p);
+    attn_block_tc_kernel<D, QT><<<grid, TcShape<D, QT>::THREADS, SMEM, stream>>>(tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], p); note_launch();
     return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
 }
 
@@ -775,7 +775,7 @@ int launch_one(const CUtensorMap* tm, const AttnParams& p, int chunks, cudaStrea
     static std::atomic<uint64_t> smem_set{0};
     if (ensure_dynamic_smem(smem_set, attn_block_kernel<D, NW, KS, KT, STAGES, CPS>, SMEM) != DARE_OK) return DARE_ERR_CUDA;
     dim3 grid(chunks, p.B * p.Hkv, p.splits);
-    attn_block_kernel<D, NW, KS, KT, STAGES, CPS><<<grid, (NW * KS + 1) * 32, SMEM, stream>>>(tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], p);
+    attn_block_kernel<D, NW, KS, KT, STAGES, CPS><<<grid, (NW * KS + 1) * 32, SMEM, stream>>>(tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], p); note_launch();
     return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
 }
 
@@ -885,6 +885,7 @@ int launch_attn(const dare_ctx* ctx, const AttnArgs& a, cudaStream_t stream) {
             attn_combine_kernel<128><<<blocks, 256, 0, stream>>>(p.part_o, p.part_lse, p.splits, n_rows, a.L, a.Hq, p.out, p.lse);
         else
             attn_combine_kernel<64><<<blocks, 256, 0, stream>>>(p.part_o, p.part_lse, p.splits, n_rows, a.L, a.Hq, p.out, p.lse);
+        note_launch();
         if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
     }
     return DARE_OK;

@@ -39,7 +39,7 @@ int launch_transpose(const void* in, int rows, int cols, void* out, cudaStream_t
     dim3 grid((cols + 31) / 32, (rows + 31) / 32, 1);
     if (grid.y > 65535u) return DARE_ERR_SHAPE;
     transpose_bf16_kernel<<<grid, 256, 0, stream>>>(static_cast<const unsigned short*>(in), rows, cols,
-                                                    static_cast<unsigned short*>(out));
+                                                    static_cast<unsigned short*>(out)); note_launch();
     return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
 }
 

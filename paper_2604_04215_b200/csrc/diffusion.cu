@@ -80,14 +80,14 @@ int launch_forward_mask(const int32_t* x0, int32_t* xt, int B, int64_t row_strid
     dim3 grid((groups + 127) / 128, B, 1);
     forward_mask_kernel<<<grid, 128, 0, stream>>>(x0, xt, row_stride, start, length, p_mask, mask_id,
                                                   static_cast<uint32_t>(seed & 0xffffffffu),
-                                                  static_cast<uint32_t>(seed >> 32), sample);
+                                                  static_cast<uint32_t>(seed >> 32), sample); note_launch();
     return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
 }
 
 int launch_masked_nelbo(const float* logprob, const int32_t* xt, int B, int64_t row_stride, int start, int length,
                         int32_t mask_id, const float* t, float* nelbo, int32_t* n_masked, cudaStream_t stream) {
     masked_nelbo_kernel<<<(B + 3) / 4, 128, 0, stream>>>(logprob, xt, B, row_stride, start, length, mask_id, t, nelbo,
-                                                         n_masked);
+                                                         n_masked); note_launch();
     return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
 }
 

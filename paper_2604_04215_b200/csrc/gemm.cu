@@ -687,6 +687,7 @@ int launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap&
         return cudaOccupancyMaxActiveClusters(max_clusters_query, gemm_pair_kernel<EPI>, &cfg) == cudaSuccess
                    ? DARE_OK : DARE_ERR_CUDA;
     }
+    note_launch();
     return cudaLaunchKernelEx(&cfg, gemm_pair_kernel<EPI>, ta, tb, tb2, g) == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
 }
 
@@ -780,6 +781,7 @@ int launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& 
         return cudaOccupancyMaxActiveClusters(max_clusters_query, gemm_bf16_kernel<EPI>, &cfg) == cudaSuccess
                    ? DARE_OK : DARE_ERR_CUDA;
     }
+    note_launch();
     return cudaLaunchKernelEx(&cfg, gemm_bf16_kernel<EPI>, ta, tb, tb2, g) == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
 }
 

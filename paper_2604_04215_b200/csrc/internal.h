@@ -44,6 +44,11 @@ struct dare_ctx {
 
 namespace dare {
 
+// Kernels this library has launched since it was loaded (counted on the host at every launch site; a launch that
+// is replayed from a CUDA graph is counted per replay by whoever replays it).
+extern std::atomic<uint64_t> g_kernel_launches;
+inline void note_launch(uint64_t n = 1) { g_kernel_launches.fetch_add(n, std::memory_order_relaxed); }
+
 // Raising a kernel's dynamic shared-memory limit is needed once per kernel and device, not per launch: `done` is a
 // static of the launching function (one per kernel instantiation), bit d = set on device d.
 template <typename Kernel>

@@ -114,19 +114,19 @@ rope_kv_write_kernel(const __nv_bfloat16* __restrict__ qkv, int Hq, int Hkv, int
 int launch_embed(const void* emb, int D, int V, const int32_t* tokens, int64_t row_stride, int start, int length,
                  int n_rows, void* x, cudaStream_t stream) {
     embed_gather_kernel<<<(n_rows + ROWS_PER_BLOCK - 1) / ROWS_PER_BLOCK, ROWS_PER_BLOCK * 32, 0, stream>>>(
-        static_cast<const uint4*>(emb), D / 8, V, tokens, row_stride, start, length, n_rows, static_cast<uint4*>(x));
+        static_cast<const uint4*>(emb), D / 8, V, tokens, row_stride, start, length, n_rows, static_cast<uint4*>(x)); note_launch();
     return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
 }
 
 int launch_rmsnorm(const void* x, int D, int n_rows, float eps, void* y, cudaStream_t stream) {
     rmsnorm_kernel<<<(n_rows + ROWS_PER_BLOCK - 1) / ROWS_PER_BLOCK, ROWS_PER_BLOCK * 32, 0, stream>>>(
-        static_cast<const uint4*>(x), D / 8, n_rows, eps, static_cast<uint4*>(y));
+        static_cast<const uint4*>(x), D / 8, n_rows, eps, static_cast<uint4*>(y)); note_launch();
     return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
 }
 
 int launch_rope_table(float* cs, int n_pos, int half, double base, cudaStream_t stream) {
     const int n = n_pos * half;
-    rope_table_kernel<<<(n + 255) / 256, 256, 0, stream>>>(reinterpret_cast<float2*>(cs), n_pos, half, base);
+    rope_table_kernel<<<(n + 255) / 256, 256, 0, stream>>>(reinterpret_cast<float2*>(cs), n_pos, half, base); note_launch();
     return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
 }
 
@@ -136,7 +136,7 @@ int launch_rope_kv_write(const void* qkv, int n_rows, int Hq, int Hkv, int d, in
                                                      reinterpret_cast<const float2*>(cs),
                                                      static_cast<__nv_bfloat16*>(q_out),
                                                      static_cast<__nv_bfloat16*>(k_cache),
-                                                     static_cast<__nv_bfloat16*>(v_cache), cap);
+                                                     static_cast<__nv_bfloat16*>(v_cache), cap); note_launch();
     return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
 }
 

@@ -775,7 +775,7 @@ int launch_partial(const dare_ctx* ctx, int grid, const CUtensorMap& tmap_x, con
         if (ensure_dynamic_smem(smem_set, lmhead_partial_kernel<MODE, false>, LM_SMEM_BYTES) != DARE_OK) return DARE_ERR_CUDA;
         lmhead_partial_kernel<MODE, false><<<grid, lm_threads(MODE), LM_SMEM_BYTES, stream>>>(
             tmap_x, tmap_w, M, live_rows, D, V, mask_col, n_tiles, part_max, part_sum, part_arg, ctx->dev_status, smp,
-            allow_pair);
+            allow_pair); note_launch();
         if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
     }
     if (run_pair) {
@@ -798,6 +798,7 @@ int launch_partial(const dare_ctx* ctx, int grid, const CUtensorMap& tmap_x, con
         if (cudaLaunchKernelEx(&cfg, lmhead_partial_kernel<MODE, true>, tmap_x, tmap_wh, M, live_rows, D, V, mask_col,
                                n_tiles, part_max, part_sum, part_arg, ctx->dev_status, smp, allow_pair) != cudaSuccess)
             return DARE_ERR_CUDA;
+        note_launch();
     }
     return DARE_OK;
 }
@@ -839,7 +840,7 @@ int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M,
         x_gemm = xc;
         lmhead_compact_kernel<<<(M + CP_ROWS - 1) / CP_ROWS, CP_ROWS * 32, 0, stream>>>(
             static_cast<const uint4*>(hidden), M, D / 8, row_tokens, tok_L, tok_row_stride, mask_id,
-            static_cast<uint4*>(xc), idx, live_rows, pred, conf);
+            static_cast<uint4*>(xc), idx, live_rows, pred, conf); note_launch();
         if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
     }
     size_t groups_max = static_cast<size_t>(ctx->sm_count);
@@ -868,10 +869,10 @@ int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M,
             sel.n_committed = select->n_committed; sel.n_remaining = select->n_remaining;
             lmhead_merge_select_kernel<<<select->B, 32 * tok_L, 0, stream>>>(part_max, part_sum, part_arg, grid, n_tiles,
                                                                              tok_L, live_rows, idx, mask_id, pred, conf,
-                                                                             allow_pair, sel);
+                                                                             allow_pair, sel); note_launch();
         } else {
             lmhead_merge_kernel<<<(M + rows_per_block - 1) / rows_per_block, rows_per_block * 32, 0, stream>>>(
-                part_max, part_sum, part_arg, grid, n_tiles, M, live_rows, idx, pred, conf, allow_pair);
+                part_max, part_sum, part_arg, grid, n_tiles, M, live_rows, idx, pred, conf, allow_pair); note_launch();
         }
     } else {
         smp.inv_temperature = 1.0f / sample->temperature;
@@ -887,7 +888,7 @@ int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M,
         if (rc != DARE_OK) return rc;
         lmhead_merge_sample_kernel<<<(M + rows_per_block - 1) / rows_per_block, rows_per_block * 32, 0, stream>>>(
             part_max, part_sum, part_arg, smp.part_y, smp.part_zb, grid, n_tiles, M, live_rows, idx, pred, conf,
-            allow_pair, sample->step_dev);
+            allow_pair, sample->step_dev); note_launch();
     }
     if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
     return DARE_OK;
@@ -918,7 +919,7 @@ int launch_lmhead_logprob(const dare_ctx* ctx, void* scratch, const void* hidden
     if (rc != DARE_OK) return rc;
     const int rows_per_block = 8;
     lmhead_merge_logprob_kernel<<<(M + rows_per_block - 1) / rows_per_block, rows_per_block * 32, 0, stream>>>(
-        part_max, part_sum, part_zt, grid, n_tiles, M, logprob, lse_out, allow_pair);
+        part_max, part_sum, part_zt, grid, n_tiles, M, logprob, lse_out, allow_pair); note_launch();
     return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
 }
 

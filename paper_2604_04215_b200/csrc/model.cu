@@ -217,7 +217,7 @@ int dare_model_set_sampling(dare_model* m, float temperature, uint64_t seed, uin
     if (!(temperature >= 0.f) || isinf(temperature)) return DARE_ERR_RANGE;
     m->sample_temperature = temperature;
     m->sample_seed = seed;
-    set_word_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(m->step_counter, first_step);
+    set_word_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(m->step_counter, first_step); dare::note_launch();
     return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
 }
 
@@ -326,8 +326,11 @@ int run_block(dare_model* m, int32_t* tokens, int B, int64_t row_stride, int sta
     cudaStream_t s = m->work;
     BlockGraph cur;
     if (cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal) != cudaSuccess) return DARE_ERR_CUDA;
+    const uint64_t launches_before = dare::g_kernel_launches.load();      // the capture itself launches nothing:
     int rc = step_rows(m, tokens, B, row_stride, start, L, kv_len, k_cache, v_cache, cap, mode, threshold, k, pred, conf,
                        nullptr, n_remaining, s);
+    const uint64_t per_replay = dare::g_kernel_launches.load() - launches_before;
+    dare::g_kernel_launches.fetch_sub(per_replay);                        // ... its kernels are counted per replay
     const cudaError_t end = cudaStreamEndCapture(s, &cur.graph);      // always ends the capture, also after an error
     if (rc == DARE_OK && (end != cudaSuccess || cur.graph == nullptr)) rc = DARE_ERR_CUDA;
     if (rc == DARE_OK && cudaGraphInstantiate(&cur.exec, cur.graph, 0) != cudaSuccess) rc = DARE_ERR_CUDA;
@@ -343,6 +346,7 @@ int run_block(dare_model* m, int32_t* tokens, int B, int64_t row_stride, int sta
             break;
         }
         ++issued;
+        dare::note_launch(per_replay);
         if (issued >= 2) {
             const int prev = (issued - 2) & 1;
             if (cudaEventSynchronize(m->ev[prev]) != cudaSuccess) { rc = DARE_ERR_CUDA; break; }
@@ -403,8 +407,10 @@ int dare_generate(dare_model* m, int32_t* tokens, int B, int64_t row_stride, int
     for (int b = 0; b < gen_len / L && rc == DARE_OK; ++b) {
         const int start = prompt_len + b * L;
         int taken = -1;
-        if (m->sample_temperature > 0.f)       // step n of block b draws with the counter (b << 16) + n
+        if (m->sample_temperature > 0.f) {     // step n of block b draws with the counter (b << 16) + n
             set_word_kernel<<<1, 1, 0, m->work>>>(m->step_counter, static_cast<uint32_t>(b) << 16);
+            dare::note_launch();
+        }
         rc = run_block(m, tokens, B, row_stride, start, L, start + L, k_cache, v_cache, cache_cap, mode, threshold, k,
                        pred, conf, n_remaining, &old, &taken);
         if (rc == DARE_OK && steps_per_block) steps_per_block[b] = taken;
@@ -430,8 +436,10 @@ int dare_generate_dual(dare_model* m, int32_t* tokens, int B, int64_t row_stride
         rc = forward_rows(m, tokens, B, row_stride, 0, T, T, k_cache, v_cache, cache_cap, nullptr, m->work);
         if (rc != DARE_OK) break;
         int taken = -1;
-        if (m->sample_temperature > 0.f)
+        if (m->sample_temperature > 0.f) {
             set_word_kernel<<<1, 1, 0, m->work>>>(m->step_counter, static_cast<uint32_t>(b) << 16);
+            dare::note_launch();
+        }
         rc = run_block(m, tokens, B, row_stride, start, L, T, k_cache, v_cache, cache_cap, mode, threshold, k, pred, conf,
                        n_remaining, &old, &taken);
         if (rc == DARE_OK && steps_per_block) steps_per_block[b] = taken;

@@ -75,7 +75,7 @@ int launch_unmask_select(int32_t* tokens, int B, int64_t row_stride, int block_s
     if (L > SEL_MAX_L) return DARE_ERR_SHAPE;
     unmask_select_kernel<<<B, SEL_THREADS, L * sizeof(float), stream>>>(tokens, row_stride, block_start, L, pred, conf,
                                                                         mask_id, mode, threshold, k, n_committed,
-                                                                        n_remaining);
+                                                                        n_remaining); note_launch();
     return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
 }
 

@@ -60,3 +60,28 @@ def test_two_ranks_shard_rollouts_and_reduce(tmp_path):
     world = 2
     mp.spawn(_worker, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
     assert open(tmp_path / "ok").read() == "1"
+
+
+def test_bench_starts_its_own_ranks_when_no_launcher_set_the_environment(tmp_path):
+    """`python bench.py --gpus 2` with no WORLD_SIZE in the environment must start two ranks by itself (one process
+    per GPU through torch.distributed.run on 127.0.0.1).  Checked on the CPU with the oracle arm standing in for the
+    step: the two ranks meet over gloo, rank 0 alone prints the line, the other exits 0."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items()
+           if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    res = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--impl", "reference", "--gpus", "2",
+                          "--workload", "tiny", "--steps", "2", "--warmup", "1"],
+                         env=env, capture_output=True, text=True, timeout=600)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [json.loads(l) for l in res.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                              # rank 0 alone reports
+    assert lines[0]["impl"] == "reference" and lines[0]["n_gpus"] == 2 and lines[0]["value"] > 0
+    # a rank count that contradicts the launcher's is refused instead of silently timing another job
+    env1 = dict(env, WORLD_SIZE="1", RANK="0", LOCAL_RANK="0")
+    bad = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--impl", "reference", "--gpus", "2",
+                          "--workload", "tiny", "--steps", "1", "--warmup", "0"],
+                         env=env1, capture_output=True, text=True, timeout=600)
+    assert bad.returncode != 0 and "does not match WORLD_SIZE" in bad.stderr
