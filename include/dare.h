@@ -150,8 +150,8 @@ int dare_attn_varlen(dare_ctx* ctx, int total_tokens, int n_seqs, int max_seqlen
  *                pred = that token, conf = -inf
  *   pred         int32 [M] out      conf  fp32 [M] out
  * Only rows that are still masked are evaluated (they are compacted on the device first).
- * Supported: D % 8 == 0, D >= 8; V >= 2; M >= 1.  Needs ctx workspace of 12 * M * min(#SMs, ceil(V/256))
- * bytes, plus 2*M*D + 4*M + 2048 bytes when row_tokens is given.
+ * Supported: D % 8 == 0, D >= 8; V >= 2; M >= 1.  Needs ctx workspace of 12 * M * min(#SMs, 2 * ceil(V/256))
+ * bytes (partial (max, sum, argmax) triples per row), plus 2*M*D + 4*M + 2048 bytes when row_tokens is given.
  */
 int dare_lmhead_confidence(dare_ctx* ctx,
                            const void* hidden, int M, int D, const void* w, int V,
@@ -168,7 +168,7 @@ int dare_lmhead_confidence(dare_ctx* ctx,
  * (v / 4, m, step, 0x44415245) where m is the row's index in `hidden`; element v uses output word v % 4, whose top
  * 23 bits k give u_v = (2 k + 1) / 2^24.  The same (seed, step) reproduces the same tokens; callers advance `step`
  * from one denoising step to the next.  Other arguments, skipped rows and limits as dare_lmhead_confidence;
- * temperature > 0; the workspace need is 20 instead of 12 bytes per (row, vocabulary group).
+ * temperature > 0; the workspace need is 20 * M * min(#SMs, ceil(V/256)) bytes (+ the row_tokens part).
  */
 int dare_lmhead_sample(dare_ctx* ctx,
                        const void* hidden, int M, int D, const void* w, int V,
@@ -185,7 +185,7 @@ int dare_lmhead_sample(dare_ctx* ctx,
  *
  *   targets   int32 [M]: a target outside [0, V) (or the excluded column) gives logprob = -inf
  *   logprob   fp32 [M] out          lse  fp32 [M] out or NULL: logsumexp z
- * Every row is evaluated.  Workspace and limits as dare_lmhead_confidence without row_tokens.
+ * Every row is evaluated.  Limits as dare_lmhead_confidence; workspace 12 * M * min(#SMs, ceil(V/256)) bytes.
  */
 int dare_lmhead_logprob(dare_ctx* ctx,
                         const void* hidden, int M, int D, const void* w, int V,
@@ -445,7 +445,7 @@ int dare_generate_dual(dare_model* model, int32_t* tokens, int B, int64_t row_st
  *
  * Same arguments, results and arithmetic as dare_lmhead_confidence, without the ctx; it runs on the
  * CURRENT device.  Limits and rules:
- *   - The scratch the call needs (12 * M * min(#SMs, ceil(V/256)) bytes, plus 2*M*D + 4*M + 2048 bytes when
+ *   - The scratch the call needs (12 * M * min(#SMs, 2 * ceil(V/256)) bytes, plus 2*M*D + 4*M + 2048 bytes when
  *     row_tokens is given) must not exceed DARE_LMHEAD_STATIC_SCRATCH_BYTES, else DARE_ERR_WORKSPACE is
  *     returned and nothing is launched (use the ctx variant for larger problems).
  *   - The first call on each device looks up the device address of the scratch array and a driver entry

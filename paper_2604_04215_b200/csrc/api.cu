@@ -14,17 +14,29 @@ int make_tmap_bf16_2d(const dare_ctx* ctx, CUtensorMap* out, const void* base, u
                       uint32_t box_rows, uint32_t box_cols) {
     TmapCache::Slot* slot = nullptr;
     if (ctx->tmaps) {
-        uint64_t h = (reinterpret_cast<uintptr_t>(base) >> 4) * 0x9E3779B97F4A7C15ull;
-        h ^= (rows * 0xC2B2AE3D27D4EB4Full) ^ (cols << 17) ^ (static_cast<uint64_t>(box_rows) << 7) ^ box_cols;
-        h ^= h >> 29;
-        slot = &ctx->tmaps->slot[h % TmapCache::SLOTS];
-        if (slot->valid && slot->base == base && slot->rows == rows && slot->cols == cols &&
-            slot->box_rows == box_rows && slot->box_cols == box_cols) {
-            *out = slot->map;
-            ++ctx->tmaps->hits;
-            return DARE_OK;
+        // 64-bit finaliser over the whole key (allocations are aligned to hundreds of bytes, shapes are round numbers:
+        // the raw low bits carry almost nothing)
+        uint64_t h = reinterpret_cast<uintptr_t>(base) ^ (rows * 0x9E3779B97F4A7C15ull) ^ (cols * 0xC2B2AE3D27D4EB4Full) ^
+                     (static_cast<uint64_t>(box_rows) << 40) ^ (static_cast<uint64_t>(box_cols) << 52);
+        h ^= h >> 30; h *= 0xBF58476D1CE4E5B9ull;
+        h ^= h >> 27; h *= 0x94D049BB133111EBull;
+        h ^= h >> 31;
+        const int set = static_cast<int>(h % TmapCache::SETS);
+        TmapCache::Slot* ways = &ctx->tmaps->slot[set * TmapCache::WAYS];
+        for (int i = 0; i < TmapCache::WAYS; ++i) {
+            TmapCache::Slot& s = ways[i];
+            if (s.valid && s.base == base && s.rows == rows && s.cols == cols && s.box_rows == box_rows &&
+                s.box_cols == box_cols) {
+                *out = s.map;
+                ++ctx->tmaps->hits;
+                return DARE_OK;
+            }
         }
         ++ctx->tmaps->misses;
+        slot = &ways[ctx->tmaps->next_way[set]];
+        for (int i = 0; i < TmapCache::WAYS; ++i)       // an empty way first, else the set's next one in turn
+            if (!ways[i].valid) { slot = &ways[i]; break; }
+        if (slot->valid) ctx->tmaps->next_way[set] = static_cast<uint8_t>((ctx->tmaps->next_way[set] + 1) % TmapCache::WAYS);
     }
     cuuint64_t dims[2] = {cols, rows};
     cuuint64_t strides[1] = {cols * 2};   // bytes, dimension 1

@@ -16,9 +16,9 @@ typedef CUresult (*dare_encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuui
 // Encoded tensor maps, kept per context.  A map is a pure function of (base address, rows, columns, box): it holds no
 // state of the memory it describes, so an entry can never go stale -- a buffer that was freed and allocated again at
 // the same address with the same shape gets the same, still correct, map.  The rollout passes the same buffers every
-// step, so after the first step no call encodes anything.  Direct-mapped, a colliding key overwrites.
+// step, so after the first step no call encodes anything.  Four-way set associative; a full set evicts in turn.
 struct TmapCache {
-    static constexpr int SLOTS = 1024;
+    static constexpr int SETS = 256, WAYS = 4, SLOTS = SETS * WAYS;
     struct Slot {
         const void* base;
         uint64_t rows, cols;
@@ -27,6 +27,7 @@ struct TmapCache {
         CUtensorMap map;
     };
     Slot slot[SLOTS];
+    uint8_t next_way[SETS];
     uint64_t hits, misses;
 };
 

@@ -78,14 +78,16 @@ __host__ __device__ inline int lm_groups(int grid, int m_tiles, int n_tiles) {
     return g;
 }
 
-// Pairs pay when the row tiles come in twos (an odd tile would drag an empty partner along).  The row count is
-// only known on the device, so both kernels are launched and the one whose mode does not apply returns at once.
+// Pairs pay when the row tiles come in twos (an odd tile would drag an empty partner along: measured at 3584 x
+// 152064, five tiles take 544 us on single CTAs and 600 to 660 us on pairs with the sixth tile empty).  The row
+// count is only known on the device, so both kernels are launched and the one whose mode does not apply returns
+// at once.
 __host__ __device__ inline bool lm_pair_mode(int m_tiles, int allow_pair) {
     return allow_pair && m_tiles >= 2 && (m_tiles & 1) == 0;
 }
 // Vocabulary groups in the mode that applies: pairs count as one CTA and two row tiles as one.
 __host__ __device__ inline int lm_groups_mode(int grid, int m_tiles, int n_tiles, int allow_pair) {
-    return lm_pair_mode(m_tiles, allow_pair) ? lm_groups(grid / 2, m_tiles / 2, n_tiles) : lm_groups(grid, m_tiles, n_tiles);
+    return lm_pair_mode(m_tiles, allow_pair) ? lm_groups(grid / 2, (m_tiles + 1) / 2, n_tiles) : lm_groups(grid, m_tiles, n_tiles);
 }
 
 __device__ __forceinline__ int32_t row_token(const int32_t* row_tokens, int tok_L, int64_t tok_row_stride, int m) {
@@ -178,12 +180,13 @@ __device__ __forceinline__ float gumbel_from_word(uint32_t w) {
 // bf16 in both orientations (the two products of the backward pass take it from there); no partials.
 constexpr int LM_GREEDY = 0, LM_SAMPLE = 1, LM_LOGPROB = 2, LM_GRAD = 3;
 
+// swap_small: this launch leaves steps with at most SW_NMAX live rows to the swapped-operand path (further down).
 template <int MODE, bool PAIR>
-__global__ void __launch_bounds__(lm_threads(MODE), 1)
-lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
-                      int M, const int32_t* __restrict__ live_rows, int D, int V, int mask_col, int n_tiles,
-                      float* __restrict__ part_max, float* __restrict__ part_sum, int32_t* __restrict__ part_arg,
-                      uint32_t* __restrict__ dev_status, const LmSampling smp, int allow_pair) {
+__device__ __forceinline__ void
+lm_rowmajor_body(const CUtensorMap& tmap_x, const CUtensorMap& tmap_w,
+                 int M, const int32_t* __restrict__ live_rows, int D, int V, int mask_col, int n_tiles,
+                 float* __restrict__ part_max, float* __restrict__ part_sum, int32_t* __restrict__ part_arg,
+                 uint32_t* __restrict__ dev_status, const LmSampling& smp, int allow_pair, int swap_small) {
     constexpr int NSTAGES = PAIR ? PSTAGES : STAGES;
     constexpr int STAGE_SZ = PAIR ? PSTAGE_BYTES : STAGE_BYTES;
     using Barriers = typename std::conditional<PAIR, LmPairBarriers, LmBarriers>::type;
@@ -195,12 +198,13 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     const int Mc = live_rows ? *live_rows : M;          // rows that need logits (uniform over the grid)
     const int m_tiles = (Mc + BM - 1) / BM;
     if (m_tiles == 0) return;
+    if (swap_small && Mc <= 256) return;                          // the swapped-operand path does this launch's work
     if (lm_pair_mode(m_tiles, allow_pair) != PAIR) return;        // the other kernel does this launch's work
     // PAIR: a work unit is a cluster of two CTAs, an item two row tiles (one per CTA) and a vocabulary group
     const int rank = PAIR ? static_cast<int>(cluster_cta_rank()) : 0;
     const int unit = PAIR ? blockIdx.x >> 1 : blockIdx.x;
     const int n_units = PAIR ? gridDim.x >> 1 : gridDim.x;
-    const int item_rows = PAIR ? m_tiles >> 1 : m_tiles;             // row tiles (pairs of them) to walk
+    const int item_rows = PAIR ? (m_tiles + 1) >> 1 : m_tiles;       // row tiles (pairs of them) to walk
     const int groups = lm_groups(n_units, item_rows, n_tiles);
     const int n_items = item_rows * groups;
     if (unit >= n_items) return;                                    // (both CTAs of a pair alike)
@@ -510,6 +514,354 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     }
 }
 
+template <int MODE, bool PAIR>
+__global__ void __launch_bounds__(lm_threads(MODE), 1)
+lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
+                      int M, const int32_t* __restrict__ live_rows, int D, int V, int mask_col, int n_tiles,
+                      float* __restrict__ part_max, float* __restrict__ part_sum, int32_t* __restrict__ part_arg,
+                      uint32_t* __restrict__ dev_status, const LmSampling smp, int allow_pair, int swap_small) {
+    lm_rowmajor_body<MODE, PAIR>(tmap_x, tmap_w, M, live_rows, D, V, mask_col, n_tiles, part_max, part_sum, part_arg,
+                                 dev_status, smp, allow_pair, swap_small);
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Greedy head with the operands swapped: the VOCABULARY sits on the accumulator's lanes (W is the MMA's A operand,
+// 128 rows per CTA, 256 per CTA pair) and the live ROWS are its columns (the compacted X is the B operand,
+// N = the number of rows, any multiple of 16 up to 256).  What that buys over the row-major kernel above:
+//   * no padding to 128-row tiles: a step with 96 masked rows issues MMAs of N = 96, not of 128 padded rows;
+//   * every work item is a CTA pair whatever the row count, and the 128-row vocabulary tiles per CTA spread evenly
+//     over the SMs: with few rows left the W stream is the bound and the kernel reads it at the copy bandwidth.
+// It is used while at most SW_NMAX rows are live.  Above that the step is bound by the tensor pipe, where it does
+// not pay: an MMA reads its 128 x 16 A operand from shared memory in ~116 cycles whatever N is, so two chunks of
+// N = 144 cost what two chunks of N = 256 cost (measured: 319 us for 288 rows, 350 us for 512), and the row-major
+// kernel above, whose A operand is the row tile, does the same work in as many or fewer MMAs.
+// The price is the epilogue: a thread's TMEM lane is now a vocabulary entry and the softmax runs ACROSS lanes.
+// Each epilogue warp turns its 32 x 32 block of logits through shared memory (padded rows, conflict-free) so that
+// a thread again holds 32 consecutive vocabulary entries of ONE row, and keeps that row's running
+// (max, sum, argmax) in registers across the group's tiles: 8 column blocks x 3 values per thread.  At the end of
+// an item the four epilogue warps fold their values through the same shared memory, and one partial per (row,
+// vocabulary group, CTA of the pair) goes to the merge kernel.
+constexpr int SW_BV = 128;                               // vocabulary rows per CTA and tile
+constexpr int SW_NMAX = 256;                             // rows (accumulator columns) per chunk
+constexpr int SW_STAGES = 6;
+constexpr int SW_W_BYTES = SW_BV * BK * 2;               // 16 KB
+constexpr int SW_X_BYTES = (SW_NMAX / 2) * BK * 2;       // each CTA loads half of the chunk's rows: up to 16 KB
+constexpr int SW_STAGE_BYTES = SW_W_BYTES + SW_X_BYTES;
+constexpr int SW_XP_FLOATS = 32 * 33;                    // per epilogue warp: one 32 x 32 block, rows padded to 33
+constexpr int SW_PARTS_PER_GROUP = 2;                    // one per CTA of the pair
+struct SwBarriers {
+    uint64_t full[SW_STAGES];
+    uint64_t empty[SW_STAGES];
+    uint64_t tmem_full[2];
+    uint64_t tmem_empty[2];
+    uint64_t fold_full, fold_empty;                      // the epilogue warps' exchange at the end of an item
+    uint32_t tmem_base;
+    uint32_t abort_flag;
+};
+constexpr int SW_SMEM_BYTES = SW_STAGES * SW_STAGE_BYTES + 4 * SW_XP_FLOATS * 4 + static_cast<int>(sizeof(SwBarriers)) + 1024;
+// X tiles of 128, 64, 32, 16 and 8 rows: a CTA's share of a chunk (a multiple of 8 rows) is covered by one or two
+// of them, stacked in shared memory (each a whole number of 1 KB swizzle atoms); a few rows too many may be loaded,
+// the MMA reads only its own.  (Exact covers of up to four boxes were measured slower: 432 us for 480 rows, where
+// each CTA loaded 64 + 32 + 16 + 8 rows per stage, against 350 us for 512 rows with one box.)
+struct SwXMaps { CUtensorMap m[5]; };
+struct SwBoxes { int i1, i2, rows; };      // indices into SwXMaps::m (i2 < 0: one box), rows loaded in all
+__device__ __forceinline__ SwBoxes sw_boxes(int rows_half) {
+    int single = 0;                        // smallest box that holds the rows
+    while ((128 >> single) >= 2 * rows_half && single < 4) ++single;
+    int first = single + 1;                // largest box below that, plus the smallest box for the remainder
+    SwBoxes b = {single, -1, 128 >> single};
+    if (first <= 4) {
+        const int rem = rows_half - (128 >> first);
+        if (rem > 0) {
+            int second = 4;
+            while ((128 >> second) < rem) --second;
+            if ((128 >> first) + (128 >> second) < (128 >> single)) { b.i1 = first; b.i2 = second; b.rows = (128 >> first) + (128 >> second); }
+        }
+    }
+    return b;
+}
+
+// How `rows` live rows are cut up for a grid of n_units CTA pairs and n_vt vocabulary tiles of 256 (the same
+// formula on the host, in the GEMM and in the merge kernels).
+struct SwPlan { int n_chunks, nc, groups, parts; };
+__host__ __device__ inline SwPlan sw_plan(int rows, int n_units, int n_vt) {
+    SwPlan p;
+    p.n_chunks = (rows + SW_NMAX - 1) / SW_NMAX;
+    if (p.n_chunks < 1) p.n_chunks = 1;
+    const int per = (rows + p.n_chunks - 1) / p.n_chunks;
+    p.nc = (per + 15) & ~15;                             // rows per chunk: N of the pair's MMA
+    if (p.nc < 16) p.nc = 16;
+    p.groups = lm_groups(n_units, p.n_chunks, n_vt);
+    p.parts = SW_PARTS_PER_GROUP * p.groups;
+    return p;
+}
+
+__device__ __forceinline__ void
+lm_swapped_body(const CUtensorMap& tmap_w, const SwXMaps& xmaps, int Mc, int D, int V, int mask_col, int n_vt,
+                float* __restrict__ part_max, float* __restrict__ part_sum, int32_t* __restrict__ part_arg,
+                uint32_t* __restrict__ dev_status) {
+    if (Mc <= 0) return;
+    const int rank = static_cast<int>(cluster_cta_rank());
+    const int unit = blockIdx.x >> 1;
+    const int n_units = gridDim.x >> 1;
+    const SwPlan plan = sw_plan(Mc, n_units, n_vt);
+    const int n_items = plan.n_chunks * plan.groups;
+    if (unit >= n_items) return;                         // (both CTAs of a pair alike)
+    const int nc = plan.nc, groups = plan.groups;
+    const int rows_half = nc >> 1;                       // this CTA's share of a chunk's rows (multiple of 8)
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    float* xpose = reinterpret_cast<float*>(tiles + SW_STAGES * SW_STAGE_BYTES);
+    SwBarriers* bars = reinterpret_cast<SwBarriers*>(xpose + 4 * SW_XP_FLOATS);
+    volatile uint32_t* abort_flag = &bars->abort_flag;
+
+    const int warp = warp_index_uniform();
+    const int lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < SW_STAGES; ++s) {
+            mbar_init(&bars->full[s], 1);
+            mbar_init(&bars->empty[s], 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(&bars->tmem_full[a], 1);
+            mbar_init(&bars->tmem_empty[a], 8);          // one arrival per epilogue warp of both CTAs
+        }
+        mbar_init(&bars->fold_full, 128);
+        mbar_init(&bars->fold_empty, 128);
+        bars->abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) { tmem_alloc_pair(&bars->tmem_base, TMEM_COLS); tmem_relinquish_pair(); }
+    tc_fence_before_sync();
+    cluster_sync_all();                                  // both CTAs' barriers exist before either signals the other's
+    tc_fence_after_sync();
+    const uint32_t tmem_base = bars->tmem_base;
+    const int num_k = (D + BK - 1) / BK;
+
+    // item w -> chunk w % n_chunks, vocabulary group w / n_chunks; the group's tiles are g, g + groups, ...
+    if (warp == 0) {
+        if (lane == 0) {
+            prefetch_tensormap(&tmap_w);
+#pragma unroll
+            for (int i = 0; i < 5; ++i) prefetch_tensormap(&xmaps.m[i]);
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            const uint32_t full0 = cluster_map_shared(smem_u32(&bars->full[0]), 0);   // the even CTA's barriers count both CTAs' bytes
+            const SwBoxes box = sw_boxes(rows_half);
+            const uint32_t stage_tx = 2u * static_cast<uint32_t>(SW_W_BYTES + box.rows * 128);
+            for (int item = unit; item < n_items && ok; item += n_units) {
+                const int x_row0 = (item % plan.n_chunks) * nc + rank * rows_half;
+                for (int vt = item / plan.n_chunks; vt < n_vt && ok; vt += groups) {
+                    const int w_row0 = vt * (2 * SW_BV) + rank * SW_BV;
+                    for (int kb = 0; kb < num_k; ++kb) {
+                        if (!mbar_wait(&bars->empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
+                        uint8_t* w_dst = tiles + stage * SW_STAGE_BYTES;
+                        uint8_t* x_dst = w_dst + SW_W_BYTES;
+                        const uint32_t full = full0 + stage * static_cast<uint32_t>(sizeof(uint64_t));
+                        if (rank == 0) mbar_arrive_expect_tx(&bars->full[stage], stage_tx);
+                        tma_load_2d_pair(w_dst, &tmap_w, full, kb * BK, w_row0);
+                        tma_load_2d_pair(x_dst, &xmaps.m[box.i1], full, kb * BK, x_row0);
+                        if (box.i2 >= 0)
+                            tma_load_2d_pair(x_dst + (128 >> box.i1) * 128, &xmaps.m[box.i2], full, kb * BK,
+                                             x_row0 + (128 >> box.i1));
+                        if (++stage == SW_STAGES) { stage = 0; phase ^= 1; }
+                    }
+                }
+            }
+        }
+    } else if (warp == 1 && rank == 0) {
+        // all lanes run the loops, one elected lane issues the MMAs of the pair and their commits
+        const bool leader = elect_one_sync();
+        const uint32_t idesc = umma_idesc_bf16(2 * SW_BV, nc);
+        int stage = 0;
+        uint32_t phase = 0;
+        int it = 0;
+        bool ok = true;
+        for (int item = unit; item < n_items && ok; item += n_units) {
+            for (int vt = item / plan.n_chunks; vt < n_vt && ok; vt += groups, ++it) {
+                const int acc = it & 1;
+                const uint32_t acc_phase = (it >> 1) & 1;
+                ok = __all_sync(0xffffffffu, mbar_wait(&bars->tmem_empty[acc], acc_phase ^ 1, abort_flag));
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + acc * SW_NMAX;
+                for (int kb = 0; kb < num_k; ++kb) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(&bars->full[stage], phase, abort_flag));
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const uint32_t w_addr = smem_u32(tiles + stage * SW_STAGE_BYTES);
+                    const uint64_t a_desc = umma_desc_sw128_kmajor(w_addr);
+                    const uint64_t b_desc = umma_desc_sw128_kmajor(w_addr + SW_W_BYTES);
+                    if (leader) {
+#pragma unroll
+                        for (int kk = 0; kk < BK / 16; ++kk)
+                            umma_bf16_pair(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (kb | kk) != 0);
+                        umma_commit_pair(&bars->empty[stage], 3);      // frees the stage in both CTAs
+                    }
+                    __syncwarp();
+                    if (++stage == SW_STAGES) { stage = 0; phase ^= 1; }
+                }
+                if (ok && leader) umma_commit_pair(&bars->tmem_full[acc], 3);
+                __syncwarp();
+            }
+        }
+    } else if (warp >= 2) {
+        // epilogue: warp w may touch TMEM lanes [32 * (w % 4), +32) = 32 consecutive vocabulary entries of the tile
+        const int lq = warp & 3;
+        float* xp = xpose + lq * SW_XP_FLOATS;
+        int it = 0;
+        uint32_t items_done = 0;
+        bool ok = true;
+        for (int item = unit; item < n_items && ok; item += n_units, ++items_done) {
+            const int chunk = item % plan.n_chunks;
+            const int group = item / plan.n_chunks;
+            float run_max[SW_NMAX / 32], run_sum[SW_NMAX / 32];
+            int run_arg[SW_NMAX / 32];
+#pragma unroll
+            for (int cb = 0; cb < SW_NMAX / 32; ++cb) { run_max[cb] = -INFINITY; run_sum[cb] = 0.f; run_arg[cb] = ARG_NONE; }
+            for (int vt = group; vt < n_vt && ok; vt += groups, ++it) {
+                const int acc = it & 1;
+                const uint32_t acc_phase = (it >> 1) & 1;
+                ok = __all_sync(0xffffffffu, mbar_wait(&bars->tmem_full[acc], acc_phase, abort_flag));
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t taddr = tmem_base + (static_cast<uint32_t>(lq * 32) << 16) + acc * SW_NMAX;
+                const int vbase = vt * (2 * SW_BV) + rank * SW_BV + lq * 32;     // first vocabulary entry of this warp's lanes
+                const bool edge = (vbase + 32 > V) || (mask_col >= vbase && mask_col < vbase + 32);
+                if (vbase < V) {
+#pragma unroll
+                    for (int cb = 0; cb < SW_NMAX / 32; ++cb) {
+                        if (cb * 32 < nc) {
+                            uint32_t v[32];
+                            tmem_ld_32cols(taddr + cb * 32, v);
+                            tmem_ld_wait();
+                            // turn the block: in, thread = vocabulary entry with 32 rows; out, thread = row with 32 entries
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) xp[lane * 33 + c] = __uint_as_float(v[c]);
+                            __syncwarp();
+                            float z[32];
+#pragma unroll
+                            for (int l = 0; l < 32; ++l) z[l] = xp[l * 33 + lane];
+                            __syncwarp();
+                            if (edge) {
+#pragma unroll
+                                for (int l = 0; l < 32; ++l)
+                                    if (vbase + l >= V || vbase + l == mask_col) z[l] = -INFINITY;
+                            }
+                            float cmax = -INFINITY;
+                            int carg = ARG_NONE;
+#pragma unroll
+                            for (int l = 0; l < 32; ++l)
+                                if (z[l] > cmax) { cmax = z[l]; carg = vbase + l; }       // strict '>' keeps the lowest id
+                            if (cmax > -INFINITY) {
+                                if (cmax > run_max[cb]) {     // tiles of a group come in ascending order: '>' keeps the lowest id
+                                    run_sum[cb] *= fast_exp2((run_max[cb] - cmax) * LOG2E);   // exp2(-inf) = 0 the first time
+                                    run_max[cb] = cmax;
+                                    run_arg[cb] = carg;
+                                }
+                                const float mb = run_max[cb] * LOG2E;
+                                float sum = 0.f;
+#pragma unroll
+                                for (int l = 0; l < 32; ++l) sum += fast_exp2(fmaf(z[l], LOG2E, -mb));
+                                run_sum[cb] += sum;
+                            }
+                        }
+                    }
+                }
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(&bars->tmem_empty[acc], 0);   // one arrival per warp, on the even CTA's barrier
+            }
+            if (ok) {
+                // fold the four warps' values (each saw a quarter of every tile's vocabulary entries): every warp
+                // leaves its own in its block of shared memory, then warp q folds column blocks 2 q and 2 q + 1
+#pragma unroll
+                for (int cb = 0; cb < SW_NMAX / 32; ++cb) {
+                    xp[(cb * 3 + 0) * 32 + lane] = run_max[cb];
+                    xp[(cb * 3 + 1) * 32 + lane] = run_sum[cb];
+                    xp[(cb * 3 + 2) * 32 + lane] = __int_as_float(run_arg[cb]);
+                }
+                mbar_arrive(&bars->fold_full);            // (release: the values above are visible to the waiters)
+                ok = __all_sync(0xffffffffu, mbar_wait(&bars->fold_full, items_done & 1, abort_flag));
+                if (ok) {
+                    for (int cb = 2 * lq; cb < 2 * lq + 2; ++cb) {
+                        const int col = cb * 32 + lane;
+                        const int row = chunk * nc + col;
+                        if (col < nc && row < Mc) {
+                            float m = -INFINITY, sum = 0.f;
+                            int a = ARG_NONE;
+                            for (int q = 0; q < 4; ++q) {
+                                const float* src = xpose + q * SW_XP_FLOATS + cb * 96 + lane;
+                                const float m2 = src[0], s2 = src[32];
+                                const int a2 = __float_as_int(src[64]);
+                                if (m2 > -INFINITY) {
+                                    if (m2 > m) { sum = sum * fast_exp2((m - m2) * LOG2E) + s2; m = m2; a = a2; }
+                                    else { sum += s2 * fast_exp2((m2 - m) * LOG2E); if (m2 == m && a2 < a) a = a2; }
+                                }
+                            }
+                            const size_t o = static_cast<size_t>(row) * plan.parts + group * 2 + rank;
+                            part_max[o] = m;
+                            part_sum[o] = sum;
+                            part_arg[o] = a;
+                        }
+                    }
+                    mbar_arrive(&bars->fold_empty);       // the blocks may be written again once all have read
+                    ok = __all_sync(0xffffffffu, mbar_wait(&bars->fold_empty, items_done & 1, abort_flag));
+                }
+            }
+        }
+    }
+
+    // teardown: neither CTA leaves while its partner can still signal its barriers or read its tiles
+    tc_fence_before_sync();
+    cluster_sync_all();
+    if (*abort_flag) {
+        // give copies still in flight time to land before the shared memory is released
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) {}
+        if (threadIdx.x == 0) atomicOr(dev_status, DEV_WAIT_EXPIRED);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc_pair(tmem_base, TMEM_COLS);
+    }
+}
+
+// The greedy head on CTA pairs: while few rows are live the swapped-operand path, otherwise the row-major pair
+// path (which returns at once when the row tiles call for single CTAs: that kernel is enqueued behind this one).
+// The W tile is the same for both: 128 rows per CTA.
+__global__ void __launch_bounds__(LM_THREADS, 1)
+lmhead_greedy_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ SwXMaps xmaps, int M,
+                          const int32_t* __restrict__ live_rows, int D, int V, int mask_col, int n_tiles,
+                          float* __restrict__ part_max, float* __restrict__ part_sum, int32_t* __restrict__ part_arg,
+                          uint32_t* __restrict__ dev_status) {
+    const int Mc = live_rows ? *live_rows : M;          // rows that need logits (uniform over the grid)
+    if (Mc <= SW_NMAX) {
+        lm_swapped_body(tmap_w, xmaps, Mc, D, V, mask_col, n_tiles, part_max, part_sum, part_arg, dev_status);
+    } else {
+        const LmSampling none = {};
+        lm_rowmajor_body<LM_GREEDY, true>(xmaps.m[0], tmap_w, M, live_rows, D, V, mask_col, n_tiles, part_max, part_sum,
+                                          part_arg, dev_status, none, 1, 1);
+    }
+}
+
+// Partials per live row, as the GEMM that ran wrote them.  layout 0 / 1: the row-major kernel (single CTAs only /
+// CTA pairs where they pay), one partial per vocabulary group.  layout 2: the greedy head's pair of kernels: the
+// swapped path (two partials per vocabulary group of a CTA pair) while at most SW_NMAX rows are live, the
+// row-major kernels above that.  `grid` = CTAs of the GEMM launch, n_tiles = vocabulary tiles of 256.
+constexpr int LM_LAYOUT_HYBRID = 2;
+__host__ __device__ inline int lm_partials_per_row(int layout, int grid, int rows, int n_tiles) {
+    if (layout == LM_LAYOUT_HYBRID) {
+        if (rows <= SW_NMAX) return sw_plan(rows, grid >> 1, n_tiles).parts;
+        layout = 1;
+    }
+    return lm_groups_mode(grid, (rows + BM - 1) / BM, n_tiles, layout);
+}
+
 // Fold of one row's partial triples by a warp: returns (argmax token, sum of exp relative to the maximum) in all
 // lanes.  Ties of the maximum go to the lowest token id.
 __device__ __forceinline__ void merge_row_partials(const float* __restrict__ part_max, const float* __restrict__ part_sum,
@@ -517,13 +869,28 @@ __device__ __forceinline__ void merge_row_partials(const float* __restrict__ par
                                                    int& a_out, float& s_out) {
     float m = -INFINITY, s = 0.f;
     int a = ARG_NONE;
-    for (int t = lane; t < groups; t += 32) {
-        const float m2 = part_max[base + t];
-        const float s2 = part_sum[base + t];
-        const int a2 = part_arg[base + t];
-        if (m2 > -INFINITY) {
-            if (m2 > m) { s = s * exp2f((m - m2) * LOG2E) + s2; m = m2; a = a2; }
-            else { s += s2 * exp2f((m2 - m) * LOG2E); if (m2 == m && a2 < a) a = a2; }
+    // the loads of a batch are issued together (five per lane cover 160 partials: one round trip to memory for the
+    // usual case), then folded
+    constexpr int BATCH = 5;
+    for (int t0 = lane; t0 < groups; t0 += 32 * BATCH) {
+        float bm[BATCH], bs[BATCH];
+        int ba[BATCH];
+#pragma unroll
+        for (int u = 0; u < BATCH; ++u) {
+            const int t = t0 + 32 * u;
+            const bool in = t < groups;
+            bm[u] = in ? part_max[base + t] : -INFINITY;
+            bs[u] = in ? part_sum[base + t] : 0.f;
+            ba[u] = in ? part_arg[base + t] : ARG_NONE;
+        }
+#pragma unroll
+        for (int u = 0; u < BATCH; ++u) {
+            const float m2 = bm[u], s2 = bs[u];
+            const int a2 = ba[u];
+            if (m2 > -INFINITY) {
+                if (m2 > m) { s = s * exp2f((m - m2) * LOG2E) + s2; m = m2; a = a2; }
+                else { s += s2 * exp2f((m2 - m) * LOG2E); if (m2 == m && a2 < a) a = a2; }
+            }
         }
     }
 #pragma unroll
@@ -550,7 +917,7 @@ __global__ void lmhead_merge_kernel(const float* __restrict__ part_max, const fl
     const int lane = threadIdx.x & 31;
     const int Mc = live_rows ? *live_rows : M;
     if (c >= Mc) return;
-    const int groups = lm_groups_mode(grid_gemm, (Mc + BM - 1) / BM, n_tiles, allow_pair);
+    const int groups = lm_partials_per_row(allow_pair, grid_gemm, Mc, n_tiles);
     int a;
     float s;
     merge_row_partials(part_max, part_sum, part_arg, static_cast<size_t>(c) * groups, groups, lane, a, s);
@@ -603,7 +970,7 @@ lmhead_merge_select_kernel(const float* __restrict__ part_max, const float* __re
     if (masked) {
         int c = s_before;
         for (int i = 0; i < warp; ++i) c += s_flag[i];
-        const int groups = lm_groups_mode(grid_gemm, (Mc + BM - 1) / BM, n_tiles, allow_pair);
+        const int groups = lm_partials_per_row(allow_pair, grid_gemm, Mc, n_tiles);
         int a;
         float s;
         merge_row_partials(part_max, part_sum, part_arg, static_cast<size_t>(c) * groups, groups, lane, a, s);
@@ -775,7 +1142,7 @@ int launch_partial(const dare_ctx* ctx, int grid, const CUtensorMap& tmap_x, con
         if (ensure_dynamic_smem(smem_set, lmhead_partial_kernel<MODE, false>, LM_SMEM_BYTES) != DARE_OK) return DARE_ERR_CUDA;
         lmhead_partial_kernel<MODE, false><<<grid, lm_threads(MODE), LM_SMEM_BYTES, stream>>>(
             tmap_x, tmap_w, M, live_rows, D, V, mask_col, n_tiles, part_max, part_sum, part_arg, ctx->dev_status, smp,
-            allow_pair); note_launch();
+            allow_pair, 0); note_launch();
         if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
     }
     if (run_pair) {
@@ -796,7 +1163,7 @@ int launch_partial(const dare_ctx* ctx, int grid, const CUtensorMap& tmap_x, con
         cfg.attrs = &attr;
         cfg.numAttrs = 1;
         if (cudaLaunchKernelEx(&cfg, lmhead_partial_kernel<MODE, true>, tmap_x, tmap_wh, M, live_rows, D, V, mask_col,
-                               n_tiles, part_max, part_sum, part_arg, ctx->dev_status, smp, allow_pair) != cudaSuccess)
+                               n_tiles, part_max, part_sum, part_arg, ctx->dev_status, smp, allow_pair, 0) != cudaSuccess)
             return DARE_ERR_CUDA;
         note_launch();
     }
@@ -810,6 +1177,10 @@ size_t lmhead_workspace_bytes(int M, int D, int V, int sm_count, bool with_row_t
     const size_t n_tiles = (static_cast<size_t>(V) + BN - 1) / BN;
     size_t groups = static_cast<size_t>(sm_count);
     if (groups > n_tiles) groups = n_tiles;
+    if (!sampling) {      // the greedy head's swapped path: two partials per vocabulary group of a CTA pair
+        groups = static_cast<size_t>(sm_count);
+        if (groups > 2 * n_tiles) groups = 2 * n_tiles;
+    }
     size_t bytes = (sampling ? 5 : 3) * sizeof(float) * groups * static_cast<size_t>(M);
     if (with_row_tokens)
         bytes += round_up(static_cast<size_t>(M) * D * 2, 1024) + round_up(static_cast<size_t>(M) * 4 + 4, 1024);
@@ -845,17 +1216,82 @@ int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M,
     }
     size_t groups_max = static_cast<size_t>(ctx->sm_count);
     if (groups_max > static_cast<size_t>(n_tiles)) groups_max = n_tiles;
+    const bool hybrid = sample == nullptr && grid >= 2 && lm_pair_available();
+    if (hybrid && groups_max < static_cast<size_t>(2 * n_tiles))      // the swapped path: two partials per group
+        groups_max = static_cast<size_t>(2 * n_tiles) < static_cast<size_t>(ctx->sm_count) ? 2 * n_tiles : ctx->sm_count;
     const size_t n_part = static_cast<size_t>(M) * groups_max;
     float* part_max = reinterpret_cast<float*>(cur);
     float* part_sum = part_max + n_part;
     int32_t* part_arg = reinterpret_cast<int32_t*>(part_sum + n_part);
 
-    CUtensorMap tmap_x;
-    int rc = make_tmap_bf16_2d(ctx, &tmap_x, x_gemm, static_cast<uint64_t>(M), static_cast<uint64_t>(D), BM, BK);
-    if (rc != DARE_OK) return rc;
-
     const int mask_col = (exclude_mask_column && mask_id >= 0 && mask_id < V) ? mask_id : -1;
     const int rows_per_block = 8;
+    int rc = DARE_OK;
+    if (hybrid) {
+        // which kernels can have work: known when the row count is (no row_tokens), otherwise both are enqueued
+        const bool rows_known = live_rows == nullptr;
+        const bool need_pair = !rows_known || M <= SW_NMAX || lm_pair_mode(m_tiles_max, 1);
+        const bool need_single = !rows_known ? m_tiles_max >= 3 : (M > SW_NMAX && !lm_pair_mode(m_tiles_max, 1));
+        CUtensorMap tmap_w;
+        SwXMaps xm;
+        rc = make_tmap_bf16_2d(ctx, &tmap_w, w, static_cast<uint64_t>(V), static_cast<uint64_t>(D), SW_BV, BK);
+        for (int i = 0; i < 5 && rc == DARE_OK; ++i)
+            rc = make_tmap_bf16_2d(ctx, &xm.m[i], x_gemm, static_cast<uint64_t>(M), static_cast<uint64_t>(D), 128u >> i, BK);
+        if (rc != DARE_OK) return rc;
+        const int grid_pair = grid & ~1;
+        if (need_pair) {
+            constexpr int SMEM = SW_SMEM_BYTES > LM_PAIR_SMEM_BYTES ? SW_SMEM_BYTES : LM_PAIR_SMEM_BYTES;
+            static std::atomic<uint64_t> smem_set_hybrid{0};
+            if (ensure_dynamic_smem(smem_set_hybrid, lmhead_greedy_pair_kernel, SMEM) != DARE_OK) return DARE_ERR_CUDA;
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(static_cast<unsigned>(grid_pair), 1, 1);
+            cfg.blockDim = dim3(LM_THREADS, 1, 1);
+            cfg.dynamicSmemBytes = SMEM;
+            cfg.stream = stream;
+            cudaLaunchAttribute attr;
+            attr.id = cudaLaunchAttributeClusterDimension;
+            attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+            cfg.attrs = &attr;
+            cfg.numAttrs = 1;
+            if (cudaLaunchKernelEx(&cfg, lmhead_greedy_pair_kernel, tmap_w, xm, M, static_cast<const int32_t*>(live_rows), D,
+                                   V, mask_col, n_tiles, part_max, part_sum, part_arg, ctx->dev_status) != cudaSuccess)
+                return DARE_ERR_CUDA;
+            note_launch();
+        }
+        if (need_single) {
+            CUtensorMap tmap_w256;
+            rc = make_tmap_bf16_2d(ctx, &tmap_w256, w, static_cast<uint64_t>(V), static_cast<uint64_t>(D), BN, BK);
+            if (rc != DARE_OK) return rc;
+            static std::atomic<uint64_t> smem_set_single{0};
+            if (ensure_dynamic_smem(smem_set_single, lmhead_partial_kernel<LM_GREEDY, false>, LM_SMEM_BYTES) != DARE_OK)
+                return DARE_ERR_CUDA;
+            const LmSampling none = {};
+            lmhead_partial_kernel<LM_GREEDY, false><<<grid_pair, LM_THREADS, LM_SMEM_BYTES, stream>>>(
+                xm.m[0], tmap_w256, M, live_rows, D, V, mask_col, n_tiles, part_max, part_sum, part_arg, ctx->dev_status,
+                none, 1, 1);
+            if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
+            note_launch();
+        }
+        if (select) {
+            LmSelect sel;
+            sel.tokens_block = select->tokens_block; sel.row_stride = tok_row_stride; sel.mode = select->mode;
+            sel.threshold = select->threshold; sel.k = select->k;
+            sel.n_committed = select->n_committed; sel.n_remaining = select->n_remaining;
+            lmhead_merge_select_kernel<<<select->B, 32 * tok_L, 0, stream>>>(part_max, part_sum, part_arg, grid_pair, n_tiles,
+                                                                             tok_L, live_rows, idx, mask_id, pred, conf,
+                                                                             LM_LAYOUT_HYBRID, sel);
+        } else {
+            lmhead_merge_kernel<<<(M + rows_per_block - 1) / rows_per_block, rows_per_block * 32, 0, stream>>>(
+                part_max, part_sum, part_arg, grid_pair, n_tiles, M, live_rows, idx, pred, conf, LM_LAYOUT_HYBRID);
+        }
+        note_launch();
+        return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
+    }
+
+    CUtensorMap tmap_x;
+    rc = make_tmap_bf16_2d(ctx, &tmap_x, x_gemm, static_cast<uint64_t>(M), static_cast<uint64_t>(D), BM, BK);
+    if (rc != DARE_OK) return rc;
+
     LmSampling smp = {};
     int allow_pair = 0;
     if (sample == nullptr) {

@@ -107,15 +107,20 @@ def test_lmhead_without_exclusion_and_with_committed_rows(ctx):
 
 
 @pytest.mark.parametrize("M,D,V,mu,with_rows", [
-    (256, 320, 2600, 7, False),        # two row tiles known on the host: the CTA-pair kernel alone is launched
-    (500, 128, 1000, 999, False),      # four row tiles, ragged last one
-    (600, 256, 2048, 5, True),         # 200 masked rows = two tiles, known only on the device: pairs do the work
-    (1400, 64, 1200, 3, True),         # 467 masked rows = four tiles
+    (256, 320, 2600, 7, False),        # 256 rows known on the host: the swapped-operand path (vocabulary on the lanes)
+    (500, 128, 1000, 999, False),      # four row tiles, ragged last one: row-major CTA pairs
+    (600, 256, 2048, 5, True),         # 200 masked rows, known only on the device: swapped path, N = 208
+    (1400, 64, 1200, 3, True),         # 467 masked rows = four tiles: pairs
     (900, 64, 1200, 3, True),          # 300 masked rows = three tiles: the single-CTA kernel does the work
+    (640, 128, 1000, 999, False),      # five row tiles known on the host: single CTAs
+    (1900, 64, 1200, 3, True),         # ~634 masked rows = five tiles, known only on the device
+    (72, 200, 700, 0, False),          # swapped path, each CTA of a pair loads 40 rows as boxes of 32 + 8
+    (330, 64, 520, 519, True),         # 110 masked rows: N = 112, one box of 64 rows per CTA covers its 56
 ])
 def test_lmhead_single_and_pair_modes(ctx, M, D, V, mu, with_rows):
-    """The LM-head GEMM has a single-CTA and a CTA-pair instantiation; which one works depends on the number of
-    128-row tiles of masked rows (even: pairs), decided on the device when rows are skipped."""
+    """The greedy head has three GEMM paths, picked by the number of live rows (on the device when rows are skipped):
+    up to 256 rows the swapped-operand path on CTA pairs; above that row-major tiles of 128 rows, on CTA pairs when
+    the tiles come in twos, on single CTAs otherwise."""
     _lm_case(ctx, M, D, V, mu, seed=M + D, with_rows=with_rows)
 
 
