@@ -234,17 +234,20 @@ attn_block_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_cons
                         mma_bf16_16816(sacc[nb], qf[2 * kq + 1], r2, r3);
                     }
                 }
-                // scale into the log2 domain, mask keys that do not exist, row max
+                // mask keys that do not exist (only a segment's last tile has any), row max.  The scores stay
+                // unscaled: the softmax scale (times log2 e) goes into the exponent's multiply-add below, and
+                // the running max m0 / m1 is kept in score units until the tiles are done.
+                if (ti.valid < koff + KPW) {
+#pragma unroll
+                    for (int nb = 0; nb < KPW / 8; ++nb) {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            if (koff + nb * 8 + tq * 2 + (e & 1) >= ti.valid) sacc[nb][e] = -INFINITY;
+                    }
+                }
                 float tmax0 = -INFINITY, tmax1 = -INFINITY;
 #pragma unroll
                 for (int nb = 0; nb < KPW / 8; ++nb) {
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int key = koff + nb * 8 + tq * 2 + (e & 1);
-                        float sv = sacc[nb][e] * p.scale_log2;
-                        if (key >= ti.valid) sv = -INFINITY;
-                        sacc[nb][e] = sv;
-                    }
                     tmax0 = fmaxf(tmax0, fmaxf(sacc[nb][0], sacc[nb][1]));
                     tmax1 = fmaxf(tmax1, fmaxf(sacc[nb][2], sacc[nb][3]));
                 }
@@ -253,26 +256,33 @@ attn_block_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_cons
                 tmax1 = fmaxf(tmax1, __shfl_xor_sync(0xffffffffu, tmax1, 1));
                 tmax1 = fmaxf(tmax1, __shfl_xor_sync(0xffffffffu, tmax1, 2));
                 const float mn0 = fmaxf(m0, tmax0), mn1 = fmaxf(m1, tmax1);   // finite: the slice has >= 1 key
-                const float a0 = fast_exp2(m0 - mn0), a1 = fast_exp2(m1 - mn1);
-                m0 = mn0; m1 = mn1;
+                const bool moved = __any_sync(0xffffffffu, mn0 != m0 || mn1 != m1);
+                const float c = p.scale_log2;
+                const float nb0 = -mn0 * c, nb1 = -mn1 * c;
                 float ps0 = 0.f, ps1 = 0.f;
                 uint32_t pa[KPW / 16][4];
 #pragma unroll
                 for (int nb = 0; nb < KPW / 8; ++nb) {
-                    const float e0 = fast_exp2(sacc[nb][0] - mn0), e1 = fast_exp2(sacc[nb][1] - mn0);
-                    const float e2 = fast_exp2(sacc[nb][2] - mn1), e3 = fast_exp2(sacc[nb][3] - mn1);
+                    const float e0 = fast_exp2(fmaf(sacc[nb][0], c, nb0)), e1 = fast_exp2(fmaf(sacc[nb][1], c, nb0));
+                    const float e2 = fast_exp2(fmaf(sacc[nb][2], c, nb1)), e3 = fast_exp2(fmaf(sacc[nb][3], c, nb1));
                     ps0 += e0 + e1;
                     ps1 += e2 + e3;
                     pa[nb >> 1][(nb & 1) * 2 + 0] = pack_bf16(e0, e1);
                     pa[nb >> 1][(nb & 1) * 2 + 1] = pack_bf16(e2, e3);
                 }
-                l0 = l0 * a0 + ps0;
-                l1 = l1 * a1 + ps1;
+                if (moved) {   // (rare after the first tiles: a row's max over hundreds of keys settles early)
+                    const float a0 = fast_exp2((m0 - mn0) * c), a1 = fast_exp2((m1 - mn1) * c);
+                    m0 = mn0; m1 = mn1;
+                    l0 *= a0;
+                    l1 *= a1;
 #pragma unroll
-                for (int n = 0; n < D / 8; ++n) {
-                    oacc[n][0] *= a0; oacc[n][1] *= a0;
-                    oacc[n][2] *= a1; oacc[n][3] *= a1;
+                    for (int n = 0; n < D / 8; ++n) {
+                        oacc[n][0] *= a0; oacc[n][1] *= a0;
+                        oacc[n][2] *= a1; oacc[n][3] *= a1;
+                    }
                 }
+                l0 += ps0;
+                l1 += ps1;
                 // O += P V
 #pragma unroll
                 for (int kk = 0; kk < KPW / 16; ++kk) {
@@ -296,6 +306,8 @@ attn_block_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_cons
         l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
         l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
         l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+        m0 *= p.scale_log2;      // from here on the max is in the log2 domain (-inf stays -inf: the scale is > 0)
+        m1 *= p.scale_log2;
     }
 
     // ---------------- merge the key slices of a row group (through the now idle tile ring), then write out

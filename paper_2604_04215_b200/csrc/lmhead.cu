@@ -180,13 +180,18 @@ __device__ __forceinline__ float gumbel_from_word(uint32_t w) {
 // bf16 in both orientations (the two products of the backward pass take it from there); no partials.
 constexpr int LM_GREEDY = 0, LM_SAMPLE = 1, LM_LOGPROB = 2, LM_GRAD = 3;
 
-// swap_small: this launch leaves steps with at most SW_NMAX live rows to the swapped-operand path (further down).
-template <int MODE, bool PAIR>
+// The work of one launch, or of the part of a launch that runs this body: `n_units` units (CTAs, or CTA pairs with
+// PAIR), of which this CTA belongs to unit `unit`, walk the row tiles [tile0, tile0 + m_tiles) against all
+// vocabulary tiles; a row's partials start at row * parts_stride (parts_stride < 0: at row * groups, the packed
+// layout of the stand-alone kernels).  W_HALF_BOX: the W tensor map's box is 128 rows (half a tile), so a single
+// CTA fetches its 256-row tile as two boxes.
+struct LmUnits { int unit, n_units, tile0, m_tiles, parts_stride; };
+template <int MODE, bool PAIR, bool W_HALF_BOX = false>
 __device__ __forceinline__ void
 lm_rowmajor_body(const CUtensorMap& tmap_x, const CUtensorMap& tmap_w,
-                 int M, const int32_t* __restrict__ live_rows, int D, int V, int mask_col, int n_tiles,
+                 int Mc, int D, int V, int mask_col, int n_tiles,
                  float* __restrict__ part_max, float* __restrict__ part_sum, int32_t* __restrict__ part_arg,
-                 uint32_t* __restrict__ dev_status, const LmSampling& smp, int allow_pair, int swap_small) {
+                 uint32_t* __restrict__ dev_status, const LmSampling& smp, const LmUnits u) {
     constexpr int NSTAGES = PAIR ? PSTAGES : STAGES;
     constexpr int STAGE_SZ = PAIR ? PSTAGE_BYTES : STAGE_BYTES;
     using Barriers = typename std::conditional<PAIR, LmPairBarriers, LmBarriers>::type;
@@ -195,19 +200,16 @@ lm_rowmajor_body(const CUtensorMap& tmap_x, const CUtensorMap& tmap_w,
     constexpr bool GRAD = MODE == LM_GRAD;
     constexpr int EPI_SETS = SAMPLE ? 2 : 1;                 // sets of four epilogue warps
     __shared__ float s_exch[5][BM];                          // (max, sum, best y, its logit, its column) per row
-    const int Mc = live_rows ? *live_rows : M;          // rows that need logits (uniform over the grid)
-    const int m_tiles = (Mc + BM - 1) / BM;
-    if (m_tiles == 0) return;
-    if (swap_small && Mc <= 256) return;                          // the swapped-operand path does this launch's work
-    if (lm_pair_mode(m_tiles, allow_pair) != PAIR) return;        // the other kernel does this launch's work
+    if (u.m_tiles <= 0) return;
     // PAIR: a work unit is a cluster of two CTAs, an item two row tiles (one per CTA) and a vocabulary group
     const int rank = PAIR ? static_cast<int>(cluster_cta_rank()) : 0;
-    const int unit = PAIR ? blockIdx.x >> 1 : blockIdx.x;
-    const int n_units = PAIR ? gridDim.x >> 1 : gridDim.x;
-    const int item_rows = PAIR ? (m_tiles + 1) >> 1 : m_tiles;       // row tiles (pairs of them) to walk
+    const int unit = u.unit;
+    const int n_units = u.n_units;
+    const int item_rows = PAIR ? (u.m_tiles + 1) >> 1 : u.m_tiles;   // row tiles (pairs of them) to walk
     const int groups = lm_groups(n_units, item_rows, n_tiles);
     const int n_items = item_rows * groups;
     if (unit >= n_items) return;                                    // (both CTAs of a pair alike)
+    const int parts_stride = u.parts_stride < 0 ? groups : u.parts_stride;
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -254,7 +256,7 @@ lm_rowmajor_body(const CUtensorMap& tmap_x, const CUtensorMap& tmap_w,
             // PAIR: the even CTA's "full" barriers count the bytes of both CTAs' copies
             const uint32_t full0 = PAIR ? cluster_map_shared(smem_u32(&bars->full[0]), 0) : 0u;
             for (int item = unit; item < n_items && ok; item += n_units) {
-                const int m_tile = PAIR ? 2 * (item % item_rows) + rank : item % item_rows;
+                const int m_tile = u.tile0 + (PAIR ? 2 * (item % item_rows) + rank : item % item_rows);
                 for (int n_tile = item / item_rows; n_tile < n_tiles && ok; n_tile += groups) {
                     for (int kb = 0; kb < num_k; ++kb) {
                         if (!mbar_wait(&bars->empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
@@ -269,6 +271,8 @@ lm_rowmajor_body(const CUtensorMap& tmap_x, const CUtensorMap& tmap_w,
                             mbar_arrive_expect_tx(&bars->full[stage], STAGE_SZ);
                             tma_load_2d(a_dst, &tmap_x, &bars->full[stage], kb * BK, m_tile * BM);
                             tma_load_2d(b_dst, &tmap_w, &bars->full[stage], kb * BK, n_tile * BN);
+                            if (W_HALF_BOX)
+                                tma_load_2d(b_dst + (BN / 2) * BK * 2, &tmap_w, &bars->full[stage], kb * BK, n_tile * BN + BN / 2);
                         }
                         if (++stage == NSTAGES) { stage = 0; phase ^= 1; }
                     }
@@ -330,7 +334,7 @@ lm_rowmajor_body(const CUtensorMap& tmap_x, const CUtensorMap& tmap_w,
         int items_done = 0;
         bool ok = true;
         for (int item = unit; item < n_items && ok; item += n_units, ++items_done) {
-            const int m_tile = PAIR ? 2 * (item % item_rows) + rank : item % item_rows;
+            const int m_tile = u.tile0 + (PAIR ? 2 * (item % item_rows) + rank : item % item_rows);
             const int group = item / item_rows;
             float run_max = -INFINITY;
             float run_sum = 0.f;
@@ -487,7 +491,7 @@ lm_rowmajor_body(const CUtensorMap& tmap_x, const CUtensorMap& tmap_w,
             }
             const int row = m_tile * BM + row_in_tile;
             if (!GRAD && ok && row < Mc && set == 0) {
-                const size_t o = static_cast<size_t>(row) * groups + group;
+                const size_t o = static_cast<size_t>(row) * parts_stride + group;
                 part_max[o] = run_max;
                 part_sum[o] = run_sum;
                 part_arg[o] = LOGPROB ? __float_as_int(target_z) : run_arg;
@@ -519,9 +523,14 @@ __global__ void __launch_bounds__(lm_threads(MODE), 1)
 lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                       int M, const int32_t* __restrict__ live_rows, int D, int V, int mask_col, int n_tiles,
                       float* __restrict__ part_max, float* __restrict__ part_sum, int32_t* __restrict__ part_arg,
-                      uint32_t* __restrict__ dev_status, const LmSampling smp, int allow_pair, int swap_small) {
-    lm_rowmajor_body<MODE, PAIR>(tmap_x, tmap_w, M, live_rows, D, V, mask_col, n_tiles, part_max, part_sum, part_arg,
-                                 dev_status, smp, allow_pair, swap_small);
+                      uint32_t* __restrict__ dev_status, const LmSampling smp, int allow_pair) {
+    const int Mc = live_rows ? *live_rows : M;          // rows that need logits (uniform over the grid)
+    const int m_tiles = (Mc + BM - 1) / BM;
+    if (lm_pair_mode(m_tiles, allow_pair) != PAIR) return;        // the other kernel does this launch's work
+    const LmUnits u = {static_cast<int>(PAIR ? blockIdx.x >> 1 : blockIdx.x),
+                       static_cast<int>(PAIR ? gridDim.x >> 1 : gridDim.x), 0, m_tiles, -1};
+    lm_rowmajor_body<MODE, PAIR>(tmap_x, tmap_w, Mc, D, V, mask_col, n_tiles, part_max, part_sum, part_arg, dev_status,
+                                 smp, u);
 }
 
 // ---------------------------------------------------------------------------------------------------------
@@ -599,7 +608,7 @@ __host__ __device__ inline SwPlan sw_plan(int rows, int n_units, int n_vt) {
 __device__ __forceinline__ void
 lm_swapped_body(const CUtensorMap& tmap_w, const SwXMaps& xmaps, int Mc, int D, int V, int mask_col, int n_vt,
                 float* __restrict__ part_max, float* __restrict__ part_sum, int32_t* __restrict__ part_arg,
-                uint32_t* __restrict__ dev_status) {
+                uint32_t* __restrict__ dev_status, int parts_stride) {
     if (Mc <= 0) return;
     const int rank = static_cast<int>(cluster_cta_rank());
     const int unit = blockIdx.x >> 1;
@@ -802,7 +811,7 @@ lm_swapped_body(const CUtensorMap& tmap_w, const SwXMaps& xmaps, int Mc, int D, 
                                     else { sum += s2 * fast_exp2((m2 - m) * LOG2E); if (m2 == m && a2 < a) a = a2; }
                                 }
                             }
-                            const size_t o = static_cast<size_t>(row) * plan.parts + group * 2 + rank;
+                            const size_t o = static_cast<size_t>(row) * parts_stride + group * 2 + rank;
                             part_max[o] = m;
                             part_sum[o] = sum;
                             part_arg[o] = a;
@@ -831,35 +840,75 @@ lm_swapped_body(const CUtensorMap& tmap_w, const SwXMaps& xmaps, int Mc, int D, 
     }
 }
 
-// The greedy head on CTA pairs: while few rows are live the swapped-operand path, otherwise the row-major pair
-// path (which returns at once when the row tiles call for single CTAs: that kernel is enqueued behind this one).
-// The W tile is the same for both: 128 rows per CTA.
+// An odd number of row tiles, 2 p + 1, on n_clusters CTA pairs: the first lm_mixed_pair_clusters() clusters run the
+// row-major pair path on the tiles [0, 2 p), and the CTAs of the remaining clusters each run the single-CTA path on
+// the last tile.  The split balances the two parts: an item of two row tiles costs a pair one unit of time, an item
+// of one row tile costs a single CTA about 1.2 (its tensor pipe is busy 83 % of the time against 97 %), i.e. a
+// cluster of two such CTAs 0.6 per item.  (Same formula on the host, in the GEMM and in the merge kernels.)
+__host__ __device__ inline int lm_mixed_pair_clusters(int n_clusters, int p) {
+    int up = (n_clusters * 10 * p + 5 * p + 3) / (10 * p + 6);      // round(n_clusters * p / (p + 0.6))
+    if (up > n_clusters - 1) up = n_clusters - 1;
+    if (up < 1) up = 1;
+    return up;
+}
+
+// The greedy head, one launch on CTA pairs whatever the number of live rows (known only on the device when rows are
+// skipped): up to SW_NMAX rows the swapped-operand path; above that row-major tiles of 128 rows, on CTA pairs when
+// the tiles come in twos, and for an odd count on pairs plus single CTAs for the last tile (see above).  The W
+// tile box is 128 rows for all of them.  A row's partials start at row * parts_stride; how many there are follows
+// from the same rules in lm_row_partials.
 __global__ void __launch_bounds__(LM_THREADS, 1)
-lmhead_greedy_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ SwXMaps xmaps, int M,
-                          const int32_t* __restrict__ live_rows, int D, int V, int mask_col, int n_tiles,
-                          float* __restrict__ part_max, float* __restrict__ part_sum, int32_t* __restrict__ part_arg,
-                          uint32_t* __restrict__ dev_status) {
+lmhead_greedy_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ SwXMaps xmaps, int M,
+                     const int32_t* __restrict__ live_rows, int D, int V, int mask_col, int n_tiles,
+                     float* __restrict__ part_max, float* __restrict__ part_sum, int32_t* __restrict__ part_arg,
+                     uint32_t* __restrict__ dev_status, int parts_stride) {
     const int Mc = live_rows ? *live_rows : M;          // rows that need logits (uniform over the grid)
     if (Mc <= SW_NMAX) {
-        lm_swapped_body(tmap_w, xmaps, Mc, D, V, mask_col, n_tiles, part_max, part_sum, part_arg, dev_status);
+        lm_swapped_body(tmap_w, xmaps, Mc, D, V, mask_col, n_tiles, part_max, part_sum, part_arg, dev_status, parts_stride);
+        return;
+    }
+    const LmSampling none = {};
+    const int m_tiles = (Mc + BM - 1) / BM;
+    const int cluster = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
+    if ((m_tiles & 1) == 0) {
+        const LmUnits u = {cluster, n_clusters, 0, m_tiles, parts_stride};
+        lm_rowmajor_body<LM_GREEDY, true>(xmaps.m[0], tmap_w, Mc, D, V, mask_col, n_tiles, part_max, part_sum, part_arg,
+                                          dev_status, none, u);
+    } else if (n_clusters < 2) {
+        const LmUnits u = {static_cast<int>(blockIdx.x), static_cast<int>(gridDim.x), 0, m_tiles, parts_stride};
+        lm_rowmajor_body<LM_GREEDY, false, true>(xmaps.m[0], tmap_w, Mc, D, V, mask_col, n_tiles, part_max, part_sum,
+                                                 part_arg, dev_status, none, u);
     } else {
-        const LmSampling none = {};
-        lm_rowmajor_body<LM_GREEDY, true>(xmaps.m[0], tmap_w, M, live_rows, D, V, mask_col, n_tiles, part_max, part_sum,
-                                          part_arg, dev_status, none, 1, 1);
+        const int p = m_tiles >> 1;
+        const int up = lm_mixed_pair_clusters(n_clusters, p);
+        if (cluster < up) {
+            const LmUnits u = {cluster, up, 0, 2 * p, parts_stride};
+            lm_rowmajor_body<LM_GREEDY, true>(xmaps.m[0], tmap_w, Mc, D, V, mask_col, n_tiles, part_max, part_sum,
+                                              part_arg, dev_status, none, u);
+        } else {
+            const LmUnits u = {static_cast<int>(blockIdx.x) - 2 * up, static_cast<int>(gridDim.x) - 2 * up, 2 * p, 1,
+                               parts_stride};
+            lm_rowmajor_body<LM_GREEDY, false, true>(xmaps.m[0], tmap_w, Mc, D, V, mask_col, n_tiles, part_max, part_sum,
+                                                     part_arg, dev_status, none, u);
+        }
     }
 }
 
-// Partials per live row, as the GEMM that ran wrote them.  layout 0 / 1: the row-major kernel (single CTAs only /
-// CTA pairs where they pay), one partial per vocabulary group.  layout 2: the greedy head's pair of kernels: the
-// swapped path (two partials per vocabulary group of a CTA pair) while at most SW_NMAX rows are live, the
-// row-major kernels above that.  `grid` = CTAs of the GEMM launch, n_tiles = vocabulary tiles of 256.
-constexpr int LM_LAYOUT_HYBRID = 2;
-__host__ __device__ inline int lm_partials_per_row(int layout, int grid, int rows, int n_tiles) {
-    if (layout == LM_LAYOUT_HYBRID) {
-        if (rows <= SW_NMAX) return sw_plan(rows, grid >> 1, n_tiles).parts;
-        layout = 1;
-    }
-    return lm_groups_mode(grid, (rows + BM - 1) / BM, n_tiles, layout);
+// Partials of live row `row`, as the GEMM that ran wrote them (they start at row * stride).  layout 0 / 1: the
+// stand-alone row-major kernels (single CTAs only / CTA pairs where they apply), one partial per vocabulary group,
+// packed (stride = count).  layout 2: lmhead_greedy_kernel's rules.  `grid` = CTAs of the GEMM launch, n_tiles =
+// vocabulary tiles of 256.
+constexpr int LM_LAYOUT_GREEDY = 2;
+__host__ __device__ inline int lm_row_partials(int layout, int grid, int rows, int n_tiles, int row) {
+    const int m_tiles = (rows + BM - 1) / BM;
+    if (layout != LM_LAYOUT_GREEDY) return lm_groups_mode(grid, m_tiles, n_tiles, layout);
+    const int n_clusters = grid >> 1;
+    if (rows <= SW_NMAX) return sw_plan(rows, n_clusters, n_tiles).parts;
+    if ((m_tiles & 1) == 0) return lm_groups(n_clusters, m_tiles >> 1, n_tiles);
+    if (n_clusters < 2) return lm_groups(grid, m_tiles, n_tiles);
+    const int p = m_tiles >> 1;
+    const int up = lm_mixed_pair_clusters(n_clusters, p);
+    return row < 2 * p * BM ? lm_groups(up, p, n_tiles) : lm_groups(grid - 2 * up, 1, n_tiles);
 }
 
 // Fold of one row's partial triples by a warp: returns (argmax token, sum of exp relative to the maximum) in all
@@ -912,15 +961,17 @@ __device__ __forceinline__ void merge_row_partials(const float* __restrict__ par
 __global__ void lmhead_merge_kernel(const float* __restrict__ part_max, const float* __restrict__ part_sum,
                                     const int32_t* __restrict__ part_arg, int grid_gemm, int n_tiles, int M,
                                     const int32_t* __restrict__ live_rows, const int32_t* __restrict__ idx,
-                                    int32_t* __restrict__ pred, float* __restrict__ conf, int allow_pair) {
+                                    int32_t* __restrict__ pred, float* __restrict__ conf, int allow_pair,
+                                    int parts_stride) {
     const int c = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     const int Mc = live_rows ? *live_rows : M;
     if (c >= Mc) return;
-    const int groups = lm_partials_per_row(allow_pair, grid_gemm, Mc, n_tiles);
+    const int groups = lm_row_partials(allow_pair, grid_gemm, Mc, n_tiles, c);
     int a;
     float s;
-    merge_row_partials(part_max, part_sum, part_arg, static_cast<size_t>(c) * groups, groups, lane, a, s);
+    merge_row_partials(part_max, part_sum, part_arg, static_cast<size_t>(c) * (parts_stride < 0 ? groups : parts_stride),
+                       groups, lane, a, s);
     if (lane == 0) {
         const int row = idx ? idx[c] : c;
         pred[row] = a;
@@ -946,7 +997,8 @@ __global__ void __launch_bounds__(1024)
 lmhead_merge_select_kernel(const float* __restrict__ part_max, const float* __restrict__ part_sum,
                            const int32_t* __restrict__ part_arg, int grid_gemm, int n_tiles, int L,
                            const int32_t* __restrict__ live_rows, const int32_t* __restrict__ idx, int32_t mask_id,
-                           int32_t* __restrict__ pred, float* __restrict__ conf, int allow_pair, const LmSelect sel) {
+                           int32_t* __restrict__ pred, float* __restrict__ conf, int allow_pair, int parts_stride,
+                           const LmSelect sel) {
     __shared__ int s_before;
     __shared__ int s_flag[32];
     __shared__ float s_conf[32];
@@ -970,10 +1022,11 @@ lmhead_merge_select_kernel(const float* __restrict__ part_max, const float* __re
     if (masked) {
         int c = s_before;
         for (int i = 0; i < warp; ++i) c += s_flag[i];
-        const int groups = lm_partials_per_row(allow_pair, grid_gemm, Mc, n_tiles);
+        const int groups = lm_row_partials(allow_pair, grid_gemm, Mc, n_tiles, c);
         int a;
         float s;
-        merge_row_partials(part_max, part_sum, part_arg, static_cast<size_t>(c) * groups, groups, lane, a, s);
+        merge_row_partials(part_max, part_sum, part_arg, static_cast<size_t>(c) * (parts_stride < 0 ? groups : parts_stride),
+                           groups, lane, a, s);
         if (lane == 0) {
             float cf = 1.0f / s;
             pred[b * L + warp] = a;
@@ -1142,7 +1195,7 @@ int launch_partial(const dare_ctx* ctx, int grid, const CUtensorMap& tmap_x, con
         if (ensure_dynamic_smem(smem_set, lmhead_partial_kernel<MODE, false>, LM_SMEM_BYTES) != DARE_OK) return DARE_ERR_CUDA;
         lmhead_partial_kernel<MODE, false><<<grid, lm_threads(MODE), LM_SMEM_BYTES, stream>>>(
             tmap_x, tmap_w, M, live_rows, D, V, mask_col, n_tiles, part_max, part_sum, part_arg, ctx->dev_status, smp,
-            allow_pair, 0); note_launch();
+            allow_pair); note_launch();
         if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
     }
     if (run_pair) {
@@ -1163,7 +1216,7 @@ int launch_partial(const dare_ctx* ctx, int grid, const CUtensorMap& tmap_x, con
         cfg.attrs = &attr;
         cfg.numAttrs = 1;
         if (cudaLaunchKernelEx(&cfg, lmhead_partial_kernel<MODE, true>, tmap_x, tmap_wh, M, live_rows, D, V, mask_col,
-                               n_tiles, part_max, part_sum, part_arg, ctx->dev_status, smp, allow_pair, 0) != cudaSuccess)
+                               n_tiles, part_max, part_sum, part_arg, ctx->dev_status, smp, allow_pair) != cudaSuccess)
             return DARE_ERR_CUDA;
         note_launch();
     }
@@ -1216,9 +1269,11 @@ int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M,
     }
     size_t groups_max = static_cast<size_t>(ctx->sm_count);
     if (groups_max > static_cast<size_t>(n_tiles)) groups_max = n_tiles;
-    const bool hybrid = sample == nullptr && grid >= 2 && lm_pair_available();
-    if (hybrid && groups_max < static_cast<size_t>(2 * n_tiles))      // the swapped path: two partials per group
-        groups_max = static_cast<size_t>(2 * n_tiles) < static_cast<size_t>(ctx->sm_count) ? 2 * n_tiles : ctx->sm_count;
+    const bool greedy_pairs = sample == nullptr && grid >= 2 && lm_pair_available();
+    if (greedy_pairs) {      // lmhead_greedy_kernel: a fixed stride, at most min(#CTAs, 2 per vocabulary tile) partials
+        groups_max = static_cast<size_t>(grid & ~1);
+        if (groups_max > static_cast<size_t>(2 * n_tiles)) groups_max = 2 * n_tiles;
+    }
     const size_t n_part = static_cast<size_t>(M) * groups_max;
     float* part_max = reinterpret_cast<float*>(cur);
     float* part_sum = part_max + n_part;
@@ -1227,11 +1282,7 @@ int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M,
     const int mask_col = (exclude_mask_column && mask_id >= 0 && mask_id < V) ? mask_id : -1;
     const int rows_per_block = 8;
     int rc = DARE_OK;
-    if (hybrid) {
-        // which kernels can have work: known when the row count is (no row_tokens), otherwise both are enqueued
-        const bool rows_known = live_rows == nullptr;
-        const bool need_pair = !rows_known || M <= SW_NMAX || lm_pair_mode(m_tiles_max, 1);
-        const bool need_single = !rows_known ? m_tiles_max >= 3 : (M > SW_NMAX && !lm_pair_mode(m_tiles_max, 1));
+    if (greedy_pairs) {
         CUtensorMap tmap_w;
         SwXMaps xm;
         rc = make_tmap_bf16_2d(ctx, &tmap_w, w, static_cast<uint64_t>(V), static_cast<uint64_t>(D), SW_BV, BK);
@@ -1239,39 +1290,25 @@ int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M,
             rc = make_tmap_bf16_2d(ctx, &xm.m[i], x_gemm, static_cast<uint64_t>(M), static_cast<uint64_t>(D), 128u >> i, BK);
         if (rc != DARE_OK) return rc;
         const int grid_pair = grid & ~1;
-        if (need_pair) {
-            constexpr int SMEM = SW_SMEM_BYTES > LM_PAIR_SMEM_BYTES ? SW_SMEM_BYTES : LM_PAIR_SMEM_BYTES;
-            static std::atomic<uint64_t> smem_set_hybrid{0};
-            if (ensure_dynamic_smem(smem_set_hybrid, lmhead_greedy_pair_kernel, SMEM) != DARE_OK) return DARE_ERR_CUDA;
-            cudaLaunchConfig_t cfg = {};
-            cfg.gridDim = dim3(static_cast<unsigned>(grid_pair), 1, 1);
-            cfg.blockDim = dim3(LM_THREADS, 1, 1);
-            cfg.dynamicSmemBytes = SMEM;
-            cfg.stream = stream;
-            cudaLaunchAttribute attr;
-            attr.id = cudaLaunchAttributeClusterDimension;
-            attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
-            cfg.attrs = &attr;
-            cfg.numAttrs = 1;
-            if (cudaLaunchKernelEx(&cfg, lmhead_greedy_pair_kernel, tmap_w, xm, M, static_cast<const int32_t*>(live_rows), D,
-                                   V, mask_col, n_tiles, part_max, part_sum, part_arg, ctx->dev_status) != cudaSuccess)
-                return DARE_ERR_CUDA;
-            note_launch();
-        }
-        if (need_single) {
-            CUtensorMap tmap_w256;
-            rc = make_tmap_bf16_2d(ctx, &tmap_w256, w, static_cast<uint64_t>(V), static_cast<uint64_t>(D), BN, BK);
-            if (rc != DARE_OK) return rc;
-            static std::atomic<uint64_t> smem_set_single{0};
-            if (ensure_dynamic_smem(smem_set_single, lmhead_partial_kernel<LM_GREEDY, false>, LM_SMEM_BYTES) != DARE_OK)
-                return DARE_ERR_CUDA;
-            const LmSampling none = {};
-            lmhead_partial_kernel<LM_GREEDY, false><<<grid_pair, LM_THREADS, LM_SMEM_BYTES, stream>>>(
-                xm.m[0], tmap_w256, M, live_rows, D, V, mask_col, n_tiles, part_max, part_sum, part_arg, ctx->dev_status,
-                none, 1, 1);
-            if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
-            note_launch();
-        }
+        const int parts_stride = static_cast<int>(groups_max);
+        constexpr int SMEM_A = SW_SMEM_BYTES > LM_PAIR_SMEM_BYTES ? SW_SMEM_BYTES : LM_PAIR_SMEM_BYTES;
+        constexpr int SMEM = SMEM_A > LM_SMEM_BYTES ? SMEM_A : LM_SMEM_BYTES;
+        static std::atomic<uint64_t> smem_set_greedy{0};
+        if (ensure_dynamic_smem(smem_set_greedy, lmhead_greedy_kernel, SMEM) != DARE_OK) return DARE_ERR_CUDA;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(static_cast<unsigned>(grid_pair), 1, 1);
+        cfg.blockDim = dim3(LM_THREADS, 1, 1);
+        cfg.dynamicSmemBytes = SMEM;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, lmhead_greedy_kernel, tmap_w, xm, M, static_cast<const int32_t*>(live_rows), D, V,
+                               mask_col, n_tiles, part_max, part_sum, part_arg, ctx->dev_status, parts_stride) != cudaSuccess)
+            return DARE_ERR_CUDA;
+        note_launch();
         if (select) {
             LmSelect sel;
             sel.tokens_block = select->tokens_block; sel.row_stride = tok_row_stride; sel.mode = select->mode;
@@ -1279,10 +1316,11 @@ int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M,
             sel.n_committed = select->n_committed; sel.n_remaining = select->n_remaining;
             lmhead_merge_select_kernel<<<select->B, 32 * tok_L, 0, stream>>>(part_max, part_sum, part_arg, grid_pair, n_tiles,
                                                                              tok_L, live_rows, idx, mask_id, pred, conf,
-                                                                             LM_LAYOUT_HYBRID, sel);
+                                                                             LM_LAYOUT_GREEDY, parts_stride, sel);
         } else {
             lmhead_merge_kernel<<<(M + rows_per_block - 1) / rows_per_block, rows_per_block * 32, 0, stream>>>(
-                part_max, part_sum, part_arg, grid_pair, n_tiles, M, live_rows, idx, pred, conf, LM_LAYOUT_HYBRID);
+                part_max, part_sum, part_arg, grid_pair, n_tiles, M, live_rows, idx, pred, conf, LM_LAYOUT_GREEDY,
+                parts_stride);
         }
         note_launch();
         return cudaGetLastError() == cudaSuccess ? DARE_OK : DARE_ERR_CUDA;
@@ -1305,10 +1343,10 @@ int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M,
             sel.n_committed = select->n_committed; sel.n_remaining = select->n_remaining;
             lmhead_merge_select_kernel<<<select->B, 32 * tok_L, 0, stream>>>(part_max, part_sum, part_arg, grid, n_tiles,
                                                                              tok_L, live_rows, idx, mask_id, pred, conf,
-                                                                             allow_pair, sel); note_launch();
+                                                                             allow_pair, -1, sel); note_launch();
         } else {
             lmhead_merge_kernel<<<(M + rows_per_block - 1) / rows_per_block, rows_per_block * 32, 0, stream>>>(
-                part_max, part_sum, part_arg, grid, n_tiles, M, live_rows, idx, pred, conf, allow_pair); note_launch();
+                part_max, part_sum, part_arg, grid, n_tiles, M, live_rows, idx, pred, conf, allow_pair, -1); note_launch();
         }
     } else {
         smp.inv_temperature = 1.0f / sample->temperature;
