@@ -391,33 +391,45 @@ attn_block_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_cons
 // tcgen05 path: used when the query rows that share a KV head fill 128-row tensor-core tiles well (GQA
 // groups, long blocks such as the prefill).  One CTA per (one or two tiles of packed query rows, rollout x
 // KV head); the two query tiles share every K/V tile:
-//   warp 0        TMA producer: 64-key K and V tiles through a shared-memory ring (as above)
-//   warp 1 (and the last warp for the second query tile)
-//                 UMMA issuer:  S = Q K^T (128 x 64, K-major operands) into one of two TMEM buffers per query
-//                 tile, then O += P V (128 x D; V is the MN-major operand, straight from the TMA tile),
-//                 accumulated in TMEM over the whole key range
+//   warp 0        TMA producer: 128-key K and V tiles through a shared-memory ring (as above)
+//   warp 1        UMMA issuer (one thread, so that the order of its MMAs is the order they run in):
+//                 S = Q K^T (128 x 128, K-major operands from shared memory) into tensor memory, then
+//                 O += P V (128 x D) with P, the A operand, read from TENSOR memory and V, the MN-major B operand,
+//                 straight from the TMA tile; O stays in tensor memory over the whole key range
 //   warps 2..5    softmax of query tile 0 (warps 6..9: tile 1): one TMEM lane = one query row per thread;
-//                 reads S, keeps the row's reference max and sum, writes P as a bf16 K-major tile into
-//                 shared memory for the second MMA
+//                 reads S twice (tile max, then exponentials), keeps the row's reference max and sum, and writes
+//                 P as packed bf16 over the columns S came from: P never touches shared memory
+// An MMA whose A operand sits in shared memory costs ~80 to 120 cycles whatever its N (the 128 x 16 A slab is
+// read at ~32 bytes per cycle); with P in tensor memory the second product runs at its N / 2 cycles, and with
+// 128-key tiles the first product's MMAs have N = 128 instead of 64: per 64 keys and query tile ~740 cycles of
+// tensor pipe instead of ~1120.
+// With two query tiles each has ONE S/P buffer and the issuer interleaves them: while the softmax warps of one
+// tile work, the pipe runs the other tile's products (S_a(t), S_b(t), then per tile P V(t) and S(t + 1), which may
+// overwrite P(t) because the pipe runs the issuer's MMAs in order).  With one query tile there are two S/P buffers.
 // O stays in TMEM, so it cannot be rescaled for free when a row's max grows.  The exponentials are therefore
 // taken relative to a reference max that is only moved when the true max has run more than 2^8 ahead of it;
 // then (rarely, mostly in the first tiles) the warp waits for the MMAs in flight, multiplies its rows of O by
 // the correction factor in place and moves the reference.  The sum uses the same reference, so O / l is exact.
 // A tile holds floor(128 / g) block positions x g heads so that a position's heads never straddle two tiles.
-constexpr int TC_KT = 64;                 // keys per tile
+constexpr int TC_KT = 128;                // keys per tile
 constexpr float TC_RESCALE_GAP = 8.0f;    // log2 units the true max may run ahead of the reference
 
 template <int D, int QT>
 struct TcShape {
     static constexpr int Q_BYTES = 128 * D * 2;                        // per query tile
     static constexpr int KV_STAGE = 2 * TC_KT * D * 2;                 // K tile + V tile
-    static constexpr int P_BYTES = 128 * TC_KT * 2;                    // per query tile and buffer
-    static constexpr int FIXED = QT * Q_BYTES + QT * 2 * P_BYTES;
-    static constexpr int STAGES = (226 * 1024 - 2048 - FIXED) / KV_STAGE > 6 ? 6 : (226 * 1024 - 2048 - FIXED) / KV_STAGE;
+    static constexpr int NBUF = QT == 2 ? 1 : 2;                       // S / P buffers per query tile
+    static constexpr int FIXED = QT * Q_BYTES;
+    static constexpr int FIT = (226 * 1024 - 2048 - FIXED) / KV_STAGE;
+    static constexpr int STAGES = FIT > 4 ? 4 : FIT;
     static constexpr int SMEM = FIXED + STAGES * KV_STAGE + 1024 + 512;
-    static constexpr int THREADS = (2 + 4 * QT + 1) * 32;             // TMA warp, MMA warp, softmax warps, second MMA warp
-    static constexpr uint32_t TMEM_COLS = QT * 256;                    // per query tile: S 2 x 64 columns, O D columns
-    static_assert(STAGES >= 2, "K/V ring too small");
+    static constexpr int THREADS = (2 + 4 * QT) * 32;                  // TMA warp, MMA warp, softmax warps
+    static constexpr uint32_t TMEM_COLS = 512;
+    // tensor-memory columns: two query tiles: tile j has S/P at j * 256 and O at j * 256 + 128;
+    // one query tile: S/P buffers at 0 and 128, O at 256
+    __host__ __device__ static constexpr uint32_t s_col(int j, int b) { return QT == 2 ? j * 256 : b * 128; }
+    __host__ __device__ static constexpr uint32_t o_col(int j) { return QT == 2 ? j * 256 + 128 : 256; }
+    static_assert(STAGES >= NBUF + 1, "K/V ring too small");
 };
 
 template <int STAGES, int QT>
@@ -425,7 +437,7 @@ struct TcBarriers {
     uint64_t full[STAGES];
     uint64_t empty[STAGES];
     uint64_t q_ready;
-    uint64_t s_full[QT][2], s_free[QT][2], p_full[QT][2], o_done[QT][2];
+    uint64_t s_full[QT][2], p_full[QT][2], pv_done[QT][2];     // indexed by the key tile's parity
     uint32_t tmem_base;
     uint32_t abort_flag;
 };
@@ -438,16 +450,16 @@ attn_block_tc_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_c
                      const AttnParams p) {
     using S = TcShape<D, QT>;
     constexpr int STAGES = S::STAGES;
+    constexpr int NBUF = S::NBUF;
     constexpr int NHALF = D / 64;
-    constexpr int HALF_K = TC_KT * 128;            // one 64-column half of a K or V tile: 64 rows x 128 bytes
+    constexpr int HALF_K = TC_KT * 128;            // one 64-column half of a K or V tile: 128 rows x 128 bytes
     constexpr int KV_BYTES = TC_KT * D * 2;
     constexpr int HALF_Q = 128 * 128;              // one 64-column half of a Q tile: 128 rows x 128 bytes
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* q_s = base;                                   // [QT][Q_BYTES]
-    uint8_t* p_s = q_s + QT * S::Q_BYTES;                  // [QT][2][P_BYTES]
-    uint8_t* kv_s = p_s + QT * 2 * S::P_BYTES;             // [STAGES][KV_STAGE]
+    uint8_t* kv_s = q_s + QT * S::Q_BYTES;                 // [STAGES][KV_STAGE]
     TcBarriers<STAGES, QT>* bars = reinterpret_cast<TcBarriers<STAGES, QT>*>(kv_s + STAGES * S::KV_STAGE);
     volatile uint32_t* abort_flag = &bars->abort_flag;
 
@@ -468,15 +480,14 @@ attn_block_tc_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_c
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(&bars->full[s], 1);
-            mbar_init(&bars->empty[s], QT);                // one release per query tile's MMA thread
+            mbar_init(&bars->empty[s], 1);                 // released by the issuer once both query tiles are done with it
         }
         mbar_init(&bars->q_ready, 128 * QT);
         for (int j = 0; j < QT; ++j)
             for (int i = 0; i < 2; ++i) {
                 mbar_init(&bars->s_full[j][i], 1);
-                mbar_init(&bars->s_free[j][i], 128);
                 mbar_init(&bars->p_full[j][i], 128);
-                mbar_init(&bars->o_done[j][i], 1);
+                mbar_init(&bars->pv_done[j][i], 1);
             }
         bars->abort_flag = 0;
         fence_barrier_init();
@@ -488,7 +499,7 @@ attn_block_tc_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_c
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    const uint32_t tmem_base = bars->tmem_base;    // query tile j: S buffers at columns j*256 + {0, 64}, O at j*256 + 128
+    const uint32_t tmem_base = bars->tmem_base;
 
     // lengths and tiles of this unit (same bookkeeping as the warp-level kernel)
     int P = p.prefix_len ? p.prefix_len[b]
@@ -532,50 +543,49 @@ attn_block_tc_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_c
                 if (++stage == STAGES) { stage = 0; phase ^= 1; }
             }
         }
-    } else if (warp == 1 || warp == S::THREADS / 32 - 1) {
-        // One issuing thread per query tile (warp 1: tile 0; with two tiles the last warp: tile 1): the fixed
-        // cost of issuing a tcgen05.mma is paid per thread, so two threads keep the tensor pipe twice as busy.
-        const int j = warp == 1 ? 0 : 1;
-        if (lane == 0 && j < QT) {
+    } else if (warp == 1) {
+        if (lane == 0) {
             constexpr uint32_t idesc_s = umma_idesc_bf16(128, TC_KT);
             constexpr uint32_t idesc_o = umma_idesc_bf16(128, D) | UMMA_B_MN_MAJOR;
             // descriptor lower words (address >> 4 [| leading byte offset]); the upper word is a constant
-            const uint32_t q_lo = (smem_u32(q_s) >> 4) + j * (S::Q_BYTES >> 4);
-            const uint32_t kv_lo = smem_u32(kv_s) >> 4, p_lo = (smem_u32(p_s) >> 4) + j * 2 * (S::P_BYTES >> 4);
+            const uint32_t q_lo = smem_u32(q_s) >> 4, kv_lo = smem_u32(kv_s) >> 4;
             const uint32_t v_lbo = static_cast<uint32_t>(HALF_K >> 4) << 16;   // second 64 head-dim columns: one half tile on
-            const uint32_t tm_j = tmem_base + j * 256;
             bool ok = mbar_wait(&bars->q_ready, 0, abort_flag);
-            // S(t) = Q K_t^T into S buffer t & 1 once the softmax warps have read what it held
-            auto issue_s = [&](int t) -> bool {
-                const int stage = t % STAGES, buf = t & 1;
+            // S_j(t) = Q_j K_t^T into tile j's buffer t % NBUF (whatever that buffer held has been consumed: the P V
+            // product that read it was issued before this, and the pipe keeps the issue order)
+            auto issue_s = [&](int j, int t) -> bool {
+                const int stage = t % STAGES;
                 if (!mbar_wait(&bars->full[stage], (t / STAGES) & 1, abort_flag)) return false;
-                if (!mbar_wait(&bars->s_free[j][buf], ((t >> 1) & 1) ^ 1, abort_flag)) return false;
                 tc_fence_after_sync();
-                const uint32_t k_lo = kv_lo + stage * (S::KV_STAGE >> 4), sd = tm_j + buf * TC_KT;
-                umma_bf16_lo<false>(sd, q_lo, k_lo, idesc_s);
+                const uint32_t k_lo = kv_lo + stage * (S::KV_STAGE >> 4), qj = q_lo + j * (S::Q_BYTES >> 4);
+                const uint32_t sd = tmem_base + S::s_col(j, t % NBUF);
+                umma_bf16_lo<false>(sd, qj, k_lo, idesc_s);
 #pragma unroll
                 for (int kk = 1; kk < D / 16; ++kk)     // 16 channels = 32 bytes along the swizzled row: +2
-                    umma_bf16_lo<true>(sd, q_lo + (kk >> 2) * (HALF_Q >> 4) + 2 * (kk & 3),
+                    umma_bf16_lo<true>(sd, qj + (kk >> 2) * (HALF_Q >> 4) + 2 * (kk & 3),
                                        k_lo + (kk >> 2) * (HALF_K >> 4) + 2 * (kk & 3), idesc_s);
-                umma_commit(&bars->s_full[j][buf]);
+                umma_commit(&bars->s_full[j][t & 1]);
                 return true;
             };
-            if (ok && n_tiles > 0) ok = issue_s(0);
+            for (int t = 0; t < NBUF && t < n_tiles && ok; ++t)
+                for (int j = 0; j < QT && ok; ++j) ok = issue_s(j, t);
             for (int t = 0; t < n_tiles && ok; ++t) {
-                if (t + 1 < n_tiles && !issue_s(t + 1)) { ok = false; break; }
-                const int stage = t % STAGES, buf = t & 1;
+                const int stage = t % STAGES;
                 const uint32_t v_lo = (kv_lo + stage * (S::KV_STAGE >> 4) + (KV_BYTES >> 4)) | v_lbo;
-                if (!mbar_wait(&bars->p_full[j][buf], (t >> 1) & 1, abort_flag)) { ok = false; break; }
-                tc_fence_after_sync();
-                // A: 16 keys further along the 128-byte row of P (+2); B: 16 key rows (2 KB) further down V
-                const uint32_t pa = p_lo + buf * (S::P_BYTES >> 4), od = tm_j + 128;
-                if (t == 0) umma_bf16_lo<false>(od, pa, v_lo, idesc_o);
-                else umma_bf16_lo<true>(od, pa, v_lo, idesc_o);
+                for (int j = 0; j < QT && ok; ++j) {
+                    if (!mbar_wait(&bars->p_full[j][t & 1], (t >> 1) & 1, abort_flag)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    // A: P in tensor memory, 16 keys = 8 columns per MMA; B: 16 key rows (2 KB) further down V
+                    const uint32_t pa = tmem_base + S::s_col(j, t % NBUF), od = tmem_base + S::o_col(j);
+                    if (t == 0) umma_bf16_ts_lo<false>(od, pa, v_lo, idesc_o);
+                    else umma_bf16_ts_lo<true>(od, pa, v_lo, idesc_o);
 #pragma unroll
-                for (int kk = 1; kk < TC_KT / 16; ++kk)
-                    umma_bf16_lo<true>(od, pa + 2 * kk, v_lo + kk * (2048 >> 4), idesc_o);
-                umma_commit(&bars->o_done[j][buf]);    // P buffer free again; O holds tiles 0..t
-                umma_commit(&bars->empty[stage]);      // this query tile is done with K and V of the tile
+                    for (int kk = 1; kk < TC_KT / 16; ++kk)
+                        umma_bf16_ts_lo<true>(od, pa + 8 * kk, v_lo + kk * (2048 >> 4), idesc_o);
+                    umma_commit(&bars->pv_done[j][t & 1]);     // O holds tiles 0..t
+                    if (t + NBUF < n_tiles) ok = issue_s(j, t + NBUF);
+                }
+                if (ok) umma_commit(&bars->empty[stage]);      // every product that reads this K/V tile has been issued
             }
         }
     } else {
@@ -602,78 +612,102 @@ attn_block_tc_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_c
         }
         float m_ref = -INFINITY, l = 0.f;              // reference max (log2 domain) and sum of exp2(s - m_ref)
         const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
-        const uint32_t tm_s = tmem_base + j * 256 + lane_off;
-        const uint32_t tm_o = tmem_base + j * 256 + 128 + lane_off;
+        const uint32_t tm_o = tmem_base + S::o_col(j) + lane_off;
+        const float c2 = p.scale_log2;
         bool ok = true;
         for (int t = 0; t < n_tiles; ++t) {
             const TileInfo ti = tile_info<TC_KT>(t, n_pre, n_blk, len_pre, len_blk, Sx, base_pre, base_blk, base_suf);
             const int buf = t & 1, stage = t % STAGES;
             if (!mbar_wait(&bars->s_full[j][buf], (t >> 1) & 1, abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
-            uint32_t sv[TC_KT];
-            {
-                uint32_t (&lo)[32] = *reinterpret_cast<uint32_t (*)[32]>(&sv[0]);
-                uint32_t (&hi)[32] = *reinterpret_cast<uint32_t (*)[32]>(&sv[32]);
-                tmem_ld_32cols(tm_s + buf * TC_KT, lo);
-                tmem_ld_32cols(tm_s + buf * TC_KT + 32, hi);
-                tmem_ld_wait();
-            }
-            tc_fence_before_sync();
-            mbar_arrive(&bars->s_free[j][buf]);
-            // scores -> log2 domain, keys past the segment's end masked out, tile max
+            const uint32_t tm_s = tmem_base + S::s_col(j, t % NBUF) + lane_off;
+            // first pass over S: the tile's largest score (keys past the segment's end do not count).  The load of
+            // the next 32 columns is in flight while the current ones are looked at.  (A single pass that keeps P in
+            // registers until the reference is known to hold was measured no faster: 37.2 against 35.4 us.)
             float tmax = -INFINITY;
+            {
+                uint32_t sa[32], sb[32];
+                tmem_ld_32cols(tm_s, sa);
+                tmem_ld_wait();
 #pragma unroll
-            for (int c = 0; c < TC_KT; ++c) {
-                float sc = __uint_as_float(sv[c]) * p.scale_log2;
-                if (c >= ti.valid) sc = -INFINITY;
-                sv[c] = __float_as_uint(sc);
-                tmax = fmaxf(tmax, sc);
+                for (int c = 0; c < TC_KT / 32; ++c) {
+                    uint32_t (&cur)[32] = (c & 1) ? sb : sa;
+                    uint32_t (&nxt)[32] = (c & 1) ? sa : sb;
+                    if (c + 1 < TC_KT / 32) tmem_ld_32cols(tm_s + (c + 1) * 32, nxt);
+                    if (ti.valid >= (c + 1) * 32) {
+#pragma unroll
+                        for (int k = 0; k < 32; ++k) tmax = fmaxf(tmax, __uint_as_float(cur[k]));
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < 32; ++k)
+                            if (c * 32 + k < ti.valid) tmax = fmaxf(tmax, __uint_as_float(cur[k]));
+                    }
+                    if (c + 1 < TC_KT / 32) tmem_ld_wait();
+                }
             }
+            tmax *= c2;                                 // log2 domain (the scale is > 0); finite: every tile has a key
             // move the reference only when the true max has run away from it (decided per warp, so that the
             // TMEM loads and stores below are executed by whole warps)
             const bool move = __any_sync(0xffffffffu, tmax > m_ref + TC_RESCALE_GAP);
-            float factor = 1.f;
             if (move) {
-                const float m_new = fmaxf(m_ref, tmax);         // finite: every tile has at least one key
-                factor = fast_exp2(m_ref - m_new);              // exp2(-inf) = 0 on the first tile
+                const float m_new = fmaxf(m_ref, tmax);
+                const float factor = fast_exp2(m_ref - m_new);   // exp2(-inf) = 0 on the first tile
                 m_ref = m_new;
                 l *= factor;
+                if (t >= 1) {
+                    // every MMA that adds to O must have landed before O is rescaled in place: tile t - 1 is the last
+                    if (!mbar_wait(&bars->pv_done[j][(t - 1) & 1], ((t - 1) >> 1) & 1, abort_flag)) { ok = false; break; }
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t ov[32];
+                        tmem_ld_32cols(tm_o + c * 32, ov);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int k = 0; k < 32; ++k) ov[k] = __float_as_uint(__uint_as_float(ov[k]) * factor);
+                        tmem_st_32cols(tm_o + c * 32, ov);
+                    }
+                }
             }
+            // second pass: P = exp2(s - m_ref) as packed bf16 over the columns S came from.  The 16 columns written
+            // for keys [32 c, 32 c + 32) lie below column 16 c + 16, which this pass has already read.
+            const float nm = -m_ref;
             float psum = 0.f;
-            if (t >= 2) {   // P buffer `buf` was read by the second MMA of tile t - 2
-                if (!mbar_wait(&bars->o_done[j][buf], ((t >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
-            }
-            uint8_t* prow = p_s + (j * 2 + buf) * S::P_BYTES + r * 128;
+            {
+                uint32_t sa[32], sb[32];
+                tmem_ld_32cols(tm_s, sa);
+                tmem_ld_wait();
 #pragma unroll
-            for (int c = 0; c < TC_KT / 8; ++c) {
-                float e[8];
+                for (int c = 0; c < TC_KT / 32; ++c) {
+                    uint32_t (&cur)[32] = (c & 1) ? sb : sa;
+                    uint32_t (&nxt)[32] = (c & 1) ? sa : sb;
+                    if (c + 1 < TC_KT / 32) tmem_ld_32cols(tm_s + (c + 1) * 32, nxt);
+                    uint32_t pk[16];
+                    if (ti.valid >= (c + 1) * 32) {
 #pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    e[k] = fast_exp2(__uint_as_float(sv[c * 8 + k]) - m_ref);
-                    psum += e[k];
+                        for (int k = 0; k < 32; k += 2) {
+                            const float e0 = fast_exp2(fmaf(__uint_as_float(cur[k]), c2, nm));
+                            const float e1 = fast_exp2(fmaf(__uint_as_float(cur[k + 1]), c2, nm));
+                            psum += e0 + e1;
+                            pk[k >> 1] = pack_bf16(e0, e1);
+                        }
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < 32; k += 2) {
+                            float e0 = fast_exp2(fmaf(__uint_as_float(cur[k]), c2, nm));
+                            float e1 = fast_exp2(fmaf(__uint_as_float(cur[k + 1]), c2, nm));
+                            if (c * 32 + k >= ti.valid) e0 = 0.f;
+                            if (c * 32 + k + 1 >= ti.valid) e1 = 0.f;
+                            psum += e0 + e1;
+                            pk[k >> 1] = pack_bf16(e0, e1);
+                        }
+                    }
+                    if (c + 1 < TC_KT / 32) tmem_ld_wait();      // (the next columns, [32 c + 32, +32), lie above the store below)
+                    tmem_st_16cols(tm_s + c * 16, pk);
                 }
-                uint4 o;
-                o.x = pack_bf16(e[0], e[1]); o.y = pack_bf16(e[2], e[3]);
-                o.z = pack_bf16(e[4], e[5]); o.w = pack_bf16(e[6], e[7]);
-                *reinterpret_cast<uint4*>(prow + ((c ^ (r & 7)) << 4)) = o;
             }
+            tmem_st_wait();
             l += psum;
-            if (move && t >= 1) {
-                // every MMA that adds to O must have landed before O is rescaled in place: tile t - 1 is the last
-                if (!mbar_wait(&bars->o_done[j][(t - 1) & 1], ((t - 1) >> 1) & 1, abort_flag)) { ok = false; break; }
-                tc_fence_after_sync();
-#pragma unroll
-                for (int c = 0; c < D / 32; ++c) {
-                    uint32_t ov[32];
-                    tmem_ld_32cols(tm_o + c * 32, ov);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int k = 0; k < 32; ++k) ov[k] = __float_as_uint(__uint_as_float(ov[k]) * factor);
-                    tmem_st_32cols(tm_o + c * 32, ov);
-                }
-                tmem_st_wait();
-                tc_fence_before_sync();
-            }
             if (ti.valid < TC_KT) {
                 // V rows past the segment's end hold whatever lies behind it in memory: zero them so that
                 // probability 0 times garbage cannot make a NaN (thread r clears 16-byte pieces of those rows;
@@ -683,11 +717,12 @@ attn_block_tc_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_c
                 for (int h2 = 0; h2 < NHALF; ++h2)
                     for (int q = r; q < n_bad; q += 128)
                         *reinterpret_cast<uint4*>(vt + h2 * HALF_K + ti.valid * 128 + q * 16) = make_uint4(0, 0, 0, 0);
+                fence_proxy_async_smem();
             }
-            fence_proxy_async_smem();
+            tc_fence_before_sync();
             mbar_arrive(&bars->p_full[j][buf]);
         }
-        if (ok && n_tiles > 0) ok = mbar_wait(&bars->o_done[j][(n_tiles - 1) & 1], ((n_tiles - 1) >> 1) & 1, abort_flag);
+        if (ok && n_tiles > 0) ok = mbar_wait(&bars->pv_done[j][(n_tiles - 1) & 1], ((n_tiles - 1) >> 1) & 1, abort_flag);
         tc_fence_after_sync();
         const float inv = l > 0.f ? 1.f / l : 0.f;
         __nv_bfloat16* dst = p.out + qrow;
