@@ -131,6 +131,7 @@ int dare_create(dare_ctx** out, int device, size_t workspace_bytes) {
     ctx->workspace_bytes = workspace_bytes ? workspace_bytes : (size_t(256) << 20);
     ctx->workspace = nullptr;
     ctx->dev_status = nullptr;
+    ctx->aux = nullptr; ctx->ev_fork = nullptr; ctx->ev_join = nullptr;
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
@@ -142,9 +143,15 @@ int dare_create(dare_ctx** out, int device, size_t workspace_bytes) {
     ctx->encode_tiled = reinterpret_cast<dare_encode_tiled_fn>(fn);
     if (cudaMalloc(&ctx->workspace, ctx->workspace_bytes) != cudaSuccess ||
         cudaMalloc(reinterpret_cast<void**>(&ctx->dev_status), sizeof(uint32_t)) != cudaSuccess ||
-        cudaMemset(ctx->dev_status, 0, sizeof(uint32_t)) != cudaSuccess) {
+        cudaMemset(ctx->dev_status, 0, sizeof(uint32_t)) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&ctx->aux, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming) != cudaSuccess) {
         if (ctx->workspace) cudaFree(ctx->workspace);
         if (ctx->dev_status) cudaFree(ctx->dev_status);
+        if (ctx->aux) cudaStreamDestroy(ctx->aux);
+        if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+        if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
         delete ctx->tmaps;
         delete ctx;
         return DARE_ERR_CUDA;
@@ -158,6 +165,9 @@ int dare_destroy(dare_ctx* ctx) {
     dare::DeviceScope scope(ctx->device);
     cudaFree(ctx->workspace);
     cudaFree(ctx->dev_status);
+    if (ctx->aux) cudaStreamDestroy(ctx->aux);
+    if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+    if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
     delete ctx->tmaps;
     delete ctx;
     return DARE_OK;
@@ -287,17 +297,27 @@ int dare_denoise_block(dare_ctx* ctx, int B, int L, int Hq, int Hkv, int d, int 
     rc = check_select(tokens, B, row_stride, block_start, L, pred, conf, mode, threshold, k);
     if (rc != DARE_OK) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    rc = dare::launch_attn(ctx, a, s);
-    if (rc != DARE_OK) return rc;
+    // The LM head's row compaction reads the token state and `hidden`, not the attention's output: it is enqueued on
+    // the context's side stream, ordered after everything already on `stream` and joined back before the head's
+    // GEMM, so that it runs beside the attention kernel.  (Not when the attention splits K/V: its partials and the
+    // compacted rows share the workspace.)
+    cudaStream_t side = nullptr;
+    if (ctx->aux && dare::attn_plan_splits(ctx, a) == 1) {
+        if (cudaEventRecord(ctx->ev_fork, s) != cudaSuccess || cudaStreamWaitEvent(ctx->aux, ctx->ev_fork, 0) != cudaSuccess)
+            return DARE_ERR_CUDA;
+        side = ctx->aux;
+    }
     // The LM head reads each row's current token straight from the token state: row m = (r, i) lives at
     // tokens[r * row_stride + block_start + i].
+    rc = dare::launch_attn(ctx, a, s);
+    if (rc != DARE_OK) return rc;
     if (L <= dare::LMHEAD_SELECT_MAX_L) {      // short blocks: the selection rides on the head's merge kernel
         const dare::LmSelectArgs sel = {tokens + block_start, B, mode, threshold, k, n_committed, n_remaining};
         return dare::launch_lmhead(ctx, ctx->workspace, hidden, M, D, w, V, tokens + block_start, L, row_stride, mask_id,
-                                   exclude_mask_column, pred, conf, s, nullptr, &sel);
+                                   exclude_mask_column, pred, conf, s, nullptr, &sel, side);
     }
     rc = dare::launch_lmhead(ctx, ctx->workspace, hidden, M, D, w, V, tokens + block_start, L, row_stride, mask_id,
-                             exclude_mask_column, pred, conf, s, nullptr);
+                             exclude_mask_column, pred, conf, s, nullptr, nullptr, side);
     if (rc != DARE_OK) return rc;
     return dare::launch_unmask_select(tokens, B, row_stride, block_start, L, pred, conf, mask_id, mode, threshold, k,
                                       n_committed, n_remaining, s);

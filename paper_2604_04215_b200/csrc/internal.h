@@ -39,6 +39,10 @@ struct dare_ctx {
     uint32_t* dev_status;   // device word, bits DARE_DEV_*
     dare_encode_tiled_fn encode_tiled;
     TmapCache* tmaps;       // host memory; NULL = encode on every call
+    // side stream of dare_denoise_block: the LM head's row compaction does not depend on the attention kernel, so
+    // it runs beside it (forked from and joined back into the caller's stream with the two events); NULL = none
+    cudaStream_t aux;
+    cudaEvent_t ev_fork, ev_join;
 };
 
 #include <atomic>
@@ -113,7 +117,9 @@ constexpr int LMHEAD_SELECT_MAX_L = 32;
 struct LmSelectArgs { int32_t* tokens_block; int B; int mode; float threshold; int k; int32_t* n_committed; int32_t* n_remaining; };
 int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M, int D, const void* w, int V,
                   const int32_t* row_tokens, int tok_L, int64_t tok_row_stride, int32_t mask_id, int exclude_mask_column, int32_t* pred, float* conf,
-                  cudaStream_t stream, const LmSampleArgs* sample, const LmSelectArgs* select = nullptr);
+                  cudaStream_t stream, const LmSampleArgs* sample, const LmSelectArgs* select = nullptr,
+                  cudaStream_t compact_stream = nullptr);     // non-NULL: the row compaction is enqueued there (the caller
+                                                              // has ordered that stream after `stream`; it is joined back here)
 
 struct AttnArgs {
     int B, L, Hq, Hkv, d, prefix_cap, suffix_cap;
