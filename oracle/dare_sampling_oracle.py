@@ -15,7 +15,11 @@ v takes output word v % 4; its top 23 bits k give u = (2 k + 1) / 2^24, which is
 
 Pins (tests/test_oracle_sampling.py): the generator against the known-answer vectors distributed with its
 reference implementation; the uniforms' range and exactness in float32; the Gumbel moments; the sampling law
-(token frequencies follow softmax(z / T)); T -> 0 recovers the greedy head; determinism in (seed, row, step).
+(token frequencies follow softmax(z / T)); T -> 0 recovers the greedy head; determinism in (seed, row, step);
+perturbed_score against the sampled head's own winning score, rebuilt from the uniforms, and its row / step / seed
+keys; denoise_step_sampled as the composition of the separately pinned attention, sampled head and selection, its
+step invariants, and its T -> 0 limit (the greedy step); the forward process' marginals and window; the bound's
+term on a hand-worked case.
 """
 from __future__ import annotations
 

@@ -6,7 +6,11 @@
   * the Gumbel transform: closed-form values, mean = Euler's constant, variance = pi^2 / 6;
   * the sampling law (Gumbel-max): token frequencies follow softmax(z / T), checked on a small vocabulary;
   * limits: T -> 0 gives the greedy head's token; the confidence is the temperature-1 probability of the token;
-    committed rows are skipped; the mask column is never sampled.
+    committed rows are skipped; the mask column is never sampled;
+  * perturbed_score (which judges near-ties in the GPU tests): equals the sampled head's winning score at its token,
+    stays below it elsewhere, is rebuilt from the uniforms, and depends on the row, step and seed keys;
+  * denoise_step_sampled: equals attention + sampled head + selection on the same inputs, keeps committed tokens and
+    everything outside the block, and turns into the greedy step as T -> 0.
 """
 import os
 
