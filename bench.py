@@ -419,6 +419,16 @@ def bench_step_workload(dare, ctx, wl, steps, warmup, rank, world, sampler, with
                 bufs[t & 1][1].copy_(xh, non_blocking=True)
                 uploaded[t & 1].record(copy_stream)
 
+        # the upload alone (no compute beside it): what the host link delivers for one step's inputs
+        up0, up1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(copy_stream):
+            up0.record(copy_stream)
+            for i in range(8):
+                bufs[i & 1][0].copy_(pool_h[i % NPOOL][0], non_blocking=True)
+                bufs[i & 1][1].copy_(pool_h[i % NPOOL][1], non_blocking=True)
+            up1.record(copy_stream)
+        torch.cuda.synchronize()
+        upload_ms = up0.elapsed_time(up1) / 8
         _barrier(world)
         for ev_ in consumed:
             ev_.record(stream)
@@ -448,7 +458,8 @@ def bench_step_workload(dare, ctx, wl, steps, warmup, rank, world, sampler, with
         h2d = pool_h[0][0].numel() * 2 + pool_h[0][1].numel() * 2
         d2h = 4 * (B + B + B * L)
         out["e2e"] = {"value": e2e_n / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
-                      "d2h_bytes_per_step": d2h, "steps": n_e2e}
+                      "d2h_bytes_per_step": d2h, "steps": n_e2e, "ms_per_step": e2e_s / n_e2e * 1e3,
+                      "h2d_ms_per_step_alone": upload_ms, "h2d_GBps_alone": h2d / (upload_ms * 1e-3) / 1e9}
     return out
 
 
