@@ -217,14 +217,15 @@ def bench_step_workload(dare, ctx, wl, steps, warmup, rank, world, sampler, with
     nr = torch.zeros(B, dtype=torch.int32, device="cuda")
     stream = torch.cuda.current_stream()
 
-    def step(t, q, x, nc):
+    def step(t, q, x, nc, nr_out=None):
         g = t % steps_per_gen
         b = g // steps_per_block
         if g == 0:
             tokens.copy_(tok0)                                  # new generation: re-mask (one small copy)
         dare.dare_denoise_block(ctx, q, k_pre, v_pre, plen_blocks[b], None, None, k_suf, v_suf, suffix_len,
                                 attn_out, None, x, w, wl.mask_id, True, tokens, wl.prompt_len + b * L,
-                                wl.mode, wl.threshold, wl.k, pred, conf, nc, nr, stream=stream)
+                                wl.mode, wl.threshold, wl.k, pred, conf, nc, nr if nr_out is None else nr_out,
+                                stream=stream)
 
     # ---- device-resident timed region
     for t in range(warmup):
@@ -398,14 +399,15 @@ def bench_step_workload(dare, ctx, wl, steps, warmup, rank, world, sampler, with
     if with_e2e:
         n_e2e = min(steps, 4 * steps_per_gen)
         # Double-buffered both ways: a copy stream uploads step t + 1's activations while step t computes, and the
-        # host reads step t's counts and tokens (copied to pinned memory right behind the step) while step t + 1
-        # runs: the step does not depend on the host, so the host stays one step behind, as dare_generate does.
+        # host reads step t's counts and tokens while step t + 1 runs: the step does not depend on the host, so the
+        # host stays one step behind, as dare_generate does.  The two count vectors are page-locked host tensors that
+        # the step's last kernel writes directly (three small copies behind every step cost ~40 us of stream time,
+        # one costs ~15); the block's tokens are copied to pinned memory right behind the step.
         # Every step still uploads its own inputs from pinned memory and every step's results are read on the host.
         bufs = [(torch.empty_like(pool[0][0]), torch.empty_like(pool[0][1])) for _ in range(2)]
         nc_h = [torch.zeros(B, dtype=torch.int32).pin_memory() for _ in range(2)]
         nr_h = [torch.zeros(B, dtype=torch.int32).pin_memory() for _ in range(2)]
         tok_blk_h = [torch.zeros(B, L, dtype=torch.int32).pin_memory() for _ in range(2)]
-        nc_d = [torch.zeros(B, dtype=torch.int32, device="cuda") for _ in range(2)]
         read_back = [torch.cuda.Event(), torch.cuda.Event()]
         copy_stream = torch.cuda.Stream()
         uploaded = [torch.cuda.Event(), torch.cuda.Event()]
@@ -439,12 +441,10 @@ def bench_step_workload(dare, ctx, wl, steps, warmup, rank, world, sampler, with
             if t + 1 < n_e2e:
                 upload(t + 1)
             stream.wait_event(uploaded[t & 1])
-            step(t, bufs[t & 1][0], bufs[t & 1][1], nc_d[t & 1])
+            step(t, bufs[t & 1][0], bufs[t & 1][1], nc_h[t & 1], nr_h[t & 1])
             consumed[t & 1].record(stream)
             g = t % steps_per_gen
             bs = wl.prompt_len + (g // steps_per_block) * L
-            nc_h[t & 1].copy_(nc_d[t & 1], non_blocking=True)
-            nr_h[t & 1].copy_(nr, non_blocking=True)
             tok_blk_h[t & 1].copy_(tokens[:, bs:bs + L], non_blocking=True)
             read_back[t & 1].record(stream)
             if t >= 1:

@@ -224,7 +224,11 @@ int dare_masked_nelbo(dare_ctx* ctx, const float* logprob, const int32_t* xt, in
  * Comparisons are in fp32; NaN counts as -inf.
  *
  *   tokens       int32 [B, row_stride] in/out     pred int32 [B, L]     conf fp32 [B, L]
- *   n_committed, n_remaining   int32 [B] out, each may be NULL
+ *   n_committed, n_remaining   int32 [B] out, each may be NULL.  Here, in dare_denoise_block(_sampled) and in
+ *                dare_model_step(_dual) these two may also point to page-locked host memory that the device can
+ *                address (cudaHostAlloc / cudaHostRegister under unified addressing): the kernel stores the B
+ *                integers with plain writes, so the host reads them after synchronising with the stream, without
+ *                a copy back.  dare_generate(_dual) need device memory for n_remaining.
  * Supported: 1 <= L <= 4096; 0 <= block_start, block_start + L <= row_stride.
  */
 int dare_unmask_select(dare_ctx* ctx,

@@ -151,6 +151,18 @@ def _ptr(t: Optional[torch.Tensor], dtype=None):
     return C.c_void_p(t.data_ptr())
 
 
+def _count_ptr(t: Optional[torch.Tensor]):
+    """The per-rollout count outputs (n_committed, n_remaining): a device tensor, or a page-locked host tensor (the
+    kernel then stores its B integers straight into host memory and the caller needs no copy back)."""
+    if t is not None and not t.is_cuda:
+        if not t.is_pinned() or not t.is_contiguous():
+            raise ValueError("a host tensor for the counts must be page-locked (pin_memory()) and contiguous")
+        if t.dtype != torch.int32:
+            raise ValueError(f"expected dtype {torch.int32}, got {t.dtype}")
+        return C.c_void_p(t.data_ptr())
+    return _ptr(t, torch.int32)
+
+
 def _stream(stream) -> C.c_void_p:
     if stream is None:
         stream = torch.cuda.current_stream()
@@ -385,8 +397,8 @@ def dare_unmask_select(ctx: Context, tokens, block_start: int, L: int, pred, con
     B, row_stride = tokens.shape
     rc = load().dare_unmask_select(ctx.handle, _ptr(tokens, torch.int32), B, row_stride, int(block_start), int(L),
                                    _ptr(pred, torch.int32), _ptr(conf, torch.float32), int(mask_id), int(mode),
-                                   float(threshold), int(k), _ptr(n_committed, torch.int32),
-                                   _ptr(n_remaining, torch.int32), _stream(stream))
+                                   float(threshold), int(k), _count_ptr(n_committed),
+                                   _count_ptr(n_remaining), _stream(stream))
     if rc != 0 and check:
         raise DareError(rc, "dare_unmask_select")
     return rc
@@ -408,8 +420,8 @@ def dare_denoise_block(ctx: Context, q, k_pre, v_pre, prefix_len, k_blk, v_blk, 
         _ptr(k_suf, bf), _ptr(v_suf, bf), _ptr(suffix_len, torch.int32), _ptr(attn_out, bf), _ptr(lse, torch.float32),
         _ptr(hidden, bf), D, _ptr(w, bf), V, int(mask_id), int(bool(exclude_mask_column)),
         _ptr(tokens, torch.int32), tokens.shape[1], int(block_start), int(mode), float(threshold), int(k),
-        _ptr(pred, torch.int32), _ptr(conf, torch.float32), _ptr(n_committed, torch.int32),
-        _ptr(n_remaining, torch.int32), _stream(stream))
+        _ptr(pred, torch.int32), _ptr(conf, torch.float32), _count_ptr(n_committed),
+        _count_ptr(n_remaining), _stream(stream))
     if rc != 0 and check:
         raise DareError(rc, "dare_denoise_block")
     return rc
@@ -433,8 +445,8 @@ def dare_denoise_block_sampled(ctx: Context, q, k_pre, v_pre, prefix_len, k_blk,
         _ptr(hidden, bf), D, _ptr(w, bf), V, int(mask_id), int(bool(exclude_mask_column)), float(temperature),
         int(seed) & 0xFFFFFFFFFFFFFFFF, int(step) & 0xFFFFFFFF,
         _ptr(tokens, torch.int32), tokens.shape[1], int(block_start), int(mode), float(threshold), int(k),
-        _ptr(pred, torch.int32), _ptr(conf, torch.float32), _ptr(n_committed, torch.int32),
-        _ptr(n_remaining, torch.int32), _stream(stream))
+        _ptr(pred, torch.int32), _ptr(conf, torch.float32), _count_ptr(n_committed),
+        _count_ptr(n_remaining), _stream(stream))
     if rc != 0 and check:
         raise DareError(rc, "dare_denoise_block_sampled")
     return rc
@@ -542,7 +554,7 @@ def dare_model_step(model: Model, tokens, block_start: int, L: int, k_cache, v_c
     rc = load().dare_model_step(model.handle, _ptr(tokens, torch.int32), B, row_stride, int(block_start), int(L),
                                 _ptr(k_cache, bf), _ptr(v_cache, bf), k_cache.shape[3], int(mode), float(threshold),
                                 int(k), _ptr(pred, torch.int32), _ptr(conf, torch.float32),
-                                _ptr(n_committed, torch.int32), _ptr(n_remaining, torch.int32), _stream(stream))
+                                _count_ptr(n_committed), _count_ptr(n_remaining), _stream(stream))
     if rc != 0 and check:
         raise DareError(rc, "dare_model_step")
     return rc
@@ -584,7 +596,7 @@ def dare_model_step_window(model: Model, tokens, block_start: int, L: int, kv_le
     rc = load().dare_model_step_window(model.handle, _ptr(tokens, torch.int32), B, row_stride, int(block_start), int(L),
                                        int(kv_len), _ptr(k_cache, bf), _ptr(v_cache, bf), k_cache.shape[3], int(mode),
                                        float(threshold), int(k), _ptr(pred, torch.int32), _ptr(conf, torch.float32),
-                                       _ptr(n_committed, torch.int32), _ptr(n_remaining, torch.int32), _stream(stream))
+                                       _count_ptr(n_committed), _count_ptr(n_remaining), _stream(stream))
     if rc != 0 and check:
         raise DareError(rc, "dare_model_step_window")
     return rc

@@ -241,8 +241,11 @@ def test_tiny_workload_eight_iterations(ctx):
             attn_out = torch.empty_like(si.q, device="cuda")
             pred = torch.empty(wl.M, dtype=torch.int32, device="cuda")
             conf = torch.empty(wl.M, dtype=torch.float32, device="cuda")
-            nc = torch.zeros(wl.batch, dtype=torch.int32, device="cuda")
-            nr = torch.zeros(wl.batch, dtype=torch.int32, device="cuda")
+            # the planted pass takes the counts in page-locked host memory, which the step's last kernel writes itself
+            nc = torch.full((wl.batch,), -1, dtype=torch.int32, device="cuda")
+            nr = torch.full((wl.batch,), -1, dtype=torch.int32, device="cuda")
+            if planted:
+                nc, nr = nc.cpu().pin_memory(), nr.cpu().pin_memory()
             dare.dare_denoise_block(ctx, si.q.cuda(), kp, vp, si.prefix_len.cuda(), si.k_blk.cuda(), si.v_blk.cuda(),
                                     None, None, None, attn_out, None, si.x.cuda(), wd, wl.mask_id, True, tok_d,
                                     si.block_start, wl.mode, wl.threshold, wl.k, pred, conf, nc, nr)

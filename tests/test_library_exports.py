@@ -3,6 +3,9 @@ import ctypes
 import os
 import re
 
+import pytest
+import torch
+
 from paper_2604_04215_b200 import binding, build
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
@@ -72,6 +75,14 @@ def test_binding_refuses_a_tensor_that_is_not_on_the_current_device(monkeypatch)
         binding._ptr(FakeTensor(), torch.int32)
     monkeypatch.setattr(torch.cuda, "current_device", lambda: 1)
     assert binding._ptr(FakeTensor(), torch.int32).value == 0x1000
+
+
+def test_count_outputs_on_the_host_must_be_page_locked():
+    """n_committed / n_remaining may live in pinned host memory (the kernel writes them there); pageable host memory,
+    which the device cannot address, is refused in the binding."""
+    assert binding._count_ptr(None) is None
+    with pytest.raises(ValueError, match="page-locked"):
+        binding._count_ptr(torch.zeros(4, dtype=torch.int32))
 
 
 def test_null_context_is_refused_before_anything_else():
