@@ -108,21 +108,61 @@ attn_block_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_cons
     const int b = unit / p.Hkv;
     const int kvh = unit % p.Hkv;
 
-    if (threadIdx.x == 0) {
+    // A CTA lives for a handful of tiles, so what it does before its first tile arrives counts.  Nothing below waits
+    // for anything else: the row's lengths are requested first (needed only after the barrier below), the producer
+    // lane sets up the barriers itself and, where the first tile's place does not depend on the lengths (in-place
+    // cache: the prefix segment holds at least the block's L >= 1 keys and starts at the unit's base), sends for that
+    // tile at once; the consumers' Q rows are requested beside it.
+    int P = p.prefix_len ? p.prefix_len[b]
+                         : (p.uniform_P >= 0 ? p.uniform_P : (p.inplace ? p.prefix_cap - p.L : p.prefix_cap));
+    int S = p.has_suffix ? (p.suffix_len ? p.suffix_len[b] : p.suffix_cap) : 0;
+    // (only without a K/V split: a CTA of a split launch may own no tile at all, and a tile sent for must be waited for)
+    const bool early_tile = p.inplace && p.splits == 1;     // tile 0 of this CTA is tile 0 of the prefix segment
+    if (threadIdx.x == NCW * 32) {
         for (int s = 0; s < ATT_STAGES; ++s) {
             mbar_init(&bars->full[s], 1);
             mbar_init(&bars->empty[s], NCW);
         }
         bars->abort_flag = 0;
         fence_barrier_init();
+        prefetch_tensormap(&tm_kpre);
+        prefetch_tensormap(&tm_vpre);
+        if (early_tile) {
+            mbar_arrive_expect_tx(&bars->full[0], 2 * KV_BYTES);
+#pragma unroll
+            for (int h = 0; h < NHALF; ++h) {
+                tma_load_2d(tiles + h * HALF, &tm_kpre, &bars->full[0], h * 64, unit * p.prefix_cap);
+                tma_load_2d(tiles + KV_BYTES + h * HALF, &tm_vpre, &bars->full[0], h * 64, unit * p.prefix_cap);
+            }
+        }
+    }
+
+    // per-thread state of the consumers (declared here so that the final merge can see it)
+    const int rg = warp % NW;              // row group
+    const int ks = warp / NW;              // key slice (NW*KS == producer warp: unused there)
+    const int quad = lane >> 2;            // row inside the 16-row tile (and +8)
+    const int tq = lane & 3;
+    const int rho0 = chunk * (NW * 16) + rg * 16 + quad;
+    const int rho1 = rho0 + 8;
+    const bool live0 = rho0 < p.R, live1 = rho1 < p.R;
+    const int i0 = live0 ? rho0 / p.g : 0, h0 = kvh * p.g + (live0 ? rho0 % p.g : 0);
+    const int i1 = live1 ? rho1 / p.g : 0, h1 = kvh * p.g + (live1 ? rho1 % p.g : 0);
+    uint32_t qf[D / 16][4];
+    if (warp < NCW) {
+        const uint32_t* q0 = reinterpret_cast<const uint32_t*>(p.q + ((static_cast<size_t>(b) * p.L + i0) * p.Hq + h0) * D);
+        const uint32_t* q1 = reinterpret_cast<const uint32_t*>(p.q + ((static_cast<size_t>(b) * p.L + i1) * p.Hq + h1) * D);
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+            qf[kk][0] = live0 ? q0[kk * 8 + tq] : 0u;
+            qf[kk][1] = live1 ? q1[kk * 8 + tq] : 0u;
+            qf[kk][2] = live0 ? q0[kk * 8 + 4 + tq] : 0u;
+            qf[kk][3] = live1 ? q1[kk * 8 + 4 + tq] : 0u;
+        }
     }
     __syncthreads();
 
     // lengths (clamped to capacity; a clamp is reported, never trapped on)
-    int P = p.prefix_len ? p.prefix_len[b]
-                         : (p.uniform_P >= 0 ? p.uniform_P : (p.inplace ? p.prefix_cap - p.L : p.prefix_cap));
     const int p_max = p.inplace ? p.prefix_cap - p.L : p.prefix_cap;
-    int S = p.has_suffix ? (p.suffix_len ? p.suffix_len[b] : p.suffix_cap) : 0;
     if (P < 0 || P > p_max || S < 0 || S > p.suffix_cap) {
         P = max(0, min(P, p_max));
         S = max(0, min(S, p.suffix_cap));
@@ -140,16 +180,6 @@ attn_block_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_cons
     const int base_blk = unit * p.L;
     const int base_suf = unit * p.suffix_cap;
 
-    // per-thread state of the consumers (declared here so that the final merge can see it)
-    const int rg = warp % NW;              // row group
-    const int ks = warp / NW;              // key slice (NW*KS == producer warp: unused there)
-    const int quad = lane >> 2;            // row inside the 16-row tile (and +8)
-    const int tq = lane & 3;
-    const int rho0 = chunk * (NW * 16) + rg * 16 + quad;
-    const int rho1 = rho0 + 8;
-    const bool live0 = rho0 < p.R, live1 = rho1 < p.R;
-    const int i0 = live0 ? rho0 / p.g : 0, h0 = kvh * p.g + (live0 ? rho0 % p.g : 0);
-    const int i1 = live1 ? rho1 / p.g : 0, h1 = kvh * p.g + (live1 ? rho1 % p.g : 0);
     float oacc[D / 8][4];
 #pragma unroll
     for (int n = 0; n < D / 8; ++n) { oacc[n][0] = oacc[n][1] = oacc[n][2] = oacc[n][3] = 0.f; }
@@ -159,11 +189,14 @@ attn_block_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_cons
     if (warp == NCW) {
         // ---------------- producer
         if (lane == 0) {
-            prefetch_tensormap(&tm_kpre);
-            prefetch_tensormap(&tm_vpre);
             int stage = 0;
             uint32_t phase = 0;
-            for (int t = t_begin; t < t_end; ++t) {
+            int t = t_begin;
+            if (early_tile) {                         // tile 0 is on its way already (no split: t_begin = 0, t_end = n_tiles >= 1)
+                ++t;
+                if (++stage == ATT_STAGES) { stage = 0; phase ^= 1; }
+            }
+            for (; t < t_end; ++t) {
                 const TileInfo ti = tile_info<KT>(t, n_pre, n_blk, len_pre, len_blk, S, base_pre, base_blk, base_suf);
                 const CUtensorMap* mk = ti.seg == 0 ? &tm_kpre : (ti.seg == 1 ? &tm_kblk : &tm_ksuf);
                 const CUtensorMap* mv = ti.seg == 0 ? &tm_vpre : (ti.seg == 1 ? &tm_vblk : &tm_vsuf);
@@ -181,20 +214,6 @@ attn_block_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_cons
         }
     } else {
         // ---------------- consumers
-        const size_t qoff0 = ((static_cast<size_t>(b) * p.L + i0) * p.Hq + h0) * D;
-        const size_t qoff1 = ((static_cast<size_t>(b) * p.L + i1) * p.Hq + h1) * D;
-        uint32_t qf[D / 16][4];
-        {
-            const uint32_t* q0 = reinterpret_cast<const uint32_t*>(p.q + qoff0);
-            const uint32_t* q1 = reinterpret_cast<const uint32_t*>(p.q + qoff1);
-#pragma unroll
-            for (int kk = 0; kk < D / 16; ++kk) {
-                qf[kk][0] = live0 ? q0[kk * 8 + tq] : 0u;
-                qf[kk][1] = live1 ? q1[kk * 8 + tq] : 0u;
-                qf[kk][2] = live0 ? q0[kk * 8 + 4 + tq] : 0u;
-                qf[kk][3] = live1 ? q1[kk * 8 + 4 + tq] : 0u;
-            }
-        }
         int stage = 0;
         uint32_t phase = 0;
         const int mi = lane >> 3, rin = lane & 7;
@@ -477,6 +496,15 @@ attn_block_tc_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_c
     if (static_cast<int>(blockIdx.x) * QT * pos_per_tile >= L_eff) return;   // (whole CTA, before anything is set up)
     const int kv_col0 = packed ? kvh * D : 0;      // first column of this KV head in the 2-D view of K / V
 
+    // Set-up, with nothing waiting for anything else (a launch is a single wave of CTAs that live for about ten key
+    // tiles, so the time to the first product counts): the lengths are requested first; thread 0, which is also the
+    // TMA producer, sets up the barriers and sends for key tile 0 at once where its place does not depend on the
+    // lengths (packed sequences and the in-place cache: the first segment is not empty and starts at the unit's
+    // base); warp 1 allocates tensor memory; the softmax threads stage their Q rows.
+    int P = p.prefix_len ? p.prefix_len[b]
+                         : (p.uniform_P >= 0 ? p.uniform_P : (p.inplace ? p.prefix_cap - p.L : p.prefix_cap));
+    int Sx = p.has_suffix ? (p.suffix_len ? p.suffix_len[b] : p.suffix_cap) : 0;
+    const bool early_tile = packed || p.inplace;
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(&bars->full[s], 1);
@@ -491,10 +519,39 @@ attn_block_tc_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_c
             }
         bars->abort_flag = 0;
         fence_barrier_init();
+        prefetch_tensormap(&tm_kpre);
+        prefetch_tensormap(&tm_vpre);
+        if (early_tile) {
+            const int row0 = packed ? seq_base : unit * p.prefix_cap;
+            mbar_arrive_expect_tx(&bars->full[0], 2 * KV_BYTES);
+#pragma unroll
+            for (int h = 0; h < NHALF; ++h) {
+                tma_load_2d(kv_s + h * HALF_K, &tm_kpre, &bars->full[0], kv_col0 + h * 64, row0);
+                tma_load_2d(kv_s + KV_BYTES + h * HALF_K, &tm_vpre, &bars->full[0], kv_col0 + h * 64, row0);
+            }
+        }
     }
     if (warp == 1) {
         tmem_alloc(&bars->tmem_base, S::TMEM_COLS);
         tmem_relinquish();
+    }
+    if (warp >= 2) {
+        // Q row -> shared memory, K-major with the 128-byte swizzle (16-byte chunk c of row r sits at c ^ (r & 7));
+        // thread = packed query row r of query tile j
+        const int j = (warp - 2) >> 2;
+        const int r = (warp & 3) * 32 + lane;
+        const int i = (blockIdx.x * QT + j) * pos_per_tile + r / p.g;
+        const int h = kvh * p.g + r % p.g;
+        const bool live = r < pos_per_tile * p.g && i < L_eff;
+        const size_t q_token = packed ? static_cast<size_t>(seq_base) : static_cast<size_t>(b) * p.L;
+        const uint4* src = reinterpret_cast<const uint4*>(p.q + ((q_token + (live ? i : 0)) * p.Hq + (live ? h : 0)) * D);
+        uint8_t* qt = q_s + j * S::Q_BYTES;
+#pragma unroll
+        for (int c = 0; c < D / 8; ++c) {
+            const uint4 v = live ? src[c] : make_uint4(0, 0, 0, 0);
+            *reinterpret_cast<uint4*>(qt + (c >> 3) * HALF_Q + r * 128 + (((c & 7) ^ (r & 7)) << 4)) = v;
+        }
+        fence_proxy_async_smem();
     }
     tc_fence_before_sync();
     __syncthreads();
@@ -502,10 +559,7 @@ attn_block_tc_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_c
     const uint32_t tmem_base = bars->tmem_base;
 
     // lengths and tiles of this unit (same bookkeeping as the warp-level kernel)
-    int P = p.prefix_len ? p.prefix_len[b]
-                         : (p.uniform_P >= 0 ? p.uniform_P : (p.inplace ? p.prefix_cap - p.L : p.prefix_cap));
     const int p_max = p.inplace ? p.prefix_cap - p.L : p.prefix_cap;
-    int Sx = p.has_suffix ? (p.suffix_len ? p.suffix_len[b] : p.suffix_cap) : 0;
     if (!packed && (P < 0 || P > p_max || Sx < 0 || Sx > p.suffix_cap)) {
         P = max(0, min(P, p_max));
         Sx = max(0, min(Sx, p.suffix_cap));
@@ -523,11 +577,14 @@ attn_block_tc_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_c
 
     if (warp == 0) {
         if (lane == 0) {
-            prefetch_tensormap(&tm_kpre);
-            prefetch_tensormap(&tm_vpre);
             int stage = 0;
             uint32_t phase = 0;
-            for (int t = 0; t < n_tiles; ++t) {
+            int t = 0;
+            if (early_tile) {                               // key tile 0 is on its way already (n_tiles >= 1 here)
+                ++t;
+                if (++stage == STAGES) { stage = 0; phase ^= 1; }
+            }
+            for (; t < n_tiles; ++t) {
                 const TileInfo ti = tile_info<TC_KT>(t, n_pre, n_blk, len_pre, len_blk, Sx, base_pre, base_blk, base_suf);
                 const CUtensorMap* mk = ti.seg == 0 ? &tm_kpre : (ti.seg == 1 ? &tm_kblk : &tm_ksuf);
                 const CUtensorMap* mv = ti.seg == 0 ? &tm_vpre : (ti.seg == 1 ? &tm_vblk : &tm_vsuf);
@@ -598,18 +655,7 @@ attn_block_tc_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_c
         const bool live = r < rows_in_tile && i < L_eff;
         const size_t q_token = packed ? static_cast<size_t>(seq_base) : static_cast<size_t>(b) * p.L;   // first token of b
         const size_t qrow = ((q_token + (live ? i : 0)) * p.Hq + (live ? h : 0)) * D;
-        // Q row -> shared memory, K-major with the 128-byte swizzle (16-byte chunk c of row r sits at c ^ (r & 7))
-        {
-            const uint4* src = reinterpret_cast<const uint4*>(p.q + qrow);
-            uint8_t* qt = q_s + j * S::Q_BYTES;
-#pragma unroll
-            for (int c = 0; c < D / 8; ++c) {
-                const uint4 v = live ? src[c] : make_uint4(0, 0, 0, 0);
-                *reinterpret_cast<uint4*>(qt + (c >> 3) * HALF_Q + r * 128 + (((c & 7) ^ (r & 7)) << 4)) = v;
-            }
-            fence_proxy_async_smem();
-            mbar_arrive(&bars->q_ready);
-        }
+        mbar_arrive(&bars->q_ready);                   // (this thread's Q row was staged before the barrier above)
         float m_ref = -INFINITY, l = 0.f;              // reference max (log2 domain) and sum of exp2(s - m_ref)
         const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
         const uint32_t tm_o = tmem_base + S::o_col(j) + lane_off;
