@@ -536,20 +536,27 @@ attn_block_tc_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_c
         tmem_relinquish();
     }
     if (warp >= 2) {
-        // Q row -> shared memory, K-major with the 128-byte swizzle (16-byte chunk c of row r sits at c ^ (r & 7));
-        // thread = packed query row r of query tile j
+        // Q rows -> shared memory, K-major with the 128-byte swizzle (16-byte chunk c of row r sits at c ^ (r & 7)).
+        // A warp copies the 32 rows whose softmax it runs, coalesced: one instruction reads 32 / CPR whole rows
+        // (a lane per 16-byte chunk), so that a request touches 2 to 4 cache lines, not one per lane.
+        constexpr int CPR = D / 8;                     // 16-byte chunks per row
         const int j = (warp - 2) >> 2;
-        const int r = (warp & 3) * 32 + lane;
-        const int i = (blockIdx.x * QT + j) * pos_per_tile + r / p.g;
-        const int h = kvh * p.g + r % p.g;
-        const bool live = r < pos_per_tile * p.g && i < L_eff;
+        const int c = lane % CPR;
         const size_t q_token = packed ? static_cast<size_t>(seq_base) : static_cast<size_t>(b) * p.L;
-        const uint4* src = reinterpret_cast<const uint4*>(p.q + ((q_token + (live ? i : 0)) * p.Hq + (live ? h : 0)) * D);
         uint8_t* qt = q_s + j * S::Q_BYTES;
+        uint4 v[CPR];
 #pragma unroll
-        for (int c = 0; c < D / 8; ++c) {
-            const uint4 v = live ? src[c] : make_uint4(0, 0, 0, 0);
-            *reinterpret_cast<uint4*>(qt + (c >> 3) * HALF_Q + r * 128 + (((c & 7) ^ (r & 7)) << 4)) = v;
+        for (int k = 0; k < CPR; ++k) {
+            const int r = (warp & 3) * 32 + k * (32 / CPR) + lane / CPR;
+            const int i = (blockIdx.x * QT + j) * pos_per_tile + r / p.g;
+            const int h = kvh * p.g + r % p.g;
+            const bool live = r < pos_per_tile * p.g && i < L_eff;
+            v[k] = live ? reinterpret_cast<const uint4*>(p.q + ((q_token + i) * p.Hq + h) * D)[c] : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int k = 0; k < CPR; ++k) {
+            const int r = (warp & 3) * 32 + k * (32 / CPR) + lane / CPR;
+            *reinterpret_cast<uint4*>(qt + (c >> 3) * HALF_Q + r * 128 + (((c & 7) ^ (r & 7)) << 4)) = v[k];
         }
         fence_proxy_async_smem();
     }
@@ -654,8 +661,7 @@ attn_block_tc_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_c
         const int h = kvh * p.g + r % p.g;                              // query head
         const bool live = r < rows_in_tile && i < L_eff;
         const size_t q_token = packed ? static_cast<size_t>(seq_base) : static_cast<size_t>(b) * p.L;   // first token of b
-        const size_t qrow = ((q_token + (live ? i : 0)) * p.Hq + (live ? h : 0)) * D;
-        mbar_arrive(&bars->q_ready);                   // (this thread's Q row was staged before the barrier above)
+        mbar_arrive(&bars->q_ready);                   // (the warp's Q rows were staged before the barrier above)
         float m_ref = -INFINITY, l = 0.f;              // reference max (log2 domain) and sum of exp2(s - m_ref)
         const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
         const uint32_t tm_o = tmem_base + S::o_col(j) + lane_off;
@@ -771,22 +777,41 @@ attn_block_tc_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_c
         if (ok && n_tiles > 0) ok = mbar_wait(&bars->pv_done[j][(n_tiles - 1) & 1], ((n_tiles - 1) >> 1) & 1, abort_flag);
         tc_fence_after_sync();
         const float inv = l > 0.f ? 1.f / l : 0.f;
-        __nv_bfloat16* dst = p.out + qrow;
+        // O rows leave through shared memory so that the global stores are coalesced (a thread holds one whole row,
+        // and 32 lanes storing 16 bytes each to 32 different rows cost a request per lane).  The tile's Q rows are
+        // no longer read (every S product has completed: the pipe runs the issuer's MMAs in order and the last P V
+        // has landed), so each warp turns its 32 rows in the place its Q rows had, in the same swizzled layout.
+        uint8_t* ot = q_s + j * S::Q_BYTES;
 #pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-            uint32_t ov[32];
-            tmem_ld_32cols(tm_o + c * 32, ov);          // (whole warp, also for rows that are not stored)
+        for (int c2 = 0; c2 < D / 64; ++c2) {
+            uint32_t oa[32], ob[32];
+            tmem_ld_32cols(tm_o + c2 * 64, oa);          // (whole warp, also for rows that are not stored)
+            tmem_ld_32cols(tm_o + c2 * 64 + 32, ob);
             tmem_ld_wait();
-            if (ok && live) {
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    uint4 o;
-                    o.x = pack_bf16(__uint_as_float(ov[k * 8 + 0]) * inv, __uint_as_float(ov[k * 8 + 1]) * inv);
-                    o.y = pack_bf16(__uint_as_float(ov[k * 8 + 2]) * inv, __uint_as_float(ov[k * 8 + 3]) * inv);
-                    o.z = pack_bf16(__uint_as_float(ov[k * 8 + 4]) * inv, __uint_as_float(ov[k * 8 + 5]) * inv);
-                    o.w = pack_bf16(__uint_as_float(ov[k * 8 + 6]) * inv, __uint_as_float(ov[k * 8 + 7]) * inv);
-                    reinterpret_cast<uint4*>(dst)[c * 4 + k] = o;
-                }
+            for (int k = 0; k < 8; ++k) {
+                const uint32_t (&ov)[32] = k < 4 ? oa : ob;
+                const int k8 = (k & 3) * 8, cc = c2 * 8 + k;
+                uint4 o;
+                o.x = pack_bf16(__uint_as_float(ov[k8 + 0]) * inv, __uint_as_float(ov[k8 + 1]) * inv);
+                o.y = pack_bf16(__uint_as_float(ov[k8 + 2]) * inv, __uint_as_float(ov[k8 + 3]) * inv);
+                o.z = pack_bf16(__uint_as_float(ov[k8 + 4]) * inv, __uint_as_float(ov[k8 + 5]) * inv);
+                o.w = pack_bf16(__uint_as_float(ov[k8 + 6]) * inv, __uint_as_float(ov[k8 + 7]) * inv);
+                *reinterpret_cast<uint4*>(ot + (cc >> 3) * HALF_Q + r * 128 + (((cc & 7) ^ (r & 7)) << 4)) = o;
+            }
+        }
+        __syncwarp();
+        {
+            constexpr int CPR = D / 8;
+            const int c = lane % CPR;
+#pragma unroll
+            for (int k = 0; k < CPR; ++k) {
+                const int r2 = (warp & 3) * 32 + k * (32 / CPR) + lane / CPR;
+                const int i2 = (blockIdx.x * QT + j) * pos_per_tile + r2 / p.g;
+                const int h2 = kvh * p.g + r2 % p.g;
+                if (ok && r2 < rows_in_tile && i2 < L_eff)
+                    reinterpret_cast<uint4*>(p.out + ((q_token + i2) * p.Hq + h2) * D)[c] =
+                        *reinterpret_cast<const uint4*>(ot + (c >> 3) * HALF_Q + r2 * 128 + (((c & 7) ^ (r2 & 7)) << 4));
             }
         }
         if (ok && live && p.lse != nullptr)
