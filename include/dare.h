@@ -10,8 +10,7 @@
  *     dare_lmhead_confidence  LM head + vocabulary softmax -> (argmax token, max probability) per row,
  *                             logits never written to memory
  *     dare_unmask_select      confidence-threshold / per-block top-k commit on the int32 token state
- *     dare_denoise_block      the three above, enqueued back to back (dare_denoise_block_sampled: with the
- *                             sampled head)
+ *     dare_denoise_block      the three above in one call (dare_denoise_block_sampled: with the sampled head)
  *     dare_model_* / dare_generate   the same step with a stack of transformer layers in between, and the
  *                             whole block-by-block loop (dare_linear, dare_rmsnorm, dare_rope_kv_write: its parts)
  *     dare_model_*_window / dare_generate_dual   the same with a cached suffix behind the block (dual cache)
@@ -238,10 +237,18 @@ int dare_unmask_select(dare_ctx* ctx,
                        int32_t* n_committed, int32_t* n_remaining, void* stream);
 
 /*
- * One whole denoising step: dare_attn_block, then dare_lmhead_confidence on the block's rows
+ * One whole denoising step: dare_attn_block, dare_lmhead_confidence on the block's rows
  * (row_tokens taken from tokens[:, block_start : block_start + L], M = B * L), then
  * dare_unmask_select.  `hidden` is the LM-head input for the B*L block positions.  pred/conf are
  * caller-provided [B*L] buffers that also serve as the step's intermediate results.
+ *
+ * Ordering: everything the step reads is taken as `stream` has it when the call is made, and everything it
+ * writes (attn_out, lse, pred, conf, tokens, the counts) is complete for whatever is enqueued on `stream`
+ * afterwards.  Inside the step the attention and the head, neither of which reads what the other writes, are
+ * not kept in sequence: the head runs on a stream of the context, forked from and joined back to `stream` by
+ * events, and the attention's CTAs fill the SMs that the head's GEMM leaves early.  `hidden` and attn_out must
+ * therefore not overlap (nor any other input of one half with an output of the other).  The fork and the join are
+ * capturable in a CUDA graph like any event fork / join.
  */
 int dare_denoise_block(dare_ctx* ctx,
                        int B, int L, int Hq, int Hkv, int d, int prefix_cap, int suffix_cap, float scale,

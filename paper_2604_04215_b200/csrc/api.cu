@@ -131,7 +131,7 @@ int dare_create(dare_ctx** out, int device, size_t workspace_bytes) {
     ctx->workspace_bytes = workspace_bytes ? workspace_bytes : (size_t(256) << 20);
     ctx->workspace = nullptr;
     ctx->dev_status = nullptr;
-    ctx->aux = nullptr; ctx->ev_fork = nullptr; ctx->ev_join = nullptr;
+    ctx->aux = nullptr; ctx->ev_fork = nullptr; ctx->ev_mid = nullptr; ctx->ev_join = nullptr;
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
@@ -141,16 +141,20 @@ int dare_create(dare_ctx** out, int device, size_t workspace_bytes) {
         return DARE_ERR_CUDA;
     }
     ctx->encode_tiled = reinterpret_cast<dare_encode_tiled_fn>(fn);
+    int prio_low = 0, prio_high = 0;      // the side stream takes the highest priority (see dare_denoise_block)
+    if (cudaDeviceGetStreamPriorityRange(&prio_low, &prio_high) != cudaSuccess) prio_high = 0;
     if (cudaMalloc(&ctx->workspace, ctx->workspace_bytes) != cudaSuccess ||
         cudaMalloc(reinterpret_cast<void**>(&ctx->dev_status), sizeof(uint32_t)) != cudaSuccess ||
         cudaMemset(ctx->dev_status, 0, sizeof(uint32_t)) != cudaSuccess ||
-        cudaStreamCreateWithFlags(&ctx->aux, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaStreamCreateWithPriority(&ctx->aux, cudaStreamNonBlocking, prio_high) != cudaSuccess ||
         cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->ev_mid, cudaEventDisableTiming) != cudaSuccess ||
         cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming) != cudaSuccess) {
         if (ctx->workspace) cudaFree(ctx->workspace);
         if (ctx->dev_status) cudaFree(ctx->dev_status);
         if (ctx->aux) cudaStreamDestroy(ctx->aux);
         if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+        if (ctx->ev_mid) cudaEventDestroy(ctx->ev_mid);
         if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
         delete ctx->tmaps;
         delete ctx;
@@ -167,6 +171,7 @@ int dare_destroy(dare_ctx* ctx) {
     cudaFree(ctx->dev_status);
     if (ctx->aux) cudaStreamDestroy(ctx->aux);
     if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+    if (ctx->ev_mid) cudaEventDestroy(ctx->ev_mid);
     if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
     delete ctx->tmaps;
     delete ctx;
@@ -297,30 +302,50 @@ int dare_denoise_block(dare_ctx* ctx, int B, int L, int Hq, int Hkv, int d, int 
     rc = check_select(tokens, B, row_stride, block_start, L, pred, conf, mode, threshold, k);
     if (rc != DARE_OK) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    // The LM head's row compaction reads the token state and `hidden`, not the attention's output: it is enqueued on
-    // the context's side stream, ordered after everything already on `stream` and joined back before the head's
-    // GEMM, so that it runs beside the attention kernel.  (Not when the attention splits K/V: its partials and the
-    // compacted rows share the workspace.)
-    cudaStream_t side = nullptr;
-    if (ctx->aux && dare::attn_plan_splits(ctx, a) == 1) {
-        if (cudaEventRecord(ctx->ev_fork, s) != cudaSuccess || cudaStreamWaitEvent(ctx->aux, ctx->ev_fork, 0) != cudaSuccess)
-            return DARE_ERR_CUDA;
-        side = ctx->aux;
-    }
     // The LM head reads each row's current token straight from the token state: row m = (r, i) lives at
     // tokens[r * row_stride + block_start + i].
-    rc = dare::launch_attn(ctx, a, s);
-    if (rc != DARE_OK) return rc;
+    //
+    // Neither of the step's two halves reads what the other writes: the attention takes q and the caches and writes
+    // attn_out (and lse); the head takes `hidden` and the token state and writes pred, conf and the tokens.  The
+    // head's GEMM is a single wave of CTAs, one per SM, that finish up to a tenth of its duration apart (a CTA owns
+    // 13 or 14 vocabulary tiles, and a tile is the unit of its work), and in that tail a third to a half of the SMs
+    // have nothing to do.  So the head goes first, on the context's side stream (highest priority, ordered after
+    // everything already on `stream`), and the attention is enqueued on `stream` behind the head's row compaction:
+    // both the GEMM and the attention become ready at that point, the GEMM's CTAs take every SM, and the attention's
+    // CTAs (which do not fit beside them) move into the SMs that the GEMM's early finishers leave.  `stream` joins
+    // the side stream at the end, so everything the step wrote is ordered before what the caller enqueues next.
+    // (Not when the attention splits K/V: its partials and the head's scratch share the workspace.)
+    const bool overlap = ctx->aux && dare::attn_plan_splits(ctx, a) == 1;
+    cudaStream_t head = s;
+    if (overlap) {
+        if (cudaEventRecord(ctx->ev_fork, s) != cudaSuccess || cudaStreamWaitEvent(ctx->aux, ctx->ev_fork, 0) != cudaSuccess)
+            return DARE_ERR_CUDA;
+        head = ctx->aux;
+    } else {
+        rc = dare::launch_attn(ctx, a, s);
+        if (rc != DARE_OK) return rc;
+    }
     if (L <= dare::LMHEAD_SELECT_MAX_L) {      // short blocks: the selection rides on the head's merge kernel
         const dare::LmSelectArgs sel = {tokens + block_start, B, mode, threshold, k, n_committed, n_remaining};
-        return dare::launch_lmhead(ctx, ctx->workspace, hidden, M, D, w, V, tokens + block_start, L, row_stride, mask_id,
-                                   exclude_mask_column, pred, conf, s, nullptr, &sel, side);
+        rc = dare::launch_lmhead(ctx, ctx->workspace, hidden, M, D, w, V, tokens + block_start, L, row_stride, mask_id,
+                                 exclude_mask_column, pred, conf, head, nullptr, &sel, overlap ? ctx->ev_mid : nullptr);
+    } else {
+        rc = dare::launch_lmhead(ctx, ctx->workspace, hidden, M, D, w, V, tokens + block_start, L, row_stride, mask_id,
+                                 exclude_mask_column, pred, conf, head, nullptr, nullptr, overlap ? ctx->ev_mid : nullptr);
+        if (rc == DARE_OK)
+            rc = dare::launch_unmask_select(tokens, B, row_stride, block_start, L, pred, conf, mask_id, mode, threshold, k,
+                                            n_committed, n_remaining, head);
     }
-    rc = dare::launch_lmhead(ctx, ctx->workspace, hidden, M, D, w, V, tokens + block_start, L, row_stride, mask_id,
-                             exclude_mask_column, pred, conf, s, nullptr, nullptr, side);
-    if (rc != DARE_OK) return rc;
-    return dare::launch_unmask_select(tokens, B, row_stride, block_start, L, pred, conf, mask_id, mode, threshold, k,
-                                      n_committed, n_remaining, s);
+    if (overlap) {
+        // (also after an error above: `stream` must not be left without its join once the fork has been enqueued)
+        int rc2 = DARE_OK;
+        if (cudaStreamWaitEvent(s, ctx->ev_mid, 0) != cudaSuccess) rc2 = DARE_ERR_CUDA;
+        if (rc == DARE_OK && rc2 == DARE_OK) rc2 = dare::launch_attn(ctx, a, s);
+        if (cudaEventRecord(ctx->ev_join, ctx->aux) != cudaSuccess || cudaStreamWaitEvent(s, ctx->ev_join, 0) != cudaSuccess)
+            rc2 = DARE_ERR_CUDA;
+        if (rc == DARE_OK) rc = rc2;
+    }
+    return rc;
 }
 
 // The step with the sampled head: as dare_denoise_block, the token of every masked row drawn by temperature +

@@ -42,7 +42,7 @@ struct dare_ctx {
     // side stream of dare_denoise_block: the LM head's row compaction does not depend on the attention kernel, so
     // it runs beside it (forked from and joined back into the caller's stream with the two events); NULL = none
     cudaStream_t aux;
-    cudaEvent_t ev_fork, ev_join;
+    cudaEvent_t ev_fork, ev_mid, ev_join;
 };
 
 #include <atomic>
@@ -118,8 +118,8 @@ struct LmSelectArgs { int32_t* tokens_block; int B; int mode; float threshold; i
 int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M, int D, const void* w, int V,
                   const int32_t* row_tokens, int tok_L, int64_t tok_row_stride, int32_t mask_id, int exclude_mask_column, int32_t* pred, float* conf,
                   cudaStream_t stream, const LmSampleArgs* sample, const LmSelectArgs* select = nullptr,
-                  cudaStream_t compact_stream = nullptr);     // non-NULL: the row compaction is enqueued there (the caller
-                                                              // has ordered that stream after `stream`; it is joined back here)
+                  cudaEvent_t after_compaction = nullptr);    // non-NULL: recorded on `stream` behind the row compaction,
+                                                              // i.e. just before the head's GEMM becomes ready to run
 
 struct AttnArgs {
     int B, L, Hq, Hkv, d, prefix_cap, suffix_cap;

@@ -1243,7 +1243,7 @@ size_t lmhead_workspace_bytes(int M, int D, int V, int sm_count, bool with_row_t
 int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M, int D, const void* w, int V,
                   const int32_t* row_tokens, int tok_L, int64_t tok_row_stride, int32_t mask_id,
                   int exclude_mask_column, int32_t* pred, float* conf, cudaStream_t stream, const LmSampleArgs* sample,
-                  const LmSelectArgs* select, cudaStream_t compact_stream) {
+                  const LmSelectArgs* select, cudaEvent_t after_compaction) {
     if (select && (sample || !row_tokens || tok_L > LMHEAD_SELECT_MAX_L || tok_L < 1 || M != select->B * tok_L))
         return DARE_ERR_SHAPE;
     const int n_tiles = (V + BN - 1) / BN;
@@ -1262,16 +1262,12 @@ int launch_lmhead(const dare_ctx* ctx, void* scratch, const void* hidden, int M,
         live_rows = idx + M;
         cur += round_up(static_cast<size_t>(M) * 4 + 4, 1024);
         x_gemm = xc;
-        lmhead_compact_kernel<<<(M + CP_ROWS - 1) / CP_ROWS, CP_ROWS * 32, 0, compact_stream ? compact_stream : stream>>>(
+        lmhead_compact_kernel<<<(M + CP_ROWS - 1) / CP_ROWS, CP_ROWS * 32, 0, stream>>>(
             static_cast<const uint4*>(hidden), M, D / 8, row_tokens, tok_L, tok_row_stride, mask_id,
             static_cast<uint4*>(xc), idx, live_rows, pred, conf); note_launch();
         if (cudaGetLastError() != cudaSuccess) return DARE_ERR_CUDA;
-        if (compact_stream) {     // the rest of the head, on `stream`, comes after the compaction on its side stream
-            if (cudaEventRecord(ctx->ev_join, compact_stream) != cudaSuccess ||
-                cudaStreamWaitEvent(stream, ctx->ev_join, 0) != cudaSuccess)
-                return DARE_ERR_CUDA;
-        }
     }
+    if (after_compaction && cudaEventRecord(after_compaction, stream) != cudaSuccess) return DARE_ERR_CUDA;
     size_t groups_max = static_cast<size_t>(ctx->sm_count);
     if (groups_max > static_cast<size_t>(n_tiles)) groups_max = n_tiles;
     const bool greedy_pairs = sample == nullptr && grid >= 2 && lm_pair_available();
@@ -1517,7 +1513,7 @@ extern "C" int dare_lmhead_confidence_static(const void* hidden, int M, int D, c
     // a context-shaped view of the static state for the shared launcher; nothing here is allocated
     dare_ctx view;
     view.tmaps = nullptr;
-    view.aux = nullptr; view.ev_fork = nullptr; view.ev_join = nullptr;
+    view.aux = nullptr; view.ev_fork = nullptr; view.ev_mid = nullptr; view.ev_join = nullptr;
     view.device = st->device;
     view.sm_count = st->sm_count;
     view.workspace = st->scratch;
