@@ -265,10 +265,11 @@ int dare_denoise_block(dare_ctx* ctx,
                        int32_t* n_committed, int32_t* n_remaining, void* stream);
 
 /*
- * The same step with the sampled head (Section 4.2: several different rollouts per prompt): dare_attn_block, then
+ * The same step with the sampled head (Section 4.2: several different rollouts per prompt): dare_attn_block,
  * dare_lmhead_sample on the block's rows (temperature, seed and step counter as there), then dare_unmask_select on
- * the sampled tokens and their temperature-1 probabilities.  Same buffers and rules as dare_denoise_block;
- * temperature must be finite and > 0 (DARE_ERR_RANGE otherwise).
+ * the sampled tokens and their temperature-1 probabilities.  Same buffers, rules and ordering as dare_denoise_block
+ * (the head on the context's stream, the attention beside it); temperature must be finite and > 0 (DARE_ERR_RANGE
+ * otherwise).
  */
 int dare_denoise_block_sampled(dare_ctx* ctx, int B, int L, int Hq, int Hkv, int d, int prefix_cap, int suffix_cap,
                                float scale, const void* q, const void* k_pre, const void* v_pre,

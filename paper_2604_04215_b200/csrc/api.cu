@@ -282,26 +282,12 @@ int dare_unmask_select(dare_ctx* ctx, int32_t* tokens, int B, int64_t row_stride
                                       n_committed, n_remaining, static_cast<cudaStream_t>(stream));
 }
 
-int dare_denoise_block(dare_ctx* ctx, int B, int L, int Hq, int Hkv, int d, int prefix_cap, int suffix_cap,
-                       float scale, const void* q, const void* k_pre, const void* v_pre, const int32_t* prefix_len,
-                       const void* k_blk, const void* v_blk, const void* k_suf, const void* v_suf,
-                       const int32_t* suffix_len, void* attn_out, float* lse, const void* hidden, int D, const void* w,
-                       int V, int32_t mask_id, int exclude_mask_column, int32_t* tokens, int64_t row_stride,
-                       int block_start, int mode, float threshold, int k, int32_t* pred, float* conf,
-                       int32_t* n_committed, int32_t* n_remaining, void* stream) {
-    // validate everything first: on any error nothing is launched
-    dare::AttnArgs a;
-    int rc = check_attn(ctx, B, L, Hq, Hkv, d, prefix_cap, suffix_cap, scale, q, k_pre, v_pre, k_blk, v_blk, k_suf,
-                        v_suf, attn_out, &a);
-    if (rc != DARE_OK) return rc;
-    a.prefix_len = prefix_len; a.suffix_len = suffix_len; a.lse = lse;
-    if (static_cast<long long>(B) * L > 0x7fffffffLL) return DARE_ERR_SHAPE;
-    const int M = B * L;
-    rc = check_lmhead(ctx, hidden, M, D, w, V, true, pred, conf);
-    if (rc != DARE_OK) return rc;
-    rc = check_select(tokens, B, row_stride, block_start, L, pred, conf, mode, threshold, k);
-    if (rc != DARE_OK) return rc;
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
+// The launches of one step, shared by the greedy and the sampled entry point (every argument has been validated).
+static int enqueue_step(dare_ctx* ctx, const dare::AttnArgs& a, const void* hidden, int M, int D, const void* w, int V,
+                        int32_t mask_id, int exclude_mask_column, const dare::LmSampleArgs* sample, int32_t* tokens,
+                        int B, int L, int64_t row_stride, int block_start, int mode, float threshold, int k,
+                        int32_t* pred, float* conf, int32_t* n_committed, int32_t* n_remaining, cudaStream_t s) {
+    int rc = DARE_OK;
     // The LM head reads each row's current token straight from the token state: row m = (r, i) lives at
     // tokens[r * row_stride + block_start + i].
     //
@@ -325,13 +311,13 @@ int dare_denoise_block(dare_ctx* ctx, int B, int L, int Hq, int Hkv, int d, int 
         rc = dare::launch_attn(ctx, a, s);
         if (rc != DARE_OK) return rc;
     }
-    if (L <= dare::LMHEAD_SELECT_MAX_L) {      // short blocks: the selection rides on the head's merge kernel
+    if (sample == nullptr && L <= dare::LMHEAD_SELECT_MAX_L) {      // short blocks: the selection rides on the greedy head's merge kernel
         const dare::LmSelectArgs sel = {tokens + block_start, B, mode, threshold, k, n_committed, n_remaining};
         rc = dare::launch_lmhead(ctx, ctx->workspace, hidden, M, D, w, V, tokens + block_start, L, row_stride, mask_id,
                                  exclude_mask_column, pred, conf, head, nullptr, &sel, overlap ? ctx->ev_mid : nullptr);
     } else {
         rc = dare::launch_lmhead(ctx, ctx->workspace, hidden, M, D, w, V, tokens + block_start, L, row_stride, mask_id,
-                                 exclude_mask_column, pred, conf, head, nullptr, nullptr, overlap ? ctx->ev_mid : nullptr);
+                                 exclude_mask_column, pred, conf, head, sample, nullptr, overlap ? ctx->ev_mid : nullptr);
         if (rc == DARE_OK)
             rc = dare::launch_unmask_select(tokens, B, row_stride, block_start, L, pred, conf, mask_id, mode, threshold, k,
                                             n_committed, n_remaining, head);
@@ -346,6 +332,30 @@ int dare_denoise_block(dare_ctx* ctx, int B, int L, int Hq, int Hkv, int d, int 
         if (rc == DARE_OK) rc = rc2;
     }
     return rc;
+}
+
+int dare_denoise_block(dare_ctx* ctx, int B, int L, int Hq, int Hkv, int d, int prefix_cap, int suffix_cap,
+                       float scale, const void* q, const void* k_pre, const void* v_pre, const int32_t* prefix_len,
+                       const void* k_blk, const void* v_blk, const void* k_suf, const void* v_suf,
+                       const int32_t* suffix_len, void* attn_out, float* lse, const void* hidden, int D, const void* w,
+                       int V, int32_t mask_id, int exclude_mask_column, int32_t* tokens, int64_t row_stride,
+                       int block_start, int mode, float threshold, int k, int32_t* pred, float* conf,
+                       int32_t* n_committed, int32_t* n_remaining, void* stream) {
+    // validate everything first: on any error nothing is launched
+    dare::AttnArgs a;
+    int rc = check_attn(ctx, B, L, Hq, Hkv, d, prefix_cap, suffix_cap, scale, q, k_pre, v_pre, k_blk, v_blk, k_suf,
+                        v_suf, attn_out, &a);
+    if (rc != DARE_OK) return rc;
+    a.prefix_len = prefix_len; a.suffix_len = suffix_len; a.lse = lse;
+    if (static_cast<long long>(B) * L > 0x7fffffffLL) return DARE_ERR_SHAPE;
+    const int M = B * L;
+    rc = check_lmhead(ctx, hidden, M, D, w, V, true, pred, conf);
+    if (rc != DARE_OK) return rc;
+    rc = check_select(tokens, B, row_stride, block_start, L, pred, conf, mode, threshold, k);
+    if (rc != DARE_OK) return rc;
+    return enqueue_step(ctx, a, hidden, M, D, w, V, mask_id, exclude_mask_column, nullptr, tokens, B, L, row_stride,
+                        block_start, mode, threshold, k, pred, conf, n_committed, n_remaining,
+                        static_cast<cudaStream_t>(stream));
 }
 
 // The step with the sampled head: as dare_denoise_block, the token of every masked row drawn by temperature +
@@ -370,15 +380,10 @@ int dare_denoise_block_sampled(dare_ctx* ctx, int B, int L, int Hq, int Hkv, int
     if (!(temperature > 0.f) || isinf(temperature)) return DARE_ERR_RANGE;
     rc = check_select(tokens, B, row_stride, block_start, L, pred, conf, mode, threshold, k);
     if (rc != DARE_OK) return rc;
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    rc = dare::launch_attn(ctx, a, s);
-    if (rc != DARE_OK) return rc;
     const dare::LmSampleArgs smp = {temperature, seed, step};
-    rc = dare::launch_lmhead(ctx, ctx->workspace, hidden, M, D, w, V, tokens + block_start, L, row_stride, mask_id,
-                             exclude_mask_column, pred, conf, s, &smp);
-    if (rc != DARE_OK) return rc;
-    return dare::launch_unmask_select(tokens, B, row_stride, block_start, L, pred, conf, mask_id, mode, threshold, k,
-                                      n_committed, n_remaining, s);
+    return enqueue_step(ctx, a, hidden, M, D, w, V, mask_id, exclude_mask_column, &smp, tokens, B, L, row_stride,
+                        block_start, mode, threshold, k, pred, conf, n_committed, n_remaining,
+                        static_cast<cudaStream_t>(stream));
 }
 
 }  // extern "C"
