@@ -135,7 +135,16 @@ lmhead_compact_kernel(const uint4* __restrict__ x, int M, int D8, const int32_t*
     if (lane == 0) idx[before] = row;
     const uint4* src = x + static_cast<size_t>(row) * D8;
     uint4* dst = xc + static_cast<size_t>(before) * D8;
-    for (int i = lane; i < D8; i += 32) dst[i] = src[i];
+    // eight loads in flight per lane before the first store: the copy of a row is a chain of latencies otherwise
+    int i = lane;
+    for (; i + 7 * 32 < D8; i += 8 * 32) {
+        uint4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v[u] = src[i + u * 32];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) dst[i + u * 32] = v[u];
+    }
+    for (; i < D8; i += 32) dst[i] = src[i];
 }
 
 // Sampling epilogue (temperature + Gumbel-max): token = argmax_v (z_v / T + g_v), g_v = -ln(-ln u_v), with u_v from
