@@ -561,15 +561,16 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
 // vocabulary group, CTA of the pair) goes to the merge kernel.
 constexpr int SW_BV = 128;                               // vocabulary rows per CTA and tile
 constexpr int SW_NMAX = 256;                             // rows (accumulator columns) per chunk
-constexpr int SW_STAGES = 6;
+constexpr int SW_STAGES = 6;                             // ring slots when a CTA's X tile has its full 128 rows
+constexpr int SW_MAX_STAGES = 11;                        // ... and when it is small: the ring's bytes are cut into more slots
 constexpr int SW_W_BYTES = SW_BV * BK * 2;               // 16 KB
 constexpr int SW_X_BYTES = (SW_NMAX / 2) * BK * 2;       // each CTA loads half of the chunk's rows: up to 16 KB
 constexpr int SW_STAGE_BYTES = SW_W_BYTES + SW_X_BYTES;
 constexpr int SW_XP_FLOATS = 32 * 33;                    // per epilogue warp: one 32 x 32 block, rows padded to 33
 constexpr int SW_PARTS_PER_GROUP = 2;                    // one per CTA of the pair
 struct SwBarriers {
-    uint64_t full[SW_STAGES];
-    uint64_t empty[SW_STAGES];
+    uint64_t full[SW_MAX_STAGES];
+    uint64_t empty[SW_MAX_STAGES];
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
     uint64_t fold_full, fold_empty;                      // the epilogue warps' exchange at the end of an item
@@ -637,8 +638,14 @@ lm_swapped_body(const CUtensorMap& tmap_w, const SwXMaps& xmaps, int Mc, int D, 
     const int warp = warp_index_uniform();
     const int lane = threadIdx.x & 31;
 
+    // A ring slot holds a 16 KB W tile and the X rows this CTA loads.  With few live rows the X part is small and the
+    // ring's bytes make more slots: while W streams from HBM, what a CTA has in flight is what bounds its share of the
+    // bandwidth (6 slots per CTA, 14 MB over the GPU, covered ~2 us of HBM latency at 6.3 TB/s and no more).
+    const SwBoxes xbox = sw_boxes(rows_half);
+    const int stage_bytes = SW_W_BYTES + ((xbox.rows * 128 + 1023) & ~1023);
+    const int n_stages = min(SW_MAX_STAGES, SW_STAGES * SW_STAGE_BYTES / stage_bytes);
     if (threadIdx.x == 0) {
-        for (int s = 0; s < SW_STAGES; ++s) {
+        for (int s = 0; s < n_stages; ++s) {
             mbar_init(&bars->full[s], 1);
             mbar_init(&bars->empty[s], 1);
         }
@@ -668,7 +675,7 @@ lm_swapped_body(const CUtensorMap& tmap_w, const SwXMaps& xmaps, int Mc, int D, 
             uint32_t phase = 0;
             bool ok = true;
             const uint32_t full0 = cluster_map_shared(smem_u32(&bars->full[0]), 0);   // the even CTA's barriers count both CTAs' bytes
-            const SwBoxes box = sw_boxes(rows_half);
+            const SwBoxes box = xbox;
             const uint32_t stage_tx = 2u * static_cast<uint32_t>(SW_W_BYTES + box.rows * 128);
             for (int item = unit; item < n_items && ok; item += n_units) {
                 const int x_row0 = (item % plan.n_chunks) * nc + rank * rows_half;
@@ -676,7 +683,7 @@ lm_swapped_body(const CUtensorMap& tmap_w, const SwXMaps& xmaps, int Mc, int D, 
                     const int w_row0 = vt * (2 * SW_BV) + rank * SW_BV;
                     for (int kb = 0; kb < num_k; ++kb) {
                         if (!mbar_wait(&bars->empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
-                        uint8_t* w_dst = tiles + stage * SW_STAGE_BYTES;
+                        uint8_t* w_dst = tiles + stage * stage_bytes;
                         uint8_t* x_dst = w_dst + SW_W_BYTES;
                         const uint32_t full = full0 + stage * static_cast<uint32_t>(sizeof(uint64_t));
                         if (rank == 0) mbar_arrive_expect_tx(&bars->full[stage], stage_tx);
@@ -685,7 +692,7 @@ lm_swapped_body(const CUtensorMap& tmap_w, const SwXMaps& xmaps, int Mc, int D, 
                         if (box.i2 >= 0)
                             tma_load_2d_pair(x_dst + (128 >> box.i1) * 128, &xmaps.m[box.i2], full, kb * BK,
                                              x_row0 + (128 >> box.i1));
-                        if (++stage == SW_STAGES) { stage = 0; phase ^= 1; }
+                        if (++stage == n_stages) { stage = 0; phase ^= 1; }
                     }
                 }
             }
@@ -710,7 +717,7 @@ lm_swapped_body(const CUtensorMap& tmap_w, const SwXMaps& xmaps, int Mc, int D, 
                     ok = __all_sync(0xffffffffu, mbar_wait(&bars->full[stage], phase, abort_flag));
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const uint32_t w_addr = smem_u32(tiles + stage * SW_STAGE_BYTES);
+                    const uint32_t w_addr = smem_u32(tiles + stage * stage_bytes);
                     const uint64_t a_desc = umma_desc_sw128_kmajor(w_addr);
                     const uint64_t b_desc = umma_desc_sw128_kmajor(w_addr + SW_W_BYTES);
                     if (leader) {
@@ -720,7 +727,7 @@ lm_swapped_body(const CUtensorMap& tmap_w, const SwXMaps& xmaps, int Mc, int D, 
                         umma_commit_pair(&bars->empty[stage], 3);      // frees the stage in both CTAs
                     }
                     __syncwarp();
-                    if (++stage == SW_STAGES) { stage = 0; phase ^= 1; }
+                    if (++stage == n_stages) { stage = 0; phase ^= 1; }
                 }
                 if (ok && leader) umma_commit_pair(&bars->tmem_full[acc], 3);
                 __syncwarp();
