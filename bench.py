@@ -381,7 +381,10 @@ def bench_step_workload(dare, ctx, wl, steps, warmup, rank, world, sampler, with
     torch.cuda.synchronize()
     i1 = time.time()
     del spacer
-    inst_clocks = sampler.window(i0, i1) if sampler else None
+    # Clock samples for the pass: its own window, and, when it carried on directly behind a long timed region (no idle
+    # in between), that region's samples as well: a pass of 0.2 s catches two or three samples, taken between launches,
+    # and the GPU's state is the one the seconds of the same load before it left.
+    inst_clocks = (sampler.window(w0 if settle_s == 0.0 else i0, i1)) if sampler else None
     lm_each = np.array([ev[t][1].elapsed_time(ev[t][2]) for t in range(n_inst)])
     attn_each = np.array([ev[t][0].elapsed_time(ev[t][1]) for t in range(n_inst)])
     lm_ms, attn_ms_events = float(lm_each.mean()), float(attn_each.mean())
