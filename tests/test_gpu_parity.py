@@ -269,6 +269,42 @@ def test_tiny_workload_eight_iterations(ctx):
             assert total > 8           # planted confidences exercise the threshold branch
 
 
+def test_step_replays_from_a_cuda_graph(ctx):
+    """The step forks its LM head onto a stream of the context and joins it back by events: captured into a CUDA graph
+    on the caller's stream, a replay must give what the eager call gives (tokens, counts, attention output)."""
+    wl = I.WORKLOADS["tiny"]
+    w = I.make_weights(wl)
+    caches = I.make_caches(wl)
+    wd, kp, vp = w.cuda(), caches[0].cuda(), caches[1].cuda()
+    si = I.make_step(wl, step=0, planted=True, w=w, caches=caches)
+    q, plen, kb, vb, x = si.q.cuda(), si.prefix_len.cuda(), si.k_blk.cuda(), si.v_blk.cuda(), si.x.cuda()
+    tok0 = I.fresh_tokens(wl).cuda()
+    bufs = {}
+    for name in ("eager", "graph"):
+        bufs[name] = dict(tok=tok0.clone(), out=torch.zeros_like(q), pred=torch.zeros(wl.M, dtype=torch.int32, device="cuda"),
+                          conf=torch.zeros(wl.M, dtype=torch.float32, device="cuda"),
+                          nc=torch.zeros(wl.batch, dtype=torch.int32, device="cuda"),
+                          nr=torch.zeros(wl.batch, dtype=torch.int32, device="cuda"))
+
+    def step(b, stream=None):
+        dare.dare_denoise_block(ctx, q, kp, vp, plen, kb, vb, None, None, None, b["out"], None, x, wd, wl.mask_id, True,
+                                b["tok"], si.block_start, wl.mode, wl.threshold, wl.k, b["pred"], b["conf"], b["nc"], b["nr"],
+                                stream=stream)
+
+    step(bufs["eager"])                          # (also raises the kernels' shared-memory limits before the capture)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        step(bufs["graph"], stream=torch.cuda.current_stream())
+    bufs["graph"]["tok"].copy_(tok0)             # whatever ran or did not run during the capture: start over
+    g.replay()
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    for key in ("tok", "out", "pred", "conf", "nc", "nr"):
+        assert torch.equal(bufs["eager"][key], bufs["graph"][key]), key
+    assert int(bufs["graph"]["nc"].sum()) >= 1
+
+
 # ----------------------------------------------------------------------------- ABI error behaviour
 def test_bad_arguments_are_rejected_before_any_launch(ctx):
     q = torch.zeros(1, 4, 2, 64, dtype=torch.bfloat16, device="cuda")
