@@ -444,7 +444,9 @@ def bench_step_workload(dare, ctx, wl, steps, warmup, rank, world, sampler, with
                  "lmhead_ms": lm_ms, "select_ms": sel_ms, "attn_GBps": attn_roof["achieved"],
                  "attn_frac_hbm": attn_roof["frac"], "attn_tflops": attn_roof["tflops"],
                  "lmhead_tflops": lm_roof["achieved"], "lmhead_frac": lm_roof["frac"],
-                 "host_us_per_dare_denoise_block_call": host_us}
+                 "host_us_per_dare_denoise_block_call": host_us,
+                 "note": "parts timed one entry point at a time; inside dare_denoise_block the attention runs beside the "
+                         "LM head's GEMM (in the SMs its early finishers leave), so a step takes less than their sum"}
 
     # ---- the LM head's variants on all rows (sampling epilogue, log-probability head and its backward)
     if with_heads and wl.M % 8 == 0 and wl.vocab % 8 == 0:
