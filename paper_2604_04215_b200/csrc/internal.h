@@ -39,8 +39,9 @@ struct dare_ctx {
     uint32_t* dev_status;   // device word, bits DARE_DEV_*
     dare_encode_tiled_fn encode_tiled;
     TmapCache* tmaps;       // host memory; NULL = encode on every call
-    // side stream of dare_denoise_block: the LM head's row compaction does not depend on the attention kernel, so
-    // it runs beside it (forked from and joined back into the caller's stream with the two events); NULL = none
+    // side stream of the step (dare_denoise_block, highest priority): the LM head runs on it, forked from the caller's
+    // stream (ev_fork) and joined back (ev_join); ev_mid marks the end of the head's row compaction, behind which the
+    // attention is enqueued on the caller's stream.  NULL = none (the step then runs in sequence)
     cudaStream_t aux;
     cudaEvent_t ev_fork, ev_mid, ev_join;
 };
