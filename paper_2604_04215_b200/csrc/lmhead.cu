@@ -549,10 +549,11 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
 //   * no padding to 128-row tiles: a step with 96 masked rows issues MMAs of N = 96, not of 128 padded rows;
 //   * every work item is a CTA pair whatever the row count, and the 128-row vocabulary tiles per CTA spread evenly
 //     over the SMs: with few rows left the W stream is the bound and the kernel reads it at the copy bandwidth.
-// It is used while at most SW_NMAX rows are live.  Above that the step is bound by the tensor pipe, where it does
-// not pay: an MMA reads its 128 x 16 A operand from shared memory in ~116 cycles whatever N is, so two chunks of
-// N = 144 cost what two chunks of N = 256 cost (measured: 319 us for 288 rows, 350 us for 512), and the row-major
-// kernel above, whose A operand is the row tile, does the same work in as many or fewer MMAs.
+// More rows than SW_NMAX are cut into equal chunks (items = chunk x vocabulary group); lm_greedy_swapped says for
+// which counts that beats the row-major tiles.  An MMA alone takes max(N / 2, ~45) cycles whether M is 64 or 128 and
+// wherever A sits (timed in isolation), but here every MMA takes a fresh 128 x 16 slab of W as its A operand, so a
+// chunk streams all of W from L2 into the SMs whatever its N: two chunks of N = 144 cost nearly what two chunks of
+// N = 256 cost (319 us for 288 rows, 350 us for 512), and only chunks close to 256 rows are worth it.
 // The price is the epilogue: a thread's TMEM lane is now a vocabulary entry and the softmax runs ACROSS lanes.
 // Each epilogue warp turns its 32 x 32 block of logits through shared memory (padded rows, conflict-free) so that
 // a thread again holds 32 consecutive vocabulary entries of ONE row, and keeps that row's running
@@ -561,6 +562,21 @@ lmhead_partial_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
 // vocabulary group, CTA of the pair) goes to the merge kernel.
 constexpr int SW_BV = 128;                               // vocabulary rows per CTA and tile
 constexpr int SW_NMAX = 256;                             // rows (accumulator columns) per chunk
+// Row counts for which the greedy head takes this path: up to one chunk, where W is streamed once and the launch is
+// bound by HBM; and, up to 1024 rows, counts that cut into chunks of 208 to 240 rows, i.e. whose row-major tiles
+// would carry 64 or more padded rows per pair (measured in one process, us, swapped against row-major: D = 4096,
+// V = 126464: 416 rows 333 / 380, 448 rows 415 / 462, 480 rows 410 / 428, 512 rows 425 / 421; D = 3584, V = 152064:
+// 704 rows 625 / 650, 832 rows 784 / 840, 960 rows 851 / 895).  With shorter chunks the path loses (288 to 384 rows:
+// 339 to 372 against 329 to 343): every MMA of this path takes a fresh 128 x 16 slab of W as its A operand, so a
+// chunk streams all of W from L2 into the SMs whatever its N, and at N = 144 to 192 that stream (~12 TB/s over the
+// GPU), not the tensor pipe, sets the pace.
+__host__ __device__ inline bool lm_greedy_swapped(int rows) {
+    if (rows <= SW_NMAX) return true;
+    if (rows > 1024) return false;
+    const int n_chunks = (rows + SW_NMAX - 1) / SW_NMAX;
+    const int nc = ((rows + n_chunks - 1) / n_chunks + 15) & ~15;      // as in sw_plan below
+    return nc >= 208 && nc < SW_NMAX;
+}
 constexpr int SW_STAGES = 6;                             // ring slots when a CTA's X tile has its full 128 rows
 constexpr int SW_MAX_STAGES = 11;                        // ... and when it is small: the ring's bytes are cut into more slots
 constexpr int SW_W_BYTES = SW_BV * BK * 2;               // 16 KB
@@ -869,8 +885,9 @@ __host__ __device__ inline int lm_mixed_pair_clusters(int n_clusters, int p) {
 }
 
 // The greedy head, one launch on CTA pairs whatever the number of live rows (known only on the device when rows are
-// skipped): up to SW_NMAX rows the swapped-operand path; above that row-major tiles of 128 rows, on CTA pairs when
-// the tiles come in twos, and for an odd count on pairs plus single CTAs for the last tile (see above).  The W
+// skipped): the swapped-operand path for the counts lm_greedy_swapped names (up to SW_NMAX rows, and counts that
+// cut into long chunks); otherwise row-major tiles of 128 rows, on CTA pairs when the tiles come in twos, and for
+// an odd count on pairs plus single CTAs for the last tile (see above).  The W
 // tile box is 128 rows for all of them.  A row's partials start at row * parts_stride; how many there are follows
 // from the same rules in lm_row_partials.
 __global__ void __launch_bounds__(LM_THREADS, 1)
@@ -879,7 +896,7 @@ lmhead_greedy_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_co
                      float* __restrict__ part_max, float* __restrict__ part_sum, int32_t* __restrict__ part_arg,
                      uint32_t* __restrict__ dev_status, int parts_stride) {
     const int Mc = live_rows ? *live_rows : M;          // rows that need logits (uniform over the grid)
-    if (Mc <= SW_NMAX) {
+    if (lm_greedy_swapped(Mc)) {
         lm_swapped_body(tmap_w, xmaps, Mc, D, V, mask_col, n_tiles, part_max, part_sum, part_arg, dev_status, parts_stride);
         return;
     }
@@ -919,7 +936,7 @@ __host__ __device__ inline int lm_row_partials(int layout, int grid, int rows, i
     const int m_tiles = (rows + BM - 1) / BM;
     if (layout != LM_LAYOUT_GREEDY) return lm_groups_mode(grid, m_tiles, n_tiles, layout);
     const int n_clusters = grid >> 1;
-    if (rows <= SW_NMAX) return sw_plan(rows, n_clusters, n_tiles).parts;
+    if (lm_greedy_swapped(rows)) return sw_plan(rows, n_clusters, n_tiles).parts;
     if ((m_tiles & 1) == 0) return lm_groups(n_clusters, m_tiles >> 1, n_tiles);
     if (n_clusters < 2) return lm_groups(grid, m_tiles, n_tiles);
     const int p = m_tiles >> 1;

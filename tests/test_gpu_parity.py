@@ -108,22 +108,26 @@ def test_lmhead_without_exclusion_and_with_committed_rows(ctx):
 
 @pytest.mark.parametrize("M,D,V,mu,with_rows", [
     (256, 320, 2600, 7, False),        # 256 rows known on the host: the swapped-operand path (vocabulary on the lanes)
-    (500, 128, 1000, 999, False),      # four row tiles, ragged last one: row-major CTA pairs
+    (500, 128, 1000, 999, False),      # four row tiles, ragged last one (two chunks would be 256 long): row-major CTA pairs
     (600, 256, 2048, 5, True),         # 200 masked rows, known only on the device: swapped path, N = 208
-    (1400, 64, 1200, 3, True),         # 467 masked rows = four tiles: pairs
+    (1500, 64, 1200, 3, True),         # 500 masked rows = four tiles, known only on the device: pairs
+    (1400, 64, 1200, 3, True),         # 467 masked rows: swapped path, two chunks of N = 240
     (900, 64, 1200, 3, True),          # 300 masked rows = three tiles: one pair of tiles and a single tile
-    (640, 128, 1000, 999, False),      # five row tiles known on the host: pairs for four, single CTAs for the fifth
-    (1900, 64, 1200, 3, True),         # ~634 masked rows = five tiles, known only on the device
-    (2560, 64, 1200, 3, True),         # ~855 masked rows = seven tiles: three tile pairs and a single tile
+    (560, 128, 1000, 999, False),      # five row tiles known on the host: pairs for four, single CTAs for the fifth
+    (640, 128, 1000, 999, False),      # 640 rows known on the host: swapped path, three chunks of N = 224
+    (1900, 64, 1200, 3, True),         # ~634 masked rows, known only on the device: three chunks
+    (2560, 64, 1200, 3, True),         # ~855 masked rows: four chunks of N = 224
+    (1100, 64, 1200, 3, False),        # nine row tiles (beyond the swapped path's range): four tile pairs and a single tile
     (300, 1024, 2600, 2599, False),    # three tiles on a small grid (16 clusters: 10 run the pair, 12 CTAs the third tile)
     (72, 200, 700, 0, False),          # swapped path, each CTA of a pair loads 40 rows as boxes of 32 + 8
     (330, 64, 520, 519, True),         # 110 masked rows: N = 112, one box of 64 rows per CTA covers its 56
 ])
 def test_lmhead_single_and_pair_modes(ctx, M, D, V, mu, with_rows):
     """The greedy head's one kernel has three GEMM paths, picked by the number of live rows (on the device when rows
-    are skipped): up to 256 rows the swapped-operand path on CTA pairs; above that row-major tiles of 128 rows, on
-    CTA pairs when the tiles come in twos, and for an odd count on pairs for all but the last tile while the CTAs of
-    the remaining clusters work on that one singly."""
+    are skipped): the swapped-operand path on CTA pairs up to 256 rows and, in chunks, for counts up to 1024 that cut
+    into chunks of 208 to 240 rows; otherwise row-major tiles of 128 rows, on CTA pairs when the tiles come in twos,
+    and for an odd count on pairs for all but the last tile while the CTAs of the remaining clusters work on that one
+    singly."""
     _lm_case(ctx, M, D, V, mu, seed=M + D, with_rows=with_rows)
 
 
