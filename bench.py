@@ -47,7 +47,7 @@ NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the workload's dominant kernel, from the ncu
 # captures summarised under profiles/ (LM head: W leaves HBM once; dual-cache attention: the quarter-batch capture
 # scaled by the batch, traffic grows in proportion to the rollouts)
-DOMINANT_TRAFFIC_BYTES = {"llada8b": 1.0638e9, "dualcache": 4 * (1.3595e9 + 4.8e6)}
+DOMINANT_TRAFFIC_BYTES = {"llada8b": 1.0681e9, "dualcache": 4 * (1.3595e9 + 4.8e6)}
 EXTRA_WORKLOADS = ("dream7b", "dualcache", "llada_loop")
 
 
