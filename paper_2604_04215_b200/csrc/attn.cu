@@ -608,49 +608,57 @@ attn_block_tc_kernel(const __grid_constant__ CUtensorMap tm_kpre, const __grid_c
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            constexpr uint32_t idesc_s = umma_idesc_bf16(128, TC_KT);
-            constexpr uint32_t idesc_o = umma_idesc_bf16(128, D) | UMMA_B_MN_MAJOR;
-            // descriptor lower words (address >> 4 [| leading byte offset]); the upper word is a constant
-            const uint32_t q_lo = smem_u32(q_s) >> 4, kv_lo = smem_u32(kv_s) >> 4;
-            const uint32_t v_lbo = static_cast<uint32_t>(HALF_K >> 4) << 16;   // second 64 head-dim columns: one half tile on
-            bool ok = mbar_wait(&bars->q_ready, 0, abort_flag);
-            // S_j(t) = Q_j K_t^T into tile j's buffer t % NBUF (whatever that buffer held has been consumed: the P V
-            // product that read it was issued before this, and the pipe keeps the issue order)
-            auto issue_s = [&](int j, int t) -> bool {
-                const int stage = t % STAGES;
-                if (!mbar_wait(&bars->full[stage], (t / STAGES) & 1, abort_flag)) return false;
-                tc_fence_after_sync();
-                const uint32_t k_lo = kv_lo + stage * (S::KV_STAGE >> 4), qj = q_lo + j * (S::Q_BYTES >> 4);
-                const uint32_t sd = tmem_base + S::s_col(j, t % NBUF);
+        // All 32 lanes run the loops (waits, counters and descriptors stay warp-uniform, in the registers the MMA
+        // instruction takes its operands from); one elected lane issues the MMAs and their commits.
+        const bool leader = elect_one_sync();
+        constexpr uint32_t idesc_s = umma_idesc_bf16(128, TC_KT);
+        constexpr uint32_t idesc_o = umma_idesc_bf16(128, D) | UMMA_B_MN_MAJOR;
+        // descriptor lower words (address >> 4 [| leading byte offset]); the upper word is a constant
+        const uint32_t q_lo = smem_u32(q_s) >> 4, kv_lo = smem_u32(kv_s) >> 4;
+        const uint32_t v_lbo = static_cast<uint32_t>(HALF_K >> 4) << 16;   // second 64 head-dim columns: one half tile on
+        bool ok = __all_sync(0xffffffffu, mbar_wait(&bars->q_ready, 0, abort_flag));
+        // S_j(t) = Q_j K_t^T into tile j's buffer t % NBUF (whatever that buffer held has been consumed: the P V
+        // product that read it was issued before this, and the pipe keeps the issue order)
+        auto issue_s = [&](int j, int t) -> bool {
+            const int stage = t % STAGES;
+            if (!__all_sync(0xffffffffu, mbar_wait(&bars->full[stage], (t / STAGES) & 1, abort_flag))) return false;
+            tc_fence_after_sync();
+            const uint32_t k_lo = kv_lo + stage * (S::KV_STAGE >> 4), qj = q_lo + j * (S::Q_BYTES >> 4);
+            const uint32_t sd = tmem_base + S::s_col(j, t % NBUF);
+            if (leader) {
                 umma_bf16_lo<false>(sd, qj, k_lo, idesc_s);
 #pragma unroll
                 for (int kk = 1; kk < D / 16; ++kk)     // 16 channels = 32 bytes along the swizzled row: +2
                     umma_bf16_lo<true>(sd, qj + (kk >> 2) * (HALF_Q >> 4) + 2 * (kk & 3),
                                        k_lo + (kk >> 2) * (HALF_K >> 4) + 2 * (kk & 3), idesc_s);
                 umma_commit(&bars->s_full[j][t & 1]);
-                return true;
-            };
-            for (int t = 0; t < NBUF && t < n_tiles && ok; ++t)
-                for (int j = 0; j < QT && ok; ++j) ok = issue_s(j, t);
-            for (int t = 0; t < n_tiles && ok; ++t) {
-                const int stage = t % STAGES;
-                const uint32_t v_lo = (kv_lo + stage * (S::KV_STAGE >> 4) + (KV_BYTES >> 4)) | v_lbo;
-                for (int j = 0; j < QT && ok; ++j) {
-                    if (!mbar_wait(&bars->p_full[j][t & 1], (t >> 1) & 1, abort_flag)) { ok = false; break; }
-                    tc_fence_after_sync();
-                    // A: P in tensor memory, 16 keys = 8 columns per MMA; B: 16 key rows (2 KB) further down V
-                    const uint32_t pa = tmem_base + S::s_col(j, t % NBUF), od = tmem_base + S::o_col(j);
+            }
+            __syncwarp();
+            return true;
+        };
+        for (int t = 0; t < NBUF && t < n_tiles && ok; ++t)
+            for (int j = 0; j < QT && ok; ++j) ok = issue_s(j, t);
+        for (int t = 0; t < n_tiles && ok; ++t) {
+            const int stage = t % STAGES;
+            const uint32_t v_lo = (kv_lo + stage * (S::KV_STAGE >> 4) + (KV_BYTES >> 4)) | v_lbo;
+            for (int j = 0; j < QT && ok; ++j) {
+                if (!__all_sync(0xffffffffu, mbar_wait(&bars->p_full[j][t & 1], (t >> 1) & 1, abort_flag))) { ok = false; break; }
+                tc_fence_after_sync();
+                // A: P in tensor memory, 16 keys = 8 columns per MMA; B: 16 key rows (2 KB) further down V
+                const uint32_t pa = tmem_base + S::s_col(j, t % NBUF), od = tmem_base + S::o_col(j);
+                if (leader) {
                     if (t == 0) umma_bf16_ts_lo<false>(od, pa, v_lo, idesc_o);
                     else umma_bf16_ts_lo<true>(od, pa, v_lo, idesc_o);
 #pragma unroll
                     for (int kk = 1; kk < TC_KT / 16; ++kk)
                         umma_bf16_ts_lo<true>(od, pa + 8 * kk, v_lo + kk * (2048 >> 4), idesc_o);
                     umma_commit(&bars->pv_done[j][t & 1]);     // O holds tiles 0..t
-                    if (t + NBUF < n_tiles) ok = issue_s(j, t + NBUF);
                 }
-                if (ok) umma_commit(&bars->empty[stage]);      // every product that reads this K/V tile has been issued
+                __syncwarp();
+                if (t + NBUF < n_tiles) ok = issue_s(j, t + NBUF);
             }
+            if (ok && leader) umma_commit(&bars->empty[stage]);      // every product that reads this K/V tile has been issued
+            __syncwarp();
         }
     } else {
         // ---------------- softmax warps: set j = query tile, thread = packed query row r of that tile = TMEM lane r
